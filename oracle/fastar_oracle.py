@@ -1,0 +1,394 @@
+"""CPU oracle for the FAST-AR attention step (TempCache, AnnSA, AnnCA).
+
+TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, fp64 restatement of what
+the paper's method computes, written from the paper and sharing no code with
+the CUDA path.  Only tests, the smoke check and the bench's CPU-baseline leg may
+import it; the product path never does.
+
+Every function works on ONE head (the paper's formulas are per head:
+q in R^{d_k}, Lemma 1) and on float64 arrays whose values are the bf16-rounded
+inputs the GPU reads.  numpy matmul / argmax / lexsort are used as plain library
+steps; there is no blocking, fusion or reordering beyond the stated algorithm.
+
+Paper passages followed
+  * Eq. 1 (Section 3)            dense cached attention            -> dense_attention
+  * Section 5.1                  attention over a candidate set    -> sparse_attention
+  * Section 5.2 "Finding temporal correspondences"  top-1 key      -> top1_cosine
+  * Section 5.2 / Appendix C     threshold merge, last-key representative,
+                                 mean value, multiplicity m        -> tempcache_update
+  * Lemma 1 (Section 5.2, Appendix A)  + log m bias                -> sparse_attention
+  * Section 5.1 "LSH"            shared random projection, buckets -> lsh_codes
+  * Section 5.4 (AnnSA)          same-bucket rule, block-sparse    -> block_histograms,
+                                                                      block_scores, topk_lowest_index
+  * Section 5.3 (AnnCA)          prompt token kept iff a current-frame query
+                                 is its neighbour                  -> prompt_relevance, annca
+  * Section 4 / Section 6 "Metrics"  recall, density              -> attention_recall, density
+
+Pinned by tests/test_oracle_pins.py: Lemma exactness, brute-force nearest
+neighbour, cache invariants, reduction to dense attention (checked against
+torch's scaled_dot_product_attention), brute-force collision counts, hand-made
+eviction and top-k cases, closed-form fixtures under tests/golden/.
+Parity unpinned: the paper's recall/density/speed-up values (they need the
+paper's models and prompts) — nothing here reproduces them.
+
+Readings taken where the paper is silent (each listed in the design notes):
+key->key cosine matching against every live slot of the pre-call cache; ties to
+the lowest index; representative = newest frame, then highest similarity, then
+lowest token index; unmatched tokens appended in token order; at capacity the
+least-recently-touched slots (smallest (stamp, slot)) are overwritten; sign
+random projections with T tables of b bits; tile score = number of same-bucket
+(query, key, table) triples; fixed budgets with ties to the lower index; AnnCA
+relevance = max over the frame's queries of the scaled dot product.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+class CapacityError(RuntimeError):
+    """An update needed more eviction victims than the cache can offer; the cache is unchanged."""
+
+
+# --------------------------------------------------------------------------- #
+# storage rounding
+# --------------------------------------------------------------------------- #
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest bf16 value (8 significant bits, ties to even) of float64 x, as float64.
+    Sub-normal and overflow ranges are not treated (inputs are O(1))."""
+    x = np.asarray(x, dtype=np.float64)
+    mant, exp = np.frexp(x)
+    return np.ldexp(np.rint(mant * 256.0) / 256.0, exp)
+
+
+# --------------------------------------------------------------------------- #
+# cache state of one head
+# --------------------------------------------------------------------------- #
+@dataclass
+class HeadCache:
+    capacity: int
+    head_dim: int
+    n_sink: int = 0
+    store_bf16: bool = True                      # round merged values to the cache dtype
+    K: np.ndarray = field(init=False)            # [CAP][d] representative keys
+    V: np.ndarray = field(init=False)            # [CAP][d] group-mean values
+    m: np.ndarray = field(init=False)            # [CAP] multiplicity (Lemma 1: m_t)
+    stamp: np.ndarray = field(init=False)        # [CAP] update index of the last touch
+    L: int = 0                                   # live slots
+    now: int = 0                                 # update counter
+    evicted_tokens: int = 0
+    inserted_tokens: int = 0
+
+    def __post_init__(self):
+        self.K = np.zeros((self.capacity, self.head_dim), dtype=np.float64)
+        self.V = np.zeros((self.capacity, self.head_dim), dtype=np.float64)
+        self.m = np.zeros(self.capacity, dtype=np.int64)
+        self.stamp = np.zeros(self.capacity, dtype=np.int64)
+
+    def copy(self) -> "HeadCache":
+        c = HeadCache(self.capacity, self.head_dim, self.n_sink, self.store_bf16)
+        c.K, c.V, c.m, c.stamp = self.K.copy(), self.V.copy(), self.m.copy(), self.stamp.copy()
+        c.L, c.now, c.evicted_tokens, c.inserted_tokens = self.L, self.now, self.evicted_tokens, self.inserted_tokens
+        return c
+
+    def load(self, K, V, m=None, stamp=None, now: Optional[int] = None) -> None:
+        """Import a state (e.g. a checkpoint exported elsewhere)."""
+        n = K.shape[0]
+        self.K[:n], self.V[:n] = K, V
+        self.m[:n] = 1 if m is None else m
+        self.stamp[:n] = 0 if stamp is None else stamp
+        self.L = n
+        self.now = (int(self.stamp[:n].max()) + 1 if n else 0) if now is None else now
+        self.inserted_tokens = int(self.m[:n].sum())
+
+
+# --------------------------------------------------------------------------- #
+# TempCache (Section 5.2)
+# --------------------------------------------------------------------------- #
+def cosine_matrix(A: np.ndarray, B: np.ndarray) -> np.ndarray:
+    """c_ij = <a_i, b_j> / (|a_i| |b_j|), 0 where a norm is 0."""
+    A = np.asarray(A, np.float64)
+    B = np.asarray(B, np.float64)
+    na = np.sqrt(np.sum(A * A, axis=1))
+    nb = np.sqrt(np.sum(B * B, axis=1))
+    den = na[:, None] * nb[None, :]
+    dots = A @ B.T
+    return np.where(den > 0, dots / np.where(den > 0, den, 1.0), 0.0)
+
+
+def top1_cosine(K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.ndarray]:
+    """Temporal correspondence: for each new key its most similar live cached key
+    (ties -> smallest slot).  Returns (j*, c*); j* = -1 and c* = 0 on an empty cache."""
+    n = K_new.shape[0]
+    if cache.L == 0:
+        return np.full(n, -1, np.int64), np.zeros(n, np.float64)
+    c = cosine_matrix(K_new, cache.K[: cache.L])
+    j = np.argmax(c, axis=1)
+    return j.astype(np.int64), c[np.arange(n), j]
+
+
+def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
+                     forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None) -> Dict[str, np.ndarray]:
+    """One TempCache update of one head.
+
+    forced = (j*, c*, matched) replaces steps 1-2 by decisions taken elsewhere
+    (staged parity: near-ties have several correct answers)."""
+    K_new = np.asarray(K_new, np.float64)
+    V_new = np.asarray(V_new, np.float64)
+    n = K_new.shape[0]
+    L, CAP, now = cache.L, cache.capacity, cache.now
+
+    # 1. top-1 correspondence against the pre-call cache; 2. threshold
+    if forced is None:
+        jstar, cstar = top1_cosine(K_new, cache)
+        matched = (cstar >= tau) & (jstar >= 0)
+    else:
+        jstar, cstar, matched = (np.asarray(a) for a in forced)
+        matched = matched.astype(bool)
+
+    # plan the unmatched tokens before touching anything (validate, then commit)
+    unmatched = np.flatnonzero(~matched)
+    n_app = min(unmatched.size, CAP - L)
+    n_evict = unmatched.size - n_app
+    touched = np.unique(jstar[matched])
+    victims = np.zeros(0, np.int64)
+    if n_evict > 0:
+        evictable = cache.stamp[:L] < now                      # not written by this update ...
+        evictable[touched] = False                             # ... nor merged into by it
+        evictable[: cache.n_sink] = False                      # protected prefix
+        cand = np.flatnonzero(evictable).astype(np.int64)
+        if cand.size < n_evict:
+            raise CapacityError(f"need {n_evict} victims, only {cand.size} evictable")
+        order = np.lexsort((cand, cache.stamp[cand]))          # by stamp, then slot
+        victims = cand[order[:n_evict]]
+
+    dest = np.full(n, -1, np.int64)
+    frame_of = np.arange(n) // frame_len
+
+    # 3. merge every group into its slot
+    midx = np.flatnonzero(matched)
+    by_slot = midx[np.argsort(jstar[midx], kind="stable")]     # grouped by slot, ascending token index inside
+    bounds = np.flatnonzero(np.diff(jstar[by_slot], prepend=-2, append=-3))
+    for s0, s1 in zip(bounds[:-1], bounds[1:]):
+        G = by_slot[s0:s1]                                     # G_j, ascending token index
+        j = int(jstar[G[0]])
+        g = G.size
+        acc = cache.m[j] * cache.V[j]
+        for i in G:
+            acc = acc + V_new[i]
+        vbar = acc / (cache.m[j] + g)
+        cache.V[j] = round_to_bf16(vbar) if cache.store_bf16 else vbar
+        rep = min(G, key=lambda i: (-frame_of[i], -cstar[i], i))
+        cache.K[j] = K_new[rep]
+        cache.m[j] += g
+        cache.stamp[j] = now
+        dest[G] = j
+
+    # 4. unmatched tokens: append in token order, then overwrite victims
+    slots = np.concatenate([np.arange(L, L + n_app, dtype=np.int64), victims])
+    evicted_now = int(cache.m[victims].sum()) if victims.size else 0
+    for i, s in zip(unmatched, slots):
+        cache.K[s] = K_new[i]
+        cache.V[s] = V_new[i]
+        cache.m[s] = 1
+        cache.stamp[s] = now
+        dest[i] = s
+    cache.L = L + n_app
+    cache.evicted_tokens += evicted_now
+    cache.inserted_tokens += n
+
+    # 5. advance the clock
+    cache.now = now + 1
+    stats = dict(matched=int(matched.sum()), touched=int(touched.size), appended=int(n_app),
+                 evicted_slots=int(victims.size), evicted_tokens=evicted_now, length=int(cache.L))
+    match_out = np.where(matched, jstar, -1).astype(np.int64)
+    return dict(match=match_out, sim=np.asarray(cstar, np.float64), matched=matched, dest=dest, stats=stats,
+                jstar=np.asarray(jstar, np.int64))
+
+
+# --------------------------------------------------------------------------- #
+# LSH block selection (Sections 5.1, 5.4)
+# --------------------------------------------------------------------------- #
+def lsh_projections(X: np.ndarray, R: np.ndarray) -> np.ndarray:
+    """<x, r_c> for every row x and every direction r_c (R is [T*b][d])."""
+    return np.asarray(X, np.float64) @ np.asarray(R, np.float64).T
+
+
+def lsh_codes(X: np.ndarray, R: np.ndarray, tables: int, bits: int) -> np.ndarray:
+    """code_t(x) = sum_u [<x, R[t*b+u]> > 0] * 2^u   ->  [n][T] int64."""
+    proj = lsh_projections(X, R)
+    sign = (proj > 0).astype(np.int64).reshape(X.shape[0], tables, bits)
+    return (sign << np.arange(bits, dtype=np.int64)).sum(axis=2)
+
+
+def block_histograms(codes: np.ndarray, n_live: int, block: int, bits: int) -> np.ndarray:
+    """H[blk][t][w] = number of rows r < n_live of block blk with code_t = w."""
+    tables = codes.shape[1]
+    nblk = -(-n_live // block) if n_live > 0 else 0
+    H = np.zeros((nblk, tables, 1 << bits), dtype=np.int64)
+    rows = np.arange(n_live)
+    for t in range(tables):
+        np.add.at(H, (rows // block, t, codes[:n_live, t]), 1)
+    return H
+
+
+def block_scores(HQ: np.ndarray, HK: np.ndarray) -> np.ndarray:
+    """S[a][b] = sum_t sum_w HQ[a][t][w] * HK[b][t][w]  (same-bucket triples in tile (a,b))."""
+    a, b = HQ.shape[0], HK.shape[0]
+    return HQ.reshape(a, -1) @ HK.reshape(b, -1).T
+
+
+def topk_lowest_index(scores: np.ndarray, keep: int) -> np.ndarray:
+    """Per row, the min(keep, n) columns with the largest score (ties -> lower column),
+    listed in ascending column order.  -> [rows][min(keep, n)] int64."""
+    scores = np.asarray(scores)
+    rows, ncol = scores.shape
+    k = min(keep, ncol)
+    out = np.zeros((rows, k), dtype=np.int64)
+    cols = np.arange(ncol)
+    for r in range(rows):
+        order = np.lexsort((cols, -scores[r]))                 # by -score, then column
+        out[r] = np.sort(order[:k])
+    return out
+
+
+def sparse_attention(Q: np.ndarray, cache: HeadCache, sel: np.ndarray, block_q: int, block_k: int,
+                     return_probs: bool = False):
+    """o_i = sum_j softmax_j(<q_i, k_j>/sqrt(d) + ln m_j) V_j over the live slots j of the key
+    blocks sel[a(i)]  (candidate-set attention of Section 5.1 with Lemma 1's bias)."""
+    Q = np.asarray(Q, np.float64)
+    nq, d = Q.shape
+    O = np.zeros((nq, d), dtype=np.float64)
+    probs = [] if return_probs else None
+    if cache.L == 0:
+        return (O, probs) if return_probs else O
+    scale = 1.0 / np.sqrt(d)
+    for a in range(-(-nq // block_q)):
+        rows = np.arange(a * block_q, min((a + 1) * block_q, nq))
+        slots = np.concatenate([np.arange(b * block_k, min((b + 1) * block_k, cache.L)) for b in sel[a]]
+                               + [np.zeros(0, np.int64)]).astype(np.int64)
+        if slots.size == 0:
+            continue
+        logits = (Q[rows] @ cache.K[slots].T) * scale + np.log(cache.m[slots].astype(np.float64))[None, :]
+        logits -= logits.max(axis=1, keepdims=True)
+        p = np.exp(logits)
+        p /= p.sum(axis=1, keepdims=True)
+        O[rows] = p @ cache.V[slots]
+        if return_probs:
+            probs.append((rows, slots, p))
+    return (O, probs) if return_probs else O
+
+
+def annsa(Q: np.ndarray, cache: HeadCache, R: np.ndarray, tables: int, bits: int, block_q: int, block_k: int,
+          keep: int, qcodes: Optional[np.ndarray] = None, kcodes: Optional[np.ndarray] = None,
+          sel: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """AnnSA of one head.  qcodes/kcodes/sel, when given, replace the corresponding
+    stage by decisions taken elsewhere (staged parity)."""
+    nq = Q.shape[0]
+    if qcodes is None:
+        qcodes = lsh_codes(Q, R, tables, bits)
+    if kcodes is None:
+        kcodes = lsh_codes(cache.K[: cache.L], R, tables, bits) if cache.L else np.zeros((0, tables), np.int64)
+    HQ = block_histograms(qcodes, nq, block_q, bits)
+    HK = block_histograms(kcodes, cache.L, block_k, bits)
+    S = block_scores(HQ, HK) if cache.L else np.zeros((HQ.shape[0], 0), np.int64)
+    if sel is None:
+        sel = topk_lowest_index(S, keep) if cache.L else np.zeros((HQ.shape[0], 0), np.int64)
+    O = sparse_attention(Q, cache, sel, block_q, block_k)
+    return dict(out=O, sel=sel, scores=S, qcodes=qcodes, kcodes=kcodes)
+
+
+# --------------------------------------------------------------------------- #
+# AnnCA (Section 5.3)
+# --------------------------------------------------------------------------- #
+def prompt_relevance(Q: np.ndarray, K_p: np.ndarray, frame_len: int) -> np.ndarray:
+    """r[f][p] = max over the queries i of frame f of <q_i, k_p>/sqrt(d)."""
+    Q = np.asarray(Q, np.float64)
+    K_p = np.asarray(K_p, np.float64)
+    nq, d = Q.shape
+    F = -(-nq // frame_len)
+    s = (Q @ K_p.T) / np.sqrt(d)
+    return np.stack([s[f * frame_len: min((f + 1) * frame_len, nq)].max(axis=0) for f in range(F)])
+
+
+def annca(Q: np.ndarray, K_p: np.ndarray, V_p: np.ndarray, frame_len: int, keep: int,
+          sel: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """AnnCA of one head: per frame keep the `keep` most relevant prompt tokens, then
+    o_i = softmax_{p in sel[f(i)]}(<q_i, k_p>/sqrt(d)) v_p."""
+    Q = np.asarray(Q, np.float64)
+    K_p = np.asarray(K_p, np.float64)
+    V_p = np.asarray(V_p, np.float64)
+    nq, d = Q.shape
+    r = prompt_relevance(Q, K_p, frame_len)
+    if sel is None:
+        sel = topk_lowest_index(r, keep)
+    O = np.zeros((nq, d))
+    for f in range(r.shape[0]):
+        rows = np.arange(f * frame_len, min((f + 1) * frame_len, nq))
+        P = np.asarray(sel[f], np.int64)
+        logits = (Q[rows] @ K_p[P].T) / np.sqrt(d)
+        logits -= logits.max(axis=1, keepdims=True)
+        p = np.exp(logits)
+        p /= p.sum(axis=1, keepdims=True)
+        O[rows] = p @ V_p[P]
+    return dict(out=O, sel=sel, relevance=r)
+
+
+# --------------------------------------------------------------------------- #
+# Eq. 1 and the diagnostics of Sections 4 / 6
+# --------------------------------------------------------------------------- #
+def dense_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, return_probs: bool = False):
+    """O = softmax(Q K^T / sqrt(d)) V   (Eq. 1)."""
+    Q, K, V = (np.asarray(a, np.float64) for a in (Q, K, V))
+    logits = (Q @ K.T) / np.sqrt(Q.shape[1])
+    logits -= logits.max(axis=1, keepdims=True)
+    p = np.exp(logits)
+    p /= p.sum(axis=1, keepdims=True)
+    return (p @ V, p) if return_probs else p @ V
+
+
+def attention_recall(Q: np.ndarray, cache: HeadCache, sel: np.ndarray, block_q: int, block_k: int) -> float:
+    """Share of the (bias-corrected) dense attention mass over the live cache that falls on
+    the keys of the selected blocks, averaged over queries."""
+    Q = np.asarray(Q, np.float64)
+    L = cache.L
+    logits = (Q @ cache.K[:L].T) / np.sqrt(Q.shape[1]) + np.log(cache.m[:L].astype(np.float64))[None, :]
+    logits -= logits.max(axis=1, keepdims=True)
+    p = np.exp(logits)
+    p /= p.sum(axis=1, keepdims=True)
+    tot = 0.0
+    for a in range(-(-Q.shape[0] // block_q)):
+        rows = slice(a * block_q, min((a + 1) * block_q, Q.shape[0]))
+        for b in sel[a]:
+            tot += p[rows, b * block_k: min((b + 1) * block_k, L)].sum()
+    return tot / Q.shape[0]
+
+
+def density(nq: int, L: int, sel: np.ndarray, block_q: int, block_k: int) -> float:
+    """Executed (query, key) pairs / dense pairs."""
+    pairs = 0
+    for a in range(-(-nq // block_q)):
+        rows = min((a + 1) * block_q, nq) - a * block_q
+        for b in sel[a]:
+            pairs += rows * (min((b + 1) * block_k, L) - b * block_k)
+    return pairs / float(nq * L)
+
+
+# --------------------------------------------------------------------------- #
+# multi-head convenience (heads are independent)
+# --------------------------------------------------------------------------- #
+class OracleCache:
+    def __init__(self, num_heads: int, head_dim: int, capacity: int, n_sink: int = 0, store_bf16: bool = True):
+        self.heads: List[HeadCache] = [HeadCache(capacity, head_dim, n_sink, store_bf16) for _ in range(num_heads)]
+
+    def update(self, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
+               forced: Optional[Sequence] = None) -> List[Dict[str, np.ndarray]]:
+        return [tempcache_update(hc, K_new[h], V_new[h], frame_len, tau, None if forced is None else forced[h])
+                for h, hc in enumerate(self.heads)]
+
+    def copy(self) -> "OracleCache":
+        c = OracleCache.__new__(OracleCache)
+        c.heads = [h.copy() for h in self.heads]
+        return c

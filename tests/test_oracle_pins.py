@@ -1,0 +1,383 @@
+"""Pins for the CPU oracle: everything here checks oracle/ against something other than
+itself -- closed forms, brute force in plain Python loops, invariants the paper states,
+special cases that reduce to a library routine (torch's fp64 scaled_dot_product_attention).
+No GPU, no CUDA library."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import fastar_oracle as O
+from paper_2602_01801_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rng(s):
+    return np.random.default_rng(s)
+
+
+def _sdpa(Q, K, V):
+    q, k, v = (torch.from_numpy(np.asarray(a, np.float64))[None, None] for a in (Q, K, V))
+    return torch.nn.functional.scaled_dot_product_attention(q, k, v)[0, 0].numpy()
+
+
+def _all_blocks(nq, L, bq, bk):
+    return np.tile(np.arange(-(-L // bk)), (-(-nq // bq), 1))
+
+
+# ----------------------------------------------------------------------------- storage
+def test_round_to_bf16_matches_torch():
+    x = _rng(0).standard_normal(20000) * np.exp(_rng(1).uniform(-8, 8, 20000))
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    # torch rounds fp64->bf16 through fp32 in places; compare only where that cannot double-round
+    f32 = x.astype(np.float32).astype(np.float64)
+    safe = np.abs(f32 - x) < 1e-12 * np.abs(x) + 1e-300
+    got = O.round_to_bf16(x)
+    assert np.array_equal(got[safe], want[safe])
+    assert np.all(np.abs(got - x) <= np.abs(x) * 2.0 ** -8)
+    xs = synth.round_bf16(x.astype(np.float32)).astype(np.float64)       # already bf16: fixed points
+    assert np.array_equal(O.round_to_bf16(xs), xs)
+
+
+def test_synth_bf16_bits_match_torch():
+    x = _rng(2).standard_normal(5000).astype(np.float32)
+    bits = synth.f32_to_bf16_bits(x)
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(bits, want)
+
+
+# ----------------------------------------------------------------------------- Lemma 1
+def _read_golden(name):
+    out = {}
+    for line in open(os.path.join(GOLDEN, name)):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, *v = line.split()
+        out[k] = np.array([float(t) for t in v])
+    return out
+
+
+def test_lemma_closed_form_fixture():
+    g = _read_golden("lemma_closed_form.txt")
+    q = g["q"][None, :]
+    K, V = g["keys"].reshape(3, 2), g["values"].reshape(3, 2)
+    assert np.allclose(O.dense_attention(q, K, V)[0], g["expected"], atol=1e-14)
+    c = O.HeadCache(4, 2, store_bf16=False)
+    c.load(K=np.array([K[0], K[2]]), V=np.array([(V[0] + V[1]) / 2, V[2]]), m=np.array([2, 1]))
+    o = O.sparse_attention(q, c, np.array([[0]]), 1, 4)
+    assert np.allclose(o[0], g["expected"], atol=1e-14)
+
+
+def _duplicate_stream(H, d, n, chunks, seed):
+    """Chunks whose keys repeat exactly (sigma = 0, no resampling); values differ."""
+    r = _rng(seed)
+    base = synth.round_bf16(r.standard_normal((n, d)).astype(np.float32)).astype(np.float64)
+    Ks = [base[r.permutation(n)] for _ in range(chunks)]
+    Vs = [synth.round_bf16(r.standard_normal((n, d)).astype(np.float32)).astype(np.float64) for _ in range(chunks)]
+    return Ks, Vs
+
+
+def test_lemma_exact_on_duplicate_keys():
+    d, n = 16, 48
+    Ks, Vs = _duplicate_stream(1, d, n, 5, 3)
+    c = O.HeadCache(64, d, store_bf16=False)
+    for K, V in zip(Ks, Vs):
+        O.tempcache_update(c, K, V, frame_len=n, tau=1 - 1e-6)
+    assert c.L == n and np.all(c.m[:n] == 5)
+    Q = _rng(4).standard_normal((20, d))
+    got = O.sparse_attention(Q, c, _all_blocks(20, c.L, 8, 16), 8, 16)
+    want = _sdpa(Q, np.concatenate(Ks), np.concatenate(Vs))
+    assert np.max(np.abs(got - want)) < 1e-12
+
+
+def test_zero_query_gives_mean_of_all_values():
+    d, n = 8, 32
+    Ks, Vs = _duplicate_stream(1, d, n, 3, 5)
+    Ks.append(synth.round_bf16(_rng(6).standard_normal((n, d)).astype(np.float32)).astype(np.float64))
+    Vs.append(_rng(7).standard_normal((n, d)))
+    c = O.HeadCache(128, d, store_bf16=False)
+    for K, V in zip(Ks, Vs):
+        O.tempcache_update(c, K, V, n, 0.999)
+    o = O.sparse_attention(np.zeros((1, d)), c, _all_blocks(1, c.L, 4, 16), 4, 16)
+    assert np.allclose(o[0], np.concatenate(Vs).mean(axis=0), atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- T1
+def test_top1_brute_force():
+    r = _rng(8)
+    d, n, L = 6, 9, 13
+    c = O.HeadCache(16, d)
+    Kc = r.standard_normal((L, d))
+    Kc[4] = Kc[2]                                                   # an exact tie -> lower slot
+    c.load(Kc, r.standard_normal((L, d)))
+    Kn = r.standard_normal((n, d))
+    Kn[3] = 2.5 * Kc[2]
+    j, s = O.top1_cosine(Kn, c)
+    for i in range(n):
+        best, bj = -2.0, -1
+        for jj in range(L):
+            dot = sum(Kn[i][t] * Kc[jj][t] for t in range(d))
+            cs = dot / (math.sqrt(sum(x * x for x in Kn[i])) * math.sqrt(sum(x * x for x in Kc[jj])))
+            if cs > best + 1e-15:
+                best, bj = cs, jj
+        assert j[i] == bj and abs(s[i] - best) < 1e-14
+    assert j[3] == 2 and abs(s[3] - 1) < 1e-14
+    je, se = O.top1_cosine(Kn, O.HeadCache(16, d))
+    assert np.all(je == -1) and np.all(se == 0)
+
+
+def test_zero_norm_key_has_zero_similarity():
+    c = O.HeadCache(4, 3)
+    c.load(np.array([[0.0, 0, 0], [1, 0, 0]]), np.zeros((2, 3)))
+    j, s = O.top1_cosine(np.array([[0.0, 0, 0], [-1, 0, 0]]), c)
+    assert s[0] == 0 and j[0] == 0
+    assert j[1] == 0 and s[1] == 0          # cos with slot 1 is -1, with the zero key 0
+
+
+# ----------------------------------------------------------------------------- T2-T4
+def _c0_like(chunks, seed=0, **kw):
+    cfg = synth.small_config(num_heads=1, head_dim=32, grid_h=8, grid_w=8, frames_per_chunk=2, clusters=12,
+                             capacity=512, block=32, seed=seed, **kw)
+    w = synth.Workload(cfg)
+    return cfg, [w.chunk(i) for i in range(chunks)]
+
+
+def test_update_invariants_and_last_key():
+    cfg, chunks = _c0_like(5)
+    c = O.HeadCache(cfg.capacity, cfg.head_dim, store_bf16=False)
+    total_v = np.zeros(cfg.head_dim)
+    inserted = 0
+    saw_merge = False
+    for (_, K, V) in chunks:
+        K, V = K[0].astype(np.float64), V[0].astype(np.float64)
+        L0, now = c.L, c.now
+        res = O.tempcache_update(c, K, V, cfg.frame_len, 0.9)
+        st = res["stats"]
+        inserted += K.shape[0]
+        total_v += V.sum(axis=0)
+        assert c.L == L0 + st["appended"] <= cfg.capacity
+        assert st["matched"] + st["appended"] + st["evicted_slots"] == K.shape[0]
+        assert int(c.m[: c.L].sum()) + c.evicted_tokens == inserted == c.inserted_tokens
+        assert np.allclose((c.m[: c.L, None] * c.V[: c.L]).sum(axis=0), total_v, atol=1e-9)
+        written = np.flatnonzero(c.stamp[: c.L] == now)
+        keyset = {K[i].tobytes() for i in range(K.shape[0])}
+        assert all(c.K[j].tobytes() in keyset for j in written)         # last-key: bit copies of new keys
+        assert np.all(c.K[res["dest"]][~res["matched"]] == K[~res["matched"]])
+        saw_merge |= st["matched"] > 0
+        assert c.now == now + 1
+    assert saw_merge and c.m[: c.L].max() > 1
+
+
+def test_tau_above_one_is_plain_append_and_length_is_monotone_in_tau():
+    cfg, chunks = _c0_like(3, seed=1)
+    lens = []
+    for tau in (1.5, 0.95, 0.9, 0.7, 0.5):
+        c = O.HeadCache(cfg.capacity, cfg.head_dim)
+        for (_, K, V) in chunks:
+            O.tempcache_update(c, K[0], V[0], cfg.frame_len, tau)
+        lens.append(c.L)
+        if tau > 1:
+            allK = np.concatenate([k[0] for (_, k, _) in chunks]).astype(np.float64)
+            allV = np.concatenate([v[0] for (_, _, v) in chunks]).astype(np.float64)
+            assert c.L == allK.shape[0] and np.all(c.m[: c.L] == 1)
+            assert np.array_equal(c.K[: c.L], allK) and np.array_equal(c.V[: c.L], allV)
+    assert all(a >= b for a, b in zip(lens, lens[1:])) and lens[0] > lens[-1]
+
+
+def test_representative_is_newest_frame_then_highest_similarity_then_lowest_index():
+    d = 4
+    c = O.HeadCache(8, d, store_bf16=False)
+    c.load(np.array([[1.0, 0, 0, 0], [0, 1.0, 0, 0]]), np.array([[10.0, 0, 0, 0], [0, 0, 0, 0]]), m=np.array([3, 1]))
+    # frame_len 2: tokens 0,1 frame 0; tokens 2,3 frame 1.  All but token 1 match slot 0.
+    K = np.array([[1.0, 0.01, 0, 0], [0, 0, 1.0, 0], [1.0, 0.2, 0, 0], [1.0, 0.1, 0, 0]])
+    V = np.array([[1.0, 0, 0, 0], [7.0, 7, 7, 7], [2.0, 0, 0, 0], [3.0, 0, 0, 0]])
+    res = O.tempcache_update(c, K, V, frame_len=2, tau=0.9)
+    assert list(res["match"]) == [0, -1, 0, 0]
+    assert np.array_equal(c.K[0], K[3])            # newest frame (tokens 2,3), higher cosine is token 3
+    assert c.m[0] == 6 and np.allclose(c.V[0], [(30 + 1 + 2 + 3) / 6, 0, 0, 0])
+    assert list(res["dest"]) == [0, 2, 0, 0] and c.L == 3 and np.array_equal(c.K[2], K[1])
+    # identical similarity inside the newest frame -> lowest token index
+    c2 = O.HeadCache(8, d, store_bf16=False)
+    c2.load(np.array([[1.0, 0, 0, 0]]), np.zeros((1, d)))
+    K2 = np.array([[2.0, 0, 0, 0], [3.0, 0, 0, 0]])
+    O.tempcache_update(c2, K2, np.zeros((2, d)), frame_len=2, tau=0.9)
+    assert np.array_equal(c2.K[0], K2[0])
+
+
+def test_eviction_takes_least_recently_touched_slots_in_order():
+    d = 3
+    c = O.HeadCache(6, d, n_sink=1, store_bf16=False)
+    e = np.eye(3)
+    K0 = np.array([e[0], e[1], e[2], -e[0], -e[1], -e[2]])
+    c.load(K0, np.arange(18.0).reshape(6, 3), m=np.array([1, 2, 3, 4, 5, 6]), stamp=np.array([0, 3, 1, 1, 2, 0]), now=4)
+    # token 0 merges into slot 2 (so slot 2 is not evictable); tokens 1..3 are new directions
+    K = np.array([e[2], [1.0, 1, 0], [0, 1.0, 1], [1.0, 0, 1]])
+    V = np.ones((4, 3))
+    res = O.tempcache_update(c, K, V, frame_len=4, tau=0.9)
+    # candidates (slot>=1, stamp<4, untouched): 1(s3) 3(s1) 4(s2) 5(s0)  -> order 5, 3, 4
+    assert list(res["dest"]) == [2, 5, 3, 4]
+    assert res["stats"]["evicted_tokens"] == 6 + 4 + 5 and c.evicted_tokens == 15
+    assert c.L == 6 and list(c.m) == [1, 2, 4, 1, 1, 1] and list(c.stamp) == [0, 3, 4, 4, 4, 4]
+    assert int(c.m.sum()) + c.evicted_tokens == c.inserted_tokens == 21 + 4
+
+
+def test_capacity_error_leaves_cache_unchanged():
+    d = 3
+    c = O.HeadCache(2, d)
+    c.load(np.eye(3)[:2], np.zeros((2, 3)), stamp=np.array([0, 0]), now=1)
+    O.tempcache_update(c, np.eye(3)[:2], np.ones((2, 3)), 2, 0.9)     # both slots touched at now=1
+    before = c.copy()
+    with pytest.raises(O.CapacityError):
+        # slot 0 is touched by token 0; slot 1 alone cannot host two unmatched tokens
+        O.tempcache_update(c, np.array([[1.0, 0, 0], [0, 0, 1.0], [1.0, 0, 1.0]]), np.ones((3, 3)), 3, 0.9)
+    for a in ("K", "V", "m", "stamp"):
+        assert np.array_equal(getattr(c, a), getattr(before, a))
+    assert (c.L, c.now, c.evicted_tokens) == (before.L, before.now, before.evicted_tokens)
+
+
+# ----------------------------------------------------------------------------- S1-S4
+def test_lsh_codes_hand_case():
+    R = np.array([[1.0, 0], [0, 1.0], [-1.0, 0], [1.0, 1.0]])          # T=2 tables x b=2 bits, d=2
+    X = np.array([[1.0, 2.0], [-1.0, 0.5], [0.0, -3.0], [0.0, 0.0]])
+    codes = O.lsh_codes(X, R, tables=2, bits=2)
+    # table 0 bits (x0>0, x1>0), table 1 bits (-x0>0, x0+x1>0); bit u has weight 2^u; 0 is not > 0
+    assert codes.tolist() == [[3, 2], [2, 1], [0, 0], [0, 0]]
+
+
+def test_block_scores_equal_brute_force_collision_count():
+    r = _rng(11)
+    T, b, bq, bk, nq, L = 3, 2, 4, 5, 10, 17
+    qc = r.integers(0, 1 << b, (nq, T))
+    kc = r.integers(0, 1 << b, (L + 3, T))                             # rows >= L are dead slots
+    S = O.block_scores(O.block_histograms(qc, nq, bq, b), O.block_histograms(kc, L, bk, b))
+    assert S.shape == (3, 4)
+    for a in range(3):
+        for bb in range(4):
+            cnt = 0
+            for i in range(a * bq, min((a + 1) * bq, nq)):
+                for j in range(bb * bk, min((bb + 1) * bk, L)):
+                    for t in range(T):
+                        cnt += int(qc[i, t] == kc[j, t])
+            assert S[a, bb] == cnt
+
+
+def test_topk_rule_against_python_sort():
+    r = _rng(12)
+    S = r.integers(0, 4, (7, 11))
+    for keep in (1, 3, 11, 20):
+        sel = O.topk_lowest_index(S, keep)
+        for a in range(7):
+            want = sorted(sorted(range(11), key=lambda c: (-S[a, c], c))[: min(keep, 11)])
+            assert sel[a].tolist() == want
+    assert O.topk_lowest_index(np.array([[5, 9, 9, 1]]), 2).tolist() == [[1, 2]]
+    assert O.topk_lowest_index(np.array([[5, 5, 5, 5]]), 2).tolist() == [[0, 1]]
+
+
+# ----------------------------------------------------------------------------- S5 / D
+def test_keep_all_and_no_merge_is_dense_attention():
+    cfg, chunks = _c0_like(3, seed=2)
+    c = O.HeadCache(cfg.capacity, cfg.head_dim)
+    for (_, K, V) in chunks:
+        O.tempcache_update(c, K[0], V[0], cfg.frame_len, tau=2.0)
+    Q = chunks[-1][0][0].astype(np.float64)
+    R = synth.Workload(cfg).lsh_projection()
+    res = O.annsa(Q, c, R, cfg.lsh_tables, cfg.lsh_bits, cfg.block, cfg.block, keep=10 ** 6)
+    nkb = -(-c.L // cfg.block)
+    assert np.array_equal(res["sel"], _all_blocks(Q.shape[0], c.L, cfg.block, cfg.block)) and res["sel"].shape[1] == nkb
+    want = _sdpa(Q, np.concatenate([k[0] for (_, k, _) in chunks]), np.concatenate([v[0] for (_, _, v) in chunks]))
+    assert np.max(np.abs(res["out"] - want)) < 1e-12
+    assert np.max(np.abs(O.dense_attention(Q, c.K[: c.L], c.V[: c.L]) - want)) < 1e-12
+
+
+def test_single_key_and_probabilities():
+    d = 8
+    c = O.HeadCache(4, d)
+    v = _rng(13).standard_normal((1, d))
+    c.load(_rng(14).standard_normal((1, d)), v, m=np.array([7]))
+    Q = _rng(15).standard_normal((5, d))
+    assert np.allclose(O.sparse_attention(Q, c, np.zeros((2, 1), np.int64), 4, 4), np.repeat(v, 5, 0), atol=1e-15)
+    c2 = O.HeadCache(64, d)
+    c2.load(_rng(16).standard_normal((37, d)), _rng(17).standard_normal((37, d)), m=_rng(18).integers(1, 9, 37))
+    sel = np.array([[0, 2], [1, 4]])
+    _, probs = O.sparse_attention(Q, c2, sel, 4, 8, return_probs=True)
+    for rows, slots, p in probs:
+        assert np.allclose(p.sum(axis=1), 1, atol=1e-14)
+    assert probs[1][1].tolist() == list(range(8, 16)) + list(range(32, 37))      # ragged last block
+    # the bias: doubling m of one slot doubles its odds
+    p0 = probs[0][2][0]
+    c2.m[3] *= 2
+    _, probs2 = O.sparse_attention(Q, c2, sel, 4, 8, return_probs=True)
+    p1 = probs2[0][2][0]
+    k = probs[0][1].tolist().index(3)
+    assert np.isclose(p1[k] / (1 - p1[k]), 2 * p0[k] / (1 - p0[k]), rtol=1e-12)
+
+
+def test_empty_cache_attention_is_zero():
+    c = O.HeadCache(8, 4)
+    out = O.annsa(np.ones((3, 4)), c, np.ones((2, 4)), 1, 2, 2, 2, keep=2)
+    assert np.all(out["out"] == 0) and out["sel"].shape == (2, 0)
+
+
+# ----------------------------------------------------------------------------- C1-C3
+def test_annca_keep_all_is_dense_cross_attention_and_brute_force_relevance():
+    r = _rng(19)
+    nq, npr, d, fl = 23, 9, 8, 10
+    Q, Kp, Vp = r.standard_normal((nq, d)), r.standard_normal((npr, d)), r.standard_normal((npr, d))
+    res = O.annca(Q, Kp, Vp, fl, keep=npr)
+    assert np.max(np.abs(res["out"] - _sdpa(Q, Kp, Vp))) < 1e-12
+    rel = res["relevance"]
+    assert rel.shape == (3, npr)
+    for f in range(3):
+        for p in range(npr):
+            best = max(sum(Q[i][t] * Kp[p][t] for t in range(d)) / math.sqrt(d) for i in range(f * fl, min((f + 1) * fl, nq)))
+            assert abs(rel[f, p] - best) < 1e-13
+    res2 = O.annca(Q, Kp, Vp, fl, keep=3)
+    for f in range(3):
+        P = sorted(sorted(range(npr), key=lambda p: (-rel[f, p], p))[:3])
+        assert res2["sel"][f].tolist() == P
+        rows = slice(f * fl, min((f + 1) * fl, nq))
+        assert np.max(np.abs(res2["out"][rows] - _sdpa(Q[rows], Kp[P], Vp[P]))) < 1e-12
+
+
+def test_annca_selects_planted_prompt_tokens():
+    cfg = synth.CONFIGS["c0"]
+    w = synth.Workload(cfg)
+    Q, _, _ = w.chunk(4)
+    Kp, Vp, planted = w.prompt(4)
+    res = O.annca(Q[0], Kp[0], Vp[0], cfg.frame_len, cfg.keep_prompt)
+    assert set(planted[0].tolist()) <= set(res["sel"][0].tolist())
+
+
+# ----------------------------------------------------------------------------- diagnostics + workload sanity
+def test_density_and_recall_definitions():
+    d = 8
+    c = O.HeadCache(64, d)
+    c.load(_rng(20).standard_normal((64, d)), _rng(21).standard_normal((64, d)))
+    Q = _rng(22).standard_normal((16, d))
+    sel = np.array([[0, 3], [1, 2]])
+    assert O.density(16, 64, sel, 8, 16) == pytest.approx(2 * 16 / 64)
+    assert O.attention_recall(Q, c, _all_blocks(16, 64, 8, 16), 8, 16) == pytest.approx(1.0)
+    assert 0 < O.attention_recall(Q, c, sel, 8, 16) < 1
+
+
+def test_c0_workload_behaves_as_designed():
+    cfg = synth.CONFIGS["c0"]
+    w = synth.Workload(cfg)
+    c = O.HeadCache(cfg.capacity, cfg.head_dim)
+    for t in range(cfg.prior_chunks):
+        _, K, V = w.chunk(t)
+        O.tempcache_update(c, K[0], V[0], cfg.frame_len, tau=2.0)
+    assert c.L == 1024
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    res = O.tempcache_update(c, K[0], V[0], cfg.frame_len, cfg.tau)
+    st = res["stats"]
+    assert 0.8 * 256 <= st["matched"] <= 0.92 * 256            # all but the ~10 % resampled tokens
+    assert st["appended"] == 256 - st["matched"] and st["touched"] <= st["matched"]
+    R = w.lsh_projection()
+    a = O.annsa(Q[0].astype(np.float64), c, R, cfg.lsh_tables, cfg.lsh_bits, cfg.block, cfg.block, cfg.keep_blocks)
+    assert a["sel"].shape == (4, 4)
+    rec = O.attention_recall(Q[0], c, a["sel"], cfg.block, cfg.block)
+    assert rec > 0.5                                            # the selector finds the mass on clustered data
