@@ -1,0 +1,186 @@
+/*
+ * fastar.h -- C ABI of the B200 (sm_100a) FAST-AR attention step.
+ *
+ * One library, three hot calls, after the three components of the method
+ * (paper Section 5):
+ *   fastar_tempcache_update   TempCache, Section 5.2 (temporal-correspondence KV compression,
+ *                             Lemma 1: multiplicity m and mean value per representative key)
+ *   fastar_annsa_attention    AnnSA, Section 5.4 over Section 5.1 (LSH buckets -> block-sparse
+ *                             self-attention over the compressed cache, logits shifted by log m)
+ *   fastar_annca_attention    AnnCA, Section 5.3 (cross-attention over the frame-relevant
+ *                             prompt tokens only)
+ * plus cache create / reset / destroy / export / import.
+ *
+ * Conventions
+ *   - Every function returns an int status: FASTAR_OK (0) or a negative FASTAR_ERR_*.
+ *     Argument errors are detected on the host before anything is launched.  Conditions only
+ *     the device can see (capacity overflow of an update, a bounded wait that ran out) are
+ *     written to a device status word, read back by fastar_last_device_status().
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory
+ *     (pinned memory makes the copies asynchronous).  `stream` is a cudaStream_t passed as
+ *     void* (0 = the legacy default stream).  All work is enqueued on that stream and the
+ *     call returns without synchronising unless stated otherwise.
+ *   - Ownership: the caller owns every tensor and the workspace buffer; the library owns only
+ *     the small host object behind fastar_cache_t.  Nothing here allocates device memory.
+ *   - Tensors are [head][token][channel] with element strides `head_stride`, `token_stride`
+ *     (channel stride 1).  Strides in bytes must be multiples of 16 and base pointers 16-byte
+ *     aligned (TMA requirement).  Element type is the cache's `dtype`: bf16, or fp32 which is
+ *     rounded to bf16 (nearest-even) on entry; outputs are written in the same type.
+ *   - Heads are independent (the paper's formulas are per head); cache lengths are ragged
+ *     across heads and live on the device, so no call needs a host round trip.
+ *   - There is no CPU fallback: a device that is not compute capability 10.x yields
+ *     FASTAR_ERR_NOT_SM100.
+ */
+#ifndef FASTAR_H_
+#define FASTAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FASTAR_OK                      0
+#define FASTAR_ERR_INVALID_ARG        -1
+#define FASTAR_ERR_UNSUPPORTED_SHAPE  -2
+#define FASTAR_ERR_CAPACITY           -3   /* update needed more eviction victims than exist; cache unchanged */
+#define FASTAR_ERR_CUDA               -4
+#define FASTAR_ERR_TIMEOUT            -5   /* a bounded device-side wait gave up */
+#define FASTAR_ERR_NOT_SM100          -6
+#define FASTAR_ERR_WORKSPACE          -7   /* workspace buffer too small or misaligned */
+
+typedef struct fastar_cache fastar_cache_t;          /* opaque host object */
+
+typedef enum { FASTAR_BF16 = 0, FASTAR_FP32 = 1 } fastar_dtype_t;
+
+typedef struct {
+  int32_t num_heads;         /* H >= 1 */
+  int32_t head_dim;          /* d = value dim: 64 or 128 */
+  int32_t capacity;          /* CAP, tokens per head; multiple of page_tokens */
+  int32_t page_tokens;       /* page size = AnnSA key block Bk: 64 or 128 */
+  int32_t n_sink;            /* first n_sink slots are never evicted (0 = off) */
+  int32_t lsh_tables;        /* T in [1,4] */
+  int32_t lsh_bits;          /* b in [1,8] */
+  int32_t max_tokens;        /* largest n / nq of any call (sizes the scratch area) */
+  int32_t max_prompt_tokens; /* largest np of any AnnCA call */
+  int32_t max_frames;        /* largest number of frames per AnnCA call */
+  int32_t dtype;             /* fastar_dtype_t of the tensors the caller passes */
+  int32_t device;            /* CUDA device ordinal */
+} fastar_cache_desc;
+
+typedef struct {
+  int32_t matched;           /* new tokens merged into an existing slot */
+  int32_t touched;           /* distinct slots they were merged into */
+  int32_t appended;          /* unmatched tokens written to fresh slots */
+  int32_t evicted_slots;     /* unmatched tokens that overwrote a victim slot */
+  int32_t evicted_tokens;    /* sum of the victims' multiplicities */
+  int32_t length;            /* live slots after the update */
+  int32_t ok;                /* 1 = applied, 0 = rejected (FASTAR_ERR_CAPACITY), cache unchanged */
+  int32_t reserved;
+} fastar_update_stats;
+
+/* Bytes of device workspace a cache with this description needs (0 on an invalid description).
+ * Layout: paged K and V pools (bf16, one page = page_tokens x d), page table, per-slot
+ * multiplicity / stamp / log2(m) / 1/|k| / LSH code, per-block bucket histograms, per-head
+ * length, and the per-call scratch area. */
+size_t fastar_cache_workspace_bytes(const fastar_cache_desc* desc);
+
+/* Create a cache over the caller's workspace `dev_buf` (>= workspace_bytes, 1024-byte aligned).
+ * `lsh_proj_host`: the shared random projection of Section 5.1, host fp32 [T*b][d] (row t*b+u is
+ * bit u of table t); rounded to bf16.  The random numbers are an input so that any generator can
+ * be used.  Synchronous: the cache is reset (empty, clock 0) on return. */
+int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc,
+                        const float* lsh_proj_host, void* dev_buf, size_t bytes);
+
+/* Empty the cache: every length 0, clock 0, multiplicities 0, K/V pools zeroed.  Asynchronous. */
+int fastar_cache_reset(fastar_cache_t* cache, void* stream);
+
+/* Free the host object.  Never frees or touches dev_buf. */
+int fastar_cache_destroy(fastar_cache_t* cache);
+
+/* Copy the cache state to host buffers (any pointer may be NULL to skip it) and synchronise
+ * the stream.  host_k/host_v: bf16 bit patterns [H][CAP][d]; count (multiplicity m), stamp,
+ * code (LSH code, 8 bits per table, table t in byte t): [H][CAP]; len: [H]; now: [1]. */
+int fastar_cache_export(fastar_cache_t* cache, uint16_t* host_k, uint16_t* host_v, int32_t* count,
+                        int32_t* stamp, uint32_t* code, int32_t* len, int32_t* now, void* stream);
+
+/* Load a state (same layouts; count/stamp NULL = all ones / all zeros).  Slots >= len[h] are
+ * cleared.  Derived per-slot data (1/|k|, log2 m, LSH codes, histograms) are recomputed on the
+ * device.  `now` must exceed every stamp.  Synchronises the stream. */
+int fastar_cache_import(fastar_cache_t* cache, const uint16_t* host_k, const uint16_t* host_v,
+                        const int32_t* count, const int32_t* stamp, const int32_t* len, int32_t now,
+                        void* stream);
+
+/* TempCache update (Section 5.2; threshold merge and last-key representative: Section 5.2 last
+ * paragraph and Appendix C).  For every head, all n new tokens are matched against the cache as
+ * it was before the call:
+ *   j*_i = argmax_j cos(k_i, K_j) over live slots (ties: lowest slot), matched iff cos >= tau;
+ *   every touched slot j takes the mean value (m_j V_j + sum v_i)/(m_j + g), the key of its
+ *   newest matching token (latest frame floor(i/frame_len), then highest cosine, then lowest i),
+ *   m_j += g, stamp = clock;
+ *   unmatched tokens are appended in token order; when the capacity is reached they overwrite
+ *   the least recently touched slots (smallest (stamp, slot), slots >= n_sink, not touched by
+ *   this call).  If there are too few such slots nothing is changed, stats.ok = 0 and the
+ *   device status becomes FASTAR_ERR_CAPACITY.
+ * k_new, v_new: dev [H][n][d].  Optional dev outputs: match_out [H][n] (slot or -1),
+ * sim_out [H][n] (best cosine, 0 on an empty cache), dest_out [H][n] (slot that now holds or
+ * absorbed token i), stats_out [H].  n <= max_tokens, n <= 16384. */
+int fastar_tempcache_update(fastar_cache_t* cache, const void* k_new, const void* v_new, int32_t n,
+                            int32_t frame_len, int64_t head_stride, int64_t token_stride, float tau,
+                            int32_t* match_out, float* sim_out, int32_t* dest_out,
+                            fastar_update_stats* stats_out, void* stream);
+
+/* AnnSA (Sections 5.1 and 5.4 with the bias of Lemma 1).  Queries are cut into blocks of block_q
+ * rows, the cache into blocks of page_tokens slots.  Each query and key gets T b-bit codes (signs
+ * of the shared random projection); tile (a, b) scores the number of (query, key, table) triples
+ * with equal code; each query block keeps its min(keep_blocks, live blocks) best key blocks (ties:
+ * lower block) and attends to them only:
+ *   o_i = sum_j softmax_j(q_i.K_j/sqrt(d) + ln m_j) V_j    over live slots j of the kept blocks.
+ * keep_blocks >= capacity/page_tokens selects everything without running the selector (dense
+ * attention, Eq. 1).  An empty cache gives zeros.
+ * q, out: dev [H][nq][d] (same strides).  block_q: 64 or 128.  Optional dev outputs:
+ * sel_out [H][nQB][keep_blocks] (ascending, padded with -1), nsel_out [H] kept blocks per head,
+ * qcode_out [H][nq], scores_out [H][nQB][capacity/page_tokens] (fp32, exact integers).
+ * sel_in (dev, same layout as sel_out, with nsel_in [H]) bypasses the selector. */
+int fastar_annsa_attention(fastar_cache_t* cache, const void* q, void* out, int32_t nq,
+                           int64_t head_stride, int64_t token_stride, int32_t block_q, int32_t keep_blocks,
+                           int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out, float* scores_out,
+                           const int32_t* sel_in, const int32_t* nsel_in, void* stream);
+
+/* AnnCA (Section 5.3).  Per head and per frame f (queries [f*frame_len, (f+1)*frame_len)):
+ *   r[f][p] = max_i q_i.k_p/sqrt(d); keep the min(keep_tokens, np) prompt tokens with the
+ *   largest r (ties: lower p); o_i = softmax over the kept p of q_i.k_p/sqrt(d), times v_p.
+ * The cache object only supplies H, d, dtype, scratch and the status word; its contents are
+ * not touched.  q, out: dev [H][nq][d]; k_prompt, v_prompt: dev [H][np][d] with their own strides.
+ * Optional dev outputs: sel_out [H][F][keep_tokens] (ascending), rel_out [H][F][np] fp32.
+ * sel_in bypasses the selection.  np <= max_prompt_tokens (<= 1024), F <= max_frames. */
+int fastar_annca_attention(fastar_cache_t* cache, const void* q, const void* k_prompt, const void* v_prompt,
+                           void* out, int32_t nq, int32_t frame_len, int32_t np, int32_t keep_tokens,
+                           int64_t head_stride, int64_t token_stride,
+                           int64_t prompt_head_stride, int64_t prompt_token_stride,
+                           int32_t* sel_out, float* rel_out, const int32_t* sel_in, void* stream);
+
+/* One whole attention step with HOST tensors (contiguous [H][n][d] / [H][np][d], cache dtype):
+ * copies the inputs to the device, runs update -> AnnSA -> AnnCA (same arguments as above, the
+ * chunk's n tokens being both the new keys/values and the queries), copies both outputs back and
+ * synchronises the stream.  Staging buffers live in the workspace. */
+int fastar_attention_step_host(fastar_cache_t* cache, const void* k_new_host, const void* v_new_host,
+                               const void* q_host, const void* k_prompt_host, const void* v_prompt_host,
+                               void* out_sa_host, void* out_ca_host, int32_t n, int32_t frame_len, int32_t np,
+                               float tau, int32_t block_q, int32_t keep_blocks, int32_t keep_tokens,
+                               void* stream);
+
+/* Synchronise the stream and return the device status word (FASTAR_OK or the first error a
+ * kernel recorded since the last reset/clear); clears it. */
+int fastar_last_device_status(fastar_cache_t* cache, void* stream);
+
+/* Number of kernels this library has launched through this cache since creation. */
+int64_t fastar_launch_count(const fastar_cache_t* cache);
+
+const char* fastar_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTAR_H_ */

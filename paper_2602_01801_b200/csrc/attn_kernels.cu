@@ -1,0 +1,412 @@
+// Candidate-set attention on tcgen05 / TMEM (paper Section 5.1: attention over N(q); Lemma 1:
+// logits shifted by log m, values are group means):
+//   paged  : AnnSA's selected-block attention and the dense Eq. 1 baseline.  A query block attends
+//            to the key blocks listed in `sel`; one key block = one cache page = one TMA box, looked
+//            up through the page table.
+//   gather : AnnCA's attention over the kept prompt tokens of the query's frame; rows of K_p / V_p
+//            are gathered by index with 128-bit loads into the same swizzled tile layout.
+//
+// One CTA = 128 query rows (TMEM lanes).  Per key tile j:
+//   S_j = Q K_j^T        (tcgen05.mma, SMEM x SMEM -> TMEM, two S buffers)
+//   P_j = exp2(S_j*scale + log2 m - m_run)   (4 softmax warps, one thread per row, two passes
+//                                             over TMEM: row max, then exponentials -> bf16 P in SMEM)
+//   O  += P_j V_j        (tcgen05.mma, V is the MN-major operand straight from its [key][d] page)
+// with lazy rescaling of O (only when a row maximum grew by more than 2^8).
+// Warp roles: warps 0-3 softmax + epilogue, warp 4 producer (TMA or gather), warp 5 MMA issue.
+#include "common.h"
+#include "ptx.cuh"
+
+namespace fastar {
+
+constexpr int kQChunk = 128 * 128;   // bytes of one 128-row x 64-column bf16 chunk
+
+template <int D, int BKT>
+struct AttnSmem {
+  static constexpr int KS = 2, VS = 2, NB = 4;
+  static constexpr int q_bytes = (D / 64) * kQChunk;
+  static constexpr int kv_bytes = (D / 64) * BKT * 128;          // one K or V tile
+  static constexpr int p_bytes = (BKT / 64) * kQChunk;           // one P tile (128 x BKT bf16)
+  static constexpr int q_off = 0;
+  static constexpr int k_off = q_off + q_bytes;
+  static constexpr int v_off = k_off + KS * kv_bytes;
+  static constexpr int p_off = v_off + VS * kv_bytes;
+  static constexpr int bias_off = p_off + 2 * p_bytes;
+  static constexpr int bar_off = bias_off + NB * BKT * 4;
+  static constexpr int total = bar_off + 256;
+  static constexpr int tmem_cols = (2 * BKT + D) <= 256 ? 256 : 512;
+};
+
+template <int D, int BKT, bool GATHER>
+__global__ void __launch_bounds__(192, 1)
+attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+            const __grid_constant__ CUtensorMap tm_v, const CacheView c, const AttnArgs a) {
+  using SM = AttnSmem<D, BKT>;
+  constexpr int KS = SM::KS, VS = SM::VS, NB = SM::NB;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t sbase = smem_u32(smem_raw);
+  uint8_t* sgen = smem_raw;
+  if (sbase & 1023u) {                  // swizzled tiles need 1024-byte alignment; uniform for the CTA
+    if (threadIdx.x == 0) record_status(c.status, FASTAR_ERR_CUDA);
+    return;
+  }
+  const uint32_t q_s = sbase + SM::q_off;
+  const uint32_t k_s = sbase + SM::k_off;
+  const uint32_t v_s = sbase + SM::v_off;
+  const uint32_t p_s = sbase + SM::p_off;
+  float* bias_g = reinterpret_cast<float*>(sgen + SM::bias_off);
+  const uint32_t bias_s = sbase + SM::bias_off;
+  const uint32_t bar = sbase + SM::bar_off;
+  const uint32_t bar_q_full = bar;
+  const uint32_t bar_k_full = bar + 8;             // [KS]
+  const uint32_t bar_k_empty = bar_k_full + 8 * KS;
+  const uint32_t bar_v_full = bar_k_empty + 8 * KS;
+  const uint32_t bar_v_empty = bar_v_full + 8 * VS;
+  const uint32_t bar_b_full = bar_v_empty + 8 * VS;   // [NB]
+  const uint32_t bar_s_full = bar_b_full + 8 * NB;    // [2]
+  const uint32_t bar_s_empty = bar_s_full + 16;       // [2]
+  const uint32_t bar_p_full = bar_s_empty + 16;       // [2]
+  const uint32_t bar_pv_done = bar_p_full + 16;       // [1]
+  constexpr int kBarBytes = 8 + 16 * KS + 16 * VS + 8 * NB + 48 + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + SM::bar_off + kBarBytes);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + SM::bar_off + kBarBytes + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.y;
+  const int L = c.len[h];
+
+  // ---- which rows and which key tiles ---------------------------------------------------------
+  int q0, valid_rows, nt;
+  const int32_t* list;
+  if (!GATHER) {
+    const int qa = blockIdx.x;
+    q0 = qa * a.block_q;
+    valid_rows = min(a.block_q, a.nq - q0);
+    if (a.sel == nullptr) {
+      nt = (L + BKT - 1) / BKT;
+      list = nullptr;
+    } else {
+      nt = a.nsel[h];
+      list = a.sel + static_cast<int64_t>(h) * a.sel_head_stride + static_cast<int64_t>(qa) * a.sel_stride;
+    }
+  } else {
+    const int f = blockIdx.z;
+    q0 = f * a.rows_per_frame + blockIdx.x * 128;
+    valid_rows = min(128, min(a.rows_per_frame - static_cast<int>(blockIdx.x) * 128, a.nq - q0));
+    nt = (a.keep + BKT - 1) / BKT;
+    list = a.sel + static_cast<int64_t>(h) * a.sel_head_stride + static_cast<int64_t>(f) * a.sel_stride;
+  }
+  if (valid_rows <= 0) return;          // uniform for the CTA; nothing allocated yet
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q_full, 1);
+    for (int s = 0; s < KS; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
+    for (int s = 0; s < VS; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
+    for (int s = 0; s < NB; ++s) mbar_init(bar_b_full + 8 * s, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_s_full + 8 * s, 1);
+      mbar_init(bar_s_empty + 8 * s, 128);
+      mbar_init(bar_p_full + 8 * s, 128);
+    }
+    mbar_init(bar_pv_done, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 4 && lane == 0) {
+    tma_prefetch_desc(&tm_q);
+    if (!GATHER) { tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); }
+  }
+  __syncthreads();
+  if (warp == 5) {
+    tmem_alloc(smem_u32(tmem_slot), SM::tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_o = tmem + 2 * BKT;
+
+  if (warp == 4) {
+    // ================================================================== producer
+    if (lane == 0 && nt > 0) {
+      mbar_arrive_expect_tx(bar_q_full, SM::q_bytes);
+      for (int kc = 0; kc < D / 64; ++kc) tma_load_3d(q_s + kc * kQChunk, &tm_q, bar_q_full, kc * 64, q0, h);
+    }
+    if (!GATHER) {
+      if (lane == 0) {
+        const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+        const float* l2m_h = c.log2m + static_cast<int64_t>(h) * c.CAP;
+        bool ok = true;
+        int blk_next = nt > 0 ? (list ? list[0] : 0) : 0;
+        int page_next = nt > 0 ? pt_h[blk_next] : 0;
+        for (int j = 0; j < nt && ok; ++j) {
+          const int blk = blk_next, page = page_next;
+          if (j + 1 < nt) {                       // look the next block up while this one is in flight
+            blk_next = list ? list[j + 1] : j + 1;
+            page_next = pt_h[blk_next];
+          }
+          const int ks = j % KS, vs = j % VS, b4 = j % NB;
+          ok = mbar_wait(bar_k_empty + 8 * ks, ((j / KS) & 1) ^ 1, abort_flag, c.status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_k_full + 8 * ks, SM::kv_bytes);
+          for (int kc = 0; kc < D / 64; ++kc)
+            tma_load_3d(k_s + ks * SM::kv_bytes + kc * BKT * 128, &tm_k, bar_k_full + 8 * ks, kc * 64, 0, page);
+          mbar_arrive_expect_tx(bar_b_full + 8 * b4, BKT * 4);
+          bulk_load_1d(bias_s + b4 * BKT * 4, l2m_h + static_cast<int64_t>(blk) * BKT, BKT * 4, bar_b_full + 8 * b4);
+          ok = mbar_wait(bar_v_empty + 8 * vs, ((j / VS) & 1) ^ 1, abort_flag, c.status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_v_full + 8 * vs, SM::kv_bytes);
+          for (int kc = 0; kc < D / 64; ++kc)
+            tma_load_3d(v_s + vs * SM::kv_bytes + kc * BKT * 128, &tm_v, bar_v_full + 8 * vs, kc * 64, 0, page);
+        }
+      }
+    } else {
+      // gather rows of K_p / V_p by index: 16-byte chunks, written at their swizzled position
+      constexpr int CPR = D / 8;                       // 16-byte chunks per row
+      const __nv_bfloat16* kp_h = a.kp + static_cast<int64_t>(h) * a.p_head_stride;
+      const __nv_bfloat16* vp_h = a.vp + static_cast<int64_t>(h) * a.p_head_stride;
+      bool ok = true;
+      for (int j = 0; j < nt && ok; ++j) {
+        const int ks = j % KS, vs = j % VS, b4 = j % NB;
+        ok = mbar_wait(bar_k_empty + 8 * ks, ((j / KS) & 1) ^ 1, abort_flag, c.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        for (int which = 0; which < 2; ++which) {
+          if (which == 1) {
+            ok = mbar_wait(bar_v_empty + 8 * vs, ((j / VS) & 1) ^ 1, abort_flag, c.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          const __nv_bfloat16* src_h = which == 0 ? kp_h : vp_h;
+          const uint32_t dst = which == 0 ? k_s + ks * SM::kv_bytes : v_s + vs * SM::kv_bytes;
+          for (int q = lane; q < BKT * CPR; q += 32) {
+            const int i = q / CPR, ch = q % CPR;
+            const int tok = j * BKT + i;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (tok < a.keep) {
+              const int idx = list[tok];
+              val = *reinterpret_cast<const uint4*>(src_h + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
+            }
+            const uint32_t off = (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + off), "r"(val.x), "r"(val.y), "r"(val.z),
+                         "r"(val.w)
+                         : "memory");
+          }
+          if (which == 0)
+            for (int i = lane; i < BKT; i += 32) bias_g[b4 * BKT + i] = (j * BKT + i < a.keep) ? 0.f : -INFINITY;
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (which == 0) { mbar_arrive(bar_k_full + 8 * ks); mbar_arrive(bar_b_full + 8 * b4); }
+            else mbar_arrive(bar_v_full + 8 * vs);
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ================================================================== MMA issue
+    if (lane == 0 && nt > 0) {
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, BKT, 0);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
+      bool ok = mbar_wait(bar_q_full, 0, abort_flag, c.status);
+      auto issue_s = [&](int j) -> bool {
+        const int ks = j % KS, sb = j & 1;
+        if (!mbar_wait(bar_k_full + 8 * ks, (j / KS) & 1, abort_flag, c.status)) return false;
+        if (!mbar_wait(bar_s_empty + 8 * sb, ((j >> 1) & 1) ^ 1, abort_flag, c.status)) return false;
+        tc_fence_after();
+        const uint32_t kt = k_s + ks * SM::kv_bytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t ad = make_smem_desc(q_s + (kk >> 2) * kQChunk + (kk & 3) * 32, 16, 1024);
+          const uint64_t bd = make_smem_desc(kt + (kk >> 2) * (BKT * 128) + (kk & 3) * 32, 16, 1024);
+          umma_ss(tmem + sb * BKT, ad, bd, idesc_qk, kk != 0);
+        }
+        umma_commit(bar_k_empty + 8 * ks);
+        umma_commit(bar_s_full + 8 * sb);
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < nt && ok; ++j) {
+        if (j + 1 < nt) { ok = issue_s(j + 1); if (!ok) break; }
+        const int vs = j % VS, pb = j & 1;
+        ok = mbar_wait(bar_p_full + 8 * pb, (j >> 1) & 1, abort_flag, c.status);
+        if (!ok) break;
+        ok = mbar_wait(bar_v_full + 8 * vs, (j / VS) & 1, abort_flag, c.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t vt = v_s + vs * SM::kv_bytes;
+        const uint32_t pt = p_s + pb * SM::p_bytes;
+#pragma unroll
+        for (int ks16 = 0; ks16 < BKT / 16; ++ks16) {
+          const uint64_t ad = make_smem_desc(pt + (ks16 >> 2) * kQChunk + (ks16 & 3) * 32, 16, 1024);
+          const uint64_t bd = make_smem_desc(vt + ks16 * 2048, BKT * 128, 1024);
+          umma_ss(tmem_o, ad, bd, idesc_pv, (j | ks16) != 0);
+        }
+        umma_commit(bar_v_empty + 8 * vs);
+        umma_commit(bar_pv_done);
+      }
+    }
+  } else {
+    // ================================================================== softmax + epilogue
+    const int r = threadIdx.x;
+    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    const float scale = rsqrtf(static_cast<float>(D)) * 1.4426950408889634f;
+    float m_used = -INFINITY, l_sum = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nt && ok; ++j) {
+      const int sb = j & 1, pb = j & 1, b4 = j % NB;
+      ok = mbar_wait(bar_b_full + 8 * b4, (j / NB) & 1, abort_flag, c.status) &&
+           mbar_wait(bar_s_full + 8 * sb, (j >> 1) & 1, abort_flag, c.status);
+      ok = __all_sync(0xffffffffu, ok);          // TMEM loads below are warp-collective
+      if (!ok) break;
+      tc_fence_after();
+      const float* bias = bias_g + b4 * BKT;
+      const uint32_t s_t = tmem + lane_addr + sb * BKT;
+      // pass 1: row maximum
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int cc = 0; cc < BKT / 32; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(s_t + cc * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int t = 0; t < 32; ++t) mx = fmaxf(mx, fmaf(__uint_as_float(v[t]), scale, bias[cc * 32 + t]));
+      }
+      float alpha = 1.f;
+      bool resc = false;
+      if (mx > m_used + 8.f || (m_used == -INFINITY && mx > -INFINITY)) {
+        alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
+        l_sum *= alpha;
+        m_used = mx;
+        resc = j > 0;
+      }
+      const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
+      // pass 2: exponentials -> bf16 P tile (K-major, 128-byte swizzle), row sum
+      const uint32_t p_row = p_s + pb * SM::p_bytes + r * 128;
+#pragma unroll 1
+      for (int cc = 0; cc < BKT / 32; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(s_t + cc * 32, v);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * t]), scale, bias[cc * 32 + 2 * t]) - m_eff);
+          const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * t + 1]), scale, bias[cc * 32 + 2 * t + 1]) - m_eff);
+          l_sum += p0 + p1;
+          pk[t] = pack_bf16x2(p0, p1);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int ch = cc * 4 + q;                   // 16-byte chunk index along the key axis
+          const uint32_t addr = p_row + (ch >> 3) * kQChunk + (((ch & 7) ^ (r & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * q]), "r"(pk[4 * q + 1]),
+                       "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3])
+                       : "memory");
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_s_empty + 8 * sb);
+      if (j > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done, (j - 1) & 1, abort_flag, c.status));
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, resc)) {
+#pragma unroll 1
+          for (int cc = 0; cc < D / 32; ++cc) {
+            uint32_t v[32];
+            tmem_ld32(tmem_o + lane_addr + cc * 32, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) * alpha);
+            tmem_st32(tmem_o + lane_addr + cc * 32, v);
+          }
+          tmem_wait_st();
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(bar_p_full + 8 * pb);
+    }
+    // epilogue: O / l -> out
+    if (ok && nt > 0) ok = mbar_wait(bar_pv_done, (nt - 1) & 1, abort_flag, c.status);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+    const bool wr = r < valid_rows;               // loads are warp-collective, only the stores are per row
+    if (ok) {
+      const float inv = (nt > 0 && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      const int64_t off = static_cast<int64_t>(h) * a.out_head_stride + static_cast<int64_t>(q0 + r) * a.out_token_stride;
+#pragma unroll 1
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t v[32];
+        if (nt > 0) {
+          tmem_ld32(tmem_o + lane_addr + cc * 32, v);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int t = 0; t < 32; ++t) v[t] = 0;
+        }
+        if (!wr) continue;
+        if (a.out_fp32) {
+          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(a.out) + off + cc * 32);
+#pragma unroll
+          for (int t = 0; t < 8; ++t)
+            dst[t] = make_float4(__uint_as_float(v[4 * t]) * inv, __uint_as_float(v[4 * t + 1]) * inv,
+                                 __uint_as_float(v[4 * t + 2]) * inv, __uint_as_float(v[4 * t + 3]) * inv);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(a.out) + off + cc * 32);
+#pragma unroll
+          for (int t = 0; t < 4; ++t)
+            dst[t] = make_uint4(pack_bf16x2(__uint_as_float(v[8 * t]) * inv, __uint_as_float(v[8 * t + 1]) * inv),
+                                pack_bf16x2(__uint_as_float(v[8 * t + 2]) * inv, __uint_as_float(v[8 * t + 3]) * inv),
+                                pack_bf16x2(__uint_as_float(v[8 * t + 4]) * inv, __uint_as_float(v[8 * t + 5]) * inv),
+                                pack_bf16x2(__uint_as_float(v[8 * t + 6]) * inv, __uint_as_float(v[8 * t + 7]) * inv));
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, SM::tmem_cols);
+  }
+}
+
+template <int D, int BKT, bool GATHER>
+static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CacheView& c,
+                       const AttnArgs& a, dim3 grid, cudaStream_t st) {
+  using SM = AttnSmem<D, BKT>;
+  auto kern = attn_kernel<D, BKT, GATHER>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+    configured = true;
+  }
+  kern<<<grid, 192, SM::total, st>>>(tq, tk, tv, c, a);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
+                           const CUtensorMap& tm_pool_v, const AttnArgs& a, cudaStream_t st) {
+  const dim3 grid((a.nq + a.block_q - 1) / a.block_q, c.H, 1);
+  if (c.D == 128 && c.PT == 128) return launch_attn<128, 128, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
+  if (c.D == 128 && c.PT == 64) return launch_attn<128, 64, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
+  if (c.D == 64 && c.PT == 128) return launch_attn<64, 128, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
+  if (c.D == 64 && c.PT == 64) return launch_attn<64, 64, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
+  return FASTAR_ERR_UNSUPPORTED_SHAPE;
+}
+
+int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st) {
+  const dim3 grid((a.rows_per_frame + 127) / 128, c.H, a.n_frames);
+  const bool small = a.keep <= 64;
+  if (c.D == 128 && !small) return launch_attn<128, 128, true>(tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 128 && small) return launch_attn<128, 64, true>(tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 64 && !small) return launch_attn<64, 128, true>(tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 64 && small) return launch_attn<64, 64, true>(tm_q, tm_q, tm_q, c, a, grid, st);
+  return FASTAR_ERR_UNSUPPORTED_SHAPE;
+}
+
+}  // namespace fastar

@@ -1,0 +1,122 @@
+// Internal view of a cache: device pointers into the caller's workspace plus shape constants.
+// Passed by value to kernels.  Logical slot s of head h lives in page page_table[h][s / PT],
+// row s % PT, of the K and V pools; one page is one AnnSA key block and one TMA box.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/fastar.h"
+
+namespace fastar {
+
+struct PlanRec {          // per head, written by the planning kernel of an update
+  int32_t ok;             // 1 = the update will be applied
+  int32_t n_matched;      // M: matched tokens (sorted positions [0, M))
+  int32_t n_seg;          // touched slots
+  int32_t n_unmatched;    // U
+  int32_t n_append;       // A
+  int32_t n_evict;        // E
+  int32_t len_old;
+  int32_t len_new;
+  int32_t evicted_tokens;
+  int32_t pad[3];
+};
+
+struct CacheView {
+  // shape
+  int32_t H, D, CAP, PT, CAPB;     // CAPB = CAP / PT
+  int32_t n_sink, T, B;            // LSH tables / bits
+  int32_t max_tokens, max_prompt, max_frames, max_qb;
+  int32_t hist_cols;               // T * 2^B rounded up to a multiple of 64
+  // persistent state
+  __nv_bfloat16* pool_k;           // [H*CAPB][PT][D]
+  __nv_bfloat16* pool_v;
+  int32_t* page_table;             // [H][CAPB]
+  int32_t* count;                  // [H][CAP]   multiplicity m (0 = dead)
+  int32_t* stamp;                  // [H][CAP]
+  float* log2m;                    // [H][CAP]   log2(m), -inf for dead slots
+  float* rnorm;                    // [H][CAP]   1/|k|
+  uint32_t* kcode;                 // [H][CAP]   table t in byte t
+  __nv_bfloat16* hk;               // [H][CAPB][hist_cols]
+  int32_t* len;                    // [H]
+  int32_t* now;                    // [1]
+  int32_t* status;                 // [1]
+  __nv_bfloat16* lsh;              // [T*B][D]
+  // per-call scratch
+  unsigned long long* best;        // [H][max_tokens]  packed (ordered score, ~slot)
+  float* rnorm_new;                // [H][max_tokens]
+  uint32_t* code_new;              // [H][max_tokens]  codes of new keys / of queries
+  int32_t* match;                  // [H][max_tokens]
+  float* sim;                      // [H][max_tokens]
+  int32_t* order;                  // [H][max_tokens]  token ids sorted by (slot, token)
+  int32_t* segpos;                 // [H][max_tokens+1] start of each segment in `order`
+  int32_t* dest;                   // [H][max_tokens]
+  int32_t* victims;                // [H][max_tokens]
+  PlanRec* plan;                   // [H]
+  __nv_bfloat16* hq;               // [H][max_qb_pad][hist_cols]
+  float* scores;                   // [H][max_qb][CAPB]
+  int32_t* sel;                    // [H][max_qb][CAPB]
+  int32_t* nsel;                   // [H]
+  uint32_t* rel;                   // [H][max_frames][max_prompt]  ordered-uint relevance
+  int32_t* selp;                   // [H][max_frames][max_prompt]
+  // staging (fp32 entry conversion and the host-tensor step)
+  __nv_bfloat16* stage[5];         // k, v, q, kp, vp  ([H][max_tokens][D] / [H][max_prompt][D])
+  void* stage_out[2];              // [H][max_tokens][D] in the caller dtype
+  void* stage_in_raw[5];           // raw caller-dtype copies for the host-tensor step (fp32 only)
+};
+
+inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
+  int page = page_table_h[slot / c.PT];
+  return (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D;
+}
+
+// ---- launchers implemented in the .cu files (all asynchronous on `st`) -----------------------
+// Each returns the number of kernels it launched (for the launch counter) or a negative status.
+
+// gemm_kernels.cu
+int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k, int n, cudaStream_t st);
+int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,
+                        int n_frames, cudaStream_t st);
+int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtensorMap& tm_hk, int nqb, cudaStream_t st);
+
+// attn_kernels.cu
+struct AttnArgs {
+  int nq;                  // query rows per head
+  int block_q;             // rows per query block (<= 128)
+  int rows_per_frame;      // gather mode: frame_len; paged mode: unused
+  int keep;                // paged: row length of sel (0 = dense: all live blocks); gather: kept prompt tokens
+  const int32_t* sel;      // paged: [H][nQB][keep]; gather: [H][F][sel_stride]
+  const int32_t* nsel;     // paged: [H] valid entries per row (nullptr in dense mode)
+  int sel_stride;          // elements between rows of sel
+  int64_t sel_head_stride; // elements between heads of sel
+  int n_frames;
+  const __nv_bfloat16* kp; // gather mode: prompt keys / values (bf16) and their strides
+  const __nv_bfloat16* vp;
+  int64_t p_head_stride, p_token_stride;
+  void* out;               // [H][nq][D] caller dtype
+  int out_fp32;
+  int64_t out_head_stride, out_token_stride;
+};
+int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
+                           const CUtensorMap& tm_pool_v, const AttnArgs& a, cudaStream_t st);
+int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st);
+
+// update_kernels.cu
+int launch_convert_f32_to_bf16(const float* src, __nv_bfloat16* dst, int H, int n, int D, int64_t hs, int64_t ts, cudaStream_t st);
+int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
+                      float* rnorm_out, cudaStream_t st);
+int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st);
+int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len,
+                  int64_t hs, int64_t ts, cudaStream_t st);
+int launch_finalize_hist(const CacheView& c, fastar_update_stats* stats_out, int advance_clock, cudaStream_t st);
+int launch_query_hist(const CacheView& c, int nq, int block_q, cudaStream_t st);
+int launch_topk_blocks(const CacheView& c, int nqb, int keep, cudaStream_t st);
+int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st);
+int launch_reset(const CacheView& c, cudaStream_t st);
+int launch_import_derive(const CacheView& c, cudaStream_t st);
+int launch_copy_outputs(const CacheView& c, int n, int32_t* match_out, float* sim_out, int32_t* dest_out, cudaStream_t st);
+int launch_decode_rel(const CacheView& c, int n_frames, int np, float scale, float* rel_out, cudaStream_t st);
+
+}  // namespace fastar

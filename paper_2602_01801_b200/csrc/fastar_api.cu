@@ -1,0 +1,492 @@
+// Host side of the C ABI declared in include/fastar.h: argument checks, workspace carving,
+// tensor-map encoding, kernel sequencing.  No device memory is allocated here.
+#include <cudaTypedefs.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.h"
+
+using namespace fastar;
+
+struct fastar_cache {
+  fastar_cache_desc desc;
+  CacheView v;
+  CUtensorMap tm_pool_k, tm_pool_v, tm_hq, tm_hk;
+  PFN_cuTensorMapEncodeTiled_v12000 encode;
+  int64_t launches;
+  size_t bytes;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool changed = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) changed = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (changed) cudaSetDevice(prev);
+  }
+};
+
+bool desc_valid(const fastar_cache_desc* d) {
+  if (!d) return false;
+  if (d->num_heads < 1 || (d->head_dim != 64 && d->head_dim != 128)) return false;
+  if (d->page_tokens != 64 && d->page_tokens != 128) return false;
+  if (d->capacity < 128 || d->capacity % 128 != 0 || d->capacity % d->page_tokens != 0) return false;
+  if (d->n_sink < 0 || d->n_sink > d->capacity) return false;
+  if (d->lsh_tables < 1 || d->lsh_tables > 4 || d->lsh_bits < 1 || d->lsh_bits > 8) return false;
+  if (d->max_tokens < 1 || d->max_tokens > 16384) return false;
+  if (d->max_prompt_tokens < 1 || d->max_prompt_tokens > 1024 || d->max_frames < 1 || d->max_frames > 64) return false;
+  if (d->dtype != FASTAR_BF16 && d->dtype != FASTAR_FP32) return false;
+  return true;
+}
+
+// Carves the workspace.  With base == nullptr only the size is computed.
+size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
+  size_t cur = 0;
+  auto take = [&](size_t bytes) -> uint8_t* {
+    cur = (cur + 1023) & ~static_cast<size_t>(1023);
+    uint8_t* p = base ? base + cur : nullptr;
+    cur += bytes;
+    return p;
+  };
+  CacheView t{};
+  t.H = d.num_heads; t.D = d.head_dim; t.CAP = d.capacity; t.PT = d.page_tokens; t.CAPB = d.capacity / d.page_tokens;
+  t.n_sink = d.n_sink; t.T = d.lsh_tables; t.B = d.lsh_bits;
+  t.max_tokens = d.max_tokens; t.max_prompt = d.max_prompt_tokens; t.max_frames = d.max_frames;
+  t.max_qb = (d.max_tokens + 63) / 64;
+  t.hist_cols = ((d.lsh_tables << d.lsh_bits) + 63) / 64 * 64;
+  const size_t H = t.H, CAP = t.CAP, D = t.D, MT = t.max_tokens, MP = t.max_prompt;
+  const size_t esz = d.dtype == FASTAR_FP32 ? 4 : 2;
+  t.pool_k = reinterpret_cast<__nv_bfloat16*>(take(H * CAP * D * 2));
+  t.pool_v = reinterpret_cast<__nv_bfloat16*>(take(H * CAP * D * 2));
+  t.page_table = reinterpret_cast<int32_t*>(take(H * t.CAPB * 4));
+  t.count = reinterpret_cast<int32_t*>(take(H * CAP * 4));
+  t.stamp = reinterpret_cast<int32_t*>(take(H * CAP * 4));
+  t.log2m = reinterpret_cast<float*>(take(H * CAP * 4));
+  t.rnorm = reinterpret_cast<float*>(take(H * CAP * 4));
+  t.kcode = reinterpret_cast<uint32_t*>(take(H * CAP * 4));
+  t.hk = reinterpret_cast<__nv_bfloat16*>(take(H * t.CAPB * t.hist_cols * 2));
+  t.len = reinterpret_cast<int32_t*>(take(H * 4));
+  t.now = reinterpret_cast<int32_t*>(take(4));
+  t.status = reinterpret_cast<int32_t*>(take(4));
+  t.lsh = reinterpret_cast<__nv_bfloat16*>(take(32 * D * 2));
+  t.best = reinterpret_cast<unsigned long long*>(take(H * MT * 8));
+  t.rnorm_new = reinterpret_cast<float*>(take(H * MT * 4));
+  t.code_new = reinterpret_cast<uint32_t*>(take(H * MT * 4));
+  t.match = reinterpret_cast<int32_t*>(take(H * MT * 4));
+  t.sim = reinterpret_cast<float*>(take(H * MT * 4));
+  t.order = reinterpret_cast<int32_t*>(take(H * MT * 4));
+  t.segpos = reinterpret_cast<int32_t*>(take(H * (MT + 1) * 4));
+  t.dest = reinterpret_cast<int32_t*>(take(H * MT * 4));
+  t.victims = reinterpret_cast<int32_t*>(take(H * MT * 4));
+  t.plan = reinterpret_cast<PlanRec*>(take(H * sizeof(PlanRec)));
+  t.hq = reinterpret_cast<__nv_bfloat16*>(take(H * t.max_qb * t.hist_cols * 2));
+  t.scores = reinterpret_cast<float*>(take(H * t.max_qb * t.CAPB * 4));
+  t.sel = reinterpret_cast<int32_t*>(take(H * t.max_qb * t.CAPB * 4));
+  t.nsel = reinterpret_cast<int32_t*>(take(H * 4));
+  t.rel = reinterpret_cast<uint32_t*>(take(H * t.max_frames * MP * 4));
+  t.selp = reinterpret_cast<int32_t*>(take(H * t.max_frames * MP * 4));
+  for (int i = 0; i < 3; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
+  for (int i = 3; i < 5; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MP * D * 2));
+  for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
+  for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
+  cur = (cur + 1023) & ~static_cast<size_t>(1023);
+  if (v) *v = t;
+  return cur;
+}
+
+// 3-D bf16 tensor map {d0 (innermost, contiguous), d1, d2}, box {64, box1, 1}, 128-byte swizzle.
+int make_map(fastar_cache* c, CUtensorMap* m, const void* ptr, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+             uint64_t stride2_bytes, uint32_t box1) {
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (stride1_bytes & 15) || (stride2_bytes & 15)) return FASTAR_ERR_INVALID_ARG;
+  const cuuint64_t dims[3] = {d0, d1, d2};
+  const cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+  const cuuint32_t box[3] = {64, box1, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+__global__ void copy_rows3_kernel(const int32_t* __restrict__ src, int64_t src_hs, int src_rs, int32_t* __restrict__ dst, int rows,
+                                  int cols) {
+  const int h = blockIdx.y;
+  for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < rows * cols; q += gridDim.x * blockDim.x) {
+    const int r = q / cols, cidx = q % cols;
+    dst[(static_cast<int64_t>(h) * rows + r) * cols + cidx] = src[h * src_hs + static_cast<int64_t>(r) * src_rs + cidx];
+  }
+}
+
+#define ACC(call)                     \
+  do {                                \
+    const int r__ = (call);           \
+    if (r__ < 0) return r__;          \
+    c->launches += r__;               \
+  } while (0)
+
+// Returns a bf16 view of a caller tensor: the tensor itself (bf16) or its converted copy in stage[slot].
+int as_bf16(fastar_cache* c, const void* src, int rows, int64_t* hs, int64_t* ts, int slot, const __nv_bfloat16** out,
+            cudaStream_t st) {
+  if (c->desc.dtype == FASTAR_BF16) {
+    *out = static_cast<const __nv_bfloat16*>(src);
+    return FASTAR_OK;
+  }
+  if ((reinterpret_cast<uintptr_t>(src) & 15) || (*hs & 3) || (*ts & 3)) return FASTAR_ERR_INVALID_ARG;
+  ACC(launch_convert_f32_to_bf16(static_cast<const float*>(src), c->v.stage[slot], c->v.H, rows, c->v.D, *hs, *ts, st));
+  *out = c->v.stage[slot];
+  *hs = static_cast<int64_t>(rows) * c->v.D;
+  *ts = c->v.D;
+  return FASTAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t fastar_cache_workspace_bytes(const fastar_cache_desc* desc) {
+  if (!desc_valid(desc)) return 0;
+  return carve(*desc, nullptr, nullptr);
+}
+
+int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, const float* lsh_proj_host, void* dev_buf,
+                        size_t bytes) {
+  if (!out || !desc_valid(desc) || !lsh_proj_host || !dev_buf) return FASTAR_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, desc->device) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (prop.major != 10) return FASTAR_ERR_NOT_SM100;
+  if ((reinterpret_cast<uintptr_t>(dev_buf) & 1023) || bytes < carve(*desc, nullptr, nullptr)) return FASTAR_ERR_WORKSPACE;
+  DeviceGuard guard(desc->device);
+  fastar_cache* c = new (std::nothrow) fastar_cache();
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  c->desc = *desc;
+  c->bytes = carve(*desc, static_cast<uint8_t*>(dev_buf), &c->v);
+  c->launches = 0;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete c;
+    return FASTAR_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  const CacheView& v = c->v;
+  const uint64_t D = v.D, PT = v.PT;
+  int r = make_map(c, &c->tm_pool_k, v.pool_k, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, v.PT);
+  if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_v, v.pool_v, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, v.PT);
+  if (r == FASTAR_OK)
+    r = make_map(c, &c->tm_hq, v.hq, v.hist_cols, v.max_qb, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
+                 static_cast<uint64_t>(v.max_qb) * v.hist_cols * 2, 128);
+  if (r == FASTAR_OK)
+    r = make_map(c, &c->tm_hk, v.hk, v.hist_cols, v.CAPB, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
+                 static_cast<uint64_t>(v.CAPB) * v.hist_cols * 2, 128);
+  if (r != FASTAR_OK) {
+    delete c;
+    return r;
+  }
+  // projection matrix: fp32 host -> bf16 (nearest even) -> device
+  std::vector<uint16_t> rb(static_cast<size_t>(32) * v.D, 0);
+  for (int i = 0; i < v.T * v.B * v.D; ++i) {
+    uint32_t u;
+    std::memcpy(&u, &lsh_proj_host[i], 4);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    rb[i] = static_cast<uint16_t>(u >> 16);
+  }
+  if (cudaMemcpy(v.lsh, rb.data(), rb.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess) {
+    delete c;
+    return FASTAR_ERR_CUDA;
+  }
+  r = fastar_cache_reset(c, nullptr);
+  if (r == FASTAR_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) r = FASTAR_ERR_CUDA;
+  if (r != FASTAR_OK) {
+    delete c;
+    return r;
+  }
+  *out = c;
+  return FASTAR_OK;
+}
+
+int fastar_cache_reset(fastar_cache_t* c, void* stream) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  ACC(launch_reset(c->v, static_cast<cudaStream_t>(stream)));
+  return FASTAR_OK;
+}
+
+int fastar_cache_destroy(fastar_cache_t* c) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  delete c;
+  return FASTAR_OK;
+}
+
+int fastar_cache_export(fastar_cache_t* c, uint16_t* host_k, uint16_t* host_v, int32_t* count, int32_t* stamp, uint32_t* code,
+                        int32_t* len, int32_t* now, void* stream) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const size_t pool = static_cast<size_t>(v.H) * v.CAP * v.D * 2, meta = static_cast<size_t>(v.H) * v.CAP * 4;
+  bool ok = true;
+  if (host_k) ok &= cudaMemcpyAsync(host_k, v.pool_k, pool, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (host_v) ok &= cudaMemcpyAsync(host_v, v.pool_v, pool, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (count) ok &= cudaMemcpyAsync(count, v.count, meta, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (stamp) ok &= cudaMemcpyAsync(stamp, v.stamp, meta, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (code) ok &= cudaMemcpyAsync(code, v.kcode, meta, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (len) ok &= cudaMemcpyAsync(len, v.len, static_cast<size_t>(v.H) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (now) ok &= cudaMemcpyAsync(now, v.now, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+int fastar_cache_import(fastar_cache_t* c, const uint16_t* host_k, const uint16_t* host_v, const int32_t* count,
+                        const int32_t* stamp, const int32_t* len, int32_t now, void* stream) {
+  if (!c || !host_k || !host_v || !len || now < 0) return FASTAR_ERR_INVALID_ARG;
+  for (int h = 0; h < c->v.H; ++h)
+    if (len[h] < 0 || len[h] > c->v.CAP) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const size_t pool = static_cast<size_t>(v.H) * v.CAP * v.D * 2, meta = static_cast<size_t>(v.H) * v.CAP * 4;
+  ACC(launch_reset(v, st));
+  bool ok = true;
+  ok &= cudaMemcpyAsync(v.pool_k, host_k, pool, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(v.pool_v, host_v, pool, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (count) ok &= cudaMemcpyAsync(v.count, count, meta, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  else {
+    std::vector<int32_t> ones(static_cast<size_t>(v.H) * v.CAP, 1);
+    ok &= cudaMemcpyAsync(v.count, ones.data(), meta, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  }
+  if (stamp) ok &= cudaMemcpyAsync(v.stamp, stamp, meta, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(v.len, len, static_cast<size_t>(v.H) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(v.now, &now, 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return FASTAR_ERR_CUDA;
+  ACC(launch_import_derive(v, st));
+  return cudaStreamSynchronize(st) == cudaSuccess ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_new, int32_t n, int32_t frame_len,
+                            int64_t head_stride, int64_t token_stride, float tau, int32_t* match_out, float* sim_out,
+                            int32_t* dest_out, fastar_update_stats* stats_out, void* stream) {
+  if (!c || !k_new || !v_new || n < 1 || frame_len < 1) return FASTAR_ERR_INVALID_ARG;
+  if (n > c->v.max_tokens || n > 16384 || n > c->v.CAP) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (token_stride < c->v.D || head_stride < 0) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const __nv_bfloat16 *kb, *vb;
+  int64_t khs = head_stride, kts = token_stride, vhs = head_stride, vts = token_stride;
+  int r = as_bf16(c, k_new, n, &khs, &kts, 0, &kb, st);
+  if (r != FASTAR_OK) return r;
+  r = as_bf16(c, v_new, n, &vhs, &vts, 1, &vb, st);
+  if (r != FASTAR_OK) return r;
+  CUtensorMap tm_a;
+  r = make_map(c, &tm_a, kb, v.D, n, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
+  if (r != FASTAR_OK) return r;
+  ACC(launch_prep_codes(v, kb, n, khs, kts, v.code_new, v.rnorm_new, st));
+  if (cudaMemsetAsync(v.best, 0, static_cast<size_t>(v.H) * v.max_tokens * 8, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  ACC(launch_t1_similarity(v, tm_a, c->tm_pool_k, n, st));
+  ACC(launch_plan(v, n, frame_len, tau, st));
+  ACC(launch_commit(v, kb, vb, n, frame_len, khs, kts, st));
+  ACC(launch_finalize_hist(v, stats_out, 1, st));
+  ACC(launch_copy_outputs(v, n, match_out, sim_out, dest_out, st));
+  return FASTAR_OK;
+}
+
+int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t nq, int64_t head_stride, int64_t token_stride,
+                           int32_t block_q, int32_t keep_blocks, int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out,
+                           float* scores_out, const int32_t* sel_in, const int32_t* nsel_in, void* stream) {
+  if (!c || !q || !out || nq < 1 || keep_blocks < 1) return FASTAR_ERR_INVALID_ARG;
+  if (block_q != 64 && block_q != 128) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (nq > c->v.max_tokens) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (token_stride < c->v.D || head_stride < 0 || (sel_in && !nsel_in)) return FASTAR_ERR_INVALID_ARG;
+  const size_t osz = c->desc.dtype == FASTAR_FP32 ? 4 : 2;
+  if ((reinterpret_cast<uintptr_t>(out) & 15) || ((head_stride * osz) & 15) || ((token_stride * osz) & 15)) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const int nqb = (nq + block_q - 1) / block_q;
+  const bool dense = !sel_in && keep_blocks >= v.CAPB;
+  const int keep = keep_blocks < v.CAPB ? keep_blocks : v.CAPB;
+  if (!dense && !sel_in && v.CAPB > 2048) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  const __nv_bfloat16* qb;
+  int64_t qhs = head_stride, qts = token_stride;
+  int r = as_bf16(c, q, nq, &qhs, &qts, 2, &qb, st);
+  if (r != FASTAR_OK) return r;
+  CUtensorMap tm_q;
+  r = make_map(c, &tm_q, qb, v.D, nq, v.H, static_cast<uint64_t>(qts) * 2, static_cast<uint64_t>(qhs) * 2, 128);
+  if (r != FASTAR_OK) return r;
+  AttnArgs a{};
+  a.nq = nq;
+  a.block_q = block_q;
+  a.out = out;
+  a.out_fp32 = c->desc.dtype == FASTAR_FP32;
+  a.out_head_stride = head_stride;
+  a.out_token_stride = token_stride;
+  if (sel_in) {
+    a.sel = sel_in;
+    a.nsel = nsel_in;
+    a.sel_stride = keep_blocks;
+    a.sel_head_stride = static_cast<int64_t>(nqb) * keep_blocks;
+    a.keep = keep_blocks;
+  } else if (!dense) {
+    ACC(launch_prep_codes(v, qb, nq, qhs, qts, v.code_new, nullptr, st));
+    ACC(launch_query_hist(v, nq, block_q, st));
+    ACC(launch_s3_scores(v, c->tm_hq, c->tm_hk, nqb, st));
+    ACC(launch_topk_blocks(v, nqb, keep, st));
+    a.sel = v.sel;
+    a.nsel = v.nsel;
+    a.sel_stride = v.CAPB;
+    a.sel_head_stride = static_cast<int64_t>(v.max_qb) * v.CAPB;
+    a.keep = keep;
+    if (sel_out) {
+      copy_rows3_kernel<<<dim3((nqb * keep + 255) / 256, v.H), 256, 0, st>>>(v.sel, a.sel_head_stride, v.CAPB, sel_out, nqb, keep);
+      if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+      c->launches += 1;
+    }
+    if (nsel_out && cudaMemcpyAsync(nsel_out, v.nsel, static_cast<size_t>(v.H) * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+    if (qcode_out && cudaMemcpy2DAsync(qcode_out, static_cast<size_t>(nq) * 4, v.code_new, static_cast<size_t>(v.max_tokens) * 4,
+                                       static_cast<size_t>(nq) * 4, v.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+    if (scores_out && cudaMemcpy2DAsync(scores_out, static_cast<size_t>(nqb) * v.CAPB * 4, v.scores,
+                                        static_cast<size_t>(v.max_qb) * v.CAPB * 4, static_cast<size_t>(nqb) * v.CAPB * 4, v.H,
+                                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+  }
+  ACC(launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, a, st));
+  return FASTAR_OK;
+}
+
+int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_prompt, const void* v_prompt, void* out, int32_t nq,
+                           int32_t frame_len, int32_t np, int32_t keep_tokens, int64_t head_stride, int64_t token_stride,
+                           int64_t prompt_head_stride, int64_t prompt_token_stride, int32_t* sel_out, float* rel_out,
+                           const int32_t* sel_in, void* stream) {
+  if (!c || !q || !k_prompt || !v_prompt || !out || nq < 1 || frame_len < 1 || np < 1 || keep_tokens < 1) return FASTAR_ERR_INVALID_ARG;
+  const int F = (nq + frame_len - 1) / frame_len;
+  if (nq > c->v.max_tokens || np > c->v.max_prompt || F > c->v.max_frames) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (token_stride < c->v.D || prompt_token_stride < c->v.D) return FASTAR_ERR_INVALID_ARG;
+  const size_t osz = c->desc.dtype == FASTAR_FP32 ? 4 : 2;
+  if ((reinterpret_cast<uintptr_t>(out) & 15) || ((head_stride * osz) & 15) || ((token_stride * osz) & 15)) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const int keep = keep_tokens < np ? keep_tokens : np;
+  const __nv_bfloat16 *qb, *kpb, *vpb;
+  int64_t qhs = head_stride, qts = token_stride, khs = prompt_head_stride, kts = prompt_token_stride, vhs = prompt_head_stride,
+          vts = prompt_token_stride;
+  int r = as_bf16(c, q, nq, &qhs, &qts, 2, &qb, st);
+  if (r == FASTAR_OK) r = as_bf16(c, k_prompt, np, &khs, &kts, 3, &kpb, st);
+  if (r == FASTAR_OK) r = as_bf16(c, v_prompt, np, &vhs, &vts, 4, &vpb, st);
+  if (r != FASTAR_OK) return r;
+  if ((reinterpret_cast<uintptr_t>(kpb) & 15) || (reinterpret_cast<uintptr_t>(vpb) & 15) || ((khs * 2) & 15) || ((kts * 2) & 15))
+    return FASTAR_ERR_INVALID_ARG;
+  CUtensorMap tm_q, tm_kp;
+  r = make_map(c, &tm_q, qb, v.D, nq, v.H, static_cast<uint64_t>(qts) * 2, static_cast<uint64_t>(qhs) * 2, 128);
+  if (r != FASTAR_OK) return r;
+  AttnArgs a{};
+  a.nq = nq;
+  a.block_q = 128;
+  a.rows_per_frame = frame_len;
+  a.keep = keep;
+  a.n_frames = F;
+  a.kp = kpb;
+  a.vp = vpb;
+  a.p_head_stride = khs;
+  a.p_token_stride = kts;
+  a.out = out;
+  a.out_fp32 = c->desc.dtype == FASTAR_FP32;
+  a.out_head_stride = head_stride;
+  a.out_token_stride = token_stride;
+  if (sel_in) {
+    a.sel = sel_in;
+    a.sel_stride = keep_tokens;
+    a.sel_head_stride = static_cast<int64_t>(F) * keep_tokens;
+  } else {
+    r = make_map(c, &tm_kp, kpb, v.D, np, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
+    if (r != FASTAR_OK) return r;
+    if (cudaMemsetAsync(v.rel, 0, static_cast<size_t>(v.H) * v.max_frames * v.max_prompt * 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+    ACC(launch_c1_relevance(v, tm_q, tm_kp, nq, np, frame_len, F, st));
+    ACC(launch_topk_prompt(v, F, np, keep, st));
+    a.sel = v.selp;
+    a.sel_stride = v.max_prompt;
+    a.sel_head_stride = static_cast<int64_t>(v.max_frames) * v.max_prompt;
+    if (sel_out) {
+      copy_rows3_kernel<<<dim3((F * keep + 255) / 256, v.H), 256, 0, st>>>(v.selp, a.sel_head_stride, v.max_prompt, sel_out, F, keep);
+      if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+      c->launches += 1;
+    }
+    if (rel_out) ACC(launch_decode_rel(v, F, np, 1.0f / sqrtf(static_cast<float>(v.D)), rel_out, st));
+  }
+  ACC(launch_attention_gather(v, tm_q, a, st));
+  return FASTAR_OK;
+}
+
+int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const void* v_new_host, const void* q_host,
+                               const void* k_prompt_host, const void* v_prompt_host, void* out_sa_host, void* out_ca_host,
+                               int32_t n, int32_t frame_len, int32_t np, float tau, int32_t block_q, int32_t keep_blocks,
+                               int32_t keep_tokens, void* stream) {
+  if (!c || !k_new_host || !v_new_host || !q_host || !k_prompt_host || !v_prompt_host || !out_sa_host || !out_ca_host)
+    return FASTAR_ERR_INVALID_ARG;
+  if (n < 1 || n > c->v.max_tokens || np < 1 || np > c->v.max_prompt) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const bool f32 = c->desc.dtype == FASTAR_FP32;
+  const size_t esz = f32 ? 4 : 2;
+  const void* hsrc[5] = {k_new_host, v_new_host, q_host, k_prompt_host, v_prompt_host};
+  void* dsrc[5];
+  for (int i = 0; i < 5; ++i) {
+    dsrc[i] = f32 ? v.stage_in_raw[i] : static_cast<void*>(v.stage[i]);
+    const size_t bytes = static_cast<size_t>(v.H) * (i < 3 ? n : np) * v.D * esz;
+    if (cudaMemcpyAsync(dsrc[i], hsrc[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  }
+  const int64_t hs = static_cast<int64_t>(n) * v.D, ts = v.D, phs = static_cast<int64_t>(np) * v.D;
+  int r = fastar_tempcache_update(c, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, stream);
+  if (r != FASTAR_OK) return r;
+  r = fastar_annsa_attention(c, dsrc[2], v.stage_out[0], n, hs, ts, block_q, keep_blocks, nullptr, nullptr, nullptr, nullptr, nullptr,
+                             nullptr, stream);
+  if (r != FASTAR_OK) return r;
+  r = fastar_annca_attention(c, dsrc[2], dsrc[3], dsrc[4], v.stage_out[1], n, frame_len, np, keep_tokens, hs, ts, phs, ts, nullptr,
+                             nullptr, nullptr, stream);
+  if (r != FASTAR_OK) return r;
+  const size_t obytes = static_cast<size_t>(v.H) * n * v.D * esz;
+  if (cudaMemcpyAsync(out_sa_host, v.stage_out[0], obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaMemcpyAsync(out_ca_host, v.stage_out[1], obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+int fastar_last_device_status(fastar_cache_t* c, void* stream) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int status = 0;
+  if (cudaMemcpyAsync(&status, c->v.status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaMemsetAsync(c->v.status, 0, 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  return status;
+}
+
+int64_t fastar_launch_count(const fastar_cache_t* c) { return c ? c->launches : 0; }
+
+const char* fastar_status_string(int status) {
+  switch (status) {
+    case FASTAR_OK: return "ok";
+    case FASTAR_ERR_INVALID_ARG: return "invalid argument";
+    case FASTAR_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case FASTAR_ERR_CAPACITY: return "cache capacity exhausted: not enough evictable slots, update not applied";
+    case FASTAR_ERR_CUDA: return "CUDA error";
+    case FASTAR_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case FASTAR_ERR_NOT_SM100: return "device is not compute capability 10.x";
+    case FASTAR_ERR_WORKSPACE: return "workspace too small or misaligned";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,328 @@
+// tcgen05 / TMEM / TMA contraction kernel with three fused epilogues:
+//   T1  key-similarity + row arg-max   (TempCache temporal correspondence, paper Section 5.2)
+//   C1  prompt relevance, column max per frame   (AnnCA, Section 5.3)
+//   S3  bucket-collision scores HQ x HK^T        (AnnSA block selection, Sections 5.1 / 5.4)
+// The score matrix is never written to memory for T1 and C1.
+//
+// One CTA = one 128-row tile of A and a range of 128-row tiles of B; D[128 x 128] fp32 lives in
+// TMEM, double buffered so the epilogue of tile t overlaps the MMAs of tile t+1.
+// Warp roles: warps 0-3 epilogue (thread r <-> TMEM lane r <-> A row r), warp 4 TMA producer,
+// warp 5 TMEM allocation + MMA issue.  Operands are bf16, K-major, 128-byte swizzled.
+#include "common.h"
+#include "ptx.cuh"
+
+namespace fastar {
+
+enum { EPI_ARGMAX = 0, EPI_COLMAX = 1, EPI_STORE = 2 };
+
+struct GemmArgs {
+  int rows_a;              // valid rows of A per head (n, nq or nqb)
+  int nkc;                 // K chunks of 64
+  int frame_len;           // COLMAX
+  int n_frames;            // COLMAX
+  int cols_b;              // COLMAX: np; STORE: unused (uses live blocks)
+};
+
+constexpr int kChunkBytes = 128 * 128;       // 128 rows x 64 bf16
+constexpr int kTmemCols = 256;
+
+template <int EPI, bool A_RES, int NST>
+struct GemmSmem {
+  static constexpr int a_bytes = A_RES ? 2 * kChunkBytes : 0;
+  static constexpr int stage_bytes = A_RES ? kChunkBytes : 2 * kChunkBytes;
+  static constexpr int ring_off = a_bytes;
+  static constexpr int rn_off = ring_off + NST * stage_bytes;
+  static constexpr int bar_off = rn_off + 2 * 128 * 4;
+  static constexpr int total = bar_off + 256;
+};
+
+template <int EPI, bool A_RES, int NST>
+__global__ void __launch_bounds__(192, A_RES ? 2 : 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c,
+            const GemmArgs g) {
+  using SM = GemmSmem<EPI, A_RES, NST>;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t sbase = smem_u32(smem_raw);
+  uint8_t* sgen = smem_raw;
+  if (sbase & 1023u) {                  // swizzled tiles need 1024-byte alignment; uniform for the CTA
+    if (threadIdx.x == 0) record_status(c.status, FASTAR_ERR_CUDA);
+    return;
+  }
+  const uint32_t a_s = sbase;
+  const uint32_t ring_s = sbase + SM::ring_off;
+  float* rn_s = reinterpret_cast<float*>(sgen + SM::rn_off);
+  const uint32_t bar_s = sbase + SM::bar_off;
+  // barrier slots (8 bytes each)
+  const uint32_t bar_full = bar_s;                   // [NST]
+  const uint32_t bar_empty = bar_s + 8 * NST;        // [NST]
+  const uint32_t bar_tfull = bar_s + 16 * NST;       // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;        // [2]
+  const uint32_t bar_afull = bar_tempty + 16;        // [1]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + SM::bar_off + 16 * NST + 40);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + SM::bar_off + 16 * NST + 44);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.y;
+  const int m0 = blockIdx.x * 128;
+  const int L = c.len[h];
+
+  // ---- tile range of this CTA ----------------------------------------------------------------
+  int n_tiles;
+  if (EPI == EPI_ARGMAX) n_tiles = (L + 127) >> 7;
+  else if (EPI == EPI_COLMAX) n_tiles = (g.cols_b + 127) >> 7;
+  else n_tiles = (((L + c.PT - 1) / c.PT) + 127) >> 7;
+  const int per = (n_tiles + gridDim.z - 1) / gridDim.z;
+  const int t0 = blockIdx.z * per;
+  const int ntl = max(0, min(n_tiles, t0 + per) - t0);
+  const int nkc = g.nkc;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NST; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8 * b, 1);
+      mbar_init(bar_tempty + 8 * b, 128);
+    }
+    mbar_init(bar_afull, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 4 && lane == 0) {
+    tma_prefetch_desc(&tm_a);
+    tma_prefetch_desc(&tm_b);
+  }
+  __syncthreads();
+  if (warp == 5) {
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (ntl > 0) {
+    if (warp == 4) {
+      // ------------------------------------------------------------------ TMA producer
+      if (lane == 0) {
+        bool ok = true;
+        if (A_RES) {
+          mbar_arrive_expect_tx(bar_afull, nkc * kChunkBytes);
+          for (int kc = 0; kc < nkc; ++kc) tma_load_3d(a_s + kc * kChunkBytes, &tm_a, bar_afull, kc * 64, m0, h);
+        }
+        const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+        const int pages_per_tile = 128 / c.PT;
+        int it = 0;
+        for (int tl = 0; tl < ntl && ok; ++tl) {
+          const int t = t0 + tl;
+          for (int kc = 0; kc < nkc; ++kc, ++it) {
+            const int s = it % NST;
+            const uint32_t ph = (it / NST) & 1;
+            ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, c.status);
+            if (!ok) break;
+            const uint32_t st_s = ring_s + s * SM::stage_bytes;
+            mbar_arrive_expect_tx(bar_full + 8 * s, SM::stage_bytes);
+            uint32_t b_s = st_s;
+            if (!A_RES) {
+              tma_load_3d(st_s, &tm_a, bar_full + 8 * s, kc * 64, m0, h);
+              b_s = st_s + kChunkBytes;
+            }
+            if (EPI == EPI_ARGMAX) {
+              for (int pg = 0; pg < pages_per_tile; ++pg) {
+                const int page = pt_h[t * pages_per_tile + pg];
+                tma_load_3d(b_s + pg * c.PT * 128, &tm_b, bar_full + 8 * s, kc * 64, 0, page);
+              }
+            } else {
+              tma_load_3d(b_s, &tm_b, bar_full + 8 * s, kc * 64, t * 128, h);
+            }
+          }
+        }
+        // drain: let the loads still in flight land before the CTA may exit
+        const int issued = it;
+        for (int k = max(0, issued - NST); k < issued; ++k) {
+          // full barriers are consumed by the MMA warp in order; waiting on the last ones is
+          // enough and cheap.  Bounded like every other wait.
+          mbar_wait(bar_full + 8 * (k % NST), (k / NST) & 1, abort_flag, c.status);
+        }
+      }
+    } else if (warp == 5) {
+      // ------------------------------------------------------------------ MMA issue
+      if (lane == 0) {
+        constexpr uint32_t idesc = make_idesc_bf16(128, 128, 0);
+        bool ok = true;
+        if (A_RES) ok = mbar_wait(bar_afull, 0, abort_flag, c.status);
+        int it = 0;
+        for (int tl = 0; tl < ntl && ok; ++tl) {
+          const int buf = tl & 1;
+          ok = mbar_wait(bar_tempty + 8 * buf, ((tl >> 1) & 1) ^ 1, abort_flag, c.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_t = tmem + buf * 128;
+          for (int kc = 0; kc < nkc; ++kc, ++it) {
+            const int s = it % NST;
+            ok = mbar_wait(bar_full + 8 * s, (it / NST) & 1, abort_flag, c.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t st_s = ring_s + s * SM::stage_bytes;
+            const uint32_t a_c = A_RES ? a_s + kc * kChunkBytes : st_s;
+            const uint32_t b_c = A_RES ? st_s : st_s + kChunkBytes;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+              const uint64_t ad = make_smem_desc(a_c + k4 * 32, 16, 1024);
+              const uint64_t bd = make_smem_desc(b_c + k4 * 32, 16, 1024);
+              umma_ss(d_t, ad, bd, idesc, (kc | k4) != 0);
+            }
+            umma_commit(bar_empty + 8 * s);
+          }
+          if (ok) umma_commit(bar_tfull + 8 * buf);
+        }
+      }
+    } else {
+      // ------------------------------------------------------------------ epilogue (128 threads)
+      const int r = threadIdx.x;                    // A row inside the tile = TMEM lane
+      const int row = m0 + r;
+      const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+      float best = -INFINITY;
+      int best_j = -1;
+      bool ok = true;
+      for (int tl = 0; tl < ntl && ok; ++tl) {
+        const int t = t0 + tl;
+        const int buf = tl & 1;
+        int valid_cols = 128;
+        if (EPI == EPI_ARGMAX) {
+          const int slot = t * 128 + r;
+          rn_s[buf * 128 + r] = slot < L ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+          valid_cols = min(128, L - t * 128);
+          named_barrier_sync(1, 128);
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
+        if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
+        tc_fence_after();
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(tmem + lane_addr + buf * 128 + cc * 32, v);
+          tmem_wait_ld();
+          if (EPI == EPI_ARGMAX) {
+            const float* rn = rn_s + buf * 128 + cc * 32;
+            const int jbase = t * 128 + cc * 32;
+            if (cc * 32 + 32 <= valid_cols) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float x = __uint_as_float(v[j]) * rn[j];
+                if (x > best) { best = x; best_j = jbase + j; }
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float x = __uint_as_float(v[j]) * rn[j];
+                if (cc * 32 + j < valid_cols && x > best) { best = x; best_j = jbase + j; }
+              }
+            }
+          } else if (EPI == EPI_COLMAX) {
+            const bool rvalid = row < g.rows_a;
+            const int f_r = rvalid ? row / g.frame_len : -1;
+            int f_lo = rvalid ? f_r : 0x7fffffff, f_hi = f_r;
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) {
+              f_lo = min(f_lo, __shfl_xor_sync(0xffffffffu, f_lo, o));
+              f_hi = max(f_hi, __shfl_xor_sync(0xffffffffu, f_hi, o));
+            }
+            for (int f = f_lo; f <= f_hi; ++f) {       // empty when the warp has no valid row
+              float x[32];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) x[j] = (f_r == f) ? __uint_as_float(v[j]) : -INFINITY;
+              // butterfly: after it, lane l holds the maximum of column l over the 32 rows
+#pragma unroll
+              for (int o = 16, w = 32; o >= 1; o >>= 1, w >>= 1) {
+                const bool up = (lane & o) != 0;
+#pragma unroll
+                for (int j = 0; j < w / 2; ++j) {
+                  const float send = up ? x[j] : x[j + w / 2];
+                  const float keep = up ? x[j + w / 2] : x[j];
+                  x[j] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, o));
+                }
+              }
+              const int col = t * 128 + cc * 32 + lane;
+              if (col < g.cols_b)
+                atomicMax(c.rel + (static_cast<int64_t>(h) * c.max_frames + f) * c.max_prompt + col,
+                          float_to_ordered(x[0]));
+            }
+          } else {  // EPI_STORE
+            if (row < g.rows_a) {
+              float* dst = c.scores + (static_cast<int64_t>(h) * c.max_qb + row) * c.CAPB + t * 128 + cc * 32;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (t * 128 + cc * 32 + j < c.CAPB) dst[j] = __uint_as_float(v[j]);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_tempty + 8 * buf);
+      }
+      if (EPI == EPI_ARGMAX && ok && row < g.rows_a && best_j >= 0) {
+        const float sim = best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
+                                       static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
+        atomicMax(c.best + static_cast<int64_t>(h) * c.max_tokens + row, key);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+template <int EPI, bool A_RES, int NST>
+static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const CacheView& c, const GemmArgs& g, dim3 grid,
+                       cudaStream_t st) {
+  using SM = GemmSmem<EPI, A_RES, NST>;
+  auto kern = gemm_kernel<EPI, A_RES, NST>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+    configured = true;
+  }
+  kern<<<grid, 192, SM::total, st>>>(tm_a, tm_b, c, g);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k, int n, cudaStream_t st) {
+  GemmArgs g{};
+  g.rows_a = n;
+  g.nkc = c.D / 64;
+  const int row_tiles = (n + 127) / 128;
+  // enough CTAs to fill the machine a few times over; every split scans a contiguous slot range
+  int splits = 1;
+  const int max_tiles = c.CAP / 128;
+  while (row_tiles * c.H * splits < 2 * 148 && splits * 2 <= max_tiles && splits < 16) splits *= 2;
+  return launch_gemm<EPI_ARGMAX, true, 4>(tm_a, tm_pool_k, c, g, dim3(row_tiles, c.H, splits), st);
+}
+
+int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,
+                        int n_frames, cudaStream_t st) {
+  GemmArgs g{};
+  g.rows_a = nq;
+  g.nkc = c.D / 64;
+  g.frame_len = frame_len;
+  g.n_frames = n_frames;
+  g.cols_b = np;
+  return launch_gemm<EPI_COLMAX, true, 4>(tm_q, tm_kp, c, g, dim3((nq + 127) / 128, c.H, 1), st);
+}
+
+int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtensorMap& tm_hk, int nqb, cudaStream_t st) {
+  GemmArgs g{};
+  g.rows_a = nqb;
+  g.nkc = c.hist_cols / 64;
+  const int col_tiles = (c.CAPB + 127) / 128;
+  return launch_gemm<EPI_STORE, false, 4>(tm_hq, tm_hk, c, g, dim3((nqb + 127) / 128, c.H, col_tiles), st);
+}
+
+}  // namespace fastar

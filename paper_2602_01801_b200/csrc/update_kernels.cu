@@ -1,0 +1,618 @@
+// HBM-bound and integer kernels of the step (plain CUDA: coalesced vector access, warp shuffles,
+// shared-memory sorts and scans):
+//   S1  sign-random-projection codes (+ 1/|x|)               paper Section 5.1 (LSH)
+//   T2  threshold, T3 grouping plan, T4 compaction / append / eviction plan   Section 5.2
+//   T3/T4 commit: count-weighted value mean, last-key copy, append            Section 5.2, Lemma 1
+//   S2  per-block bucket histograms, S4 / C2 top-k with ties to the lower index   Sections 5.3, 5.4
+#include "common.h"
+#include "ptx.cuh"
+
+namespace fastar {
+
+// ---------------------------------------------------------------------------------------------
+// block-wide helpers (blockDim.x a multiple of 32, at most 1024)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int block_sum(int v, int* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  int t = 0;
+  for (int w = 0; w < nw; ++w) t += red[w];
+  return t;
+}
+// exclusive scan of one value per thread; *total receives the block sum
+__device__ __forceinline__ int block_exscan(int v, int* red, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();
+  if (lane == 31) red[warp] = inc;
+  __syncthreads();
+  int base = 0, tot = 0;
+  for (int w = 0; w < nw; ++w) {
+    const int x = red[w];
+    if (w < warp) base += x;
+    tot += x;
+  }
+  *total = tot;
+  return base + inc - v;
+}
+__device__ __forceinline__ void bitonic_sort_smem(unsigned long long* keys, int np2) {
+  for (int k = 2; k <= np2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = threadIdx.x; t < (np2 >> 1); t += blockDim.x) {
+        const int i = ((t / j) * 2 * j) + (t % j);
+        const int p = i + j;
+        const bool up = (i & k) == 0;
+        const unsigned long long a = keys[i], b = keys[p];
+        if ((a > b) == up) { keys[i] = b; keys[p] = a; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// fp32 -> bf16 entry conversion (strided source, contiguous destination)
+// ---------------------------------------------------------------------------------------------
+__global__ void convert_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int n, int D, int64_t hs,
+                               int64_t ts) {
+  const int h = blockIdx.y;
+  const int64_t per_head = static_cast<int64_t>(n) * D / 4;
+  for (int64_t q = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; q < per_head;
+       q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t e = q * 4;
+    const int row = static_cast<int>(e / D), col = static_cast<int>(e % D);
+    const float4 v = *reinterpret_cast<const float4*>(src + h * hs + row * ts + col);
+    uint2 o;
+    o.x = pack_bf16x2(v.x, v.y);
+    o.y = pack_bf16x2(v.z, v.w);
+    *reinterpret_cast<uint2*>(dst + (static_cast<int64_t>(h) * n + row) * D + col) = o;
+  }
+}
+int launch_convert_f32_to_bf16(const float* src, __nv_bfloat16* dst, int H, int n, int D, int64_t hs, int64_t ts,
+                               cudaStream_t st) {
+  if (n <= 0) return 0;
+  const int64_t per_head = static_cast<int64_t>(n) * D / 4;
+  const int64_t want = (per_head + 255) / 256;
+  const int bx = static_cast<int>(want < 1024 ? want : 1024);
+  convert_kernel<<<dim3(bx, H), 256, 0, st>>>(src, dst, n, D, hs, ts);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// S1: codes (and reciprocal norms).  One warp per row; lane c owns projection direction c.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restrict__ x, int n, int64_t hs, int64_t ts,
+                                                   const __nv_bfloat16* __restrict__ lsh, int T, int B,
+                                                   uint32_t* __restrict__ code_out, float* __restrict__ rnorm_out,
+                                                   int64_t out_stride) {
+  __shared__ float rt[D][33];           // rt[k][c] = R[c][k]
+  __shared__ float xs[8][D];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int h = blockIdx.y;
+  const int ncol = T * B;
+  for (int q = threadIdx.x; q < D * 32; q += blockDim.x) {
+    const int cidx = q / D, k = q % D;
+    rt[k][cidx] = cidx < ncol ? __bfloat162float(lsh[cidx * D + k]) : 0.f;
+  }
+  __syncthreads();
+  constexpr int EPL = D / 32;
+  for (int row = blockIdx.x * 8 + warp; row < n; row += gridDim.x * 8) {
+    const __nv_bfloat16* xr = x + h * hs + row * ts;
+    float sq = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; e += 2) {
+      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(xr + lane * EPL + e);
+      const float a = __low2float(v), b = __high2float(v);
+      xs[warp][lane * EPL + e] = a;
+      xs[warp][lane * EPL + e + 1] = b;
+      sq = fmaf(a, a, sq);
+      sq = fmaf(b, b, sq);
+    }
+    __syncwarp();
+    float acc = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < D; ++k) acc = fmaf(xs[warp][k], rt[k][lane], acc);
+    const uint32_t bits = __ballot_sync(0xffffffffu, acc > 0.f);
+    uint32_t code = 0;
+    for (int t = 0; t < T; ++t) code |= ((bits >> (t * B)) & ((1u << B) - 1u)) << (8 * t);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if (lane == 0) {
+      code_out[h * out_stride + row] = code;
+      if (rnorm_out) rnorm_out[h * out_stride + row] = sq > 0.f ? 1.f / sqrtf(sq) : 0.f;
+    }
+    __syncwarp();
+  }
+}
+static int launch_prep_generic(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
+                               float* rnorm_out, int64_t out_stride, cudaStream_t st) {
+  if (n <= 0) return 0;
+  const dim3 grid(min((n + 7) / 8, 148 * 4), c.H);
+  if (c.D == 128) prep_kernel<128><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
+  else prep_kernel<64><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
+                      float* rnorm_out, cudaStream_t st) {
+  return launch_prep_generic(c, x, n, hs, ts, code_out, rnorm_out, c.max_tokens, st);
+}
+
+// ---------------------------------------------------------------------------------------------
+// T2-T4 planning: one CTA per head.  Sort tokens by (matched slot, token), find the groups,
+// place the unmatched tokens (append, then victims in (stamp, slot) order).  Validate, then commit.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n, int np2, float tau) {
+  extern __shared__ unsigned long long keys[];
+  __shared__ int red[32];
+  __shared__ int sh[8];
+  const int h = blockIdx.x, tid = threadIdx.x;
+  const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+  const int64_t sb = static_cast<int64_t>(h) * c.CAP;
+  const int L = c.len[h];
+  const int now = *c.now;
+
+  // T2: decode the packed arg-max, threshold
+  for (int i = tid; i < np2; i += blockDim.x) {
+    unsigned long long key = ~0ull;
+    if (i < n) {
+      const unsigned long long b = c.best[tb + i];
+      int j = -1;
+      float s = 0.f;
+      if (b != 0ull) {
+        j = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull));
+        s = ordered_to_float(static_cast<uint32_t>(b >> 32));
+      }
+      const bool matched = j >= 0 && s >= tau;
+      c.match[tb + i] = matched ? j : -1;
+      c.sim[tb + i] = s;
+      key = (static_cast<unsigned long long>(matched ? static_cast<uint32_t>(j) : 0xFFFFFFFFu) << 32) |
+            static_cast<uint32_t>(i);
+    }
+    keys[i] = key;
+  }
+  __syncthreads();
+  bitonic_sort_smem(keys, np2);
+
+  // matched count, segment heads
+  int my_m = 0, my_heads = 0, my_heads_ns = 0;
+  const int per = (np2 + blockDim.x - 1) / blockDim.x;
+  const int p_lo = tid * per, p_hi = min(n, p_lo + per);
+  for (int p = p_lo; p < p_hi; ++p) {
+    const uint32_t slot = static_cast<uint32_t>(keys[p] >> 32);
+    if (slot != 0xFFFFFFFFu) {
+      ++my_m;
+      if (p == 0 || static_cast<uint32_t>(keys[p - 1] >> 32) != slot) {
+        ++my_heads;
+        if (static_cast<int>(slot) >= c.n_sink) ++my_heads_ns;
+      }
+    }
+  }
+  const int M = block_sum(my_m, red);
+  const int touched_ns = block_sum(my_heads_ns, red);
+  int n_seg;
+  int seg_base = block_exscan(my_heads, red, &n_seg);
+  for (int p = p_lo; p < p_hi; ++p) {
+    const unsigned long long k = keys[p];
+    const uint32_t slot = static_cast<uint32_t>(k >> 32);
+    const int i = static_cast<int>(k & 0xFFFFFFFFull);
+    c.order[tb + p] = i;
+    if (slot != 0xFFFFFFFFu) {
+      c.dest[tb + i] = static_cast<int>(slot);
+      if (p == 0 || static_cast<uint32_t>(keys[p - 1] >> 32) != slot) c.segpos[static_cast<int64_t>(h) * (c.max_tokens + 1) + seg_base++] = p;
+    }
+  }
+  const int U = n - M;
+  const int A = min(U, c.CAP - L);
+  const int E = U - A;
+  int ok = 1;
+  if (E > 0) {
+    int cand = 0;
+    for (int j = tid; j < L; j += blockDim.x) cand += (j >= c.n_sink && c.stamp[sb + j] < now) ? 1 : 0;
+    cand = block_sum(cand, red) - touched_ns;
+    if (cand < E) ok = 0;
+  }
+  int evicted_tokens = 0;
+  if (ok && E > 0) {
+    // touched slots are not evictable: stamp them now (the commit writes the same value)
+    for (int p = p_lo; p < p_hi; ++p) {
+      const uint32_t slot = static_cast<uint32_t>(keys[p] >> 32);
+      if (slot != 0xFFFFFFFFu && (p == 0 || static_cast<uint32_t>(keys[p - 1] >> 32) != slot)) c.stamp[sb + slot] = now;
+    }
+    __syncthreads();
+    // smallest stamp value s* such that at least E evictable slots have stamp <= s*
+    int lo = 0, hi = now - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      int cnt = 0;
+      for (int j = tid; j < L; j += blockDim.x) cnt += (j >= c.n_sink && c.stamp[sb + j] <= mid) ? 1 : 0;
+      cnt = block_sum(cnt, red);
+      if (cnt >= E) hi = mid; else lo = mid + 1;
+    }
+    const int sstar = lo;
+    int c_less = 0;
+    for (int j = tid; j < L; j += blockDim.x) c_less += (j >= c.n_sink && c.stamp[sb + j] < sstar) ? 1 : 0;
+    c_less = block_sum(c_less, red);
+    const int need_eq = E - c_less;
+    // ordered compaction of the victims into keys[0..E)
+    int eq_run = 0, out_run = 0;
+    __syncthreads();
+    for (int j0 = 0; j0 < L; j0 += blockDim.x) {
+      const int j = j0 + tid;
+      const int stp = (j < L && j >= c.n_sink) ? c.stamp[sb + j] : 0x7fffffff;
+      const int is_eq = stp == sstar ? 1 : 0;
+      int tot_eq;
+      const int eq_rank = eq_run + block_exscan(is_eq, red, &tot_eq);
+      const int take = (stp < sstar || (is_eq && eq_rank < need_eq)) ? 1 : 0;
+      int tot_take;
+      const int pos = out_run + block_exscan(take, red, &tot_take);
+      if (take) keys[pos] = (static_cast<unsigned long long>(static_cast<uint32_t>(stp)) << 32) | static_cast<uint32_t>(j);
+      eq_run += tot_eq;
+      out_run += tot_take;
+    }
+    int e2 = 1;
+    while (e2 < E) e2 <<= 1;
+    for (int p = E + tid; p < e2; p += blockDim.x) keys[p] = ~0ull;
+    __syncthreads();
+    bitonic_sort_smem(keys, e2);
+    int ev = 0;
+    for (int k = tid; k < E; k += blockDim.x) {
+      const int v = static_cast<int>(keys[k] & 0xFFFFFFFFull);
+      c.victims[tb + k] = v;
+      ev += c.count[sb + v];
+    }
+    evicted_tokens = block_sum(ev, red);
+    __syncthreads();
+  }
+  // destinations of the unmatched tokens (sorted positions [M, n) are in token order)
+  if (ok) {
+    __syncthreads();
+    for (int p = M + tid; p < n; p += blockDim.x) {
+      const int k = p - M;
+      const int i = c.order[tb + p];
+      c.dest[tb + i] = k < A ? L + k : c.victims[tb + k - A];
+    }
+  } else {
+    for (int i = tid; i < n; i += blockDim.x) c.dest[tb + i] = -1;
+    if (tid == 0) record_status(c.status, kErrCapacity);
+  }
+  if (tid == 0) {
+    PlanRec pr;
+    pr.ok = ok;
+    pr.n_matched = M;
+    pr.n_seg = n_seg;
+    pr.n_unmatched = U;
+    pr.n_append = ok ? A : 0;
+    pr.n_evict = ok ? E : 0;
+    pr.len_old = L;
+    pr.len_new = ok ? L + A : L;
+    pr.evicted_tokens = evicted_tokens;
+    pr.pad[0] = pr.pad[1] = pr.pad[2] = 0;
+    c.plan[h] = pr;
+    (void)sh;
+  }
+}
+int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st) {
+  (void)frame_len;
+  int np2 = 1024;
+  while (np2 < n) np2 <<= 1;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 8) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+    configured = true;
+  }
+  plan_kernel<<<c.H, 1024, np2 * 8, st>>>(c, n, np2, tau);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// T3/T4 commit: one warp per touched slot or per unmatched token.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __nv_bfloat16* __restrict__ k_new,
+                                                     const __nv_bfloat16* __restrict__ v_new, int n, int frame_len, int64_t hs,
+                                                     int64_t ts) {
+  constexpr int EPL = D / 32;           // elements per lane (4 or 2), contiguous
+  const int h = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const PlanRec pr = c.plan[h];
+  if (!pr.ok) return;
+  const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+  const int64_t sb = static_cast<int64_t>(h) * c.CAP;
+  const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+  const int now = *c.now;
+  const __nv_bfloat16* kh = k_new + h * hs;
+  const __nv_bfloat16* vh = v_new + h * hs;
+
+  if (w < pr.n_seg) {
+    const int32_t* segpos = c.segpos + static_cast<int64_t>(h) * (c.max_tokens + 1);
+    const int p0 = segpos[w];
+    const int p1 = (w + 1 < pr.n_seg) ? segpos[w + 1] : pr.n_matched;
+    const int slot = c.match[tb + c.order[tb + p0]];
+    const int64_t ro = slot_row_offset(c, pt_h, slot);
+    const int m_old = c.count[sb + slot];
+    float acc[EPL];
+    {
+      const __nv_bfloat16* vr = c.pool_v + ro + lane * EPL;
+#pragma unroll
+      for (int e = 0; e < EPL; e += 2) {
+        const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(vr + e);
+        acc[e] = static_cast<float>(m_old) * __low2float(t);
+        acc[e + 1] = static_cast<float>(m_old) * __high2float(t);
+      }
+    }
+    // representative: newest frame, then highest similarity, then lowest token index
+    int best_i = -1, best_f = -1;
+    float best_s = -INFINITY;
+    for (int p = p0; p < p1; ++p) {                    // ascending token index
+      const int i = c.order[tb + p];
+      const __nv_bfloat16* vr = vh + i * ts + lane * EPL;
+#pragma unroll
+      for (int e = 0; e < EPL; e += 2) {
+        const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(vr + e);
+        acc[e] += __low2float(t);
+        acc[e + 1] += __high2float(t);
+      }
+      const int f = i / frame_len;
+      const float s = c.sim[tb + i];
+      if (f > best_f || (f == best_f && s > best_s)) { best_f = f; best_s = s; best_i = i; }
+    }
+    const int g = p1 - p0;
+    const float inv = 1.f / static_cast<float>(m_old + g);
+    {
+      __nv_bfloat16* vw = c.pool_v + ro + lane * EPL;
+      const __nv_bfloat16* kr = kh + best_i * ts + lane * EPL;
+      __nv_bfloat16* kw = c.pool_k + ro + lane * EPL;
+#pragma unroll
+      for (int e = 0; e < EPL; e += 2) {
+        *reinterpret_cast<__nv_bfloat162*>(vw + e) = __floats2bfloat162_rn(acc[e] * inv, acc[e + 1] * inv);
+        *reinterpret_cast<__nv_bfloat162*>(kw + e) = *reinterpret_cast<const __nv_bfloat162*>(kr + e);
+      }
+    }
+    if (lane == 0) {
+      c.count[sb + slot] = m_old + g;
+      c.stamp[sb + slot] = now;
+      c.log2m[sb + slot] = log2f(static_cast<float>(m_old + g));
+      c.rnorm[sb + slot] = c.rnorm_new[tb + best_i];
+      c.kcode[sb + slot] = c.code_new[tb + best_i];
+    }
+  } else if (w - pr.n_seg < pr.n_unmatched) {
+    const int i = c.order[tb + pr.n_matched + (w - pr.n_seg)];
+    const int slot = c.dest[tb + i];
+    const int64_t ro = slot_row_offset(c, pt_h, slot);
+    const __nv_bfloat16* kr = kh + i * ts + lane * EPL;
+    const __nv_bfloat16* vr = vh + i * ts + lane * EPL;
+#pragma unroll
+    for (int e = 0; e < EPL; e += 2) {
+      *reinterpret_cast<__nv_bfloat162*>(c.pool_k + ro + lane * EPL + e) = *reinterpret_cast<const __nv_bfloat162*>(kr + e);
+      *reinterpret_cast<__nv_bfloat162*>(c.pool_v + ro + lane * EPL + e) = *reinterpret_cast<const __nv_bfloat162*>(vr + e);
+    }
+    if (lane == 0) {
+      c.count[sb + slot] = 1;
+      c.stamp[sb + slot] = now;
+      c.log2m[sb + slot] = 0.f;
+      c.rnorm[sb + slot] = c.rnorm_new[tb + i];
+      c.kcode[sb + slot] = c.code_new[tb + i];
+    }
+  }
+}
+int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len, int64_t hs,
+                  int64_t ts, cudaStream_t st) {
+  if (n <= 0) return 0;
+  const dim3 grid((n + 7) / 8, c.H);
+  if (c.D == 128) commit_kernel<128><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  else commit_kernel<64><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// S2 (key side) + end of an update: bucket histogram of every key block, new lengths, stats, clock.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) key_hist_kernel(const CacheView c, int use_plan, fastar_update_stats* stats_out,
+                                                       int advance_clock) {
+  extern __shared__ int hist[];          // hist_cols counters
+  const int b = blockIdx.x, h = blockIdx.y;
+  const int L = use_plan ? c.plan[h].len_new : c.len[h];
+  for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) hist[q] = 0;
+  __syncthreads();
+  const int s0 = b * c.PT, s1 = min(L, s0 + c.PT);
+  const int nb = 1 << c.B;
+  for (int s = s0 + threadIdx.x; s < s1; s += blockDim.x) {
+    const uint32_t code = c.kcode[static_cast<int64_t>(h) * c.CAP + s];
+    for (int t = 0; t < c.T; ++t) atomicAdd(&hist[t * nb + ((code >> (8 * t)) & 0xFFu)], 1);
+  }
+  __syncthreads();
+  __nv_bfloat16* dst = c.hk + (static_cast<int64_t>(h) * c.CAPB + b) * c.hist_cols;
+  for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) dst[q] = __float2bfloat16(static_cast<float>(hist[q]));
+  if (b == 0 && threadIdx.x == 0 && use_plan) {
+    const PlanRec pr = c.plan[h];
+    c.len[h] = pr.len_new;
+    if (stats_out) {
+      fastar_update_stats s;
+      s.matched = pr.n_matched;
+      s.touched = pr.n_seg;
+      s.appended = pr.n_append;
+      s.evicted_slots = pr.n_evict;
+      s.evicted_tokens = pr.evicted_tokens;
+      s.length = pr.len_new;
+      s.ok = pr.ok;
+      s.reserved = 0;
+      stats_out[h] = s;
+    }
+    if (h == 0 && advance_clock) *c.now = *c.now + 1;
+  }
+}
+int launch_finalize_hist(const CacheView& c, fastar_update_stats* stats_out, int advance_clock, cudaStream_t st) {
+  key_hist_kernel<<<dim3(c.CAPB, c.H), 256, c.hist_cols * 4, st>>>(c, advance_clock >= 0 ? 1 : 0, stats_out,
+                                                                  advance_clock > 0 ? 1 : 0);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// S2 (query side)
+__global__ void __launch_bounds__(128) query_hist_kernel(const CacheView c, int nq, int block_q) {
+  extern __shared__ int hist[];
+  const int a = blockIdx.x, h = blockIdx.y;
+  for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) hist[q] = 0;
+  __syncthreads();
+  const int r0 = a * block_q, r1 = min(nq, r0 + block_q);
+  const int nb = 1 << c.B;
+  for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x) {
+    const uint32_t code = c.code_new[static_cast<int64_t>(h) * c.max_tokens + r];
+    for (int t = 0; t < c.T; ++t) atomicAdd(&hist[t * nb + ((code >> (8 * t)) & 0xFFu)], 1);
+  }
+  __syncthreads();
+  __nv_bfloat16* dst = c.hq + (static_cast<int64_t>(h) * c.max_qb + a) * c.hist_cols;
+  for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) dst[q] = __float2bfloat16(static_cast<float>(hist[q]));
+}
+int launch_query_hist(const CacheView& c, int nq, int block_q, cudaStream_t st) {
+  const int nqb = (nq + block_q - 1) / block_q;
+  query_hist_kernel<<<dim3(nqb, c.H), 128, c.hist_cols * 4, st>>>(c, nq, block_q);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// S4 / C2: per row keep the k largest entries (ties -> lower index), listed ascending.
+// ---------------------------------------------------------------------------------------------
+template <bool ORDERED_UINT>
+__global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src, int64_t src_head_stride, int src_row_stride,
+                                                   const int32_t* __restrict__ len, int len_div, int n_fixed, int keep,
+                                                   int32_t* __restrict__ out, int64_t out_head_stride, int out_row_stride,
+                                                   int out_fill, int32_t* __restrict__ nsel) {
+  extern __shared__ float vals[];
+  __shared__ int red[32];
+  const int row = blockIdx.x, h = blockIdx.y;
+  const int n = len ? (len[h] + len_div - 1) / len_div : n_fixed;
+  const int k = min(keep, n);
+  const int64_t so = static_cast<int64_t>(h) * src_head_stride + static_cast<int64_t>(row) * src_row_stride;
+  for (int i = threadIdx.x; i < n; i += blockDim.x)
+    vals[i] = ORDERED_UINT ? ordered_to_float(static_cast<const uint32_t*>(src)[so + i]) : static_cast<const float*>(src)[so + i];
+  __syncthreads();
+  int32_t* orow = out + static_cast<int64_t>(h) * out_head_stride + static_cast<int64_t>(row) * out_row_stride;
+  int run = 0;
+  for (int i0 = 0; i0 < n; i0 += blockDim.x) {
+    const int i = i0 + threadIdx.x;
+    int take = 0;
+    if (i < n) {
+      const float v = vals[i];
+      int rank = 0;
+      for (int j = 0; j < n; ++j) {
+        const float u = vals[j];
+        rank += (u > v || (u == v && j < i)) ? 1 : 0;
+      }
+      take = rank < k ? 1 : 0;
+    }
+    int tot;
+    const int pos = run + block_exscan(take, red, &tot);
+    if (take) orow[pos] = i;
+    run += tot;
+  }
+  for (int i = k + threadIdx.x; i < out_fill; i += blockDim.x) orow[i] = -1;
+  if (nsel && row == 0 && threadIdx.x == 0) nsel[h] = k;
+}
+int launch_topk_blocks(const CacheView& c, int nqb, int keep, cudaStream_t st) {
+  topk_kernel<false><<<dim3(nqb, c.H), 256, c.CAPB * 4, st>>>(c.scores, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB, c.len,
+                                                            c.PT, 0, keep, c.sel, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB,
+                                                            min(keep, c.CAPB), c.nsel);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st) {
+  topk_kernel<true><<<dim3(n_frames, c.H), 256, np * 4, st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
+                                                             c.max_prompt, nullptr, 1, np, keep, c.selp,
+                                                             static_cast<int64_t>(c.max_frames) * c.max_prompt, c.max_prompt,
+                                                             min(keep, np), nullptr);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// reset / import helpers, output decoding
+// ---------------------------------------------------------------------------------------------
+__global__ void reset_meta_kernel(const CacheView c) {
+  const int64_t total = static_cast<int64_t>(c.H) * c.CAP;
+  for (int64_t q = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; q < total;
+       q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    c.count[q] = 0;
+    c.stamp[q] = 0;
+    c.log2m[q] = -INFINITY;
+    c.rnorm[q] = 0.f;
+    c.kcode[q] = 0;
+    if (q < static_cast<int64_t>(c.H) * c.CAPB) c.page_table[q] = static_cast<int32_t>(q);
+    if (q < c.H) c.len[q] = 0;
+    if (q == 0) { *c.now = 0; *c.status = 0; }
+  }
+}
+int launch_reset(const CacheView& c, cudaStream_t st) {
+  const size_t pool = static_cast<size_t>(c.H) * c.CAP * c.D * sizeof(__nv_bfloat16);
+  if (cudaMemsetAsync(c.pool_k, 0, pool, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaMemsetAsync(c.pool_v, 0, pool, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaMemsetAsync(c.hk, 0, static_cast<size_t>(c.H) * c.CAPB * c.hist_cols * 2, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  reset_meta_kernel<<<296, 256, 0, st>>>(c);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// after an import: clear dead slots, derive log2 m, keep counts of dead slots at 0
+template <int D>
+__global__ void import_fix_kernel(const CacheView c) {
+  const int h = blockIdx.y;
+  const int L = c.len[h];
+  const int lane = threadIdx.x & 31;
+  const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+  for (int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); s < c.CAP; s += gridDim.x * (blockDim.x >> 5)) {
+    const int64_t q = static_cast<int64_t>(h) * c.CAP + s;
+    if (s >= L) {
+      const int64_t ro = slot_row_offset(c, pt_h, s);
+      for (int e = lane * 2; e < D; e += 64) {
+        *reinterpret_cast<uint32_t*>(c.pool_k + ro + e) = 0u;
+        *reinterpret_cast<uint32_t*>(c.pool_v + ro + e) = 0u;
+      }
+      if (lane == 0) { c.count[q] = 0; c.stamp[q] = 0; c.log2m[q] = -INFINITY; c.rnorm[q] = 0.f; c.kcode[q] = 0; }
+    } else if (lane == 0) {
+      c.log2m[q] = log2f(static_cast<float>(max(1, c.count[q])));
+    }
+  }
+}
+int launch_import_derive(const CacheView& c, cudaStream_t st) {
+  // codes and reciprocal norms of every slot (the pools are [H][CAP][D] under the identity page table)
+  int r = launch_prep_generic(c, c.pool_k, c.CAP, static_cast<int64_t>(c.CAP) * c.D, c.D, c.kcode, c.rnorm, c.CAP, st);
+  if (r < 0) return r;
+  const dim3 grid(min((c.CAP + 7) / 8, 1024), c.H);
+  if (c.D == 128) import_fix_kernel<128><<<grid, 256, 0, st>>>(c);
+  else import_fix_kernel<64><<<grid, 256, 0, st>>>(c);
+  if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+  int r2 = launch_finalize_hist(c, nullptr, -1, st);
+  if (r2 < 0) return r2;
+  return r + 1 + r2;
+}
+
+int launch_copy_outputs(const CacheView& c, int n, int32_t* match_out, float* sim_out, int32_t* dest_out, cudaStream_t st) {
+  const size_t w = static_cast<size_t>(n) * 4, sp = static_cast<size_t>(c.max_tokens) * 4;
+  if (match_out && cudaMemcpy2DAsync(match_out, w, c.match, sp, w, c.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (sim_out && cudaMemcpy2DAsync(sim_out, w, c.sim, sp, w, c.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (dest_out && cudaMemcpy2DAsync(dest_out, w, c.dest, sp, w, c.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  return 0;
+}
+
+__global__ void decode_rel_kernel(const CacheView c, int n_frames, int np, float scale, float* __restrict__ rel_out) {
+  const int h = blockIdx.y;
+  for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < n_frames * np; q += gridDim.x * blockDim.x) {
+    const int f = q / np, p = q % np;
+    rel_out[(static_cast<int64_t>(h) * n_frames + f) * np + p] =
+        ordered_to_float(c.rel[(static_cast<int64_t>(h) * c.max_frames + f) * c.max_prompt + p]) * scale;
+  }
+}
+int launch_decode_rel(const CacheView& c, int n_frames, int np, float scale, float* rel_out, cudaStream_t st) {
+  decode_rel_kernel<<<dim3((n_frames * np + 255) / 256, c.H), 256, 0, st>>>(c, n_frames, np, scale, rel_out);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+}  // namespace fastar

@@ -1,0 +1,145 @@
+"""Staged (teacher-forced) comparison of results produced elsewhere (numpy arrays) with the CPU
+oracle.  This module imports only the oracle and numpy; it never touches the CUDA binding, so the
+two implementations stay independent.  Near-ties have several correct answers, hence the stages:
+
+  T1  accept j iff cos_oracle(i, j) >= best_i - 1e-4                  (bit-equal wherever the margin is larger)
+  T2  matched flags agree wherever |best_i - tau| > 1e-4
+  T3/T4  the decisions taken are fed to the oracle's merge -> dest, len, count, stamp, K rows bit-exact,
+         V rows within one bf16 ulp
+  S1  code bits agree wherever |proj| >= 1e-4 |x||r|
+  S2-S4  the codes produced are fed to the oracle -> scores and selected blocks bit-exact
+  C1/C2  relevance within tolerance; selection correct up to 1e-4 ties
+  S5/C3/D  the selection produced is fed to the oracle attention -> max-abs 2e-2, relative L2 1e-2
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+from oracle import fastar_oracle as O
+
+MARGIN = 1e-4
+ATT_MAX_ABS = 2e-2
+ATT_REL_L2 = 1e-2
+
+
+def bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(bits, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def oracle_heads_from_export(state: Dict[str, np.ndarray], n_sink: int = 0) -> List[O.HeadCache]:
+    """Oracle caches holding exactly the exported state (teacher forcing across steps)."""
+    H, CAP, D = state["k"].shape
+    heads = []
+    for h in range(H):
+        hc = O.HeadCache(CAP, D, n_sink)
+        L = int(state["len"][h])
+        hc.load(bits_to_f64(state["k"][h, :L]), bits_to_f64(state["v"][h, :L]), m=state["count"][h, :L].astype(np.int64),
+                stamp=state["stamp"][h, :L].astype(np.int64), now=int(state["now"][0]))
+        heads.append(hc)
+    return heads
+
+
+def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float, match: np.ndarray,
+                 sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
+                 rows: Optional[np.ndarray] = None) -> O.HeadCache:
+    """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
+    exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases)."""
+    n = K_new.shape[0]
+    K64, V64 = K_new.astype(np.float64), V_new.astype(np.float64)
+    matched = match >= 0
+    idx = np.arange(n) if rows is None else rows
+    if pre.L > 0:
+        cosm = O.cosine_matrix(K64[idx], pre.K[: pre.L])
+        cbest = cosm.max(axis=1)
+        # T1: the slot reported (for matched tokens) is within the margin of the best
+        mi = np.flatnonzero(matched[idx])
+        got = cosm[mi, match[idx][mi]]
+        assert np.all(got >= cbest[mi] - MARGIN), "T1: matched slot is not a (near-)best slot"
+        uniq = (cosm >= cbest[:, None] - MARGIN).sum(axis=1) == 1
+        ui = mi[uniq[mi]]
+        assert np.array_equal(match[idx][ui], np.argmax(cosm[ui], axis=1)), "T1: index differs outside the tie window"
+        # the similarity reported is the cosine of the best slot
+        assert np.max(np.abs(sim[idx] - cbest)) <= 2e-5, "T1: similarity value"
+        # T2
+        far = np.abs(cbest - tau) > MARGIN
+        assert np.array_equal(matched[idx][far], (cbest >= tau)[far]), "T2: threshold decision"
+    else:
+        assert not matched.any() and np.all(sim == 0)
+    # T3/T4: teacher-forced merge
+    ref = pre.copy()
+    res = O.tempcache_update(ref, K64, V64, frame_len, tau, forced=(np.where(matched, match, 0), sim.astype(np.float64), matched))
+    st = res["stats"]
+    assert np.array_equal(dest, res["dest"]), "T3/T4: destination slots"
+    assert int(post["len"][h]) == ref.L == st["length"], "T4: length"
+    L = ref.L
+    assert np.array_equal(post["count"][h, :L], ref.m[:L]), "T3: multiplicities"
+    assert np.array_equal(post["stamp"][h, :L], ref.stamp[:L]), "T3/T4: stamps"
+    assert np.array_equal(bits_to_f64(post["k"][h, :L]), ref.K[:L]), "T3/T4: keys are bit copies"
+    v_got = bits_to_f64(post["v"][h, :L])
+    ulp = np.maximum(np.abs(ref.V[:L]), 2.0 ** -126) * 2.0 ** -7
+    assert np.all(np.abs(v_got - ref.V[:L]) <= ulp + 1e-6), "T3: merged values beyond one bf16 ulp"
+    assert (int(stats[0]), int(stats[1]), int(stats[2]), int(stats[3]), int(stats[4]), int(stats[5]), int(stats[6])) == (
+        st["matched"], st["touched"], st["appended"], st["evicted_slots"], st["evicted_tokens"], st["length"], 1), "stats"
+    return ref
+
+
+def unpack_codes(packed: np.ndarray, tables: int) -> np.ndarray:
+    """uint32 with table t in byte t -> [n][T]."""
+    p = packed.astype(np.uint32)
+    return np.stack([(p >> (8 * t)) & 0xFF for t in range(tables)], axis=-1).astype(np.int64)
+
+
+def check_codes(X: np.ndarray, R: np.ndarray, tables: int, bits: int, packed: np.ndarray) -> np.ndarray:
+    """S1: every code bit whose projection is clear of zero must agree.  Returns the codes [n][T]."""
+    X64, R64 = X.astype(np.float64), R.astype(np.float64)
+    proj = O.lsh_projections(X64, R64)
+    want = (proj > 0).reshape(X.shape[0], tables, bits)
+    codes = unpack_codes(packed, tables)
+    got = ((codes[:, :, None] >> np.arange(bits)) & 1).astype(bool)
+    tol = MARGIN * np.linalg.norm(X64, axis=1)[:, None] * np.linalg.norm(R64, axis=1)[None, :]
+    clear = (np.abs(proj) >= tol).reshape(want.shape)
+    assert np.array_equal(got[clear], want[clear]), "S1: code bit differs although the projection is clear of 0"
+    assert np.all(codes < (1 << bits))
+    return codes
+
+
+def check_selection(qcodes: np.ndarray, kcodes: np.ndarray, nq: int, L: int, block_q: int, block_k: int, bits: int, keep: int,
+                    scores: Optional[np.ndarray], sel: np.ndarray, nsel: int) -> np.ndarray:
+    """S2-S4 from the codes produced elsewhere: integer domain, bit-exact."""
+    HQ = O.block_histograms(qcodes, nq, block_q, bits)
+    HK = O.block_histograms(kcodes, L, block_k, bits)
+    S = O.block_scores(HQ, HK) if L else np.zeros((HQ.shape[0], 0), np.int64)
+    nkb = S.shape[1]
+    if scores is not None:
+        assert np.array_equal(scores[:, :nkb].astype(np.int64), S), "S3: block scores"
+    want = O.topk_lowest_index(S, keep) if L else np.zeros((HQ.shape[0], 0), np.int64)
+    assert nsel == want.shape[1], "S4: number of kept blocks"
+    assert np.array_equal(sel[:, :nsel], want), "S4: selected blocks"
+    assert np.all(sel[:, nsel:] == -1)
+    return want
+
+
+def check_attention(got: np.ndarray, want: np.ndarray, what: str) -> None:
+    got = got.astype(np.float64)
+    err = np.max(np.abs(got - want))
+    rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
+    assert err <= ATT_MAX_ABS and rel <= ATT_REL_L2, f"{what}: max-abs {err:.3e} (<= {ATT_MAX_ABS}), rel-L2 {rel:.3e} (<= {ATT_REL_L2})"
+
+
+def check_prompt_selection(Q: np.ndarray, K_p: np.ndarray, frame_len: int, keep: int, sel: np.ndarray,
+                           rel: Optional[np.ndarray]) -> None:
+    """C1/C2: relevance values and the kept set, up to 1e-4 ties."""
+    r = O.prompt_relevance(Q.astype(np.float64), K_p.astype(np.float64), frame_len)
+    if rel is not None:
+        assert np.max(np.abs(rel - r) / np.maximum(1.0, np.abs(r))) <= 2e-5, "C1: relevance values"
+    k = min(keep, K_p.shape[0])
+    for f in range(r.shape[0]):
+        s = sel[f]
+        assert s.shape[0] == k and np.all(np.diff(s) > 0), "C2: list not ascending / wrong length"
+        kth = np.sort(r[f])[::-1][k - 1]
+        tol = MARGIN * max(1.0, abs(kth))
+        assert np.all(r[f][s] >= kth - tol), "C2: a kept token is below the k-th relevance"
+        must = np.flatnonzero(r[f] > kth + tol)
+        assert set(must.tolist()) <= set(s.tolist()), "C2: a clearly relevant token was dropped"

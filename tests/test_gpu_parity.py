@@ -1,0 +1,256 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs, element by element (staged as described in tests/parity.py)."""
+import numpy as np
+import pytest
+
+from oracle import fastar_oracle as O
+from paper_2602_01801_b200 import synth
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu():
+    import torch
+    from paper_2602_01801_b200 import fastar
+    return torch, fastar
+
+
+def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None):
+    torch, fastar = _gpu()
+    return fastar.Cache(cfg.num_heads, cfg.head_dim, capacity or cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables,
+                        cfg.lsh_bits, max_tokens=max_tokens or cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64),
+                        max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32)
+
+
+def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False):
+    """Runs one update on the GPU and checks it against the oracle heads `heads` (advanced in place)."""
+    torch, fastar = _gpu()
+    res = cache.update(fastar.to_device(K, fp32), fastar.to_device(V, fp32), frame_len, tau)
+    assert cache.status() == 0
+    post = cache.export_state()
+    match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    for h in range(K.shape[0]):
+        heads[h] = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h)
+    return post
+
+
+def gpu_annsa_checked(cache, cfg, w, Q, post, keep, fp32=False, block_q=None):
+    torch, fastar = _gpu()
+    block_q = block_q or cfg.block
+    heads = P.oracle_heads_from_export(post)
+    res = cache.annsa(fastar.to_device(Q, fp32), block_q, keep, debug=True)
+    assert cache.status() == 0
+    out = res["out"].float().cpu().numpy()
+    R = w.lsh_projection()
+    capb = cache.CAP // cache.PT
+    for h, hc in enumerate(heads):
+        nq = Q.shape[1]
+        if keep < capb:
+            qcodes = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, res["qcode"][h].cpu().numpy().view(np.uint32))
+            kcodes = P.check_codes(P.bits_to_f64(post["k"][h, : hc.L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][h, : hc.L])
+            sel = P.check_selection(qcodes, kcodes, nq, hc.L, block_q, cfg.block, cfg.lsh_bits, keep,
+                                    res["scores"][h].cpu().numpy(), res["sel"][h].cpu().numpy(), int(res["nsel"][h]))
+        else:
+            sel = np.tile(np.arange(-(-hc.L // cfg.block)), (-(-nq // block_q), 1))
+        want = O.sparse_attention(Q[h].astype(np.float64), hc, sel, block_q, cfg.block)
+        P.check_attention(out[h], want, f"AnnSA head {h}")
+    return res
+
+
+def gpu_annca_checked(cache, cfg, Q, Kp, Vp, keep, fp32=False):
+    torch, fastar = _gpu()
+    res = cache.annca(fastar.to_device(Q, fp32), fastar.to_device(Kp, fp32), fastar.to_device(Vp, fp32), cfg.frame_len, keep,
+                      debug=True)
+    assert cache.status() == 0
+    out = res["out"].float().cpu().numpy()
+    sel, rel = res["sel"].cpu().numpy(), res["rel"].cpu().numpy()
+    for h in range(Q.shape[0]):
+        P.check_prompt_selection(Q[h], Kp[h], cfg.frame_len, keep, sel[h], rel[h])
+        want = O.annca(Q[h], Kp[h], Vp[h], cfg.frame_len, keep, sel=sel[h])["out"]
+        P.check_attention(out[h], want, f"AnnCA head {h}")
+    return res
+
+
+def full_step(cfg, fp32=False, tau=None, n_sink=0):
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, fp32, n_sink)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim, n_sink) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks):                 # prior chunks enter un-merged (tau > 1): plain append
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0, fp32)
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau if tau is None else tau, fp32)
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks, fp32)
+    Kp, Vp, planted = w.prompt(cfg.prior_chunks)
+    res = gpu_annca_checked(cache, cfg, Q, Kp, Vp, cfg.keep_prompt, fp32)
+    return cache, w, heads, post, res, planted
+
+
+def test_c0_tiny_step_fp32_entry():
+    cfg = synth.CONFIGS["c0"]
+    cache, w, heads, post, res, planted = full_step(cfg, fp32=True)
+    assert int(post["len"][0]) == heads[0].L > 1024
+    assert set(planted[0].tolist()) <= set(res["sel"][0, 0].cpu().numpy().tolist())
+
+
+def test_small_multihead_ragged_step():
+    # 2 heads, d=128, 600-token chunks (4 full 128-row tiles + a ragged tail), ragged cache lengths
+    cfg = synth.small_config()
+    cache, w, heads, post, _, _ = full_step(cfg)
+    assert len(set(int(x) for x in post["len"])) >= 1
+    # a second merging chunk on top (counts > 1 enter the bias)
+    Q, K, V = w.chunk(cfg.prior_chunks + 1)
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
+    assert post["count"].max() > 1
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+
+
+@pytest.mark.parametrize("d,pt", [(64, 128), (128, 64), (64, 64)])
+def test_other_tile_shapes(d, pt):
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=2)
+    full_step(cfg)
+
+
+def test_dense_mode_equals_eq1_on_uncompressed_cache():
+    cfg = synth.small_config(prior_chunks=2)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    Ks, Vs = [], []
+    for ci in range(3):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0)
+        Ks.append(K)
+        Vs.append(V)
+    res = cache.annsa(_gpu()[1].to_device(Q), cfg.block, 10 ** 6)
+    out = res["out"].float().cpu().numpy()
+    Kall, Vall = np.concatenate(Ks, axis=1), np.concatenate(Vs, axis=1)
+    for h in range(cfg.num_heads):
+        P.check_attention(out[h], O.dense_attention(Q[h], Kall[h], Vall[h]), "dense Eq. 1")
+
+
+def test_lemma_on_gpu_duplicate_keys():
+    # exact duplicates merged at tau ~ 1: compressed attention with log m bias == dense attention over all copies
+    torch, fastar = _gpu()
+    cfg = synth.small_config(num_heads=1, prior_chunks=0, sigma=0.0, resample=0.0, shift=0.0, frames_per_chunk=1)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim)]
+    Ks, Vs = [], []
+    for ci in range(3):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, 0.9999)
+        Ks.append(K)
+        Vs.append(V)
+    assert int(post["len"][0]) == cfg.frame_len                # every token of the later chunks merged
+    assert int(post["count"][0].sum()) == 3 * cfg.frame_len
+    Qr = synth.round_bf16(np.random.default_rng(5).standard_normal(Q.shape).astype(np.float32) * 0.3)
+    out = cache.annsa(fastar.to_device(Qr), cfg.block, 10 ** 6)["out"].float().cpu().numpy()
+    want = O.dense_attention(Qr[0], np.concatenate(Ks, axis=1)[0], np.concatenate(Vs, axis=1)[0])
+    # values are stored as bf16 means: tolerance of the attention outputs applies
+    P.check_attention(out[0], want, "Lemma 1 on the GPU")
+
+
+def test_eviction_and_sink_and_capacity_error():
+    torch, fastar = _gpu()
+    cfg = synth.small_config(num_heads=2, capacity=1536, prior_chunks=0, resample=0.5, keep_blocks=3)
+    w = synth.Workload(cfg)
+    n_sink = 100
+    cache = make_cache(cfg, w, n_sink=n_sink)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim, n_sink) for _ in range(cfg.num_heads)]
+    evicted = 0
+    for ci in range(6):                                        # 600 tokens per chunk, half of them new -> fills 1536 quickly
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
+        evicted += sum(h.evicted_tokens for h in heads)
+    assert evicted > 0 and all(h.L == cfg.capacity for h in heads)
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+    # capacity error: a tiny cache that cannot take a chunk of unrelated tokens twice in a row
+    cfg2 = synth.small_config(num_heads=1, capacity=640, prior_chunks=0, resample=1.0)
+    w2 = synth.Workload(cfg2)
+    cache2 = make_cache(cfg2, w2, n_sink=600)
+    _, K, V = w2.chunk(0)
+    cache2.update(fastar.to_device(K), fastar.to_device(V), cfg2.frame_len, 0.9)
+    assert cache2.status() == 0
+    before = cache2.export_state()
+    _, K, V = w2.chunk(1)
+    res = cache2.update(fastar.to_device(K), fastar.to_device(V), cfg2.frame_len, 0.9)
+    assert cache2.status() == fastar.ERR_CAPACITY
+    after = cache2.export_state()
+    assert int(res["stats"][0, 6]) == 0
+    for key in ("k", "v", "count", "stamp", "len"):
+        assert np.array_equal(before[key], after[key]), key
+
+
+def test_empty_cache_and_selector_bypass():
+    torch, fastar = _gpu()
+    cfg = synth.small_config(prior_chunks=1)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    Q, K, V = w.chunk(0)
+    out = cache.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks)["out"]
+    assert cache.status() == 0 and float(out.float().abs().max()) == 0.0
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0)
+    nqb = -(-Q.shape[1] // cfg.block)
+    nkb = -(-int(post["len"][0]) // cfg.block)
+    rng = np.random.default_rng(3)
+    sel = np.stack([np.stack([np.sort(rng.choice(nkb, 3, replace=False)) for _ in range(nqb)]) for _ in range(cfg.num_heads)])
+    sel_t = torch.from_numpy(sel.astype(np.int32)).cuda()
+    nsel_t = torch.full((cfg.num_heads,), 3, dtype=torch.int32).cuda()
+    out = cache.annsa(fastar.to_device(Q), cfg.block, 3, sel_in=sel_t, nsel_in=nsel_t)["out"].float().cpu().numpy()
+    hs = P.oracle_heads_from_export(post)
+    for h in range(cfg.num_heads):
+        P.check_attention(out[h], O.sparse_attention(Q[h].astype(np.float64), hs[h], sel[h], cfg.block, cfg.block), "sel_in bypass")
+
+
+def test_annca_keep_all_is_dense_cross_attention():
+    torch, fastar = _gpu()
+    cfg = synth.small_config(prompt_tokens=200)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, max_tokens=cfg.chunk_tokens)
+    Q, _, _ = w.chunk(0)
+    Kp, Vp, _ = w.prompt(0)
+    out = cache.annca(fastar.to_device(Q), fastar.to_device(Kp), fastar.to_device(Vp), cfg.frame_len, 200)["out"].float().cpu().numpy()
+    for h in range(cfg.num_heads):
+        P.check_attention(out[h], O.dense_attention(Q[h], Kp[h], Vp[h]), "AnnCA keep-all")
+
+
+def test_host_step_matches_device_calls():
+    torch, fastar = _gpu()
+    cfg = synth.small_config()
+    w = synth.Workload(cfg)
+    ca, cb = make_cache(cfg, w), make_cache(cfg, w)
+    for ci in range(cfg.prior_chunks + 1):
+        Q, K, V = w.chunk(ci)
+        Kp, Vp, _ = w.prompt(ci)
+        dq, dk, dv, dkp, dvp = (fastar.to_device(x) for x in (Q, K, V, Kp, Vp))
+        ca.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)
+        o1 = ca.annsa(dq, cfg.block, cfg.keep_blocks)["out"]
+        o2 = ca.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt)["out"]
+        hq, hk, hv, hkp, hvp = (t.cpu().pin_memory() for t in (dq, dk, dv, dkp, dvp))
+        h1, h2 = torch.empty_like(hq).pin_memory(), torch.empty_like(hq).pin_memory()
+        cb.step_host(hk, hv, hq, hkp, hvp, h1, h2, cfg.frame_len, cfg.tau, cfg.block, cfg.keep_blocks, cfg.keep_prompt)
+        assert torch.equal(o1.cpu(), h1) and torch.equal(o2.cpu(), h2)
+    assert ca.status() == 0 and cb.status() == 0
+    assert ca.launch_count() > 0
+
+
+def test_argument_errors_are_rejected_on_the_host():
+    torch, fastar = _gpu()
+    cfg = synth.small_config()
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    Q, K, V = w.chunk(0)
+    dq = fastar.to_device(Q)
+    with pytest.raises(fastar.FastarError) as e:
+        cache.annsa(dq, 96, 4)
+    assert e.value.status == fastar.ERR_UNSUPPORTED_SHAPE
+    big = torch.zeros((cfg.num_heads, cfg.chunk_tokens + 1, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(fastar.FastarError) as e:
+        cache.update(big, big, cfg.frame_len, 0.9)
+    assert e.value.status == fastar.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fastar.FastarError) as e:
+        cache.update(dq, dq, 0, 0.9)
+    assert e.value.status == fastar.ERR_INVALID_ARG
