@@ -30,8 +30,13 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False):
     assert cache.status() == 0
     post = cache.export_state()
     match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    synced = P.oracle_heads_from_export(post, heads[0].n_sink)
     for h in range(K.shape[0]):
-        heads[h] = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h)
+        ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h)
+        # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
+        # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
+        synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
+        heads[h] = synced[h]
     return post
 
 
