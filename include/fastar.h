@@ -178,6 +178,30 @@ int fastar_last_device_status(fastar_cache_t* cache, void* stream);
 /* Number of kernels this library has launched through this cache since creation. */
 int64_t fastar_launch_count(const fastar_cache_t* cache);
 
+/* Measurement aid (no counterpart in the paper).  While enabled, every hot kernel launch is bracketed
+ * by a pair of CUDA events recorded on the launching stream.  fastar_profile_read synchronises the
+ * stream, adds the elapsed milliseconds and the number of launches per kernel kind into the two
+ * caller arrays of FASTAR_K_COUNT entries, and forgets the events.  Creating events costs host time,
+ * so leave it off when timing whole steps. */
+enum {
+  FASTAR_K_CONVERT = 0,        /* fp32 -> bf16 entry conversion */
+  FASTAR_K_HASH = 1,           /* S1: LSH codes (+ 1/|k|) of new keys or queries */
+  FASTAR_K_T1_SIMILARITY = 2,  /* T1: key similarity + top-1 (tcgen05) */
+  FASTAR_K_PLAN = 3,           /* T2-T4 planning (sort, groups, append / eviction plan) */
+  FASTAR_K_COMMIT = 4,         /* T3/T4 commit (merge rows, append rows) */
+  FASTAR_K_KEY_HIST = 5,       /* S2 key-side histograms + end of update */
+  FASTAR_K_QUERY_HIST = 6,     /* S2 query side */
+  FASTAR_K_S3_SCORES = 7,      /* S3 block scores (tcgen05) */
+  FASTAR_K_TOPK_BLOCKS = 8,    /* S4 */
+  FASTAR_K_S5_ATTENTION = 9,   /* S5 / dense: selected-block attention (tcgen05) */
+  FASTAR_K_C1_RELEVANCE = 10,  /* C1 (tcgen05) */
+  FASTAR_K_TOPK_PROMPT = 11,   /* C2 */
+  FASTAR_K_C3_ATTENTION = 12,  /* C3 (tcgen05) */
+  FASTAR_K_COUNT = 13
+};
+int fastar_profile_enable(fastar_cache_t* cache, int32_t on);
+int fastar_profile_read(fastar_cache_t* cache, float* ms_by_kind, int32_t* launches_by_kind, void* stream);
+
 const char* fastar_status_string(int status);
 
 #ifdef __cplusplus

@@ -11,7 +11,14 @@
 
 using namespace fastar;
 
+struct ProfRec {
+  int kind;
+  cudaEvent_t a, b;
+};
+
 struct fastar_cache {
+  bool prof = false;
+  std::vector<ProfRec> recs;
   fastar_cache_desc desc;
   CacheView v;
   CUtensorMap tm_pool_k, tm_pool_v, tm_hq, tm_hk;
@@ -131,6 +138,25 @@ __global__ void copy_rows3_kernel(const int32_t* __restrict__ src, int64_t src_h
     c->launches += r__;               \
   } while (0)
 
+// Same, with the launch bracketed by CUDA events on the launching stream while profiling is on.
+#define ACCK(kind, call)                                   \
+  do {                                                     \
+    cudaEvent_t a__ = nullptr, b__ = nullptr;              \
+    const bool p__ = c->prof;                              \
+    if (p__) {                                             \
+      cudaEventCreate(&a__);                               \
+      cudaEventCreate(&b__);                               \
+      cudaEventRecord(a__, st);                            \
+    }                                                      \
+    const int r__ = (call);                                \
+    if (p__) {                                             \
+      cudaEventRecord(b__, st);                            \
+      c->recs.push_back(ProfRec{kind, a__, b__});          \
+    }                                                      \
+    if (r__ < 0) return r__;                               \
+    c->launches += r__;                                    \
+  } while (0)
+
 // Returns a bf16 view of a caller tensor: the tensor itself (bf16) or its converted copy in stage[slot].
 int as_bf16(fastar_cache* c, const void* src, int rows, int64_t* hs, int64_t* ts, int slot, const __nv_bfloat16** out,
             cudaStream_t st) {
@@ -139,7 +165,7 @@ int as_bf16(fastar_cache* c, const void* src, int rows, int64_t* hs, int64_t* ts
     return FASTAR_OK;
   }
   if ((reinterpret_cast<uintptr_t>(src) & 15) || (*hs & 3) || (*ts & 3)) return FASTAR_ERR_INVALID_ARG;
-  ACC(launch_convert_f32_to_bf16(static_cast<const float*>(src), c->v.stage[slot], c->v.H, rows, c->v.D, *hs, *ts, st));
+  ACCK(FASTAR_K_CONVERT, launch_convert_f32_to_bf16(static_cast<const float*>(src), c->v.stage[slot], c->v.H, rows, c->v.D, *hs, *ts, st));
   *out = c->v.stage[slot];
   *hs = static_cast<int64_t>(rows) * c->v.D;
   *ts = c->v.D;
@@ -289,12 +315,12 @@ int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_
   CUtensorMap tm_a;
   r = make_map(c, &tm_a, kb, v.D, n, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
   if (r != FASTAR_OK) return r;
-  ACC(launch_prep_codes(v, kb, n, khs, kts, v.code_new, v.rnorm_new, st));
+  ACCK(FASTAR_K_HASH, launch_prep_codes(v, kb, n, khs, kts, v.code_new, v.rnorm_new, st));
   if (cudaMemsetAsync(v.best, 0, static_cast<size_t>(v.H) * v.max_tokens * 8, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-  ACC(launch_t1_similarity(v, tm_a, c->tm_pool_k, n, st));
-  ACC(launch_plan(v, n, frame_len, tau, st));
-  ACC(launch_commit(v, kb, vb, n, frame_len, khs, kts, st));
-  ACC(launch_finalize_hist(v, stats_out, 1, st));
+  ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, n, st));
+  ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
+  ACCK(FASTAR_K_COMMIT, launch_commit(v, kb, vb, n, frame_len, khs, kts, st));
+  ACCK(FASTAR_K_KEY_HIST, launch_finalize_hist(v, stats_out, 1, st));
   ACC(launch_copy_outputs(v, n, match_out, sim_out, dest_out, st));
   return FASTAR_OK;
 }
@@ -336,10 +362,10 @@ int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t 
     a.sel_head_stride = static_cast<int64_t>(nqb) * keep_blocks;
     a.keep = keep_blocks;
   } else if (!dense) {
-    ACC(launch_prep_codes(v, qb, nq, qhs, qts, v.code_new, nullptr, st));
-    ACC(launch_query_hist(v, nq, block_q, st));
-    ACC(launch_s3_scores(v, c->tm_hq, c->tm_hk, nqb, st));
-    ACC(launch_topk_blocks(v, nqb, keep, st));
+    ACCK(FASTAR_K_HASH, launch_prep_codes(v, qb, nq, qhs, qts, v.code_new, nullptr, st));
+    ACCK(FASTAR_K_QUERY_HIST, launch_query_hist(v, nq, block_q, st));
+    ACCK(FASTAR_K_S3_SCORES, launch_s3_scores(v, c->tm_hq, c->tm_hk, nqb, st));
+    ACCK(FASTAR_K_TOPK_BLOCKS, launch_topk_blocks(v, nqb, keep, st));
     a.sel = v.sel;
     a.nsel = v.nsel;
     a.sel_stride = v.CAPB;
@@ -360,7 +386,7 @@ int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t 
                                         cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return FASTAR_ERR_CUDA;
   }
-  ACC(launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, a, st));
+  ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, a, st));
   return FASTAR_OK;
 }
 
@@ -412,8 +438,8 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
     r = make_map(c, &tm_kp, kpb, v.D, np, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
     if (r != FASTAR_OK) return r;
     if (cudaMemsetAsync(v.rel, 0, static_cast<size_t>(v.H) * v.max_frames * v.max_prompt * 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-    ACC(launch_c1_relevance(v, tm_q, tm_kp, nq, np, frame_len, F, st));
-    ACC(launch_topk_prompt(v, F, np, keep, st));
+    ACCK(FASTAR_K_C1_RELEVANCE, launch_c1_relevance(v, tm_q, tm_kp, nq, np, frame_len, F, st));
+    ACCK(FASTAR_K_TOPK_PROMPT, launch_topk_prompt(v, F, np, keep, st));
     a.sel = v.selp;
     a.sel_stride = v.max_prompt;
     a.sel_head_stride = static_cast<int64_t>(v.max_frames) * v.max_prompt;
@@ -424,7 +450,7 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
     }
     if (rel_out) ACC(launch_decode_rel(v, F, np, 1.0f / sqrtf(static_cast<float>(v.D)), rel_out, st));
   }
-  ACC(launch_attention_gather(v, tm_q, a, st));
+  ACCK(FASTAR_K_C3_ATTENTION, launch_attention_gather(v, tm_q, a, st));
   return FASTAR_OK;
 }
 
@@ -474,6 +500,29 @@ int fastar_last_device_status(fastar_cache_t* c, void* stream) {
 }
 
 int64_t fastar_launch_count(const fastar_cache_t* c) { return c ? c->launches : 0; }
+
+int fastar_profile_enable(fastar_cache_t* c, int32_t on) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  c->prof = on != 0;
+  return FASTAR_OK;
+}
+
+int fastar_profile_read(fastar_cache_t* c, float* ms_by_kind, int32_t* launches_by_kind, void* stream) {
+  if (!c || !ms_by_kind || !launches_by_kind) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return FASTAR_ERR_CUDA;
+  for (int k = 0; k < FASTAR_K_COUNT; ++k) { ms_by_kind[k] = 0.f; launches_by_kind[k] = 0; }
+  bool ok = true;
+  for (const ProfRec& r : c->recs) {
+    float ms = 0.f;
+    ok &= cudaEventSynchronize(r.b) == cudaSuccess && cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess;
+    if (r.kind >= 0 && r.kind < FASTAR_K_COUNT) { ms_by_kind[r.kind] += ms; launches_by_kind[r.kind] += 1; }
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  c->recs.clear();
+  return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
 
 const char* fastar_status_string(int status) {
   switch (status) {

@@ -49,6 +49,8 @@ SIGNATURES = {
     "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _vp]),
     "fastar_last_device_status": (C.c_int, [_vp, _vp]),
     "fastar_launch_count": (C.c_int64, [_vp]),
+    "fastar_profile_enable": (C.c_int, [_vp, _i32]),
+    "fastar_profile_read": (C.c_int, [_vp, _vp, _vp, _vp]),
     "fastar_status_string": (C.c_char_p, [C.c_int]),
 }
 
@@ -133,6 +135,18 @@ class Cache:
 
     def launch_count(self) -> int:
         return self.lib.fastar_launch_count(self.handle)
+
+    KERNEL_KINDS = ("convert", "hash", "t1_similarity", "plan", "commit", "key_hist", "query_hist", "s3_scores",
+                    "topk_blocks", "s5_attention", "c1_relevance", "topk_prompt", "c3_attention")
+
+    def profile(self, on: bool) -> None:
+        _check(self.lib.fastar_profile_enable(self.handle, 1 if on else 0), "fastar_profile_enable")
+
+    def profile_read(self) -> Dict[str, Dict[str, float]]:
+        ms = (C.c_float * len(self.KERNEL_KINDS))()
+        cnt = (C.c_int32 * len(self.KERNEL_KINDS))()
+        _check(self.lib.fastar_profile_read(self.handle, ms, cnt, _stream()), "fastar_profile_read")
+        return {k: dict(ms=float(ms[i]), launches=int(cnt[i])) for i, k in enumerate(self.KERNEL_KINDS)}
 
     def export_state(self, kv: bool = True) -> Dict[str, np.ndarray]:
         H, CAP, D = self.H, self.CAP, self.D
