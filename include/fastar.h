@@ -178,6 +178,30 @@ int fastar_last_device_status(fastar_cache_t* cache, void* stream);
 /* Number of kernels this library has launched through this cache since creation. */
 int64_t fastar_launch_count(const fastar_cache_t* cache);
 
+/* AnnCA's selection stage for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a deployment variant of the relevance + top-k stage of fastar_annca_attention).  Such callers
+ * are, for example, code that runs while its stream is being captured into a CUDA graph, plug-ins
+ * inside a host program that owns the GPU memory pool, and latency-critical loops that may not take
+ * the device-wide synchronisation cudaMalloc implies.  No cache object and no workspace are needed: the
+ * relevance accumulators live in a fixed array inside the library's device image
+ * (FASTAR_NOALLOC_MAX_WORDS 32-bit words = 2 MiB plus a 1 KiB header, reserved on every GPU that loads
+ * the library until the process exits).  The call performs no cudaMalloc / cudaFree and uses no
+ * allocating library routine.
+ *   q [H][nq][d], k_prompt [H][np][d]: dev, bf16, strides as elsewhere.  sel_out: dev [H][F][keep_tokens]
+ *   int32, F = ceil(nq / frame_len): per head and frame the keep_tokens prompt tokens with the largest
+ *   max_i q_i.k_p (ties: lower p), ascending -- identical to fastar_annca_attention's sel_out.
+ * Limits: H <= 128, np <= 1024, F <= 64, H * F * np <= FASTAR_NOALLOC_MAX_WORDS, keep_tokens <= np;
+ * anything larger returns FASTAR_ERR_UNSUPPORTED_SHAPE.  The device used is the current one.
+ * The first call on each device looks up the array's device address and clears its header with a
+ * synchronous copy; make that first call before any stream capture starts.  All calls share the one
+ * array, which keeps the previous call's contents: each call clears the part it uses on `stream`, and
+ * calls that overlap on the GPU (other streams or threads) race -- serialise them. */
+#define FASTAR_NOALLOC_MAX_WORDS (512 * 1024)
+int fastar_annca_select_noalloc(const void* q, const void* k_prompt, int32_t num_heads, int32_t head_dim, int32_t nq,
+                                int32_t frame_len, int32_t np, int32_t keep_tokens, int64_t head_stride,
+                                int64_t token_stride, int64_t prompt_head_stride, int64_t prompt_token_stride,
+                                int32_t* sel_out, void* stream);
+
 /* Measurement aid (no counterpart in the paper).  While enabled, every hot kernel launch is bracketed
  * by a pair of CUDA events recorded on the launching stream.  fastar_profile_read synchronises the
  * stream, adds the elapsed milliseconds and the number of launches per kernel kind into the two

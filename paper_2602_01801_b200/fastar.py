@@ -49,6 +49,7 @@ SIGNATURES = {
     "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _vp]),
     "fastar_last_device_status": (C.c_int, [_vp, _vp]),
     "fastar_launch_count": (C.c_int64, [_vp]),
+    "fastar_annca_select_noalloc": (C.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp]),
     "fastar_profile_enable": (C.c_int, [_vp, _i32]),
     "fastar_profile_read": (C.c_int, [_vp, _vp, _vp, _vp]),
     "fastar_status_string": (C.c_char_p, [C.c_int]),
@@ -252,6 +253,27 @@ class Cache:
                                                    k_prompt.data_ptr(), v_prompt.data_ptr(), out_sa.data_ptr(),
                                                    out_ca.data_ptr(), n, frame_len, np_, float(tau), block_q, keep_blocks,
                                                    keep_tokens, _stream()), "fastar_attention_step_host")
+
+
+def annca_select_noalloc(q, k_prompt, frame_len: int, keep_tokens: int, sel_out=None):
+    """Prompt-token selection without any device allocation inside the library (for callers that must not
+    allocate: stream capture, host-owned memory pools).  q [H][nq][d], k_prompt [H][np][d]: bf16 CUDA tensors.
+    Fills and returns sel_out [H][F][keep_tokens] int32 (pass a pre-allocated tensor to stay allocation-free
+    on the torch side too).  Calls share one fixed scratch array inside the library: do not overlap them."""
+    import torch
+    lib = load_library()
+    H, nq, D = q.shape
+    np_ = k_prompt.shape[1]
+    F = -(-nq // frame_len)
+    if sel_out is None:
+        sel_out = torch.empty((H, F, keep_tokens), dtype=torch.int32, device=q.device)
+    assert q.dtype == torch.bfloat16 and k_prompt.dtype == torch.bfloat16 and q.stride(2) == 1 and k_prompt.stride(2) == 1
+    assert sel_out.is_contiguous() and sel_out.dtype == torch.int32 and tuple(sel_out.shape) == (H, F, keep_tokens)
+    with torch.cuda.device(q.device):
+        _check(lib.fastar_annca_select_noalloc(q.data_ptr(), k_prompt.data_ptr(), H, D, nq, frame_len, np_, keep_tokens,
+                                               q.stride(0), q.stride(1), k_prompt.stride(0), k_prompt.stride(1),
+                                               sel_out.data_ptr(), _stream()), "fastar_annca_select_noalloc")
+    return sel_out
 
 
 # ---- helpers for moving synthetic numpy data (bf16-exact float32) onto the device ---------------
