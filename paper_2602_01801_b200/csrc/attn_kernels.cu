@@ -8,17 +8,19 @@
 //
 // One CTA = 128 query rows (TMEM lanes).  Per key tile j:
 //   S_j = Q K_j^T        (tcgen05.mma, SMEM x SMEM -> TMEM, two S buffers)
-//   P_j = exp2(S_j*scale + log2 m - m_run)   (4 softmax warps, one thread per row, two passes
-//                                             over TMEM: row max, then exponentials -> bf16 P in SMEM)
+//   P_j = exp2(S_j*scale + log2 m - m_run)   (8 softmax warps: two threads per row, each owning half of
+//                                             the tile's columns in registers; bf16 P tile in SMEM)
 //   O  += P_j V_j        (tcgen05.mma, V is the MN-major operand straight from its [key][d] page)
 // with lazy rescaling of O (only when a row maximum grew by more than 2^8).
-// Warp roles: warps 0-3 softmax + epilogue, warp 4 producer (TMA or gather), warp 5 MMA issue.
+// Warp roles: warps 0-7 softmax + epilogue, warp 8 producer (TMA or gather), warp 9 MMA issue.
 #include "common.h"
 #include "ptx.cuh"
 
 namespace fastar {
 
 constexpr int kQChunk = 128 * 128;   // bytes of one 128-row x 64-column bf16 chunk
+constexpr int kAttnThreads = 320;
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
 
 template <int D, int BKT>
 struct AttnSmem {
@@ -36,12 +38,23 @@ struct AttnSmem {
   static constexpr int tmem_cols = (2 * BKT + D) <= 256 ? 256 : 512;
 };
 
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+
 template <int D, int BKT, bool GATHER>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const CacheView c, const AttnArgs a) {
   using SM = AttnSmem<D, BKT>;
   constexpr int KS = SM::KS, VS = SM::VS, NB = SM::NB;
+  constexpr int HB = BKT / 2;           // key columns per softmax thread
+  constexpr int HD = D / 2;             // output columns per softmax thread
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t sbase = smem_u32(smem_raw);
   uint8_t* sgen = smem_raw;
@@ -66,7 +79,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const uint32_t bar_s_empty = bar_s_full + 16;       // [2]
   const uint32_t bar_p_full = bar_s_empty + 16;       // [2]
   const uint32_t bar_pv_done = bar_p_full + 16;       // [1]
-  constexpr int kBarBytes = 8 + 16 * KS + 16 * VS + 8 * NB + 48 + 8;
+  const uint32_t bar_xchg = bar_pv_done + 8;          // [1] row-max / row-sum exchange between the column halves
+  constexpr int kBarBytes = 8 + 16 * KS + 16 * VS + 8 * NB + 48 + 8 + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + SM::bar_off + kBarBytes);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + SM::bar_off + kBarBytes + 4);
 
@@ -104,19 +118,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     for (int s = 0; s < NB; ++s) mbar_init(bar_b_full + 8 * s, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_s_full + 8 * s, 1);
-      mbar_init(bar_s_empty + 8 * s, 128);
-      mbar_init(bar_p_full + 8 * s, 128);
+      mbar_init(bar_s_empty + 8 * s, 8);       // one arrival per softmax warp
+      mbar_init(bar_p_full + 8 * s, 8);
     }
     mbar_init(bar_pv_done, 1);
+    mbar_init(bar_xchg, 8);
     *abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 4 && lane == 0) {
+  if (warp == kProducerWarp && lane == 0) {
     tma_prefetch_desc(&tm_q);
     if (!GATHER) { tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); }
   }
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(tmem_slot), SM::tmem_cols);
     tmem_relinquish();
   }
@@ -126,7 +141,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_o = tmem + 2 * BKT;
 
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     // ================================================================== producer
     if (lane == 0 && nt > 0) {
       mbar_arrive_expect_tx(bar_q_full, SM::q_bytes);
@@ -203,16 +218,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ================================================================== MMA issue
     if (lane == 0 && nt > 0) {
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, BKT, 0);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
       bool ok = mbar_wait(bar_q_full, 0, abort_flag, c.status);
+      PT_DECL
       auto issue_s = [&](int j) -> bool {
         const int ks = j % KS, sb = j & 1;
         if (!mbar_wait(bar_k_full + 8 * ks, (j / KS) & 1, abort_flag, c.status)) return false;
+        PT_MARK(0)
         if (!mbar_wait(bar_s_empty + 8 * sb, ((j >> 1) & 1) ^ 1, abort_flag, c.status)) return false;
+        PT_MARK(1)
         tc_fence_after();
         const uint32_t kt = k_s + ks * SM::kv_bytes;
 #pragma unroll
@@ -223,6 +241,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         umma_commit(bar_k_empty + 8 * ks);
         umma_commit(bar_s_full + 8 * sb);
+        PT_MARK(2)
         return true;
       };
       if (ok) ok = issue_s(0);
@@ -231,8 +250,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const int vs = j % VS, pb = j & 1;
         ok = mbar_wait(bar_p_full + 8 * pb, (j >> 1) & 1, abort_flag, c.status);
         if (!ok) break;
+        PT_MARK(3)
         ok = mbar_wait(bar_v_full + 8 * vs, (j / VS) & 1, abort_flag, c.status);
         if (!ok) break;
+        PT_MARK(4)
         tc_fence_after();
         const uint32_t vt = v_s + vs * SM::kv_bytes;
         const uint32_t pt = p_s + pb * SM::p_bytes;
@@ -244,103 +265,144 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         umma_commit(bar_v_empty + 8 * vs);
         umma_commit(bar_pv_done);
+        PT_MARK(5)
       }
+      PT_FLUSH("attn mma", nt)
     }
   } else {
-    // ================================================================== softmax + epilogue
-    const int r = threadIdx.x;
-    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    // ================================================================== softmax + epilogue (256 threads)
+    const int wg = warp >> 2;                          // column half owned by this thread
+    const int r = (warp & 3) * 32 + lane;              // query row = TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const float scale = rsqrtf(static_cast<float>(D)) * 1.4426950408889634f;
-    float m_used = -INFINITY, l_sum = 0.f;
+    // First 16-byte chunk of each half of row r inside a P tile.  The two halves of a row exchange their
+    // partial row maximum through the *partner's* chunk: only the partner reads it, and only the partner
+    // overwrites it later with its own P data, so no extra buffer and no extra barrier are needed.
+    auto p_chunk_addr = [&](int pb, int ch) -> uint32_t {
+      return p_s + pb * SM::p_bytes + (ch >> 3) * kQChunk + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+    };
+    const int my_ch0 = wg * (HB / 8), other_ch0 = (wg ^ 1) * (HB / 8);
+    float m_used = -INFINITY;
+    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+    uint32_t xphase = 0;
     bool ok = true;
+    PT_DECL
     for (int j = 0; j < nt && ok; ++j) {
       const int sb = j & 1, pb = j & 1, b4 = j % NB;
       ok = mbar_wait(bar_b_full + 8 * b4, (j / NB) & 1, abort_flag, c.status) &&
            mbar_wait(bar_s_full + 8 * sb, (j >> 1) & 1, abort_flag, c.status);
       ok = __all_sync(0xffffffffu, ok);          // TMEM loads below are warp-collective
       if (!ok) break;
+      PT_MARK(0)
       tc_fence_after();
-      const float* bias = bias_g + b4 * BKT;
-      const uint32_t s_t = tmem + lane_addr + sb * BKT;
-      // pass 1: row maximum
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int cc = 0; cc < BKT / 32; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(s_t + cc * 32, v);
-        tmem_wait_ld();
+      // this thread's half of the logits row, kept in registers
+      float x[HB];
+      {
+        uint32_t v[HB];
 #pragma unroll
-        for (int t = 0; t < 32; ++t) mx = fmaxf(mx, fmaf(__uint_as_float(v[t]), scale, bias[cc * 32 + t]));
+        for (int cc = 0; cc < HB / 32; ++cc)
+          tmem_ld32(tmem + lane_addr + sb * BKT + wg * HB + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[cc * 32]));
+        tmem_wait_ld();
+        const float4* b4p = reinterpret_cast<const float4*>(bias_g + b4 * BKT + wg * HB);
+#pragma unroll
+        for (int t = 0; t < HB / 4; ++t) {
+          const float4 bb = b4p[t];
+          x[4 * t] = fmaf(__uint_as_float(v[4 * t]), scale, bb.x);
+          x[4 * t + 1] = fmaf(__uint_as_float(v[4 * t + 1]), scale, bb.y);
+          x[4 * t + 2] = fmaf(__uint_as_float(v[4 * t + 2]), scale, bb.z);
+          x[4 * t + 3] = fmaf(__uint_as_float(v[4 * t + 3]), scale, bb.w);
+        }
       }
+      PT_MARK(1)
+      tc_fence_before();
+      mbar_arrive_warp(bar_s_empty + 8 * sb);          // S and the bias are consumed
+      // row maximum: 4 independent chains, then across the two halves
+      float mx0 = x[0], mx1 = x[1], mx2 = x[2], mx3 = x[3];
+#pragma unroll
+      for (int t = 4; t < HB; t += 4) {
+        mx0 = fmaxf(mx0, x[t]);
+        mx1 = fmaxf(mx1, x[t + 1]);
+        mx2 = fmaxf(mx2, x[t + 2]);
+        mx3 = fmaxf(mx3, x[t + 3]);
+      }
+      float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      st_shared_f32(p_chunk_addr(pb, other_ch0), mx);
+      PT_MARK(2)
+      mbar_arrive_warp(bar_xchg);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_xchg, xphase, abort_flag, c.status));
+      xphase ^= 1;
+      if (!ok) break;
+      PT_MARK(3)
+      mx = fmaxf(mx, ld_shared_f32(p_chunk_addr(pb, my_ch0)));
       float alpha = 1.f;
       bool resc = false;
       if (mx > m_used + 8.f || (m_used == -INFINITY && mx > -INFINITY)) {
         alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
-        l_sum *= alpha;
+        l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
         m_used = mx;
         resc = j > 0;
       }
       const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
-      // pass 2: exponentials -> bf16 P tile (K-major, 128-byte swizzle), row sum
-      const uint32_t p_row = p_s + pb * SM::p_bytes + r * 128;
-#pragma unroll 1
-      for (int cc = 0; cc < BKT / 32; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(s_t + cc * 32, v);
-        tmem_wait_ld();
-        uint32_t pk[16];
+      // exponentials -> bf16 P (K-major, 128-byte swizzle); 4 independent row-sum chains
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * t]), scale, bias[cc * 32 + 2 * t]) - m_eff);
-          const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * t + 1]), scale, bias[cc * 32 + 2 * t + 1]) - m_eff);
-          l_sum += p0 + p1;
-          pk[t] = pack_bf16x2(p0, p1);
-        }
+      for (int q = 0; q < HB / 8; ++q) {
+        float p[8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int ch = cc * 4 + q;                   // 16-byte chunk index along the key axis
-          const uint32_t addr = p_row + (ch >> 3) * kQChunk + (((ch & 7) ^ (r & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * q]), "r"(pk[4 * q + 1]),
-                       "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3])
-                       : "memory");
-        }
+        for (int t = 0; t < 8; ++t) p[t] = fast_exp2(x[8 * q + t] - m_eff);
+        l0 += p[0] + p[4];
+        l1 += p[1] + p[5];
+        l2 += p[2] + p[6];
+        l3 += p[3] + p[7];
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_chunk_addr(pb, my_ch0 + q)),
+                     "r"(pack_bf16x2(p[0], p[1])), "r"(pack_bf16x2(p[2], p[3])), "r"(pack_bf16x2(p[4], p[5])),
+                     "r"(pack_bf16x2(p[6], p[7]))
+                     : "memory");
       }
-      tc_fence_before();
-      mbar_arrive(bar_s_empty + 8 * sb);
+      PT_MARK(4)
       if (j > 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done, (j - 1) & 1, abort_flag, c.status));
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, resc)) {
+        if (__any_sync(0xffffffffu, resc)) {        // both halves of a row take the same decision
 #pragma unroll 1
-          for (int cc = 0; cc < D / 32; ++cc) {
+          for (int cc = 0; cc < HD / 32; ++cc) {
             uint32_t v[32];
-            tmem_ld32(tmem_o + lane_addr + cc * 32, v);
+            tmem_ld32(tmem_o + lane_addr + wg * HD + cc * 32, v);
             tmem_wait_ld();
 #pragma unroll
             for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) * alpha);
-            tmem_st32(tmem_o + lane_addr + cc * 32, v);
+            tmem_st32(tmem_o + lane_addr + wg * HD + cc * 32, v);
           }
           tmem_wait_st();
         }
       }
+      PT_MARK(5)
       fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(bar_p_full + 8 * pb);
+      mbar_arrive_warp(bar_p_full + 8 * pb);
+      PT_MARK(6)
     }
-    // epilogue: O / l -> out
+    if (threadIdx.x == 0) { PT_FLUSH("attn softmax", nt) }
+    // epilogue: O / l -> out.  The row sum is the sum of both halves' partial sums.
     if (ok && nt > 0) ok = mbar_wait(bar_pv_done, (nt - 1) & 1, abort_flag, c.status);
     ok = __all_sync(0xffffffffu, ok);
+    float l_sum = (l0 + l1) + (l2 + l3);
+    if (ok && nt > 0) {
+      st_shared_f32(p_chunk_addr(0, other_ch0), l_sum);
+      mbar_arrive_warp(bar_xchg);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_xchg, xphase, abort_flag, c.status));
+      if (ok) l_sum += ld_shared_f32(p_chunk_addr(0, my_ch0));
+    }
     tc_fence_after();
     const bool wr = r < valid_rows;               // loads are warp-collective, only the stores are per row
     if (ok) {
       const float inv = (nt > 0 && l_sum > 0.f) ? 1.f / l_sum : 0.f;
-      const int64_t off = static_cast<int64_t>(h) * a.out_head_stride + static_cast<int64_t>(q0 + r) * a.out_token_stride;
+      const int64_t off = static_cast<int64_t>(h) * a.out_head_stride + static_cast<int64_t>(q0 + r) * a.out_token_stride + wg * HD;
 #pragma unroll 1
-      for (int cc = 0; cc < D / 32; ++cc) {
+      for (int cc = 0; cc < HD / 32; ++cc) {
         uint32_t v[32];
         if (nt > 0) {
-          tmem_ld32(tmem_o + lane_addr + cc * 32, v);
+          tmem_ld32(tmem_o + lane_addr + wg * HD + cc * 32, v);
           tmem_wait_ld();
         } else {
 #pragma unroll
@@ -368,7 +430,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, SM::tmem_cols);
   }
@@ -385,7 +447,7 @@ static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
       return FASTAR_ERR_CUDA;
     configured = true;
   }
-  kern<<<grid, 192, SM::total, st>>>(tq, tk, tv, c, a);
+  kern<<<grid, kAttnThreads, SM::total, st>>>(tq, tk, tv, c, a);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 

@@ -6,8 +6,8 @@
 //
 // One CTA = one 128-row tile of A and a range of 128-row tiles of B; D[128 x 128] fp32 lives in
 // TMEM, double buffered so the epilogue of tile t overlaps the MMAs of tile t+1.
-// Warp roles: warps 0-3 epilogue (thread r <-> TMEM lane r <-> A row r), warp 4 TMA producer,
-// warp 5 TMEM allocation + MMA issue.  Operands are bf16, K-major, 128-byte swizzled.
+// Warp roles: warps 0-7 epilogue (two threads per A row / TMEM lane, one per 64-column half), warp 8 TMA
+// producer, warp 9 TMEM allocation + MMA issue.  Operands are bf16, K-major, 128-byte swizzled.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -25,6 +25,8 @@ struct GemmArgs {
 
 constexpr int kChunkBytes = 128 * 128;       // 128 rows x 64 bf16
 constexpr int kTmemCols = 256;
+constexpr int kGemmThreads = 320;            // warps 0-7 epilogue, 8 TMA producer, 9 MMA issue
+constexpr int kGemmProducerWarp = 8, kGemmMmaWarp = 9;
 
 template <int EPI, bool A_RES, int NST>
 struct GemmSmem {
@@ -37,7 +39,7 @@ struct GemmSmem {
 };
 
 template <int EPI, bool A_RES, int NST>
-__global__ void __launch_bounds__(192, A_RES ? 2 : 1)
+__global__ void __launch_bounds__(kGemmThreads, A_RES ? 2 : 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c,
             const GemmArgs g) {
   using SM = GemmSmem<EPI, A_RES, NST>;
@@ -83,18 +85,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_tfull + 8 * b, 1);
-      mbar_init(bar_tempty + 8 * b, 128);
+      mbar_init(bar_tempty + 8 * b, 8);          // one arrival per epilogue warp
     }
     mbar_init(bar_afull, 1);
     *abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 4 && lane == 0) {
+  if (warp == kGemmProducerWarp && lane == 0) {
     tma_prefetch_desc(&tm_a);
     tma_prefetch_desc(&tm_b);
   }
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kGemmMmaWarp) {
     tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish();
   }
@@ -104,7 +106,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   const uint32_t tmem = *tmem_slot;
 
   if (ntl > 0) {
-    if (warp == 4) {
+    if (warp == kGemmProducerWarp) {
       // ------------------------------------------------------------------ TMA producer
       if (lane == 0) {
         bool ok = true;
@@ -147,23 +149,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           mbar_wait(bar_full + 8 * (k % NST), (k / NST) & 1, abort_flag, c.status);
         }
       }
-    } else if (warp == 5) {
+    } else if (warp == kGemmMmaWarp) {
       // ------------------------------------------------------------------ MMA issue
       if (lane == 0) {
         constexpr uint32_t idesc = make_idesc_bf16(128, 128, 0);
         bool ok = true;
         if (A_RES) ok = mbar_wait(bar_afull, 0, abort_flag, c.status);
         int it = 0;
+        PT_DECL
         for (int tl = 0; tl < ntl && ok; ++tl) {
           const int buf = tl & 1;
           ok = mbar_wait(bar_tempty + 8 * buf, ((tl >> 1) & 1) ^ 1, abort_flag, c.status);
           if (!ok) break;
+          PT_MARK(0)
           tc_fence_after();
           const uint32_t d_t = tmem + buf * 128;
           for (int kc = 0; kc < nkc; ++kc, ++it) {
             const int s = it % NST;
             ok = mbar_wait(bar_full + 8 * s, (it / NST) & 1, abort_flag, c.status);
             if (!ok) break;
+            PT_MARK(1)
             tc_fence_after();
             const uint32_t st_s = ring_s + s * SM::stage_bytes;
             const uint32_t a_c = A_RES ? a_s + kc * kChunkBytes : st_s;
@@ -175,51 +180,76 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
               umma_ss(d_t, ad, bd, idesc, (kc | k4) != 0);
             }
             umma_commit(bar_empty + 8 * s);
+            PT_MARK(2)
           }
           if (ok) umma_commit(bar_tfull + 8 * buf);
         }
+        PT_FLUSH("gemm mma (wait tmem, wait smem, issue)", ntl)
       }
     } else {
-      // ------------------------------------------------------------------ epilogue (128 threads)
-      const int r = threadIdx.x;                    // A row inside the tile = TMEM lane
+      // ------------------------------------------------------------------ epilogue (256 threads)
+      // Two threads per A row: warps 0-3 take columns 0-63 of every tile, warps 4-7 columns 64-127.  A TMEM
+      // load costs a few hundred cycles, so both 32-column loads of a thread are issued before the one wait.
+      const int wg = warp >> 2;
+      const int r = (warp & 3) * 32 + lane;         // A row inside the tile = TMEM lane
       const int row = m0 + r;
-      const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+      const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
       float best = -INFINITY;
       int best_j = -1;
       bool ok = true;
+      PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
         const int buf = tl & 1;
         int valid_cols = 128;
         if (EPI == EPI_ARGMAX) {
-          const int slot = t * 128 + r;
-          rn_s[buf * 128 + r] = slot < L ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+          if (wg == 0) {
+            const int slot = t * 128 + r;
+            rn_s[buf * 128 + r] = slot < L ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+          }
           valid_cols = min(128, L - t * 128);
-          named_barrier_sync(1, 128);
+          named_barrier_sync(1, 256);
         }
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
+        PT_MARK(0)
         tc_fence_after();
-#pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
-          uint32_t v[32];
-          tmem_ld32(tmem + lane_addr + buf * 128 + cc * 32, v);
-          tmem_wait_ld();
+        uint32_t vv[2][32];
+        tmem_ld32(tmem + lane_addr + buf * 128 + wg * 64, vv[0]);
+        tmem_ld32(tmem + lane_addr + buf * 128 + wg * 64 + 32, vv[1]);
+        tmem_wait_ld();
+        PT_MARK(1)
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+          const int cc = wg * 2 + c2;
+          const uint32_t(&v)[32] = vv[c2];
           if (EPI == EPI_ARGMAX) {
             const float* rn = rn_s + buf * 128 + cc * 32;
             const int jbase = t * 128 + cc * 32;
-            if (cc * 32 + 32 <= valid_cols) {
+            // Scores of the chunk, then a tree maximum (no serial compare/select chain); the index is
+            // searched only when the chunk holds a new strict maximum, which is rare after the first tiles.
+            float x[32];
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float x = __uint_as_float(v[j]) * rn[j];
-                if (x > best) { best = x; best_j = jbase + j; }
-              }
-            } else {
+            for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(v[j]) * rn[j];
+            if (cc * 32 + 32 > valid_cols) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float x = __uint_as_float(v[j]) * rn[j];
-                if (cc * 32 + j < valid_cols && x > best) { best = x; best_j = jbase + j; }
-              }
+              for (int j = 0; j < 32; ++j)
+                if (cc * 32 + j >= valid_cols) x[j] = -INFINITY;
+            }
+            float m16[16], m8[8], m4[4];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) m16[j] = fmaxf(x[2 * j], x[2 * j + 1]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) m8[j] = fmaxf(m16[2 * j], m16[2 * j + 1]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) m4[j] = fmaxf(m8[2 * j], m8[2 * j + 1]);
+            const float cm = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            if (cm > best) {
+              best = cm;
+              int idx = 31;
+#pragma unroll
+              for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;   // first (lowest) column of the maximum
+              best_j = jbase + idx;
             }
           } else if (EPI == EPI_COLMAX) {
             const bool rvalid = row < g.rows_a;
@@ -259,9 +289,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             }
           }
         }
+        PT_MARK(2)
         tc_fence_before();
-        mbar_arrive(bar_tempty + 8 * buf);
+        mbar_arrive_warp(bar_tempty + 8 * buf);
+        PT_MARK(3)
       }
+      if (threadIdx.x == 0) { PT_FLUSH("gemm epilogue (wait acc, tmem loads, compute, arrive)", ntl) }
       if (EPI == EPI_ARGMAX && ok && row < g.rows_a && best_j >= 0) {
         const float sim = best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
@@ -273,7 +306,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kGemmMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
@@ -290,7 +323,7 @@ static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const C
       return FASTAR_ERR_CUDA;
     configured = true;
   }
-  kern<<<grid, 192, SM::total, st>>>(tm_a, tm_b, c, g);
+  kern<<<grid, kGemmThreads, SM::total, st>>>(tm_a, tm_b, c, g);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
@@ -300,9 +333,23 @@ int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUte
   g.nkc = c.D / 64;
   const int row_tiles = (n + 127) / 128;
   // enough CTAs to fill the machine a few times over; every split scans a contiguous slot range
-  int splits = 1;
+  // Split the cache range so that the CTA count fills whole waves of the resident slots (2 CTAs per SM):
+  // the smallest split whose last wave is at least 90 % full, else the best one found.
+  int sm_count = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  }
+  const int slots = 2 * sm_count;
   const int max_tiles = c.CAP / 128;
-  while (row_tiles * c.H * splits < 2 * 148 && splits * 2 <= max_tiles && splits < 16) splits *= 2;
+  int splits = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= 16 && s <= max_tiles; ++s) {
+    const int total = row_tiles * c.H * s;
+    const double eff = static_cast<double>(total) / (static_cast<double>((total + slots - 1) / slots) * slots);
+    if (eff > best_eff + 1e-9) { best_eff = eff; splits = s; }
+    if (eff >= 0.9) break;
+  }
   return launch_gemm<EPI_ARGMAX, true, 4>(tm_a, tm_pool_k, c, g, dim3(row_tiles, c.H, splits), st);
 }
 

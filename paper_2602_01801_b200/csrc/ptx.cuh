@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 namespace fastar {
 
@@ -41,6 +42,13 @@ __device__ __forceinline__ void fence_mbar_init() {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// One arrival for a whole (converged) warp: the lanes' earlier accesses are ordered by the warp barrier,
+// lane 0 arrives.  Barriers fed this way are initialised with the number of warps, which avoids 32
+// serialised shared-memory atomics per warp.
+__device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -197,6 +205,24 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+
+// ---------------------------------------------------------------------------------------------
+// Optional per-phase cycle counters (compiled in only with -DFASTAR_PHASE_TIMING): CTA (0,0,0) prints the
+// cycles each role spent between marks, per loop iteration.  For finding where a tile's time goes.
+// ---------------------------------------------------------------------------------------------
+#ifdef FASTAR_PHASE_TIMING
+#define PT_DECL long long pt_t = clock64(); long long pt_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define PT_MARK(i) { const long long n__ = clock64(); pt_acc[i] += n__ - pt_t; pt_t = n__; }
+#define PT_FLUSH(name, iters)                                                                                        \
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iters) > 0)                                          \
+    printf("%s: per-iteration cycles %lld %lld %lld %lld %lld %lld %lld %lld (iterations %d)\n", name,               \
+           pt_acc[0] / (iters), pt_acc[1] / (iters), pt_acc[2] / (iters), pt_acc[3] / (iters), pt_acc[4] / (iters),  \
+           pt_acc[5] / (iters), pt_acc[6] / (iters), pt_acc[7] / (iters), static_cast<int>(iters));
+#else
+#define PT_DECL
+#define PT_MARK(i)
+#define PT_FLUSH(name, iters)
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // small numeric helpers

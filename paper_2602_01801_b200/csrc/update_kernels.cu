@@ -48,7 +48,7 @@ __device__ __forceinline__ void bitonic_sort_smem(unsigned long long* keys, int 
   for (int k = 2; k <= np2; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
       for (int t = threadIdx.x; t < (np2 >> 1); t += blockDim.x) {
-        const int i = ((t / j) * 2 * j) + (t % j);
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // j is a power of two
         const int p = i + j;
         const bool up = (i & k) == 0;
         const unsigned long long a = keys[i], b = keys[p];
@@ -95,41 +95,71 @@ __global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restri
                                                    const __nv_bfloat16* __restrict__ lsh, int T, int B,
                                                    uint32_t* __restrict__ code_out, float* __restrict__ rnorm_out,
                                                    int64_t out_stride) {
-  __shared__ float rt[D][33];           // rt[k][c] = R[c][k]
-  __shared__ float xs[8][D];
+  // rt4[k/4][c] = R[c][k..k+3]: one conflict-free 128-bit read gives lane c four consecutive k.  A warp
+  // projects 4 rows per pass so that every R value read from shared memory is used four times.
+  __shared__ float4 rt4[D / 4][32];
+  __shared__ float4 xs4[8][4][D / 4];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int h = blockIdx.y;
   const int ncol = T * B;
-  for (int q = threadIdx.x; q < D * 32; q += blockDim.x) {
-    const int cidx = q / D, k = q % D;
-    rt[k][cidx] = cidx < ncol ? __bfloat162float(lsh[cidx * D + k]) : 0.f;
+  for (int q = threadIdx.x; q < (D / 4) * 32; q += blockDim.x) {
+    const int k4 = q >> 5, cidx = q & 31;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (cidx < ncol) {
+      const __nv_bfloat16* rp = lsh + cidx * D + k4 * 4;
+      v = make_float4(__bfloat162float(rp[0]), __bfloat162float(rp[1]), __bfloat162float(rp[2]), __bfloat162float(rp[3]));
+    }
+    rt4[k4][cidx] = v;
   }
   __syncthreads();
-  constexpr int EPL = D / 32;
-  for (int row = blockIdx.x * 8 + warp; row < n; row += gridDim.x * 8) {
-    const __nv_bfloat16* xr = x + h * hs + row * ts;
-    float sq = 0.f;
+  constexpr int EPL = D / 32;                           // elements per lane: 4 (one float4) or 2
+  for (int r0 = (blockIdx.x * 8 + warp) * 4; r0 < n; r0 += gridDim.x * 32) {
+    float sq[4];
 #pragma unroll
-    for (int e = 0; e < EPL; e += 2) {
-      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(xr + lane * EPL + e);
-      const float a = __low2float(v), b = __high2float(v);
-      xs[warp][lane * EPL + e] = a;
-      xs[warp][lane * EPL + e + 1] = b;
-      sq = fmaf(a, a, sq);
-      sq = fmaf(b, b, sq);
+    for (int rr = 0; rr < 4; ++rr) {
+      const int row = min(r0 + rr, n - 1);              // rows past the end repeat the last one; never written
+      const __nv_bfloat16* xr = x + h * hs + row * ts + lane * EPL;
+      float e[EPL];
+#pragma unroll
+      for (int t = 0; t < EPL; t += 2) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(xr + t);
+        e[t] = __low2float(v);
+        e[t + 1] = __high2float(v);
+      }
+      float s2 = 0.f;
+#pragma unroll
+      for (int t = 0; t < EPL; ++t) s2 = fmaf(e[t], e[t], s2);
+      sq[rr] = s2;
+      float* dst = reinterpret_cast<float*>(&xs4[warp][rr][0]) + lane * EPL;
+#pragma unroll
+      for (int t = 0; t < EPL; ++t) dst[t] = e[t];
     }
     __syncwarp();
-    float acc = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < D; ++k) acc = fmaf(xs[warp][k], rt[k][lane], acc);
-    const uint32_t bits = __ballot_sync(0xffffffffu, acc > 0.f);
-    uint32_t code = 0;
-    for (int t = 0; t < T; ++t) code |= ((bits >> (t * B)) & ((1u << B) - 1u)) << (8 * t);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+    for (int k4 = 0; k4 < D / 4; ++k4) {
+      const float4 rv = rt4[k4][lane];
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-    if (lane == 0) {
-      code_out[h * out_stride + row] = code;
-      if (rnorm_out) rnorm_out[h * out_stride + row] = sq > 0.f ? 1.f / sqrtf(sq) : 0.f;
+      for (int rr = 0; rr < 4; ++rr) {
+        const float4 xv = xs4[warp][rr][k4];
+        acc[rr] = fmaf(xv.x, rv.x, acc[rr]);
+        acc[rr] = fmaf(xv.y, rv.y, acc[rr]);
+        acc[rr] = fmaf(xv.z, rv.z, acc[rr]);
+        acc[rr] = fmaf(xv.w, rv.w, acc[rr]);
+      }
+    }
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+      const uint32_t bits = __ballot_sync(0xffffffffu, acc[rr] > 0.f);
+      uint32_t code = 0;
+      for (int t = 0; t < T; ++t) code |= ((bits >> (t * B)) & ((1u << B) - 1u)) << (8 * t);
+      float s2 = sq[rr];
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+      if (lane == 0 && r0 + rr < n) {
+        code_out[h * out_stride + r0 + rr] = code;
+        if (rnorm_out) rnorm_out[h * out_stride + r0 + rr] = s2 > 0.f ? 1.f / sqrtf(s2) : 0.f;
+      }
     }
     __syncwarp();
   }
@@ -137,7 +167,7 @@ __global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restri
 static int launch_prep_generic(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
                                float* rnorm_out, int64_t out_stride, cudaStream_t st) {
   if (n <= 0) return 0;
-  const dim3 grid(min((n + 7) / 8, 148 * 4), c.H);
+  const dim3 grid(max(1, min((n + 31) / 32, (4 * 148 + c.H - 1) / c.H)), c.H);   // ~4 CTAs per SM, many rows each
   if (c.D == 128) prep_kernel<128><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
   else prep_kernel<64><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
