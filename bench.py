@@ -326,7 +326,17 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1", choices=["c1", "c3", "c0", "small"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="step", choices=["step", "rollout", "sweep"],
+                    help="step = the one-line contract; rollout = c2 long rollout + dense baseline; sweep = c4 roofline sweep")
+    ap.add_argument("--chunks", type=int, default=120)
+    ap.add_argument("--out", default=None)
+    ap.add_argument("--no-dense", action="store_true")
     args = ap.parse_args()
+    if args.mode != "step":
+        import bench_modes
+        args.out = args.out or os.path.join(ROOT, "gpurun_out", "c2_rollout.json" if args.mode == "rollout" else "c4_sweep.json")
+        (bench_modes.run_rollout if args.mode == "rollout" else bench_modes.run_sweep)(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = workload_config(args.workload)
     if args.impl == "reference":

@@ -49,10 +49,9 @@ __device__ __forceinline__ void bitonic_sort_smem(unsigned long long* keys, int 
     for (int j = k >> 1; j > 0; j >>= 1) {
       for (int t = threadIdx.x; t < (np2 >> 1); t += blockDim.x) {
         const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // j is a power of two
-        const int p = i + j;
         const bool up = (i & k) == 0;
-        const unsigned long long a = keys[i], b = keys[p];
-        if ((a > b) == up) { keys[i] = b; keys[p] = a; }
+        const unsigned long long a = keys[i], b = keys[i + j];
+        if ((a > b) == up) { keys[i] = b; keys[i + j] = a; }
       }
       __syncthreads();
     }
@@ -88,86 +87,101 @@ int launch_convert_f32_to_bf16(const float* src, __nv_bfloat16* dst, int H, int 
 }
 
 // ---------------------------------------------------------------------------------------------
-// S1: codes (and reciprocal norms).  One warp per row; lane c owns projection direction c.
+// S1: codes (and reciprocal norms).
 // ---------------------------------------------------------------------------------------------
+// X[n x D] . R^T[D x 32] is a skinny contraction (N = 32) bound by reading X once, so it runs on warp-level
+// mma.sync (m16n8k16, bf16 in, fp32 accumulate) with R held in registers: one warp = 16 rows per pass, no shared
+// memory, ~100 instructions per 16 rows.  Fragment layout (g = lane / 4, t = lane % 4):
+//   A: a0 = X[g][2t..], a1 = X[g+8][2t..], a2 = X[g][2t+8..], a3 = X[g+8][2t+8..]   (bf16 pairs)
+//   B: b0 = R[n = 8*nt + g][2t..], b1 = R[n][2t+8..];   C: c0,c1 = row g, cols 2t,2t+1;  c2,c3 = row g+8.
 template <int D>
 __global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restrict__ x, int n, int64_t hs, int64_t ts,
                                                    const __nv_bfloat16* __restrict__ lsh, int T, int B,
                                                    uint32_t* __restrict__ code_out, float* __restrict__ rnorm_out,
                                                    int64_t out_stride) {
-  // rt4[k/4][c] = R[c][k..k+3]: one conflict-free 128-bit read gives lane c four consecutive k.  A warp
-  // projects 4 rows per pass so that every R value read from shared memory is used four times.
-  __shared__ float4 rt4[D / 4][32];
-  __shared__ float4 xs4[8][4][D / 4];
+  constexpr int KS = D / 16;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
   const int h = blockIdx.y;
   const int ncol = T * B;
-  for (int q = threadIdx.x; q < (D / 4) * 32; q += blockDim.x) {
-    const int k4 = q >> 5, cidx = q & 31;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (cidx < ncol) {
-      const __nv_bfloat16* rp = lsh + cidx * D + k4 * 4;
-      v = make_float4(__bfloat162float(rp[0]), __bfloat162float(rp[1]), __bfloat162float(rp[2]), __bfloat162float(rp[3]));
+  uint32_t bf[KS][4][2];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const int col = 8 * nt + g;
+      const __nv_bfloat16* rp = lsh + col * D + 16 * ks + 2 * t;
+      bf[ks][nt][0] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp) : 0u;
+      bf[ks][nt][1] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp + 8) : 0u;
     }
-    rt4[k4][cidx] = v;
-  }
-  __syncthreads();
-  constexpr int EPL = D / 32;                           // elements per lane: 4 (one float4) or 2
-  for (int r0 = (blockIdx.x * 8 + warp) * 4; r0 < n; r0 += gridDim.x * 32) {
-    float sq[4];
+  for (int r0 = (blockIdx.x * 8 + warp) * 16; r0 < n; r0 += gridDim.x * 128) {
+    const int ra = min(r0 + g, n - 1), rb = min(r0 + g + 8, n - 1);   // rows past the end repeat the last one
+    const __nv_bfloat16* xa = x + h * hs + ra * ts + 2 * t;
+    const __nv_bfloat16* xb = x + h * hs + rb * ts + 2 * t;
+    float acc[4][4];
 #pragma unroll
-    for (int rr = 0; rr < 4; ++rr) {
-      const int row = min(r0 + rr, n - 1);              // rows past the end repeat the last one; never written
-      const __nv_bfloat16* xr = x + h * hs + row * ts + lane * EPL;
-      float e[EPL];
+    for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-      for (int t = 0; t < EPL; t += 2) {
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(xr + t);
-        e[t] = __low2float(v);
-        e[t + 1] = __high2float(v);
+      for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+    float sqa = 0.f, sqb = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const uint32_t a0 = *reinterpret_cast<const uint32_t*>(xa + 16 * ks);
+      const uint32_t a1 = *reinterpret_cast<const uint32_t*>(xb + 16 * ks);
+      const uint32_t a2 = *reinterpret_cast<const uint32_t*>(xa + 16 * ks + 8);
+      const uint32_t a3 = *reinterpret_cast<const uint32_t*>(xb + 16 * ks + 8);
+      {
+        const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a0));
+        const float2 f2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a2));
+        const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a1));
+        const float2 f3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a3));
+        sqa = fmaf(f0.x, f0.x, fmaf(f0.y, f0.y, fmaf(f2.x, f2.x, fmaf(f2.y, f2.y, sqa))));
+        sqb = fmaf(f1.x, f1.x, fmaf(f1.y, f1.y, fmaf(f3.x, f3.x, fmaf(f3.y, f3.y, sqb))));
       }
-      float s2 = 0.f;
 #pragma unroll
-      for (int t = 0; t < EPL; ++t) s2 = fmaf(e[t], e[t], s2);
-      sq[rr] = s2;
-      float* dst = reinterpret_cast<float*>(&xs4[warp][rr][0]) + lane * EPL;
-#pragma unroll
-      for (int t = 0; t < EPL; ++t) dst[t] = e[t];
+      for (int nt = 0; nt < 4; ++nt)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(acc[nt][0]), "+f"(acc[nt][1]), "+f"(acc[nt][2]), "+f"(acc[nt][3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bf[ks][nt][0]), "r"(bf[ks][nt][1]));
     }
-    __syncwarp();
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 4
-    for (int k4 = 0; k4 < D / 4; ++k4) {
-      const float4 rv = rt4[k4][lane];
+    // sign bits: this lane owns columns 8*nt + 2t, +1 of rows g and g+8; OR over the quad gives all 32 columns
+    uint32_t ma = 0, mb = 0;
 #pragma unroll
-      for (int rr = 0; rr < 4; ++rr) {
-        const float4 xv = xs4[warp][rr][k4];
-        acc[rr] = fmaf(xv.x, rv.x, acc[rr]);
-        acc[rr] = fmaf(xv.y, rv.y, acc[rr]);
-        acc[rr] = fmaf(xv.z, rv.z, acc[rr]);
-        acc[rr] = fmaf(xv.w, rv.w, acc[rr]);
+    for (int nt = 0; nt < 4; ++nt) {
+      const int c0 = 8 * nt + 2 * t;
+      ma |= (acc[nt][0] > 0.f ? 1u : 0u) << c0;
+      ma |= (acc[nt][1] > 0.f ? 1u : 0u) << (c0 + 1);
+      mb |= (acc[nt][2] > 0.f ? 1u : 0u) << c0;
+      mb |= (acc[nt][3] > 0.f ? 1u : 0u) << (c0 + 1);
+    }
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      ma |= __shfl_xor_sync(0xffffffffu, ma, o);
+      mb |= __shfl_xor_sync(0xffffffffu, mb, o);
+      sqa += __shfl_xor_sync(0xffffffffu, sqa, o);
+      sqb += __shfl_xor_sync(0xffffffffu, sqb, o);
+    }
+    if (t == 0) {
+      uint32_t ca = 0, cb = 0;
+      for (int tt = 0; tt < T; ++tt) {
+        ca |= ((ma >> (tt * B)) & ((1u << B) - 1u)) << (8 * tt);
+        cb |= ((mb >> (tt * B)) & ((1u << B) - 1u)) << (8 * tt);
+      }
+      if (r0 + g < n) {
+        code_out[h * out_stride + r0 + g] = ca;
+        if (rnorm_out) rnorm_out[h * out_stride + r0 + g] = sqa > 0.f ? 1.f / sqrtf(sqa) : 0.f;
+      }
+      if (r0 + g + 8 < n) {
+        code_out[h * out_stride + r0 + g + 8] = cb;
+        if (rnorm_out) rnorm_out[h * out_stride + r0 + g + 8] = sqb > 0.f ? 1.f / sqrtf(sqb) : 0.f;
       }
     }
-#pragma unroll
-    for (int rr = 0; rr < 4; ++rr) {
-      const uint32_t bits = __ballot_sync(0xffffffffu, acc[rr] > 0.f);
-      uint32_t code = 0;
-      for (int t = 0; t < T; ++t) code |= ((bits >> (t * B)) & ((1u << B) - 1u)) << (8 * t);
-      float s2 = sq[rr];
-#pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
-      if (lane == 0 && r0 + rr < n) {
-        code_out[h * out_stride + r0 + rr] = code;
-        if (rnorm_out) rnorm_out[h * out_stride + r0 + rr] = s2 > 0.f ? 1.f / sqrtf(s2) : 0.f;
-      }
-    }
-    __syncwarp();
   }
 }
 static int launch_prep_generic(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
                                float* rnorm_out, int64_t out_stride, cudaStream_t st) {
   if (n <= 0) return 0;
-  const dim3 grid(max(1, min((n + 31) / 32, (4 * 148 + c.H - 1) / c.H)), c.H);   // ~4 CTAs per SM, many rows each
+  const dim3 grid(max(1, min((n + 127) / 128, (8 * 148 + c.H - 1) / c.H)), c.H);   // 128 rows per CTA pass
   if (c.D == 128) prep_kernel<128><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
   else prep_kernel<64><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;

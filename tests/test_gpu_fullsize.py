@@ -1,0 +1,117 @@
+"""GPU parity at the benchmark's full c1 size, in the launch configuration bench.py times: the whole
+step runs on the GPU; the oracle checks sampled outputs it can compute one by one (T1 on sampled tokens,
+attention on sampled query blocks) and everything that is cheap in full (merge bookkeeping, codes, block
+scores and selections, prompt selection)."""
+import numpy as np
+import pytest
+
+from oracle import fastar_oracle as O
+from paper_2602_01801_b200 import synth
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_blocks(Q, hc, sel, blocks, bq, bk):
+    """Oracle attention for the listed query blocks only -> {block: rows x d}."""
+    out = {}
+    for a in blocks:
+        rows = slice(a * bq, min((a + 1) * bq, Q.shape[0]))
+        sub = O.sparse_attention(Q[rows].astype(np.float64), hc, sel[a: a + 1], bq, bk)
+        out[a] = sub
+    return out
+
+
+def test_c1_full_size_step_sampled():
+    import torch
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.CONFIGS["c1"]
+    w = synth.Workload(cfg)
+    H, n = cfg.num_heads, cfg.chunk_tokens
+    cache = fastar.Cache(H, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
+                         max_tokens=n, max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk)
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, 2.0, outputs=False)
+    assert cache.status() == 0
+    pre = cache.export_state()
+    assert np.all(pre["len"] == cfg.prior_chunks * n)
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    res = cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau)
+    assert cache.status() == 0
+    post = cache.export_state()
+    match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    rng = np.random.default_rng(0)
+    heads_checked = [0, 5, 11]
+    pre_heads = P.oracle_heads_from_export(pre)
+    for h in heads_checked:
+        rows = np.sort(rng.choice(n, 96, replace=False))
+        P.check_update(pre_heads[h], K[h], V[h], cfg.frame_len, cfg.tau, match[h], sim[h], dest[h], stats[h], post, h, rows=rows)
+    # every head: bookkeeping invariants from the exported state
+    for h in range(H):
+        L = int(post["len"][h])
+        assert L == int(pre["len"][h]) + int(stats[h, 2]) <= cfg.capacity
+        assert int(post["count"][h, :L].sum()) == (cfg.prior_chunks + 1) * n
+        assert int(stats[h, 0]) + int(stats[h, 2]) + int(stats[h, 3]) == n
+    # AnnSA
+    a = cache.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks, debug=True)
+    assert cache.status() == 0
+    out = a["out"].float().cpu().numpy()
+    R = w.lsh_projection()
+    post_heads = P.oracle_heads_from_export(post)
+    nqb = -(-n // cfg.block)
+    for h in heads_checked:
+        hc = post_heads[h]
+        qcodes = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, a["qcode"][h].cpu().numpy().view(np.uint32))
+        kcodes = P.check_codes(P.bits_to_f64(post["k"][h, : hc.L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][h, : hc.L])
+        sel = P.check_selection(qcodes, kcodes, n, hc.L, cfg.block, cfg.block, cfg.lsh_bits, cfg.keep_blocks,
+                                a["scores"][h].cpu().numpy(), a["sel"][h].cpu().numpy(), int(a["nsel"][h]))
+        blocks = [0, 7, nqb // 2, nqb - 1]                       # includes the ragged last block (72 rows)
+        want = _oracle_blocks(Q[h], hc, sel, blocks, cfg.block, cfg.block)
+        for blk, wnt in want.items():
+            rows = slice(blk * cfg.block, min((blk + 1) * cfg.block, n))
+            P.check_attention(out[h][rows], wnt, f"AnnSA c1 head {h} block {blk}")
+    # AnnCA
+    Kp, Vp, planted = w.prompt(cfg.prior_chunks)
+    c = cache.annca(fastar.to_device(Q), fastar.to_device(Kp), fastar.to_device(Vp), cfg.frame_len, cfg.keep_prompt, debug=True)
+    assert cache.status() == 0
+    oc = c["out"].float().cpu().numpy()
+    for h in heads_checked:
+        selp = c["sel"][h].cpu().numpy()
+        P.check_prompt_selection(Q[h], Kp[h], cfg.frame_len, cfg.keep_prompt, selp, c["rel"][h].cpu().numpy())
+        for f in range(cfg.frames_per_chunk):
+            assert set(planted[f].tolist()) <= set(selp[f].tolist())
+        P.check_attention(oc[h], O.annca(Q[h], Kp[h], Vp[h], cfg.frame_len, cfg.keep_prompt, sel=selp)["out"], f"AnnCA c1 head {h}")
+
+
+def test_c2_style_rollout_invariants():
+    """A scaled-down long rollout (slow drift, few new tokens per chunk, small capacity so that eviction sets
+    in): the cache stays bounded and the token bookkeeping holds on every chunk."""
+    import torch
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.small_config(num_heads=2, sigma=0.05, resample=0.05, shift=0.5, capacity=1024, prior_chunks=0, keep_blocks=3)
+    w = synth.Workload(cfg)
+    cache = fastar.Cache(cfg.num_heads, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
+                         max_tokens=cfg.chunk_tokens, max_prompt_tokens=128, max_frames=4)
+    n = cfg.chunk_tokens
+    evicted = np.zeros(cfg.num_heads, np.int64)
+    lens = []
+    for ci in range(24):
+        Q, K, V = w.chunk(ci)
+        res = cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau)
+        out = cache.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks)["out"]
+        assert cache.status() == 0
+        st = res["stats"].cpu().numpy()
+        evicted += st[:, 4]
+        state = cache.export_state(kv=False)
+        for h in range(cfg.num_heads):
+            L = int(state["len"][h])
+            assert L <= cfg.capacity and L == int(st[h, 5])
+            assert int(state["count"][h, :L].sum()) + int(evicted[h]) == (ci + 1) * n
+            assert np.all(state["count"][h, L:] == 0) and np.all(state["stamp"][h, :L] <= ci)
+            assert int((state["stamp"][h, :L] == ci).sum()) == int(st[h, 1]) + int(st[h, 2]) + int(st[h, 3])
+        assert bool(torch.isfinite(out.float()).all())
+        lens.append(state["len"].copy())
+    assert evicted.sum() > 0 and np.all(lens[-1] == cfg.capacity)
