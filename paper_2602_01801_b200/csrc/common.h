@@ -50,8 +50,12 @@ struct CacheView {
   uint32_t* code_new;              // [H][max_tokens]  codes of new keys / of queries
   int32_t* match;                  // [H][max_tokens]
   float* sim;                      // [H][max_tokens]
-  int32_t* order;                  // [H][max_tokens]  token ids sorted by (slot, token)
-  int32_t* segpos;                 // [H][max_tokens+1] start of each segment in `order`
+  int32_t* cnt;                    // [H][CAP]         tokens matched to each slot by this update (zeroed with `best`)
+  int32_t* cur;                    // [H][CAP]         scatter cursor of each touched slot
+  int32_t* order;                  // [H][max_tokens]  matched token ids, grouped by slot (unordered inside a group)
+  int32_t* segpos;                 // [H][max_tokens+1] start of each group in `order` (+ end sentinel)
+  int32_t* segslot;                // [H][max_tokens]  slot of each group
+  int32_t* ulist;                  // [H][max_tokens]  unmatched token ids in token order
   int32_t* dest;                   // [H][max_tokens]
   int32_t* victims;                // [H][max_tokens]
   PlanRec* plan;                   // [H]

@@ -84,6 +84,10 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.status = reinterpret_cast<int32_t*>(take(4));
   t.lsh = reinterpret_cast<__nv_bfloat16*>(take(32 * D * 2));
   t.best = reinterpret_cast<unsigned long long*>(take(H * MT * 8));
+  t.cnt = reinterpret_cast<int32_t*>(take(H * CAP * 4));            // directly after `best`: one memset clears both
+  t.cur = reinterpret_cast<int32_t*>(take(H * CAP * 4));
+  t.segslot = reinterpret_cast<int32_t*>(take(H * MT * 4));
+  t.ulist = reinterpret_cast<int32_t*>(take(H * MT * 4));
   t.rnorm_new = reinterpret_cast<float*>(take(H * MT * 4));
   t.code_new = reinterpret_cast<uint32_t*>(take(H * MT * 4));
   t.match = reinterpret_cast<int32_t*>(take(H * MT * 4));
@@ -316,7 +320,9 @@ int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_
   r = make_map(c, &tm_a, kb, v.D, n, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
   if (r != FASTAR_OK) return r;
   ACCK(FASTAR_K_HASH, launch_prep_codes(v, kb, n, khs, kts, v.code_new, v.rnorm_new, st));
-  if (cudaMemsetAsync(v.best, 0, static_cast<size_t>(v.H) * v.max_tokens * 8, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  // packed arg-max words and per-slot match counts start at zero (adjacent in the workspace: one memset)
+  if (cudaMemsetAsync(v.best, 0, reinterpret_cast<uint8_t*>(v.cnt) - reinterpret_cast<uint8_t*>(v.best) + static_cast<size_t>(v.H) * v.CAP * 4, st) != cudaSuccess)
+    return FASTAR_ERR_CUDA;
   ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, n, st));
   ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
   ACCK(FASTAR_K_COMMIT, launch_commit(v, kb, vb, n, frame_len, khs, kts, st));

@@ -192,70 +192,87 @@ int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t
 }
 
 // ---------------------------------------------------------------------------------------------
-// T2-T4 planning: one CTA per head.  Sort tokens by (matched slot, token), find the groups,
-// place the unmatched tokens (append, then victims in (stamp, slot) order).  Validate, then commit.
+// T2-T4 planning in three small kernels (all work O(n + L), no sort):
+//   match_count : decode the packed arg-max, threshold (T2), count the tokens matched to each slot
+//   plan        : one CTA per head: scan the slot counts -> groups (touched slots) and their member
+//                 ranges; scan the tokens -> unmatched tokens in token order; place them (append, then
+//                 victims in (stamp, slot) order).  Validate, then commit.
+//   scatter     : put each matched token into its group's member range
+// Members of a group land in arbitrary order; the commit walks them in ascending token order, so the
+// result does not depend on it.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n, int np2, float tau) {
-  extern __shared__ unsigned long long keys[];
+__global__ void __launch_bounds__(256) match_count_kernel(const CacheView c, int n, float tau) {
+  const int h = blockIdx.y;
+  const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const unsigned long long b = c.best[tb + i];
+    int j = -1;
+    float s = 0.f;
+    if (b != 0ull) {
+      j = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull));
+      s = ordered_to_float(static_cast<uint32_t>(b >> 32));
+    }
+    const bool matched = j >= 0 && s >= tau;
+    c.match[tb + i] = matched ? j : -1;
+    c.sim[tb + i] = s;
+    if (matched) atomicAdd(c.cnt + static_cast<int64_t>(h) * c.CAP + j, 1);
+  }
+}
+
+__global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
+  extern __shared__ unsigned long long keys[];   // victim sort buffer, only touched when evicting
   __shared__ int red[32];
-  __shared__ int sh[8];
   const int h = blockIdx.x, tid = threadIdx.x;
   const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
   const int64_t sb = static_cast<int64_t>(h) * c.CAP;
+  const int64_t gb = static_cast<int64_t>(h) * (c.max_tokens + 1);
   const int L = c.len[h];
   const int now = *c.now;
 
-  // T2: decode the packed arg-max, threshold
-  for (int i = tid; i < np2; i += blockDim.x) {
-    unsigned long long key = ~0ull;
-    if (i < n) {
-      const unsigned long long b = c.best[tb + i];
-      int j = -1;
-      float s = 0.f;
-      if (b != 0ull) {
-        j = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull));
-        s = ordered_to_float(static_cast<uint32_t>(b >> 32));
-      }
-      const bool matched = j >= 0 && s >= tau;
-      c.match[tb + i] = matched ? j : -1;
-      c.sim[tb + i] = s;
-      key = (static_cast<unsigned long long>(matched ? static_cast<uint32_t>(j) : 0xFFFFFFFFu) << 32) |
-            static_cast<uint32_t>(i);
+  // groups: 4 consecutive slots per thread and pass
+  int seg_run = 0, mem_run = 0, touched_ns = 0;
+  for (int j0 = 0; j0 < L; j0 += 4 * blockDim.x) {
+    const int j = j0 + 4 * tid;
+    int cn[4] = {0, 0, 0, 0};
+    if (j + 3 < L) {
+      const int4 v = *reinterpret_cast<const int4*>(c.cnt + sb + j);
+      cn[0] = v.x; cn[1] = v.y; cn[2] = v.z; cn[3] = v.w;
+    } else {
+      for (int u = 0; u < 4; ++u) if (j + u < L) cn[u] = c.cnt[sb + j + u];
     }
-    keys[i] = key;
+    const int my_seg = (cn[0] > 0) + (cn[1] > 0) + (cn[2] > 0) + (cn[3] > 0);
+    const int my_mem = cn[0] + cn[1] + cn[2] + cn[3];
+    int tot_seg, tot_mem;
+    int seg = seg_run + block_exscan(my_seg, red, &tot_seg);
+    int mem = mem_run + block_exscan(my_mem, red, &tot_mem);
+    for (int u = 0; u < 4; ++u) {
+      if (cn[u] > 0) {
+        c.segslot[tb + seg] = j + u;
+        c.segpos[gb + seg] = mem;
+        c.cur[sb + j + u] = mem;
+        if (j + u >= c.n_sink) ++touched_ns;
+        ++seg;
+        mem += cn[u];
+      }
+    }
+    seg_run += tot_seg;
+    mem_run += tot_mem;
   }
-  __syncthreads();
-  bitonic_sort_smem(keys, np2);
+  const int n_seg = seg_run, M = mem_run;
+  touched_ns = block_sum(touched_ns, red);
+  if (tid == 0) c.segpos[gb + n_seg] = M;
 
-  // matched count, segment heads
-  int my_m = 0, my_heads = 0, my_heads_ns = 0;
-  const int per = (np2 + blockDim.x - 1) / blockDim.x;
-  const int p_lo = tid * per, p_hi = min(n, p_lo + per);
-  for (int p = p_lo; p < p_hi; ++p) {
-    const uint32_t slot = static_cast<uint32_t>(keys[p] >> 32);
-    if (slot != 0xFFFFFFFFu) {
-      ++my_m;
-      if (p == 0 || static_cast<uint32_t>(keys[p - 1] >> 32) != slot) {
-        ++my_heads;
-        if (static_cast<int>(slot) >= c.n_sink) ++my_heads_ns;
-      }
-    }
+  // unmatched tokens in token order
+  int u_run = 0;
+  for (int i0 = 0; i0 < n; i0 += blockDim.x) {
+    const int i = i0 + tid;
+    const int un = (i < n && c.match[tb + i] < 0) ? 1 : 0;
+    int tot;
+    const int k = u_run + block_exscan(un, red, &tot);
+    if (un) c.ulist[tb + k] = i;
+    u_run += tot;
   }
-  const int M = block_sum(my_m, red);
-  const int touched_ns = block_sum(my_heads_ns, red);
-  int n_seg;
-  int seg_base = block_exscan(my_heads, red, &n_seg);
-  for (int p = p_lo; p < p_hi; ++p) {
-    const unsigned long long k = keys[p];
-    const uint32_t slot = static_cast<uint32_t>(k >> 32);
-    const int i = static_cast<int>(k & 0xFFFFFFFFull);
-    c.order[tb + p] = i;
-    if (slot != 0xFFFFFFFFu) {
-      c.dest[tb + i] = static_cast<int>(slot);
-      if (p == 0 || static_cast<uint32_t>(keys[p - 1] >> 32) != slot) c.segpos[static_cast<int64_t>(h) * (c.max_tokens + 1) + seg_base++] = p;
-    }
-  }
-  const int U = n - M;
+  const int U = u_run;
   const int A = min(U, c.CAP - L);
   const int E = U - A;
   int ok = 1;
@@ -267,32 +284,28 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n, in
   }
   int evicted_tokens = 0;
   if (ok && E > 0) {
-    // touched slots are not evictable: stamp them now (the commit writes the same value)
-    for (int p = p_lo; p < p_hi; ++p) {
-      const uint32_t slot = static_cast<uint32_t>(keys[p] >> 32);
-      if (slot != 0xFFFFFFFFu && (p == 0 || static_cast<uint32_t>(keys[p - 1] >> 32) != slot)) c.stamp[sb + slot] = now;
-    }
-    __syncthreads();
+    // evictable = live, past the sink prefix, stamp < now, not touched by this update (cnt == 0).
     // smallest stamp value s* such that at least E evictable slots have stamp <= s*
+    auto evictable_stamp = [&](int j) -> int {
+      return (j < L && j >= c.n_sink && c.cnt[sb + j] == 0) ? c.stamp[sb + j] : 0x7fffffff;
+    };
     int lo = 0, hi = now - 1;
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
-      int cnt = 0;
-      for (int j = tid; j < L; j += blockDim.x) cnt += (j >= c.n_sink && c.stamp[sb + j] <= mid) ? 1 : 0;
-      cnt = block_sum(cnt, red);
-      if (cnt >= E) hi = mid; else lo = mid + 1;
+      int cn = 0;
+      for (int j = tid; j < L; j += blockDim.x) cn += evictable_stamp(j) <= mid ? 1 : 0;
+      cn = block_sum(cn, red);
+      if (cn >= E) hi = mid; else lo = mid + 1;
     }
     const int sstar = lo;
     int c_less = 0;
-    for (int j = tid; j < L; j += blockDim.x) c_less += (j >= c.n_sink && c.stamp[sb + j] < sstar) ? 1 : 0;
+    for (int j = tid; j < L; j += blockDim.x) c_less += evictable_stamp(j) < sstar ? 1 : 0;
     c_less = block_sum(c_less, red);
     const int need_eq = E - c_less;
-    // ordered compaction of the victims into keys[0..E)
     int eq_run = 0, out_run = 0;
-    __syncthreads();
     for (int j0 = 0; j0 < L; j0 += blockDim.x) {
       const int j = j0 + tid;
-      const int stp = (j < L && j >= c.n_sink) ? c.stamp[sb + j] : 0x7fffffff;
+      const int stp = evictable_stamp(j);
       const int is_eq = stp == sstar ? 1 : 0;
       int tot_eq;
       const int eq_rank = eq_run + block_exscan(is_eq, red, &tot_eq);
@@ -315,16 +328,11 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n, in
       ev += c.count[sb + v];
     }
     evicted_tokens = block_sum(ev, red);
-    __syncthreads();
   }
-  // destinations of the unmatched tokens (sorted positions [M, n) are in token order)
+  __syncthreads();
+  // destinations (matched tokens get theirs in the scatter kernel)
   if (ok) {
-    __syncthreads();
-    for (int p = M + tid; p < n; p += blockDim.x) {
-      const int k = p - M;
-      const int i = c.order[tb + p];
-      c.dest[tb + i] = k < A ? L + k : c.victims[tb + k - A];
-    }
+    for (int k = tid; k < U; k += blockDim.x) c.dest[tb + c.ulist[tb + k]] = k < A ? L + k : c.victims[tb + k - A];
   } else {
     for (int i = tid; i < n; i += blockDim.x) c.dest[tb + i] = -1;
     if (tid == 0) record_status(c.status, kErrCapacity);
@@ -342,21 +350,36 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n, in
     pr.evicted_tokens = evicted_tokens;
     pr.pad[0] = pr.pad[1] = pr.pad[2] = 0;
     c.plan[h] = pr;
-    (void)sh;
   }
 }
+
+__global__ void __launch_bounds__(256) scatter_kernel(const CacheView c, int n) {
+  const int h = blockIdx.y;
+  if (!c.plan[h].ok) return;
+  const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int j = c.match[tb + i];
+    if (j >= 0) {
+      const int pos = atomicAdd(c.cur + static_cast<int64_t>(h) * c.CAP + j, 1);
+      c.order[tb + pos] = i;
+      c.dest[tb + i] = j;
+    }
+  }
+}
+
 int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st) {
   (void)frame_len;
-  int np2 = 1024;
-  while (np2 < n) np2 <<= 1;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 8) != cudaSuccess)
       return FASTAR_ERR_CUDA;
     configured = true;
   }
-  plan_kernel<<<c.H, 1024, np2 * 8, st>>>(c, n, np2, tau);
-  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+  const dim3 grid((n + 255) / 256, c.H);
+  match_count_kernel<<<grid, 256, 0, st>>>(c, n, tau);
+  plan_kernel<<<c.H, 1024, 16384 * 8, st>>>(c, n);
+  scatter_kernel<<<grid, 256, 0, st>>>(c, n);
+  return cudaGetLastError() == cudaSuccess ? 3 : FASTAR_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -381,9 +404,9 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
 
   if (w < pr.n_seg) {
     const int32_t* segpos = c.segpos + static_cast<int64_t>(h) * (c.max_tokens + 1);
-    const int p0 = segpos[w];
-    const int p1 = (w + 1 < pr.n_seg) ? segpos[w + 1] : pr.n_matched;
-    const int slot = c.match[tb + c.order[tb + p0]];
+    const int p0 = segpos[w], p1 = segpos[w + 1];
+    const int g = p1 - p0;
+    const int slot = c.segslot[tb + w];
     const int64_t ro = slot_row_offset(c, pt_h, slot);
     const int m_old = c.count[sb + slot];
     float acc[EPL];
@@ -396,11 +419,23 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
         acc[e + 1] = static_cast<float>(m_old) * __high2float(t);
       }
     }
+    // Walk the members in ascending token order (fixed summation order; the scatter left them unordered):
+    // each round takes the smallest token index above the previous one.  Lanes hold up to 32 members in a
+    // register, larger groups re-read the list.
+    const int mine = (p0 + lane < p1) ? c.order[tb + p0 + lane] : 0x7fffffff;
     // representative: newest frame, then highest similarity, then lowest token index
-    int best_i = -1, best_f = -1;
+    int best_i = -1, best_f = -1, last = -1;
     float best_s = -INFINITY;
-    for (int p = p0; p < p1; ++p) {                    // ascending token index
-      const int i = c.order[tb + p];
+    for (int r = 0; r < g; ++r) {
+      int cand = mine > last ? mine : 0x7fffffff;
+      for (int p = p0 + 32 + lane; p < p1; p += 32) {
+        const int i2 = c.order[tb + p];
+        if (i2 > last && i2 < cand) cand = i2;
+      }
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, o));
+      const int i = cand;
+      last = i;
       const __nv_bfloat16* vr = vh + i * ts + lane * EPL;
 #pragma unroll
       for (int e = 0; e < EPL; e += 2) {
@@ -412,7 +447,6 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
       const float s = c.sim[tb + i];
       if (f > best_f || (f == best_f && s > best_s)) { best_f = f; best_s = s; best_i = i; }
     }
-    const int g = p1 - p0;
     const float inv = 1.f / static_cast<float>(m_old + g);
     {
       __nv_bfloat16* vw = c.pool_v + ro + lane * EPL;
@@ -432,7 +466,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
       c.kcode[sb + slot] = c.code_new[tb + best_i];
     }
   } else if (w - pr.n_seg < pr.n_unmatched) {
-    const int i = c.order[tb + pr.n_matched + (w - pr.n_seg)];
+    const int i = c.ulist[tb + (w - pr.n_seg)];
     const int slot = c.dest[tb + i];
     const int64_t ro = slot_row_offset(c, pt_h, slot);
     const __nv_bfloat16* kr = kh + i * ts + lane * EPL;
