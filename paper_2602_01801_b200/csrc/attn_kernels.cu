@@ -64,17 +64,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
   const uint32_t q_s = sbase + SM::q_off;
   const uint32_t k_s = sbase + SM::k_off;
-  const uint32_t v_s = sbase + SM::v_off;
   const uint32_t p_s = sbase + SM::p_off;
   float* bias_g = reinterpret_cast<float*>(sgen + SM::bias_off);
   const uint32_t bias_s = sbase + SM::bias_off;
   const uint32_t bar = sbase + SM::bar_off;
   const uint32_t bar_q_full = bar;
-  const uint32_t bar_k_full = bar + 8;             // [KS]
-  const uint32_t bar_k_empty = bar_k_full + 8 * KS;
-  const uint32_t bar_v_full = bar_k_empty + 8 * KS;
-  const uint32_t bar_v_empty = bar_v_full + 8 * VS;
-  const uint32_t bar_b_full = bar_v_empty + 8 * VS;   // [NB]
+  constexpr int RS = KS + VS;                        // K and V tiles share one ring
+  const uint32_t ring_s = k_s;
+  const uint32_t bar_r_full = bar + 8;               // [RS]
+  const uint32_t bar_r_empty = bar_r_full + 8 * RS;  // [RS]
+  const uint32_t bar_b_full = bar_r_empty + 8 * RS;  // [NB]
   const uint32_t bar_s_full = bar_b_full + 8 * NB;    // [2]
   const uint32_t bar_s_empty = bar_s_full + 16;       // [2]
   const uint32_t bar_p_full = bar_s_empty + 16;       // [2]
@@ -113,8 +112,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q_full, 1);
-    for (int s = 0; s < KS; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
-    for (int s = 0; s < VS; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
+    for (int s = 0; s < RS; ++s) { mbar_init(bar_r_full + 8 * s, 1); mbar_init(bar_r_empty + 8 * s, 1); }
     for (int s = 0; s < NB; ++s) mbar_init(bar_b_full + 8 * s, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_s_full + 8 * s, 1);
@@ -141,38 +139,60 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_o = tmem + 2 * BKT;
 
+  // K and V tiles share one ring of RS stages, filled and consumed in the order the MMA warp needs them:
+  //   K0, K1, V0, K2, V1, K3, V2, ...   (S_{j+1} = Q K_{j+1}^T is issued before O += P_j V_j)
+  // so a key tile can be requested as soon as the tile four positions earlier has been consumed, without
+  // queueing behind a value tile whose stage frees late.
   if (warp == kProducerWarp) {
     // ================================================================== producer
     if (lane == 0 && nt > 0) {
       mbar_arrive_expect_tx(bar_q_full, SM::q_bytes);
       for (int kc = 0; kc < D / 64; ++kc) tma_load_3d(q_s + kc * kQChunk, &tm_q, bar_q_full, kc * 64, q0, h);
     }
+    bool ok = true;
+    int it = 0;
     if (!GATHER) {
-      if (lane == 0) {
-        const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
-        const float* l2m_h = c.log2m + static_cast<int64_t>(h) * c.CAP;
-        bool ok = true;
-        int blk_next = nt > 0 ? (list ? list[0] : 0) : 0;
-        int page_next = nt > 0 ? pt_h[blk_next] : 0;
-        for (int j = 0; j < nt && ok; ++j) {
-          const int blk = blk_next, page = page_next;
-          if (j + 1 < nt) {                       // look the next block up while this one is in flight
-            blk_next = list ? list[j + 1] : j + 1;
-            page_next = pt_h[blk_next];
-          }
-          const int ks = j % KS, vs = j % VS, b4 = j % NB;
-          ok = mbar_wait(bar_k_empty + 8 * ks, ((j / KS) & 1) ^ 1, abort_flag, c.status);
-          if (!ok) break;
-          mbar_arrive_expect_tx(bar_k_full + 8 * ks, SM::kv_bytes);
-          for (int kc = 0; kc < D / 64; ++kc)
-            tma_load_3d(k_s + ks * SM::kv_bytes + kc * BKT * 128, &tm_k, bar_k_full + 8 * ks, kc * 64, 0, page);
+      // block ids and page ids of 32 tiles at a time, one coalesced load each; lane 0 issues the copies
+      const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+      const float* l2m_h = c.log2m + static_cast<int64_t>(h) * c.CAP;
+      int blk_l = 0, page_l = 0;
+      auto refill = [&](int j0) {
+        if (j0 + lane < nt) {
+          blk_l = list ? list[j0 + lane] : j0 + lane;
+          page_l = pt_h[blk_l];
+        }
+      };
+      auto load_tile = [&](bool is_k, int j, int blk, int page) {
+        if (lane != 0 || !ok) return;
+        const int s = it % RS;
+        ok = mbar_wait(bar_r_empty + 8 * s, ((it / RS) & 1) ^ 1, abort_flag, c.status);
+        if (!ok) return;
+        mbar_arrive_expect_tx(bar_r_full + 8 * s, SM::kv_bytes);
+        for (int kc = 0; kc < D / 64; ++kc)
+          tma_load_3d(ring_s + s * SM::kv_bytes + kc * BKT * 128, is_k ? &tm_k : &tm_v, bar_r_full + 8 * s, kc * 64, 0, page);
+        if (is_k) {
+          const int b4 = j % NB;
           mbar_arrive_expect_tx(bar_b_full + 8 * b4, BKT * 4);
           bulk_load_1d(bias_s + b4 * BKT * 4, l2m_h + static_cast<int64_t>(blk) * BKT, BKT * 4, bar_b_full + 8 * b4);
-          ok = mbar_wait(bar_v_empty + 8 * vs, ((j / VS) & 1) ^ 1, abort_flag, c.status);
-          if (!ok) break;
-          mbar_arrive_expect_tx(bar_v_full + 8 * vs, SM::kv_bytes);
-          for (int kc = 0; kc < D / 64; ++kc)
-            tma_load_3d(v_s + vs * SM::kv_bytes + kc * BKT * 128, &tm_v, bar_v_full + 8 * vs, kc * 64, 0, page);
+        }
+        ++it;
+      };
+      if (nt > 0) {
+        refill(0);
+        int blk_cur = __shfl_sync(0xffffffffu, blk_l, 0), page_cur = __shfl_sync(0xffffffffu, page_l, 0);
+        load_tile(true, 0, blk_cur, page_cur);
+        for (int j = 0; j < nt; ++j) {
+          if (j + 1 < nt) {
+            if (((j + 1) & 31) == 0) refill(j + 1);
+            const int blk_n = __shfl_sync(0xffffffffu, blk_l, (j + 1) & 31);
+            const int page_n = __shfl_sync(0xffffffffu, page_l, (j + 1) & 31);
+            load_tile(true, j + 1, blk_n, page_n);
+            load_tile(false, j, blk_cur, page_cur);
+            blk_cur = blk_n;
+            page_cur = page_n;
+          } else {
+            load_tile(false, j, blk_cur, page_cur);
+          }
         }
       }
     } else {
@@ -180,41 +200,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       constexpr int CPR = D / 8;                       // 16-byte chunks per row
       const __nv_bfloat16* kp_h = a.kp + static_cast<int64_t>(h) * a.p_head_stride;
       const __nv_bfloat16* vp_h = a.vp + static_cast<int64_t>(h) * a.p_head_stride;
-      bool ok = true;
-      for (int j = 0; j < nt && ok; ++j) {
-        const int ks = j % KS, vs = j % VS, b4 = j % NB;
-        ok = mbar_wait(bar_k_empty + 8 * ks, ((j / KS) & 1) ^ 1, abort_flag, c.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        for (int which = 0; which < 2; ++which) {
-          if (which == 1) {
-            ok = mbar_wait(bar_v_empty + 8 * vs, ((j / VS) & 1) ^ 1, abort_flag, c.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+      auto fill_tile = [&](bool is_k, int j) {
+        if (!ok) return;
+        const int s = it % RS;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_r_empty + 8 * s, ((it / RS) & 1) ^ 1, abort_flag, c.status));
+        if (!ok) return;
+        const __nv_bfloat16* src_h = is_k ? kp_h : vp_h;
+        const uint32_t dst = ring_s + s * SM::kv_bytes;
+        for (int q = lane; q < BKT * CPR; q += 32) {
+          const int i = q / CPR, ch = q % CPR;
+          const int tok = j * BKT + i;
+          uint4 val = make_uint4(0, 0, 0, 0);
+          if (tok < a.keep) {
+            const int idx = list[tok];
+            val = *reinterpret_cast<const uint4*>(src_h + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
           }
-          const __nv_bfloat16* src_h = which == 0 ? kp_h : vp_h;
-          const uint32_t dst = which == 0 ? k_s + ks * SM::kv_bytes : v_s + vs * SM::kv_bytes;
-          for (int q = lane; q < BKT * CPR; q += 32) {
-            const int i = q / CPR, ch = q % CPR;
-            const int tok = j * BKT + i;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (tok < a.keep) {
-              const int idx = list[tok];
-              val = *reinterpret_cast<const uint4*>(src_h + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
-            }
-            const uint32_t off = (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + off), "r"(val.x), "r"(val.y), "r"(val.z),
-                         "r"(val.w)
-                         : "memory");
-          }
-          if (which == 0)
-            for (int i = lane; i < BKT; i += 32) bias_g[b4 * BKT + i] = (j * BKT + i < a.keep) ? 0.f : -INFINITY;
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            if (which == 0) { mbar_arrive(bar_k_full + 8 * ks); mbar_arrive(bar_b_full + 8 * b4); }
-            else mbar_arrive(bar_v_full + 8 * vs);
-          }
+          const uint32_t off = (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + off), "r"(val.x), "r"(val.y), "r"(val.z),
+                       "r"(val.w)
+                       : "memory");
+        }
+        const int b4 = j % NB;
+        if (is_k)
+          for (int i = lane; i < BKT; i += 32) bias_g[b4 * BKT + i] = (j * BKT + i < a.keep) ? 0.f : -INFINITY;
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar_r_full + 8 * s);
+          if (is_k) mbar_arrive(bar_b_full + 8 * b4);
+        }
+        ++it;
+      };
+      if (nt > 0) {
+        fill_tile(true, 0);
+        for (int j = 0; j < nt; ++j) {
+          if (j + 1 < nt) fill_tile(true, j + 1);
+          fill_tile(false, j);
         }
       }
     }
@@ -224,38 +245,40 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, BKT, 0);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
       bool ok = mbar_wait(bar_q_full, 0, abort_flag, c.status);
+      int it = 0;                                       // position in the K/V ring (same order as the producer)
       PT_DECL
       auto issue_s = [&](int j) -> bool {
-        const int ks = j % KS, sb = j & 1;
-        if (!mbar_wait(bar_k_full + 8 * ks, (j / KS) & 1, abort_flag, c.status)) return false;
+        const int s = it % RS, sb = j & 1;
+        if (!mbar_wait(bar_r_full + 8 * s, (it / RS) & 1, abort_flag, c.status)) return false;
         PT_MARK(0)
         if (!mbar_wait(bar_s_empty + 8 * sb, ((j >> 1) & 1) ^ 1, abort_flag, c.status)) return false;
         PT_MARK(1)
         tc_fence_after();
-        const uint32_t kt = k_s + ks * SM::kv_bytes;
+        const uint32_t kt = ring_s + s * SM::kv_bytes;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint64_t ad = make_smem_desc(q_s + (kk >> 2) * kQChunk + (kk & 3) * 32, 16, 1024);
           const uint64_t bd = make_smem_desc(kt + (kk >> 2) * (BKT * 128) + (kk & 3) * 32, 16, 1024);
           umma_ss(tmem + sb * BKT, ad, bd, idesc_qk, kk != 0);
         }
-        umma_commit(bar_k_empty + 8 * ks);
+        umma_commit(bar_r_empty + 8 * s);
         umma_commit(bar_s_full + 8 * sb);
+        ++it;
         PT_MARK(2)
         return true;
       };
       if (ok) ok = issue_s(0);
       for (int j = 0; j < nt && ok; ++j) {
         if (j + 1 < nt) { ok = issue_s(j + 1); if (!ok) break; }
-        const int vs = j % VS, pb = j & 1;
+        const int s = it % RS, pb = j & 1;
         ok = mbar_wait(bar_p_full + 8 * pb, (j >> 1) & 1, abort_flag, c.status);
         if (!ok) break;
         PT_MARK(3)
-        ok = mbar_wait(bar_v_full + 8 * vs, (j / VS) & 1, abort_flag, c.status);
+        ok = mbar_wait(bar_r_full + 8 * s, (it / RS) & 1, abort_flag, c.status);
         if (!ok) break;
         PT_MARK(4)
         tc_fence_after();
-        const uint32_t vt = v_s + vs * SM::kv_bytes;
+        const uint32_t vt = ring_s + s * SM::kv_bytes;
         const uint32_t pt = p_s + pb * SM::p_bytes;
 #pragma unroll
         for (int ks16 = 0; ks16 < BKT / 16; ++ks16) {
@@ -263,11 +286,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const uint64_t bd = make_smem_desc(vt + ks16 * 2048, BKT * 128, 1024);
           umma_ss(tmem_o, ad, bd, idesc_pv, (j | ks16) != 0);
         }
-        umma_commit(bar_v_empty + 8 * vs);
+        umma_commit(bar_r_empty + 8 * s);
         umma_commit(bar_pv_done);
+        ++it;
         PT_MARK(5)
       }
-      PT_FLUSH("attn mma", nt)
+      PT_FLUSH("attn mma (wait K, wait S buffer, issue QK, wait P, wait V, issue PV)", nt)
     }
   } else {
     // ================================================================== softmax + epilogue (256 threads)
@@ -348,7 +372,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int q = 0; q < HB / 8; ++q) {
         float p[8];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) p[t] = fast_exp2(x[8 * q + t] - m_eff);
+        for (int t = 0; t < 8; ++t)                 // half on the MUFU unit, half as a polynomial on the FMA pipe
+          p[t] = (t & 1) ? poly_exp2(x[8 * q + t] - m_eff) : fast_exp2(x[8 * q + t] - m_eff);
         l0 += p[0] + p[4];
         l1 += p[1] + p[5];
         l2 += p[2] + p[6];
@@ -382,7 +407,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       mbar_arrive_warp(bar_p_full + 8 * pb);
       PT_MARK(6)
     }
-    if (threadIdx.x == 0) { PT_FLUSH("attn softmax", nt) }
+    if (threadIdx.x == 0) { PT_FLUSH("attn softmax (wait S, load, max, exchange, exp, wait PV, arrive)", nt) }
     // epilogue: O / l -> out.  The row sum is the sum of both halves' partial sums.
     if (ok && nt > 0) ok = mbar_wait(bar_pv_done, (nt - 1) & 1, abort_flag, c.status);
     ok = __all_sync(0xffffffffu, ok);

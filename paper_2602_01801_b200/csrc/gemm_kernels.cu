@@ -108,17 +108,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   if (ntl > 0) {
     if (warp == kGemmProducerWarp) {
       // ------------------------------------------------------------------ TMA producer
-      if (lane == 0) {
-        bool ok = true;
-        if (A_RES) {
-          mbar_arrive_expect_tx(bar_afull, nkc * kChunkBytes);
-          for (int kc = 0; kc < nkc; ++kc) tma_load_3d(a_s + kc * kChunkBytes, &tm_a, bar_afull, kc * 64, m0, h);
+      // Page-table lookups are kept off the issue path: the warp fetches the page ids of 32 tiles with one
+      // coalesced load and lane 0 issues the copies from registers (a dependent global load between two TMA
+      // issues would cost about as much as the MMAs of the chunk).
+      bool ok = true;
+      if (A_RES && lane == 0) {
+        mbar_arrive_expect_tx(bar_afull, nkc * kChunkBytes);
+        for (int kc = 0; kc < nkc; ++kc) tma_load_3d(a_s + kc * kChunkBytes, &tm_a, bar_afull, kc * 64, m0, h);
+      }
+      const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+      const int pages_per_tile = 128 / c.PT;                     // 1 or 2
+      int it = 0;
+      int pg0 = 0, pg1 = 0;
+      for (int tl = 0; tl < ntl; ++tl) {
+        const int t = t0 + tl;
+        if (EPI == EPI_ARGMAX && (tl & 31) == 0 && tl + lane < ntl) {
+          pg0 = pt_h[(t + lane) * pages_per_tile];
+          pg1 = pages_per_tile == 2 ? pt_h[(t + lane) * pages_per_tile + 1] : 0;
         }
-        const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
-        const int pages_per_tile = 128 / c.PT;
-        int it = 0;
-        for (int tl = 0; tl < ntl && ok; ++tl) {
-          const int t = t0 + tl;
+        const int page0 = __shfl_sync(0xffffffffu, pg0, tl & 31);
+        const int page1 = __shfl_sync(0xffffffffu, pg1, tl & 31);
+        if (lane == 0 && ok) {
           for (int kc = 0; kc < nkc; ++kc, ++it) {
             const int s = it % NST;
             const uint32_t ph = (it / NST) & 1;
@@ -132,23 +142,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
               b_s = st_s + kChunkBytes;
             }
             if (EPI == EPI_ARGMAX) {
-              for (int pg = 0; pg < pages_per_tile; ++pg) {
-                const int page = pt_h[t * pages_per_tile + pg];
-                tma_load_3d(b_s + pg * c.PT * 128, &tm_b, bar_full + 8 * s, kc * 64, 0, page);
-              }
+              tma_load_3d(b_s, &tm_b, bar_full + 8 * s, kc * 64, 0, page0);
+              if (pages_per_tile == 2) tma_load_3d(b_s + c.PT * 128, &tm_b, bar_full + 8 * s, kc * 64, 0, page1);
             } else {
               tma_load_3d(b_s, &tm_b, bar_full + 8 * s, kc * 64, t * 128, h);
             }
           }
         }
-        // drain: let the loads still in flight land before the CTA may exit
-        const int issued = it;
-        for (int k = max(0, issued - NST); k < issued; ++k) {
-          // full barriers are consumed by the MMA warp in order; waiting on the last ones is
-          // enough and cheap.  Bounded like every other wait.
-          mbar_wait(bar_full + 8 * (k % NST), (k / NST) & 1, abort_flag, c.status);
-        }
       }
+      // drain: let the loads still in flight land before the CTA may exit.  Full barriers are consumed by the
+      // MMA warp in order; waiting on the last ones is enough and cheap.  Bounded like every other wait.
+      if (lane == 0)
+        for (int k = max(0, it - NST); k < it; ++k) mbar_wait(bar_full + 8 * (k % NST), (k / NST) & 1, abort_flag, c.status);
     } else if (warp == kGemmMmaWarp) {
       // ------------------------------------------------------------------ MMA issue
       if (lane == 0) {
