@@ -372,8 +372,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int q = 0; q < HB / 8; ++q) {
         float p[8];
 #pragma unroll
-        for (int t = 0; t < 8; ++t)                 // half on the MUFU unit, half as a polynomial on the FMA pipe
-          p[t] = (t & 1) ? poly_exp2(x[8 * q + t] - m_eff) : fast_exp2(x[8 * q + t] - m_eff);
+        for (int t = 0; t < 8; ++t) p[t] = fast_exp2(x[8 * q + t] - m_eff);
         l0 += p[0] + p[4];
         l1 += p[1] + p[5];
         l2 += p[2] + p[6];

@@ -229,33 +229,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           const int cc = wg * 2 + c2;
           const uint32_t(&v)[32] = vv[c2];
           if (EPI == EPI_ARGMAX) {
-            const float* rn = rn_s + buf * 128 + cc * 32;
-            const int jbase = t * 128 + cc * 32;
             // Scores of the chunk, then a tree maximum (no serial compare/select chain); the index is
             // searched only when the chunk holds a new strict maximum, which is rare after the first tiles.
-            float x[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(v[j]) * rn[j];
-            if (cc * 32 + 32 > valid_cols) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (cc * 32 + j >= valid_cols) x[j] = -INFINITY;
-            }
-            float m16[16], m8[8], m4[4];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) m16[j] = fmaxf(x[2 * j], x[2 * j + 1]);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) m8[j] = fmaxf(m16[2 * j], m16[2 * j + 1]);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) m4[j] = fmaxf(m8[2 * j], m8[2 * j + 1]);
-            const float cm = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-            if (cm > best) {
-              best = cm;
-              int idx = 31;
-#pragma unroll
-              for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;   // first (lowest) column of the maximum
-              best_j = jbase + idx;
-            }
+            chunk_argmax(v, reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
+                         t * 128 + cc * 32, best, best_j);
           } else if (EPI == EPI_COLMAX) {
             const bool rvalid = row < g.rows_a;
             const int f_r = rvalid ? row / g.frame_len : -1;
@@ -332,14 +309,15 @@ static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const C
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
+// T1.  A 256-row CTA tile (half the L2 traffic, one CTA per SM, sixteen epilogue warps) and an A-from-TMEM
+// variant were measured as well and were not faster (0.48 / 0.55 ms against 0.44 ms on the c1 workload): what
+// limits this kernel is moving the fp32 score tiles out of TMEM (64 KB per 128x128 tile, about as long as the
+// MMAs that produce them), not operand traffic.  Splits of the cache range fill whole waves of 2 CTAs per SM.
 int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k, int n, cudaStream_t st) {
   GemmArgs g{};
   g.rows_a = n;
   g.nkc = c.D / 64;
   const int row_tiles = (n + 127) / 128;
-  // enough CTAs to fill the machine a few times over; every split scans a contiguous slot range
-  // Split the cache range so that the CTA count fills whole waves of the resident slots (2 CTAs per SM):
-  // the smallest split whose last wave is at least 90 % full, else the best one found.
   int sm_count = 148;
   {
     int dev = 0;

@@ -88,15 +88,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-// Warp-wide bounded wait with a single poller: lane 0 waits, the result is broadcast (the shuffle is also the
-// warp barrier that orders the other lanes after the wait).  Keeps hundreds of threads from hammering the
-// barrier word while a whole warpgroup is idle.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
-  return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
 // ---------------------------------------------------------------------------------------------
 // proxy fences, named barriers
 // ---------------------------------------------------------------------------------------------
@@ -185,16 +176,6 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// A operand from TMEM (lane = row, each 32-bit column holds two consecutive K elements), B from shared memory.
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
-                                        uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 // Arrive on an mbarrier when all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -211,14 +192,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -267,18 +240,51 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// 2^x on the FMA/ALU pipes (no MUFU): round-to-nearest split x = r + f with the 1.5*2^23 trick, cubic for 2^f
-// on [-0.5, 0.5] (relative error < 7e-4, below bf16 resolution), r added into the exponent field.  Used for part
-// of the softmax exponentials so that the 16-per-clock MUFU unit is not the only path.
-__device__ __forceinline__ float poly_exp2(float x) {
-  x = fmaxf(x, -125.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(f, 0.0555041f, 0.2402265f);
-  p = fmaf(p, f, 0.6931472f);
-  p = fmaf(p, f, 1.0f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+// Three-input maximum and packed two-lane multiply (sm_100): they halve the instruction count of the arg-max
+// epilogue, which is issue-bound.
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
+__device__ __forceinline__ void fmul2(float& x0, float& x1, float a0, float a1, float b0, float b1) {
+  unsigned long long a, b, d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(b0), "f"(b1));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(d));
+}
+// Maximum of 32 scores x[j] = acc[j] * rn[j] and, only when it beats `best`, its first column.
+// acc: raw accumulator bits; rn: 32 floats (16-byte aligned, shared or registers via pointer).
+__device__ __forceinline__ void chunk_argmax(const uint32_t (&acc)[32], const float4* rn4, int valid, int jbase, float& best,
+                                             int& best_j) {
+  float x[32];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const float4 r = rn4[u];
+    fmul2(x[4 * u], x[4 * u + 1], __uint_as_float(acc[4 * u]), __uint_as_float(acc[4 * u + 1]), r.x, r.y);
+    fmul2(x[4 * u + 2], x[4 * u + 3], __uint_as_float(acc[4 * u + 2]), __uint_as_float(acc[4 * u + 3]), r.z, r.w);
+  }
+  if (valid < 32) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j >= valid) x[j] = -INFINITY;
+  }
+  float m[11];
+#pragma unroll
+  for (int j = 0; j < 10; ++j) m[j] = fmax3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
+  m[10] = fmaxf(x[30], x[31]);
+  const float a0 = fmax3(m[0], m[1], m[2]), a1 = fmax3(m[3], m[4], m[5]), a2 = fmax3(m[6], m[7], m[8]);
+  const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
+  if (cm > best) {
+    best = cm;
+    int idx = 31;
+#pragma unroll
+    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;   // first (lowest) column of the maximum
+    best_j = jbase + idx;
+  }
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
