@@ -139,6 +139,36 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_o = tmem + 2 * BKT;
 
+  // Gather mode with a single key tile (the usual AnnCA case, keep <= BKT): all threads fetch the kept rows
+  // of K_p and V_p at once, instead of leaving 2 x BKT x D x 2 bytes of 16-byte gathers to one warp.
+  bool prefilled = false;
+  if (GATHER && nt == 1) {
+    constexpr int CPR = D / 8;                         // 16-byte chunks per row
+    const __nv_bfloat16* kp_h = a.kp + static_cast<int64_t>(h) * a.p_head_stride;
+    const __nv_bfloat16* vp_h = a.vp + static_cast<int64_t>(h) * a.p_head_stride;
+    for (int q = threadIdx.x; q < 2 * BKT * CPR; q += blockDim.x) {
+      const int which = q / (BKT * CPR), qq = q % (BKT * CPR);
+      const int i = qq / CPR, ch = qq % CPR;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (i < a.keep) {
+        const int idx = list[i];
+        val = *reinterpret_cast<const uint4*>((which ? vp_h : kp_h) + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
+      }
+      const uint32_t off = which * SM::kv_bytes + (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(k_s + off), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w)
+                   : "memory");
+    }
+    for (int i = threadIdx.x; i < BKT; i += blockDim.x) bias_g[i] = (i < a.keep) ? 0.f : -INFINITY;
+    fence_proxy_async_smem();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      mbar_arrive(bar_r_full);                         // K0 -> stage 0
+      mbar_arrive(bar_r_full + 8);                     // V0 -> stage 1
+      mbar_arrive(bar_b_full);
+    }
+    prefilled = true;
+  }
+
   // K and V tiles share one ring of RS stages, filled and consumed in the order the MMA warp needs them:
   //   K0, K1, V0, K2, V1, K3, V2, ...   (S_{j+1} = Q K_{j+1}^T is issued before O += P_j V_j)
   // so a key tile can be requested as soon as the tile four positions earlier has been consumed, without
@@ -231,7 +261,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         ++it;
       };
-      if (nt > 0) {
+      if (nt > 0 && !prefilled) {
         fill_tile(true, 0);
         for (int j = 0; j < nt; ++j) {
           if (j + 1 < nt) fill_tile(true, j + 1);
