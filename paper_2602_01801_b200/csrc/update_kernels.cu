@@ -109,27 +109,32 @@ __global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restri
   for (int ks = 0; ks < KS; ++ks)
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
+      // The contraction index may be permuted freely as long as A and B agree: lane t of a quad reads 8
+      // contiguous elements (one 128-bit load) per 32-wide k block, k = 32*(ks/2) + 8t + 4*(ks%2) + {0,1 | 2,3}.
       const int col = 8 * nt + g;
-      const __nv_bfloat16* rp = lsh + col * D + 16 * ks + 2 * t;
+      const __nv_bfloat16* rp = lsh + col * D + 32 * (ks >> 1) + 8 * t + 4 * (ks & 1);
       bf[ks][nt][0] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp) : 0u;
-      bf[ks][nt][1] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp + 8) : 0u;
+      bf[ks][nt][1] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp + 2) : 0u;
     }
   for (int r0 = (blockIdx.x * 8 + warp) * 16; r0 < n; r0 += gridDim.x * 128) {
     const int ra = min(r0 + g, n - 1), rb = min(r0 + g + 8, n - 1);   // rows past the end repeat the last one
-    const __nv_bfloat16* xa = x + h * hs + ra * ts + 2 * t;
-    const __nv_bfloat16* xb = x + h * hs + rb * ts + 2 * t;
+    const __nv_bfloat16* xa = x + h * hs + ra * ts + 8 * t;
+    const __nv_bfloat16* xb = x + h * hs + rb * ts + 8 * t;
     float acc[4][4];
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
     float sqa = 0.f, sqb = 0.f;
+    uint4 va = make_uint4(0, 0, 0, 0), vb = va;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      const uint32_t a0 = *reinterpret_cast<const uint32_t*>(xa + 16 * ks);
-      const uint32_t a1 = *reinterpret_cast<const uint32_t*>(xb + 16 * ks);
-      const uint32_t a2 = *reinterpret_cast<const uint32_t*>(xa + 16 * ks + 8);
-      const uint32_t a3 = *reinterpret_cast<const uint32_t*>(xb + 16 * ks + 8);
+      if ((ks & 1) == 0) {                                // one 128-bit load per row and 32-wide k block
+        va = *reinterpret_cast<const uint4*>(xa + 32 * (ks >> 1));
+        vb = *reinterpret_cast<const uint4*>(xb + 32 * (ks >> 1));
+      }
+      const uint32_t a0 = (ks & 1) ? va.z : va.x, a2 = (ks & 1) ? va.w : va.y;
+      const uint32_t a1 = (ks & 1) ? vb.z : vb.x, a3 = (ks & 1) ? vb.w : vb.y;
       {
         const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a0));
         const float2 f2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a2));
