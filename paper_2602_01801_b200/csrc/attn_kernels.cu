@@ -6,13 +6,19 @@
 //   gather : AnnCA's attention over the kept prompt tokens of the query's frame; rows of K_p / V_p
 //            are gathered by index with 128-bit loads into the same swizzled tile layout.
 //
-// One CTA = 128 query rows (TMEM lanes).  Per key tile j:
-//   S_j = Q K_j^T        (tcgen05.mma, SMEM x SMEM -> TMEM, two S buffers)
-//   P_j = exp2(S_j*scale + log2 m - m_run)   (8 softmax warps: two threads per row, each owning half of
-//                                             the tile's columns in registers; bf16 P tile in SMEM)
-//   O  += P_j V_j        (tcgen05.mma, V is the MN-major operand straight from its [key][d] page)
-// with lazy rescaling of O (only when a row maximum grew by more than 2^8).
-// Warp roles: warps 0-7 softmax + epilogue, warp 8 producer (TMA or gather), warp 9 MMA issue.
+// One CTA = 128 query rows (TMEM lanes).  The key tiles are dealt alternately to two softmax groups
+// (g = j & 1, four warps each, one thread per row) that run a whole online softmax each, with their own
+// S buffer, P tile, running (max, sum) and O accumulator, and are combined once at the end (a split of the
+// key range inside the CTA).  While one group is in its exponentials the other is loading its logits from
+// TMEM, and the tensor core always has the next S or P.V to do:
+//   S_j = Q K_j^T                   tcgen05.mma, SMEM x SMEM -> TMEM buffer S[g]
+//   P_j = exp2(S_j*scale + log2 m - m_g)    thread r of group g: 128 logits in registers -> bf16 P[g] in SMEM
+//   O_g += P_j V_j                  tcgen05.mma, V is the MN-major operand straight from its [key][d] page
+//   O = (O_0 2^(m_0-m) + O_1 2^(m_1-m)) / (l_0 2^(m_0-m) + l_1 2^(m_1-m))
+// O_g is rescaled lazily (only when a row maximum grew by more than 2^8).
+// TMEM columns: S[0], S[1], O_0, O_1 (4 x 128 at d = 128).  K and V tiles share one TMA ring filled in the
+// order the MMA warp consumes them: K0 K1 | K2 V0 | K3 V1 | ...
+// Warp roles: warps 0-3 softmax group 0, warps 4-7 group 1, warp 8 producer (TMA or gather), warp 9 MMA issue.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -24,27 +30,24 @@ constexpr int kProducerWarp = 8, kMmaWarp = 9;
 
 template <int D, int BKT>
 struct AttnSmem {
-  static constexpr int KS = 2, VS = 2, NB = 4;
+  static constexpr int RS = 4, NB = 4;
   static constexpr int q_bytes = (D / 64) * kQChunk;
   static constexpr int kv_bytes = (D / 64) * BKT * 128;          // one K or V tile
   static constexpr int p_bytes = (BKT / 64) * kQChunk;           // one P tile (128 x BKT bf16)
   static constexpr int q_off = 0;
-  static constexpr int k_off = q_off + q_bytes;
-  static constexpr int v_off = k_off + KS * kv_bytes;
-  static constexpr int p_off = v_off + VS * kv_bytes;
+  static constexpr int ring_off = q_off + q_bytes;
+  static constexpr int p_off = ring_off + RS * kv_bytes;
   static constexpr int bias_off = p_off + 2 * p_bytes;
   static constexpr int bar_off = bias_off + NB * BKT * 4;
   static constexpr int total = bar_off + 256;
-  static constexpr int tmem_cols = (2 * BKT + D) <= 256 ? 256 : 512;
+  static constexpr int tmem_cols = (2 * BKT + 2 * D) <= 256 ? 256 : 512;
 };
 
-__device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
-  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+__device__ __forceinline__ void st_shared_f32x2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
-__device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void ld_shared_f32x2(uint32_t addr, float& a, float& b) {
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
 }
 
 template <int D, int BKT, bool GATHER>
@@ -52,9 +55,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const CacheView c, const AttnArgs a) {
   using SM = AttnSmem<D, BKT>;
-  constexpr int KS = SM::KS, VS = SM::VS, NB = SM::NB;
-  constexpr int HB = BKT / 2;           // key columns per softmax thread
-  constexpr int HD = D / 2;             // output columns per softmax thread
+  constexpr int RS = SM::RS, NB = SM::NB;
+  constexpr int HD = D / 2;             // output columns written by one thread in the epilogue
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t sbase = smem_u32(smem_raw);
   uint8_t* sgen = smem_raw;
@@ -63,23 +65,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     return;
   }
   const uint32_t q_s = sbase + SM::q_off;
-  const uint32_t k_s = sbase + SM::k_off;
+  const uint32_t ring_s = sbase + SM::ring_off;
   const uint32_t p_s = sbase + SM::p_off;
   float* bias_g = reinterpret_cast<float*>(sgen + SM::bias_off);
   const uint32_t bias_s = sbase + SM::bias_off;
   const uint32_t bar = sbase + SM::bar_off;
   const uint32_t bar_q_full = bar;
-  constexpr int RS = KS + VS;                        // K and V tiles share one ring
-  const uint32_t ring_s = k_s;
   const uint32_t bar_r_full = bar + 8;               // [RS]
   const uint32_t bar_r_empty = bar_r_full + 8 * RS;  // [RS]
   const uint32_t bar_b_full = bar_r_empty + 8 * RS;  // [NB]
-  const uint32_t bar_s_full = bar_b_full + 8 * NB;    // [2]
-  const uint32_t bar_s_empty = bar_s_full + 16;       // [2]
-  const uint32_t bar_p_full = bar_s_empty + 16;       // [2]
-  const uint32_t bar_pv_done = bar_p_full + 16;       // [1]
-  const uint32_t bar_xchg = bar_pv_done + 8;          // [1] row-max / row-sum exchange between the column halves
-  constexpr int kBarBytes = 8 + 16 * KS + 16 * VS + 8 * NB + 48 + 8 + 8;
+  const uint32_t bar_s_full = bar_b_full + 8 * NB;   // [2] per softmax group
+  const uint32_t bar_s_empty = bar_s_full + 16;      // [2]
+  const uint32_t bar_p_full = bar_s_empty + 16;      // [2]
+  const uint32_t bar_pv_done = bar_p_full + 16;      // [2]
+  const uint32_t bar_xchg = bar_pv_done + 16;        // [1] the two groups meet here before the epilogue
+  constexpr int kBarBytes = 8 + 16 * RS + 8 * NB + 64 + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + SM::bar_off + kBarBytes);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + SM::bar_off + kBarBytes + 4);
 
@@ -114,12 +114,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     mbar_init(bar_q_full, 1);
     for (int s = 0; s < RS; ++s) { mbar_init(bar_r_full + 8 * s, 1); mbar_init(bar_r_empty + 8 * s, 1); }
     for (int s = 0; s < NB; ++s) mbar_init(bar_b_full + 8 * s, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar_s_full + 8 * s, 1);
-      mbar_init(bar_s_empty + 8 * s, 8);       // one arrival per softmax warp
-      mbar_init(bar_p_full + 8 * s, 8);
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(bar_s_full + 8 * g, 1);
+      mbar_init(bar_s_empty + 8 * g, 4);       // one arrival per warp of the group
+      mbar_init(bar_p_full + 8 * g, 4);
+      mbar_init(bar_pv_done + 8 * g, 1);
     }
-    mbar_init(bar_pv_done, 1);
     mbar_init(bar_xchg, 8);
     *abort_flag = 0;
     fence_mbar_init();
@@ -137,7 +137,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_o = tmem + 2 * BKT;
+  const uint32_t tmem_o = tmem + 2 * BKT;            // O_0 at +0, O_1 at +D
 
   // Gather mode with a single key tile (the usual AnnCA case, keep <= BKT): all threads fetch the kept rows
   // of K_p and V_p at once, instead of leaving 2 x BKT x D x 2 bytes of 16-byte gathers to one warp.
@@ -155,7 +155,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         val = *reinterpret_cast<const uint4*>((which ? vp_h : kp_h) + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
       }
       const uint32_t off = which * SM::kv_bytes + (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(k_s + off), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w)
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_s + off), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w)
                    : "memory");
     }
     for (int i = threadIdx.x; i < BKT; i += blockDim.x) bias_g[i] = (i < a.keep) ? 0.f : -INFINITY;
@@ -169,10 +169,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     prefilled = true;
   }
 
-  // K and V tiles share one ring of RS stages, filled and consumed in the order the MMA warp needs them:
-  //   K0, K1, V0, K2, V1, K3, V2, ...   (S_{j+1} = Q K_{j+1}^T is issued before O += P_j V_j)
-  // so a key tile can be requested as soon as the tile four positions earlier has been consumed, without
-  // queueing behind a value tile whose stage frees late.
+  // Ring order, identical in the producer and in the MMA warp:
+  //   K0, K1, then for j = 0, 1, ...: K_{j+2} (if any), V_j
   if (warp == kProducerWarp) {
     // ================================================================== producer
     if (lane == 0 && nt > 0) {
@@ -185,11 +183,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       // block ids and page ids of 32 tiles at a time, one coalesced load each; lane 0 issues the copies
       const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
       const float* l2m_h = c.log2m + static_cast<int64_t>(h) * c.CAP;
-      int blk_l = 0, page_l = 0;
-      auto refill = [&](int j0) {
+      int blk_l = 0, page_l = 0;            // tiles [32w, 32w + 32) of the window in use
+      int blk_n = 0, page_n = 0;            // the following window (key tiles run two ahead of value tiles)
+      auto fetch = [&](int j0, int& blk, int& page) {
         if (j0 + lane < nt) {
-          blk_l = list ? list[j0 + lane] : j0 + lane;
-          page_l = pt_h[blk_l];
+          blk = list ? list[j0 + lane] : j0 + lane;
+          page = pt_h[blk];
         }
       };
       auto load_tile = [&](bool is_k, int j, int blk, int page) {
@@ -208,21 +207,27 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         ++it;
       };
       if (nt > 0) {
-        refill(0);
-        int blk_cur = __shfl_sync(0xffffffffu, blk_l, 0), page_cur = __shfl_sync(0xffffffffu, page_l, 0);
-        load_tile(true, 0, blk_cur, page_cur);
+        // two windows of 32 tiles: the low one holds the value tile in turn, key tiles may already need the next
+        fetch(0, blk_l, page_l);
+        fetch(32, blk_n, page_n);
+        auto get = [&](int j, int& blk, int& page, int base) {   // base = first tile of the low window
+          const bool hi = j >= base + 32;
+          blk = __shfl_sync(0xffffffffu, hi ? blk_n : blk_l, j & 31);
+          page = __shfl_sync(0xffffffffu, hi ? page_n : page_l, j & 31);
+        };
+        int base = 0, blk, page;
+        get(0, blk, page, base);
+        load_tile(true, 0, blk, page);
+        if (nt > 1) { get(1, blk, page, base); load_tile(true, 1, blk, page); }
         for (int j = 0; j < nt; ++j) {
-          if (j + 1 < nt) {
-            if (((j + 1) & 31) == 0) refill(j + 1);
-            const int blk_n = __shfl_sync(0xffffffffu, blk_l, (j + 1) & 31);
-            const int page_n = __shfl_sync(0xffffffffu, page_l, (j + 1) & 31);
-            load_tile(true, j + 1, blk_n, page_n);
-            load_tile(false, j, blk_cur, page_cur);
-            blk_cur = blk_n;
-            page_cur = page_n;
-          } else {
-            load_tile(false, j, blk_cur, page_cur);
+          if (j >= base + 32) {                                   // value tiles enter the next window
+            base += 32;
+            blk_l = blk_n; page_l = page_n;
+            fetch(base + 32, blk_n, page_n);
           }
+          if (j + 2 < nt) { get(j + 2, blk, page, base); load_tile(true, j + 2, blk, page); }
+          get(j, blk, page, base);
+          load_tile(false, j, blk, page);
         }
       }
     } else {
@@ -263,8 +268,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       };
       if (nt > 0 && !prefilled) {
         fill_tile(true, 0);
+        if (nt > 1) fill_tile(true, 1);
         for (int j = 0; j < nt; ++j) {
-          if (j + 1 < nt) fill_tile(true, j + 1);
+          if (j + 2 < nt) fill_tile(true, j + 2);
           fill_tile(false, j);
         }
       }
@@ -278,10 +284,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       int it = 0;                                       // position in the K/V ring (same order as the producer)
       PT_DECL
       auto issue_s = [&](int j) -> bool {
-        const int s = it % RS, sb = j & 1;
+        const int s = it % RS, g = j & 1, i = j >> 1;
         if (!mbar_wait(bar_r_full + 8 * s, (it / RS) & 1, abort_flag, c.status)) return false;
         PT_MARK(0)
-        if (!mbar_wait(bar_s_empty + 8 * sb, ((j >> 1) & 1) ^ 1, abort_flag, c.status)) return false;
+        // S[g] is free once group g holds the logits of its previous tile (j - 2) in registers
+        if (i > 0 && !mbar_wait(bar_s_empty + 8 * g, (i - 1) & 1, abort_flag, c.status)) return false;
         PT_MARK(1)
         tc_fence_after();
         const uint32_t kt = ring_s + s * SM::kv_bytes;
@@ -289,19 +296,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint64_t ad = make_smem_desc(q_s + (kk >> 2) * kQChunk + (kk & 3) * 32, 16, 1024);
           const uint64_t bd = make_smem_desc(kt + (kk >> 2) * (BKT * 128) + (kk & 3) * 32, 16, 1024);
-          umma_ss(tmem + sb * BKT, ad, bd, idesc_qk, kk != 0);
+          umma_ss(tmem + g * BKT, ad, bd, idesc_qk, kk != 0);
         }
         umma_commit(bar_r_empty + 8 * s);
-        umma_commit(bar_s_full + 8 * sb);
+        umma_commit(bar_s_full + 8 * g);
         ++it;
         PT_MARK(2)
         return true;
       };
       if (ok) ok = issue_s(0);
+      if (ok && nt > 1) ok = issue_s(1);
       for (int j = 0; j < nt && ok; ++j) {
-        if (j + 1 < nt) { ok = issue_s(j + 1); if (!ok) break; }
-        const int s = it % RS, pb = j & 1;
-        ok = mbar_wait(bar_p_full + 8 * pb, (j >> 1) & 1, abort_flag, c.status);
+        if (j + 2 < nt) { ok = issue_s(j + 2); if (!ok) break; }
+        const int s = it % RS, g = j & 1, i = j >> 1;
+        ok = mbar_wait(bar_p_full + 8 * g, i & 1, abort_flag, c.status);
         if (!ok) break;
         PT_MARK(3)
         ok = mbar_wait(bar_r_full + 8 * s, (it / RS) & 1, abort_flag, c.status);
@@ -309,57 +317,53 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         PT_MARK(4)
         tc_fence_after();
         const uint32_t vt = ring_s + s * SM::kv_bytes;
-        const uint32_t pt = p_s + pb * SM::p_bytes;
+        const uint32_t pt = p_s + g * SM::p_bytes;
 #pragma unroll
         for (int ks16 = 0; ks16 < BKT / 16; ++ks16) {
           const uint64_t ad = make_smem_desc(pt + (ks16 >> 2) * kQChunk + (ks16 & 3) * 32, 16, 1024);
           const uint64_t bd = make_smem_desc(vt + ks16 * 2048, BKT * 128, 1024);
-          umma_ss(tmem_o, ad, bd, idesc_pv, (j | ks16) != 0);
+          umma_ss(tmem_o + g * D, ad, bd, idesc_pv, (i | ks16) != 0);
         }
         umma_commit(bar_r_empty + 8 * s);
-        umma_commit(bar_pv_done);
+        umma_commit(bar_pv_done + 8 * g);
         ++it;
         PT_MARK(5)
       }
       PT_FLUSH("attn mma (wait K, wait S buffer, issue QK, wait P, wait V, issue PV)", nt)
     }
   } else {
-    // ================================================================== softmax + epilogue (256 threads)
-    const int wg = warp >> 2;                          // column half owned by this thread
-    const int r = (warp & 3) * 32 + lane;              // query row = TMEM lane
+    // ================================================================== softmax groups + epilogue (256 threads)
+    const int g = warp >> 2;                            // softmax group: key tiles j with (j & 1) == g
+    const int r = (warp & 3) * 32 + lane;               // query row = TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const float scale = rsqrtf(static_cast<float>(D)) * 1.4426950408889634f;
-    // First 16-byte chunk of each half of row r inside a P tile.  The two halves of a row exchange their
-    // partial row maximum through the *partner's* chunk: only the partner reads it, and only the partner
-    // overwrites it later with its own P data, so no extra buffer and no extra barrier are needed.
-    auto p_chunk_addr = [&](int pb, int ch) -> uint32_t {
-      return p_s + pb * SM::p_bytes + (ch >> 3) * kQChunk + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
-    };
-    const int my_ch0 = wg * (HB / 8), other_ch0 = (wg ^ 1) * (HB / 8);
+    const uint32_t s_t = tmem + lane_addr + g * BKT;
+    const uint32_t o_t = tmem_o + lane_addr + g * D;
+    const uint32_t p_row = p_s + g * SM::p_bytes + r * 128;
     float m_used = -INFINITY;
     float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-    uint32_t xphase = 0;
     bool ok = true;
+    const int n_mine = (nt - g + 1) >> 1;               // tiles of this group
     PT_DECL
-    for (int j = 0; j < nt && ok; ++j) {
-      const int sb = j & 1, pb = j & 1, b4 = j % NB;
+    for (int i = 0; i < n_mine && ok; ++i) {
+      const int j = 2 * i + g, b4 = j % NB;
       ok = mbar_wait(bar_b_full + 8 * b4, (j / NB) & 1, abort_flag, c.status) &&
-           mbar_wait(bar_s_full + 8 * sb, (j >> 1) & 1, abort_flag, c.status);
+           mbar_wait(bar_s_full + 8 * g, i & 1, abort_flag, c.status);
       ok = __all_sync(0xffffffffu, ok);          // TMEM loads below are warp-collective
       if (!ok) break;
       PT_MARK(0)
       tc_fence_after();
-      // this thread's half of the logits row, kept in registers
-      float x[HB];
+      // the whole logits row of this tile, kept in registers
+      float x[BKT];
       {
-        uint32_t v[HB];
+        uint32_t v[BKT];
 #pragma unroll
-        for (int cc = 0; cc < HB / 32; ++cc)
-          tmem_ld32(tmem + lane_addr + sb * BKT + wg * HB + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[cc * 32]));
+        for (int cc = 0; cc < BKT / 32; ++cc)
+          tmem_ld32(s_t + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[cc * 32]));
         tmem_wait_ld();
-        const float4* b4p = reinterpret_cast<const float4*>(bias_g + b4 * BKT + wg * HB);
+        const float4* b4p = reinterpret_cast<const float4*>(bias_g + b4 * BKT);
 #pragma unroll
-        for (int t = 0; t < HB / 4; ++t) {
+        for (int t = 0; t < BKT / 4; ++t) {
           const float4 bb = b4p[t];
           x[4 * t] = fmaf(__uint_as_float(v[4 * t]), scale, bb.x);
           x[4 * t + 1] = fmaf(__uint_as_float(v[4 * t + 1]), scale, bb.y);
@@ -367,39 +371,52 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           x[4 * t + 3] = fmaf(__uint_as_float(v[4 * t + 3]), scale, bb.w);
         }
       }
-      PT_MARK(1)
       tc_fence_before();
-      mbar_arrive_warp(bar_s_empty + 8 * sb);          // S and the bias are consumed
-      // row maximum: 4 independent chains, then across the two halves
+      mbar_arrive_warp(bar_s_empty + 8 * g);           // S[g] and the bias are consumed
+      PT_MARK(1)
+      // row maximum: independent chains of 3-input maxima
       float mx0 = x[0], mx1 = x[1], mx2 = x[2], mx3 = x[3];
 #pragma unroll
-      for (int t = 4; t < HB; t += 4) {
-        mx0 = fmaxf(mx0, x[t]);
-        mx1 = fmaxf(mx1, x[t + 1]);
-        mx2 = fmaxf(mx2, x[t + 2]);
-        mx3 = fmaxf(mx3, x[t + 3]);
+      for (int t = 4; t + 7 < BKT; t += 8) {
+        mx0 = fmax3(mx0, x[t], x[t + 4]);
+        mx1 = fmax3(mx1, x[t + 1], x[t + 5]);
+        mx2 = fmax3(mx2, x[t + 2], x[t + 6]);
+        mx3 = fmax3(mx3, x[t + 3], x[t + 7]);
       }
-      float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      st_shared_f32(p_chunk_addr(pb, other_ch0), mx);
-      PT_MARK(2)
-      mbar_arrive_warp(bar_xchg);
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_xchg, xphase, abort_flag, c.status));
-      xphase ^= 1;
-      if (!ok) break;
-      PT_MARK(3)
-      mx = fmaxf(mx, ld_shared_f32(p_chunk_addr(pb, my_ch0)));
+      mx0 = fmaxf(mx0, x[BKT - 4]); mx1 = fmaxf(mx1, x[BKT - 3]); mx2 = fmaxf(mx2, x[BKT - 2]); mx3 = fmaxf(mx3, x[BKT - 1]);
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       float alpha = 1.f;
       bool resc = false;
       if (mx > m_used + 8.f || (m_used == -INFINITY && mx > -INFINITY)) {
         alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
         l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
         m_used = mx;
-        resc = j > 0;
+        resc = i > 0;
       }
       const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
+      PT_MARK(2)
+      // P[g] and O_g are free once the group's previous P.V (tile j - 2) has completed
+      if (i > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + 8 * g, (i - 1) & 1, abort_flag, c.status));
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, resc)) {
+#pragma unroll 1
+          for (int cc = 0; cc < D / 32; ++cc) {
+            uint32_t v[32];
+            tmem_ld32(o_t + cc * 32, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) * alpha);
+            tmem_st32(o_t + cc * 32, v);
+          }
+          tmem_wait_st();
+        }
+      }
+      PT_MARK(3)
       // exponentials -> bf16 P (K-major, 128-byte swizzle); 4 independent row-sum chains
 #pragma unroll
-      for (int q = 0; q < HB / 8; ++q) {
+      for (int q = 0; q < BKT / 8; ++q) {
         float p[8];
 #pragma unroll
         for (int t = 0; t < 8; ++t) p[t] = fast_exp2(x[8 * q + t] - m_eff);
@@ -407,76 +424,64 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         l1 += p[1] + p[5];
         l2 += p[2] + p[6];
         l3 += p[3] + p[7];
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_chunk_addr(pb, my_ch0 + q)),
-                     "r"(pack_bf16x2(p[0], p[1])), "r"(pack_bf16x2(p[2], p[3])), "r"(pack_bf16x2(p[4], p[5])),
-                     "r"(pack_bf16x2(p[6], p[7]))
+        const uint32_t addr = p_row + (q >> 3) * kQChunk + (((q & 7) ^ (r & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16x2(p[0], p[1])),
+                     "r"(pack_bf16x2(p[2], p[3])), "r"(pack_bf16x2(p[4], p[5])), "r"(pack_bf16x2(p[6], p[7]))
                      : "memory");
       }
       PT_MARK(4)
-      if (j > 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done, (j - 1) & 1, abort_flag, c.status));
-        if (!ok) break;
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, resc)) {        // both halves of a row take the same decision
-#pragma unroll 1
-          for (int cc = 0; cc < HD / 32; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(tmem_o + lane_addr + wg * HD + cc * 32, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) * alpha);
-            tmem_st32(tmem_o + lane_addr + wg * HD + cc * 32, v);
-          }
-          tmem_wait_st();
-        }
-      }
-      PT_MARK(5)
       fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive_warp(bar_p_full + 8 * pb);
-      PT_MARK(6)
+      mbar_arrive_warp(bar_p_full + 8 * g);
+      PT_MARK(5)
     }
-    if (threadIdx.x == 0) { PT_FLUSH("attn softmax (wait S, load, max, exchange, exp, wait PV, arrive)", nt) }
-    // epilogue: O / l -> out.  The row sum is the sum of both halves' partial sums.
-    if (ok && nt > 0) ok = mbar_wait(bar_pv_done, (nt - 1) & 1, abort_flag, c.status);
+    if (threadIdx.x == 0) { PT_FLUSH("attn softmax group 0 (wait S, load, max, wait PV, exp, arrive)", n_mine) }
+    // ---- the two groups meet: (m, l) of every row through shared memory, then O = combination of O_0, O_1 ----
+    if (ok && n_mine > 0) ok = mbar_wait(bar_pv_done + 8 * g, (n_mine - 1) & 1, abort_flag, c.status);
     ok = __all_sync(0xffffffffu, ok);
-    float l_sum = (l0 + l1) + (l2 + l3);
-    if (ok && nt > 0) {
-      st_shared_f32(p_chunk_addr(0, other_ch0), l_sum);
-      mbar_arrive_warp(bar_xchg);
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_xchg, xphase, abort_flag, c.status));
-      if (ok) l_sum += ld_shared_f32(p_chunk_addr(0, my_ch0));
-    }
+    const float l_mine = (l0 + l1) + (l2 + l3);
+    // exchange area: the first bytes of P[g] (free: every P.V of this group has completed)
+    const uint32_t x_mine = p_s + g * SM::p_bytes + r * 8, x_other = p_s + (g ^ 1) * SM::p_bytes + r * 8;
+    if (ok) st_shared_f32x2(x_mine, m_used, l_mine);
+    tc_fence_after();                             // this group's last P.V is complete ...
+    tc_fence_before();                            // ... and the other group may read its accumulator after the barrier
+    mbar_arrive_warp(bar_xchg);
+    ok = ok && mbar_wait(bar_xchg, 0, abort_flag, c.status);
+    ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     const bool wr = r < valid_rows;               // loads are warp-collective, only the stores are per row
     if (ok) {
-      const float inv = (nt > 0 && l_sum > 0.f) ? 1.f / l_sum : 0.f;
-      const int64_t off = static_cast<int64_t>(h) * a.out_head_stride + static_cast<int64_t>(q0 + r) * a.out_token_stride + wg * HD;
+      float m_o, l_o;
+      ld_shared_f32x2(x_other, m_o, l_o);
+      const float m_all = fmaxf(m_used, m_o);
+      const float a_mine = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_all);
+      const float a_oth = (m_o == -INFINITY) ? 0.f : fast_exp2(m_o - m_all);
+      const float denom = l_mine * a_mine + l_o * a_oth;
+      const float inv = denom > 0.f ? 1.f / denom : 0.f;
+      const float w0 = (g == 0 ? a_mine : a_oth) * inv, w1 = (g == 0 ? a_oth : a_mine) * inv;   // weights of O_0, O_1
+      const bool has0 = nt > 0, has1 = nt > 1;    // O_1 was never written when there is a single tile
+      const int64_t off = static_cast<int64_t>(h) * a.out_head_stride + static_cast<int64_t>(q0 + r) * a.out_token_stride + g * HD;
 #pragma unroll 1
       for (int cc = 0; cc < HD / 32; ++cc) {
-        uint32_t v[32];
-        if (nt > 0) {
-          tmem_ld32(tmem_o + lane_addr + wg * HD + cc * 32, v);
-          tmem_wait_ld();
-        } else {
+        uint32_t v0[32], v1[32];
+        if (has0) tmem_ld32(tmem_o + lane_addr + g * HD + cc * 32, v0);
+        if (has1) tmem_ld32(tmem_o + lane_addr + D + g * HD + cc * 32, v1);
+        if (has0) tmem_wait_ld();
+        float o[32];
 #pragma unroll
-          for (int t = 0; t < 32; ++t) v[t] = 0;
-        }
+        for (int t = 0; t < 32; ++t)
+          o[t] = (has0 ? __uint_as_float(v0[t]) * w0 : 0.f) + (has1 ? __uint_as_float(v1[t]) * w1 : 0.f);
         if (!wr) continue;
         if (a.out_fp32) {
           float4* dst = reinterpret_cast<float4*>(static_cast<float*>(a.out) + off + cc * 32);
 #pragma unroll
-          for (int t = 0; t < 8; ++t)
-            dst[t] = make_float4(__uint_as_float(v[4 * t]) * inv, __uint_as_float(v[4 * t + 1]) * inv,
-                                 __uint_as_float(v[4 * t + 2]) * inv, __uint_as_float(v[4 * t + 3]) * inv);
+          for (int t = 0; t < 8; ++t) dst[t] = make_float4(o[4 * t], o[4 * t + 1], o[4 * t + 2], o[4 * t + 3]);
         } else {
           uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(a.out) + off + cc * 32);
 #pragma unroll
           for (int t = 0; t < 4; ++t)
-            dst[t] = make_uint4(pack_bf16x2(__uint_as_float(v[8 * t]) * inv, __uint_as_float(v[8 * t + 1]) * inv),
-                                pack_bf16x2(__uint_as_float(v[8 * t + 2]) * inv, __uint_as_float(v[8 * t + 3]) * inv),
-                                pack_bf16x2(__uint_as_float(v[8 * t + 4]) * inv, __uint_as_float(v[8 * t + 5]) * inv),
-                                pack_bf16x2(__uint_as_float(v[8 * t + 6]) * inv, __uint_as_float(v[8 * t + 7]) * inv));
+            dst[t] = make_uint4(pack_bf16x2(o[8 * t], o[8 * t + 1]), pack_bf16x2(o[8 * t + 2], o[8 * t + 3]),
+                                pack_bf16x2(o[8 * t + 4], o[8 * t + 5]), pack_bf16x2(o[8 * t + 6], o[8 * t + 7]));
         }
       }
     }

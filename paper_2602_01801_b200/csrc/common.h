@@ -80,7 +80,10 @@ inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int
 // Each returns the number of kernels it launched (for the launch counter) or a negative status.
 
 // gemm_kernels.cu
-int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k, int n, cudaStream_t st);int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,
+// tm_pool_k: one page per box; tm_pool_k_half: 64 key rows per box (what one CTA of a pair fetches)
+int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k,
+                         const CUtensorMap& tm_pool_k_half, int n, cudaStream_t st);
+int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,
                         int n_frames, cudaStream_t st);
 int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtensorMap& tm_hk, int nqb, cudaStream_t st);
 

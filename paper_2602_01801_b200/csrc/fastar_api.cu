@@ -21,7 +21,7 @@ struct fastar_cache {
   std::vector<ProfRec> recs;
   fastar_cache_desc desc;
   CacheView v;
-  CUtensorMap tm_pool_k, tm_pool_v, tm_hq, tm_hk;
+  CUtensorMap tm_pool_k, tm_pool_k_half, tm_pool_v, tm_hq, tm_hk;
   PFN_cuTensorMapEncodeTiled_v12000 encode;
   int64_t launches;
   size_t bytes;
@@ -209,6 +209,7 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
   const CacheView& v = c->v;
   const uint64_t D = v.D, PT = v.PT;
   int r = make_map(c, &c->tm_pool_k, v.pool_k, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, v.PT);
+  if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_k_half, v.pool_k, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, 64);
   if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_v, v.pool_v, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, v.PT);
   if (r == FASTAR_OK)
     r = make_map(c, &c->tm_hq, v.hq, v.hist_cols, v.max_qb, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
@@ -323,7 +324,7 @@ int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_
   // packed arg-max words and per-slot match counts start at zero (adjacent in the workspace: one memset)
   if (cudaMemsetAsync(v.best, 0, reinterpret_cast<uint8_t*>(v.cnt) - reinterpret_cast<uint8_t*>(v.best) + static_cast<size_t>(v.H) * v.CAP * 4, st) != cudaSuccess)
     return FASTAR_ERR_CUDA;
-  ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, n, st));
+  ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
   ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
   ACCK(FASTAR_K_COMMIT, launch_commit(v, kb, vb, n, frame_len, khs, kts, st));
   ACCK(FASTAR_K_KEY_HIST, launch_finalize_hist(v, stats_out, 1, st));

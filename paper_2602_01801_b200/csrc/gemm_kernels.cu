@@ -11,6 +11,9 @@
 #include "common.h"
 #include "ptx.cuh"
 
+#include <cstdlib>
+#include <cstring>
+
 namespace fastar {
 
 enum { EPI_ARGMAX = 0, EPI_COLMAX = 1, EPI_STORE = 2 };
@@ -201,6 +204,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
       float best = -INFINITY;
       int best_j = -1;
+      float rn_next = 0.f;                           // 1/|k| of the next tile's keys, loaded one tile ahead
       bool ok = true;
       PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
@@ -209,8 +213,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         int valid_cols = 128;
         if (EPI == EPI_ARGMAX) {
           if (wg == 0) {
-            const int slot = t * 128 + r;
-            rn_s[buf * 128 + r] = slot < L ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+            if (tl == 0) rn_next = (t * 128 + r < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r] : 0.f;
+            rn_s[buf * 128 + r] = rn_next;
+            const int slot = (t + 1) * 128 + r;
+            rn_next = (tl + 1 < ntl && slot < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
           }
           valid_cols = min(128, L - t * 128);
           named_barrier_sync(1, 256);
@@ -223,6 +229,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         tmem_ld32(tmem + lane_addr + buf * 128 + wg * 64, vv[0]);
         tmem_ld32(tmem + lane_addr + buf * 128 + wg * 64 + 32, vv[1]);
         tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive_warp(bar_tempty + 8 * buf);      // the scores are in registers: release the accumulator
         PT_MARK(1)
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
@@ -272,9 +280,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           }
         }
         PT_MARK(2)
-        tc_fence_before();
-        mbar_arrive_warp(bar_tempty + 8 * buf);
-        PT_MARK(3)
       }
       if (threadIdx.x == 0) { PT_FLUSH("gemm epilogue (wait acc, tmem loads, compute, arrive)", ntl) }
       if (EPI == EPI_ARGMAX && ok && row < g.rows_a && best_j >= 0) {
@@ -309,31 +314,287 @@ static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const C
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
-// T1.  A 256-row CTA tile (half the L2 traffic, one CTA per SM, sixteen epilogue warps) and an A-from-TMEM
-// variant were measured as well and were not faster (0.48 / 0.55 ms against 0.44 ms on the c1 workload): what
-// limits this kernel is moving the fp32 score tiles out of TMEM (64 KB per 128x128 tile, about as long as the
-// MMAs that produce them), not operand traffic.  Splits of the cache range fill whole waves of 2 CTAs per SM.
-int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k, int n, cudaStream_t st) {
+// ---------------------------------------------------------------------------------------------
+// T1 on CTA pairs (tcgen05 cta_group::2)
+// ---------------------------------------------------------------------------------------------
+// What paces the single-CTA kernel is shared-memory bandwidth: a 128 x 128 x 16 MMA reads 4 KB of A and 4 KB of B
+// while TMA writes the next 4 KB of B, about 12 KB per MMA at roughly 100 bytes per clock.  Two CTAs on the two
+// SMs of a TPC run one 256-row MMA instead: each keeps its own 128 rows of A, fetches only half of the key rows
+// of every B chunk (8 KB) and the tensor cores exchange the halves, so a CTA moves 8 KB per MMA.  The even CTA
+// of the pair issues; its `full`, `a_full` and `tmem_empty` barriers count the TMA bytes and epilogue arrivals
+// of both CTAs, and it signals `empty` and `tmem_full` in both with one multicast commit.  Each CTA runs its own
+// epilogue on its own 128 accumulator rows.  Two pairs are resident per TPC (2 CTAs per SM, 256 TMEM columns each).
+constexpr int kPairStages = 6;
+
+struct PairSmem {
+  static constexpr int a_bytes = 2 * kChunkBytes;               // 128 rows x up to 2 chunks of 64 columns
+  static constexpr int stage_bytes = kChunkBytes / 2;           // 64 key rows x 64 columns
+  static constexpr int ring_off = a_bytes;
+  static constexpr int rn_off = ring_off + kPairStages * stage_bytes;
+  static constexpr int bar_off = rn_off + 2 * 128 * 4;
+  static constexpr int total = bar_off + 256;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 2)
+t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b_half, const CacheView c,
+               const GemmArgs g) {
+  using SM = PairSmem;
+  constexpr int NST = kPairStages;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t sbase = smem_u32(smem_raw);
+  uint8_t* sgen = smem_raw;
+  const bool aligned = (sbase & 1023u) == 0;          // same in both CTAs of a pair (same kernel, same layout)
+  const uint32_t a_s = sbase;
+  const uint32_t ring_s = sbase + SM::ring_off;
+  float* rn_s = reinterpret_cast<float*>(sgen + SM::rn_off);
+  const uint32_t bar_s = sbase + SM::bar_off;
+  const uint32_t bar_full = bar_s;                   // [NST]  used in the even CTA: bytes of both halves
+  const uint32_t bar_empty = bar_s + 8 * NST;        // [NST]  in each CTA: multicast commit
+  const uint32_t bar_tfull = bar_s + 16 * NST;       // [2]    in each CTA: multicast commit
+  const uint32_t bar_tempty = bar_tfull + 16;        // [2]    used in the even CTA: 8 epilogue warps of each CTA
+  const uint32_t bar_afull = bar_tempty + 16;        // [1]    used in the even CTA: A of both CTAs
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + SM::bar_off + 16 * NST + 40);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + SM::bar_off + 16 * NST + 44);
+  static_assert(16 * NST + 48 <= 256, "barrier area");
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();            // 0: issues the MMAs, 1: its peer
+  const int h = blockIdx.y;
+  const int m0 = blockIdx.x * 128;
+  const int L = c.len[h];
+
+  const int n_tiles = (L + 127) >> 7;
+  const int per = (n_tiles + gridDim.z - 1) / gridDim.z;
+  const int t0 = blockIdx.z * per;
+  const int ntl = aligned ? max(0, min(n_tiles, t0 + per) - t0) : 0;
+  const int nkc = g.nkc;
+  if (!aligned && threadIdx.x == 0) record_status(c.status, FASTAR_ERR_CUDA);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NST; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8 * b, 1);
+      mbar_init(bar_tempty + 8 * b, 16);
+    }
+    mbar_init(bar_afull, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == kGemmProducerWarp && lane == 0) {
+    tma_prefetch_desc(&tm_a);
+    tma_prefetch_desc(&tm_b_half);
+  }
+  __syncthreads();
+  if (warp == kGemmMmaWarp) {
+    tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  // both CTAs' barriers are initialised and both have their TMEM columns before either touches the other
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  // barriers of the even CTA, addressed from either CTA
+  const uint32_t lead_full = map_to_cta(bar_full, 0);
+  const uint32_t lead_tempty = map_to_cta(bar_tempty, 0);
+  const uint32_t lead_afull = map_to_cta(bar_afull, 0);
+
+  if (ntl > 0) {
+    if (warp == kGemmProducerWarp) {
+      // ------------------------------------------------------------------ TMA producer (both CTAs)
+      bool ok = true;
+      if (lane == 0) {
+        if (rank == 0) mbar_arrive_expect_tx(bar_afull, 2 * nkc * kChunkBytes);
+        for (int kc = 0; kc < nkc; ++kc) tma_load_3d_pair(a_s + kc * kChunkBytes, &tm_a, lead_afull, kc * 64, m0, h);
+      }
+      // this CTA's 64 key rows of tile t: page and row offset inside the page
+      const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+      const int pages_per_tile = 128 / c.PT;                     // 1 or 2
+      const int page_sel = (static_cast<int>(rank) * 64) / c.PT;  // which page of the tile
+      const int row_off = (static_cast<int>(rank) * 64) % c.PT;   // first row inside that page
+      int it = 0;
+      int pg = 0;
+      for (int tl = 0; tl < ntl; ++tl) {
+        const int t = t0 + tl;
+        if ((tl & 31) == 0 && tl + lane < ntl) pg = pt_h[(t + lane) * pages_per_tile + page_sel];
+        const int page = __shfl_sync(0xffffffffu, pg, tl & 31);
+        if (lane == 0 && ok) {
+          for (int kc = 0; kc < nkc; ++kc, ++it) {
+            const int s = it % NST;
+            ok = mbar_wait(bar_empty + 8 * s, ((it / NST) & 1) ^ 1, abort_flag, c.status);
+            if (!ok) break;
+            if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * s, 2 * SM::stage_bytes);
+            tma_load_3d_pair(ring_s + s * SM::stage_bytes, &tm_b_half, lead_full + 8 * s, kc * 64, row_off, page);
+          }
+        }
+      }
+    } else if (warp == kGemmMmaWarp) {
+      // ------------------------------------------------------------------ MMA issue (even CTA only)
+      if (lane == 0 && rank == 0) {
+        constexpr uint32_t idesc = make_idesc_bf16(256, 128, 0);
+        bool ok = mbar_wait(bar_afull, 0, abort_flag, c.status);
+        int it = 0;
+        PT_DECL
+        for (int tl = 0; tl < ntl && ok; ++tl) {
+          const int buf = tl & 1;
+          ok = mbar_wait(bar_tempty + 8 * buf, ((tl >> 1) & 1) ^ 1, abort_flag, c.status);
+          if (!ok) break;
+          PT_MARK(0)
+          tc_fence_after();
+          const uint32_t d_t = tmem + buf * 128;
+          for (int kc = 0; kc < nkc; ++kc, ++it) {
+            const int s = it % NST;
+            ok = mbar_wait(bar_full + 8 * s, (it / NST) & 1, abort_flag, c.status);
+            if (!ok) break;
+            PT_MARK(1)
+            tc_fence_after();
+            const uint32_t a_c = a_s + kc * kChunkBytes;
+            const uint32_t b_c = ring_s + s * SM::stage_bytes;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+              const uint64_t ad = make_smem_desc(a_c + k4 * 32, 16, 1024);
+              const uint64_t bd = make_smem_desc(b_c + k4 * 32, 16, 1024);
+              umma_ss_pair(d_t, ad, bd, idesc, (kc | k4) != 0);
+            }
+            umma_commit_pair(bar_empty + 8 * s);
+            PT_MARK(2)
+          }
+          if (ok) umma_commit_pair(bar_tfull + 8 * buf);
+        }
+        PT_FLUSH("t1 pair mma (wait tmem, wait smem, issue)", ntl)
+      }
+    } else {
+      // ------------------------------------------------------------------ epilogue (256 threads, both CTAs)
+      const int wg = warp >> 2;
+      const int r = (warp & 3) * 32 + lane;         // A row inside the tile = TMEM lane
+      const int row = m0 + r;
+      const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      float best = -INFINITY;
+      int best_j = -1;
+      bool ok = true;
+      // 1/|k| of the tile's cache keys goes through shared memory; the global load runs one tile ahead so that its
+      // latency is not paid between two tiles
+      const float* rn_h = c.rnorm + static_cast<int64_t>(h) * c.CAP;
+      float rn_next = (wg == 0 && t0 * 128 + r < L) ? rn_h[t0 * 128 + r] : 0.f;
+      PT_DECL
+      for (int tl = 0; tl < ntl && ok; ++tl) {
+        const int t = t0 + tl;
+        const int buf = tl & 1;
+        if (wg == 0) {
+          rn_s[buf * 128 + r] = rn_next;
+          const int slot = (t + 1) * 128 + r;
+          rn_next = (tl + 1 < ntl && slot < L) ? rn_h[slot] : 0.f;
+        }
+        const int valid_cols = min(128, L - t * 128);
+        named_barrier_sync(1, 256);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
+        if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
+        PT_MARK(0)
+        tc_fence_after();
+        uint32_t vv[2][32];
+        const uint32_t acc = tmem + lane_addr + buf * 128 + wg * 64;
+        tmem_ld32(acc, vv[0]);
+        tmem_ld32(acc + 32, vv[1]);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {                             // the scores are in registers: release the accumulator
+          if (rank == 0) mbar_arrive(bar_tempty + 8 * buf);
+          else mbar_arrive_cluster(lead_tempty + 8 * buf);
+        }
+        PT_MARK(1)
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+          const int cc = wg * 2 + c2;
+          chunk_argmax(vv[c2], reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
+                       t * 128 + cc * 32, best, best_j);
+        }
+        PT_MARK(2)
+      }
+      if (threadIdx.x == 0 && rank == 0) { PT_FLUSH("t1 pair epilogue (wait acc, tmem loads, compute)", ntl) }
+      if (ok && row < g.rows_a && best_j >= 0) {
+        const float sim = best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
+                                       static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
+        atomicMax(c.best + static_cast<int64_t>(h) * c.max_tokens + row, key);
+      }
+    }
+  }
+
+  // Neither CTA may leave while the other can still read its shared memory, write its TMEM or signal its barriers.
+  // Every load of either CTA has landed by then: the last accumulator was committed after the MMAs that read them.
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (warp == kGemmMmaWarp) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem, kTmemCols);
+  }
+}
+
+static int launch_t1_pair(const CUtensorMap& tm_a, const CUtensorMap& tm_b_half, const CacheView& c, const GemmArgs& g,
+                          dim3 grid, cudaStream_t st) {
+  auto kern = t1_pair_kernel;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::total) != cudaSuccess)
+      return FASTAR_ERR_CUDA;
+    configured = true;
+  }
+  kern<<<grid, kGemmThreads, PairSmem::total, st>>>(tm_a, tm_b_half, c, g);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// Number of splits of the key range that fills whole waves of `slots` resident CTAs best (first one reaching 90 %),
+// and that efficiency.
+static int pick_splits(int ctas_per_split, int slots, int max_splits, double* eff_out) {
+  int splits = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= 16 && s <= max_splits; ++s) {
+    const int total = ctas_per_split * s;
+    const double eff = static_cast<double>(total) / (static_cast<double>((total + slots - 1) / slots) * slots);
+    if (eff > best_eff + 1e-9) { best_eff = eff; splits = s; }
+    if (eff >= 0.9) break;
+  }
+  *eff_out = best_eff;
+  return splits;
+}
+
+// T1.  Two kernels: single CTAs of 128 rows, and CTA pairs (256 rows, half the operand traffic per SM).  The pair
+// kernel is the faster one when both fill their waves equally well (about 10 % at 16k new keys against a 130k-key
+// cache); with few row tiles the padding to an even tile count and the coarser grid can cost more than it gains, so
+// the launcher compares the wave efficiencies.  FASTAR_T1_KERNEL=single|pair in the environment forces one (tests).
+int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k,
+                         const CUtensorMap& tm_pool_k_half, int n, cudaStream_t st) {
   GemmArgs g{};
   g.rows_a = n;
   g.nkc = c.D / 64;
-  const int row_tiles = (n + 127) / 128;
   int sm_count = 148;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
-  const int slots = 2 * sm_count;
+  const int slots = 2 * sm_count;                      // both kernels run 2 CTAs per SM
   const int max_tiles = c.CAP / 128;
-  int splits = 1;
-  double best_eff = 0.0;
-  for (int s = 1; s <= 16 && s <= max_tiles; ++s) {
-    const int total = row_tiles * c.H * s;
-    const double eff = static_cast<double>(total) / (static_cast<double>((total + slots - 1) / slots) * slots);
-    if (eff > best_eff + 1e-9) { best_eff = eff; splits = s; }
-    if (eff >= 0.9) break;
+  const int tiles_single = (n + 127) / 128;
+  const int tiles_pair = 2 * ((n + 255) / 256);        // an even number of 128-row tiles
+  double eff_single = 0.0, eff_pair = 0.0;
+  const int splits_single = pick_splits(tiles_single * c.H, slots, max_tiles, &eff_single);
+  const int splits_pair = pick_splits(tiles_pair * c.H, slots, max_tiles, &eff_pair);
+  // useful fraction of the pair grid: padded tiles do no useful work
+  eff_pair *= static_cast<double>(tiles_single) / tiles_pair;
+  bool use_pair = eff_pair >= 0.96 * eff_single;
+  if (const char* force = std::getenv("FASTAR_T1_KERNEL")) {
+    if (std::strcmp(force, "pair") == 0) use_pair = true;
+    else if (std::strcmp(force, "single") == 0) use_pair = false;
   }
-  return launch_gemm<EPI_ARGMAX, true, 4>(tm_a, tm_pool_k, c, g, dim3(row_tiles, c.H, splits), st);
+  if (use_pair) return launch_t1_pair(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st);
+  return launch_gemm<EPI_ARGMAX, true, 4>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st);
 }
 
 int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,

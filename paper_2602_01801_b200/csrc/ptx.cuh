@@ -181,6 +181,66 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// ---------------------------------------------------------------------------------------------
+// CTA pairs (cluster of two CTAs on the two SMs of a TPC, tcgen05 cta_group::2)
+// ---------------------------------------------------------------------------------------------
+// One MMA spans both SMs: each CTA supplies its own 128 rows of A and half of the rows of B from its own shared
+// memory (same offsets in both CTAs) and receives its 128 rows of D in its own TMEM.  The even CTA of the pair
+// issues the MMAs; barriers that it waits on collect arrivals and TMA bytes from both CTAs.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// arrive on a barrier given by its shared::cluster address (this CTA's or the peer's)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// 3-D tiled load into this CTA's shared memory whose bytes are counted on a barrier given by its shared::cluster
+// address (the issuing CTA's barrier of the pair).  Every CTA fetches its own tile.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst_smem, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1,
+                                                 int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// TMEM allocation for a pair: the same warp of both CTAs executes these; both get the same columns.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[256 x N] (+)= A[256 x 16] * B[N x 16]^T over the pair; issued by one thread of the even CTA.
+__device__ __forceinline__ void umma_ss_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on the barrier at this shared-memory offset in both CTAs of the pair when the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(mask)
+               : "memory");
+}
+
 // 32 lanes x 32 consecutive 32-bit columns: thread t of the warp gets lane (32*(warp%4) + t).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -211,13 +271,20 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 // cycles each role spent between marks, per loop iteration.  For finding where a tile's time goes.
 // ---------------------------------------------------------------------------------------------
 #ifdef FASTAR_PHASE_TIMING
-#define PT_DECL long long pt_t = clock64(); long long pt_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+__device__ __forceinline__ unsigned long long pt_globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define PT_DECL long long pt_t = clock64(); const long long pt_c0 = pt_t; const unsigned long long pt_g0 = pt_globaltimer(); \
+  long long pt_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #define PT_MARK(i) { const long long n__ = clock64(); pt_acc[i] += n__ - pt_t; pt_t = n__; }
 #define PT_FLUSH(name, iters)                                                                                        \
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iters) > 0)                                          \
-    printf("%s: per-iteration cycles %lld %lld %lld %lld %lld %lld %lld %lld (iterations %d)\n", name,               \
+    printf("%s: per-iteration cycles %lld %lld %lld %lld %lld %lld %lld %lld (iterations %d) total %lld cycles %llu ns\n", name, \
            pt_acc[0] / (iters), pt_acc[1] / (iters), pt_acc[2] / (iters), pt_acc[3] / (iters), pt_acc[4] / (iters),  \
-           pt_acc[5] / (iters), pt_acc[6] / (iters), pt_acc[7] / (iters), static_cast<int>(iters));
+           pt_acc[5] / (iters), pt_acc[6] / (iters), pt_acc[7] / (iters), static_cast<int>(iters),                   \
+           static_cast<long long>(clock64() - pt_c0), pt_globaltimer() - pt_g0);
 #else
 #define PT_DECL
 #define PT_MARK(i)

@@ -117,6 +117,19 @@ def test_other_tile_shapes(d, pt):
     full_step(cfg)
 
 
+@pytest.mark.parametrize("kernel", ["single", "pair"])
+@pytest.mark.parametrize("d,pt", [(128, 128), (64, 64)])
+def test_both_similarity_kernels(kernel, d, pt, monkeypatch):
+    # The launcher picks the single-CTA or the CTA-pair similarity kernel from the grid's wave efficiency; force each
+    # one in turn so that both are checked against the oracle (ragged row tiles, ragged cache lengths, two updates).
+    monkeypatch.setenv("FASTAR_T1_KERNEL", kernel)
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    cache, w, heads, post, _, _ = full_step(cfg)
+    Q, K, V = w.chunk(cfg.prior_chunks + 1)
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
+    assert post["count"].max() > 1
+
+
 def test_dense_mode_equals_eq1_on_uncompressed_cache():
     cfg = synth.small_config(prior_chunks=2)
     w = synth.Workload(cfg)
