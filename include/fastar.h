@@ -21,7 +21,8 @@
  *     void* (0 = the legacy default stream).  All work is enqueued on that stream and the
  *     call returns without synchronising unless stated otherwise.
  *   - Ownership: the caller owns every tensor and the workspace buffer; the library owns only
- *     the small host object behind fastar_cache_t.  Nothing here allocates device memory.
+ *     the small host object behind fastar_cache_t (with a CUDA stream and three events created and
+ *     destroyed with it).  Nothing here allocates device memory.
  *   - Tensors are [head][token][channel] with element strides `head_stride`, `token_stride`
  *     (channel stride 1).  Strides in bytes must be multiples of 16 and base pointers 16-byte
  *     aligned (TMA requirement).  Element type is the cache's `dtype`: bf16, or fp32 which is
@@ -152,7 +153,10 @@ int fastar_annsa_attention(fastar_cache_t* cache, const void* q, void* out, int3
  *   r[f][p] = max_i q_i.k_p/sqrt(d); keep the min(keep_tokens, np) prompt tokens with the
  *   largest r (ties: lower p); o_i = softmax over the kept p of q_i.k_p/sqrt(d), times v_p.
  * The cache object only supplies H, d, dtype, scratch and the status word; its contents are
- * not touched.  q, out: dev [H][nq][d]; k_prompt, v_prompt: dev [H][np][d] with their own strides.
+ * not touched, and the scratch it uses is its own.  One AnnCA call may therefore run on another
+ * stream at the same time as an update or an AnnSA call of the same cache (the step's three calls
+ * are otherwise issued on one stream, or ordered by the caller; two calls of the same kind never
+ * overlap).  q, out: dev [H][nq][d]; k_prompt, v_prompt: dev [H][np][d] with their own strides.
  * Optional dev outputs: sel_out [H][F][keep_tokens] (ascending), rel_out [H][F][np] fp32.
  * sel_in bypasses the selection.  np <= max_prompt_tokens (<= 1024), F <= max_frames. */
 int fastar_annca_attention(fastar_cache_t* cache, const void* q, const void* k_prompt, const void* v_prompt,
@@ -164,7 +168,10 @@ int fastar_annca_attention(fastar_cache_t* cache, const void* q, const void* k_p
 /* One whole attention step with HOST tensors (contiguous [H][n][d] / [H][np][d], cache dtype):
  * copies the inputs to the device, runs update -> AnnSA -> AnnCA (same arguments as above, the
  * chunk's n tokens being both the new keys/values and the queries), copies both outputs back and
- * synchronises the stream.  Staging buffers live in the workspace. */
+ * synchronises the stream.  Staging buffers live in the workspace.  The uploads of q and of the
+ * prompt, AnnCA and the download of its output run on a second stream owned by the cache object,
+ * beside the update; that stream starts after the work already queued on `stream` and is idle
+ * again when the call returns. */
 int fastar_attention_step_host(fastar_cache_t* cache, const void* k_new_host, const void* v_new_host,
                                const void* q_host, const void* k_prompt_host, const void* v_prompt_host,
                                void* out_sa_host, void* out_ca_host, int32_t n, int32_t frame_len, int32_t np,

@@ -66,7 +66,7 @@ struct CacheView {
   uint32_t* rel;                   // [H][max_frames][max_prompt]  ordered-uint relevance
   int32_t* selp;                   // [H][max_frames][max_prompt]
   // staging (fp32 entry conversion and the host-tensor step)
-  __nv_bfloat16* stage[5];         // k, v, q, kp, vp  ([H][max_tokens][D] / [H][max_prompt][D])
+  __nv_bfloat16* stage[6];         // k, v, q (AnnSA), kp, vp, q (AnnCA)  ([H][max_tokens][D] / [H][max_prompt][D])
   void* stage_out[2];              // [H][max_tokens][D] in the caller dtype
   void* stage_in_raw[5];           // raw caller-dtype copies for the host-tensor step (fp32 only)
 };

@@ -25,6 +25,15 @@ struct fastar_cache {
   PFN_cuTensorMapEncodeTiled_v12000 encode;
   int64_t launches;
   size_t bytes;
+  // second stream of the host-tensor step (uploads of q and the prompt, AnnCA, its download) and its fork/join events
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_q = nullptr, ev_join = nullptr;
+  ~fastar_cache() {
+    if (ev_fork) cudaEventDestroy(ev_fork);
+    if (ev_q) cudaEventDestroy(ev_q);
+    if (ev_join) cudaEventDestroy(ev_join);
+    if (side) cudaStreamDestroy(side);
+  }
 };
 
 namespace {
@@ -105,6 +114,7 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.selp = reinterpret_cast<int32_t*>(take(H * t.max_frames * MP * 4));
   for (int i = 0; i < 3; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
   for (int i = 3; i < 5; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MP * D * 2));
+  t.stage[5] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
   for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
   for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
   cur = (cur + 1023) & ~static_cast<size_t>(1023);
@@ -217,6 +227,12 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
   if (r == FASTAR_OK)
     r = make_map(c, &c->tm_hk, v.hk, v.hist_cols, v.CAPB, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
                  static_cast<uint64_t>(v.CAPB) * v.hist_cols * 2, 128);
+  if (r == FASTAR_OK &&
+      (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+       cudaEventCreateWithFlags(&c->ev_q, cudaEventDisableTiming) != cudaSuccess ||
+       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
+    r = FASTAR_ERR_CUDA;
   if (r != FASTAR_OK) {
     delete c;
     return r;
@@ -252,6 +268,7 @@ int fastar_cache_reset(fastar_cache_t* c, void* stream) {
 
 int fastar_cache_destroy(fastar_cache_t* c) {
   if (!c) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
   delete c;
   return FASTAR_OK;
 }
@@ -414,7 +431,7 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
   const __nv_bfloat16 *qb, *kpb, *vpb;
   int64_t qhs = head_stride, qts = token_stride, khs = prompt_head_stride, kts = prompt_token_stride, vhs = prompt_head_stride,
           vts = prompt_token_stride;
-  int r = as_bf16(c, q, nq, &qhs, &qts, 2, &qb, st);
+  int r = as_bf16(c, q, nq, &qhs, &qts, 5, &qb, st);   // own staging slot: may run beside an AnnSA call on another stream
   if (r == FASTAR_OK) r = as_bf16(c, k_prompt, np, &khs, &kts, 3, &kpb, st);
   if (r == FASTAR_OK) r = as_bf16(c, v_prompt, np, &vhs, &vts, 4, &vpb, st);
   if (r != FASTAR_OK) return r;
@@ -475,24 +492,42 @@ int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const 
   const size_t esz = f32 ? 4 : 2;
   const void* hsrc[5] = {k_new_host, v_new_host, q_host, k_prompt_host, v_prompt_host};
   void* dsrc[5];
-  for (int i = 0; i < 5; ++i) {
-    dsrc[i] = f32 ? v.stage_in_raw[i] : static_cast<void*>(v.stage[i]);
+  for (int i = 0; i < 5; ++i) dsrc[i] = f32 ? v.stage_in_raw[i] : static_cast<void*>(v.stage[i]);
+  auto upload = [&](int i, cudaStream_t s) {
     const size_t bytes = static_cast<size_t>(v.H) * (i < 3 ? n : np) * v.D * esz;
-    if (cudaMemcpyAsync(dsrc[i], hsrc[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-  }
+    return cudaMemcpyAsync(dsrc[i], hsrc[i], bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  };
+  // Two streams, so that the copies and the two attentions overlap the cache update instead of queueing behind it:
+  //   caller's stream : upload K, V -> update -> (q uploaded) AnnSA -> download its output
+  //   side stream     : upload q, prompt K/V -> AnnCA (reads no cache state) -> download its output
+  // The side stream starts after everything already queued on the caller's stream and is joined before returning.
+  cudaStream_t sd = c->side;
   const int64_t hs = static_cast<int64_t>(n) * v.D, ts = v.D, phs = static_cast<int64_t>(np) * v.D;
-  int r = fastar_tempcache_update(c, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, stream);
-  if (r != FASTAR_OK) return r;
-  r = fastar_annsa_attention(c, dsrc[2], v.stage_out[0], n, hs, ts, block_q, keep_blocks, nullptr, nullptr, nullptr, nullptr, nullptr,
-                             nullptr, stream);
-  if (r != FASTAR_OK) return r;
-  r = fastar_annca_attention(c, dsrc[2], dsrc[3], dsrc[4], v.stage_out[1], n, frame_len, np, keep_tokens, hs, ts, phs, ts, nullptr,
-                             nullptr, nullptr, stream);
-  if (r != FASTAR_OK) return r;
   const size_t obytes = static_cast<size_t>(v.H) * n * v.D * esz;
-  if (cudaMemcpyAsync(out_sa_host, v.stage_out[0], obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-  if (cudaMemcpyAsync(out_ca_host, v.stage_out[1], obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-  return cudaStreamSynchronize(st) == cudaSuccess ? FASTAR_OK : FASTAR_ERR_CUDA;
+  if (cudaEventRecord(c->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(sd, c->ev_fork, 0) != cudaSuccess) return FASTAR_ERR_CUDA;
+  int r = FASTAR_OK;
+  bool copies_ok = upload(0, st) && upload(1, st) && upload(2, sd);
+  copies_ok = copies_ok && cudaEventRecord(c->ev_q, sd) == cudaSuccess && upload(3, sd) && upload(4, sd);
+  if (!copies_ok) r = FASTAR_ERR_CUDA;
+  if (r == FASTAR_OK)
+    r = fastar_tempcache_update(c, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, st);
+  if (r == FASTAR_OK)
+    r = fastar_annca_attention(c, dsrc[2], dsrc[3], dsrc[4], v.stage_out[1], n, frame_len, np, keep_tokens, hs, ts, phs, ts, nullptr,
+                               nullptr, nullptr, sd);
+  if (r == FASTAR_OK && cudaMemcpyAsync(out_ca_host, v.stage_out[1], obytes, cudaMemcpyDeviceToHost, sd) != cudaSuccess) r = FASTAR_ERR_CUDA;
+  if (r == FASTAR_OK && cudaStreamWaitEvent(st, c->ev_q, 0) != cudaSuccess) r = FASTAR_ERR_CUDA;
+  if (r == FASTAR_OK)
+    r = fastar_annsa_attention(c, dsrc[2], v.stage_out[0], n, hs, ts, block_q, keep_blocks, nullptr, nullptr, nullptr, nullptr, nullptr,
+                               nullptr, st);
+  if (r == FASTAR_OK && cudaMemcpyAsync(out_sa_host, v.stage_out[0], obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) r = FASTAR_ERR_CUDA;
+  // always join: the side stream must be idle when this call returns, whatever happened above
+  const bool joined = cudaEventRecord(c->ev_join, sd) == cudaSuccess && cudaStreamWaitEvent(st, c->ev_join, 0) == cudaSuccess &&
+                      cudaStreamSynchronize(st) == cudaSuccess;
+  if (!joined) {
+    cudaStreamSynchronize(sd);
+    return r != FASTAR_OK ? r : FASTAR_ERR_CUDA;
+  }
+  return r;
 }
 
 int fastar_last_device_status(fastar_cache_t* c, void* stream) {

@@ -95,15 +95,24 @@ int launch_convert_f32_to_bf16(const float* src, __nv_bfloat16* dst, int H, int 
 //   A: a0 = X[g][2t..], a1 = X[g+8][2t..], a2 = X[g][2t+8..], a3 = X[g+8][2t+8..]   (bf16 pairs)
 //   B: b0 = R[n = 8*nt + g][2t..], b1 = R[n][2t+8..];   C: c0,c1 = row g, cols 2t,2t+1;  c2,c3 = row g+8.
 template <int D>
-__global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restrict__ x, int n, int64_t hs, int64_t ts,
+__global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restrict__ x, int H, int n, int64_t hs, int64_t ts,
                                                    const __nv_bfloat16* __restrict__ lsh, int T, int B,
                                                    uint32_t* __restrict__ code_out, float* __restrict__ rnorm_out,
                                                    int64_t out_stride) {
   constexpr int KS = D / 16;
+  constexpr int RP = D + 8;                    // padded row of the staged projection matrix (bank-conflict free)
+  __shared__ __align__(16) __nv_bfloat16 r_s[32 * RP];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int h = blockIdx.y;
   const int ncol = T * B;
+  // the projection matrix goes through shared memory once per CTA (coalesced 128-bit loads), then into registers
+  for (int q = threadIdx.x; q < 32 * (D / 8); q += blockDim.x) {
+    const int col = q / (D / 8), ch = q % (D / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (col < ncol) v = *reinterpret_cast<const uint4*>(lsh + col * D + ch * 8);
+    *reinterpret_cast<uint4*>(r_s + col * RP + ch * 8) = v;
+  }
+  __syncthreads();
   uint32_t bf[KS][4][2];
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks)
@@ -112,11 +121,16 @@ __global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restri
       // The contraction index may be permuted freely as long as A and B agree: lane t of a quad reads 8
       // contiguous elements (one 128-bit load) per 32-wide k block, k = 32*(ks/2) + 8t + 4*(ks%2) + {0,1 | 2,3}.
       const int col = 8 * nt + g;
-      const __nv_bfloat16* rp = lsh + col * D + 32 * (ks >> 1) + 8 * t + 4 * (ks & 1);
-      bf[ks][nt][0] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp) : 0u;
-      bf[ks][nt][1] = col < ncol ? *reinterpret_cast<const uint32_t*>(rp + 2) : 0u;
+      const __nv_bfloat16* rp = r_s + col * RP + 32 * (ks >> 1) + 8 * t + 4 * (ks & 1);
+      bf[ks][nt][0] = *reinterpret_cast<const uint32_t*>(rp);
+      bf[ks][nt][1] = *reinterpret_cast<const uint32_t*>(rp + 2);
     }
-  for (int r0 = (blockIdx.x * 8 + warp) * 16; r0 < n; r0 += gridDim.x * 128) {
+  // 16-row groups of all heads, dealt to the warps of a grid that fills the SMs once
+  const int groups_per_head = (n + 15) / 16;
+  const int total_groups = groups_per_head * H;
+  for (int grp = blockIdx.x * 8 + warp; grp < total_groups; grp += gridDim.x * 8) {
+    const int h = grp / groups_per_head;
+    const int r0 = (grp - h * groups_per_head) * 16;
     const int ra = min(r0 + g, n - 1), rb = min(r0 + g + 8, n - 1);   // rows past the end repeat the last one
     const __nv_bfloat16* xa = x + h * hs + ra * ts + 8 * t;
     const __nv_bfloat16* xb = x + h * hs + rb * ts + 8 * t;
@@ -186,9 +200,10 @@ __global__ void __launch_bounds__(256) prep_kernel(const __nv_bfloat16* __restri
 static int launch_prep_generic(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
                                float* rnorm_out, int64_t out_stride, cudaStream_t st) {
   if (n <= 0) return 0;
-  const dim3 grid(max(1, min((n + 127) / 128, (8 * 148 + c.H - 1) / c.H)), c.H);   // 128 rows per CTA pass
-  if (c.D == 128) prep_kernel<128><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
-  else prep_kernel<64><<<grid, 256, 0, st>>>(x, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
+  const int groups = ((n + 15) / 16) * c.H;                      // 16 rows per warp pass
+  const dim3 grid(max(1, min((groups + 7) / 8, 2 * 148)));
+  if (c.D == 128) prep_kernel<128><<<grid, 256, 0, st>>>(x, c.H, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
+  else prep_kernel<64><<<grid, 256, 0, st>>>(x, c.H, n, hs, ts, c.lsh, c.T, c.B, code_out, rnorm_out, out_stride);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
@@ -234,23 +249,34 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
   const int L = c.len[h];
   const int now = *c.now;
 
-  // groups: 4 consecutive slots per thread and pass
+  // groups: 16 consecutive slots per thread and pass (four 128-bit loads in flight; counts past the live length
+  // are zero and the capacity is a multiple of 128, so whole vectors can be read up to the capacity).  The
+  // numbers of groups and of members are scanned together, packed into one word (both stay below 2^16).
   int seg_run = 0, mem_run = 0, touched_ns = 0;
-  for (int j0 = 0; j0 < L; j0 += 4 * blockDim.x) {
-    const int j = j0 + 4 * tid;
-    int cn[4] = {0, 0, 0, 0};
-    if (j + 3 < L) {
-      const int4 v = *reinterpret_cast<const int4*>(c.cnt + sb + j);
-      cn[0] = v.x; cn[1] = v.y; cn[2] = v.z; cn[3] = v.w;
+  for (int j0 = 0; j0 < L; j0 += 16 * blockDim.x) {
+    const int j = j0 + 16 * tid;
+    int cn[16];
+    if (j < c.CAP) {
+      const int4* p = reinterpret_cast<const int4*>(c.cnt + sb + j);
+      const int4 v0 = p[0], v1 = p[1], v2 = p[2], v3 = p[3];
+      cn[0] = v0.x; cn[1] = v0.y; cn[2] = v0.z; cn[3] = v0.w;
+      cn[4] = v1.x; cn[5] = v1.y; cn[6] = v1.z; cn[7] = v1.w;
+      cn[8] = v2.x; cn[9] = v2.y; cn[10] = v2.z; cn[11] = v2.w;
+      cn[12] = v3.x; cn[13] = v3.y; cn[14] = v3.z; cn[15] = v3.w;
     } else {
-      for (int u = 0; u < 4; ++u) if (j + u < L) cn[u] = c.cnt[sb + j + u];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) cn[u] = 0;
     }
-    const int my_seg = (cn[0] > 0) + (cn[1] > 0) + (cn[2] > 0) + (cn[3] > 0);
-    const int my_mem = cn[0] + cn[1] + cn[2] + cn[3];
-    int tot_seg, tot_mem;
-    int seg = seg_run + block_exscan(my_seg, red, &tot_seg);
-    int mem = mem_run + block_exscan(my_mem, red, &tot_mem);
-    for (int u = 0; u < 4; ++u) {
+    int my_seg = 0, my_mem = 0;
+#pragma unroll
+    for (int u = 0; u < 16; ++u) { my_seg += cn[u] > 0; my_mem += cn[u]; }
+    int tot;
+    const int ex = block_exscan((my_seg << 16) | my_mem, red, &tot);
+    const int tot_seg = tot >> 16, tot_mem = tot & 0xFFFF;
+    int seg = seg_run + (ex >> 16);
+    int mem = mem_run + (ex & 0xFFFF);
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
       if (cn[u] > 0) {
         c.segslot[tb + seg] = j + u;
         c.segpos[gb + seg] = mem;
@@ -269,12 +295,16 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
 
   // unmatched tokens in token order
   int u_run = 0;
-  for (int i0 = 0; i0 < n; i0 += blockDim.x) {
-    const int i = i0 + tid;
-    const int un = (i < n && c.match[tb + i] < 0) ? 1 : 0;
+  for (int i0 = 0; i0 < n; i0 += 4 * blockDim.x) {
+    const int i = i0 + 4 * tid;
+    int un[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) un[u] = (i + u < n && c.match[tb + i + u] < 0) ? 1 : 0;
     int tot;
-    const int k = u_run + block_exscan(un, red, &tot);
-    if (un) c.ulist[tb + k] = i;
+    int k = u_run + block_exscan(un[0] + un[1] + un[2] + un[3], red, &tot);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (un[u]) c.ulist[tb + k++] = i + u;
     u_run += tot;
   }
   const int U = u_run;
