@@ -1,0 +1,154 @@
+// T3/T4 commit of a TempCache update (paper Section 5.2): every touched slot takes the count-weighted mean of
+// its old value and the values of the tokens merged into it, the key of its representative token (newest frame,
+// then highest similarity, then lowest index) and the new multiplicity; every unmatched token is written to the
+// slot the plan gave it.  The values are summed in ascending token order, in fp32, and rounded to bf16 once.
+//
+// A row of d bf16 is d/8 lanes of one 128-bit access each, so a warp serves 32/(d/8) work items (2 at d = 128,
+// 4 at d = 64) side by side.  The kernel is a chain of dependent lookups (plan -> group -> slot -> page -> rows),
+// so what it needs is many items in flight and no lookup that waits for one it does not depend on: the group
+// tables are read before the plan record is known, and a group of one member (the usual case) fetches its
+// value row, key row and metadata together.
+#include "common.h"
+#include "ptx.cuh"
+
+namespace fastar {
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 t = __bfloat1622float2(p[e]);
+    f[2 * e] = t.x;
+    f[2 * e + 1] = t.y;
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __nv_bfloat16* __restrict__ k_new,
+                                                     const __nv_bfloat16* __restrict__ v_new, int n, int frame_len, int64_t hs,
+                                                     int64_t ts) {
+  constexpr int LPR = D / 8;            // lanes per row
+  constexpr int GPW = 32 / LPR;         // work items per warp
+  const int h = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int sub = lane / LPR, sl = lane % LPR;
+  const unsigned mask = ((LPR == 32) ? 0xffffffffu : ((1u << LPR) - 1u)) << (sub * LPR);
+  const int w = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * GPW + sub;
+  if (w >= n) return;                   // groups + unmatched tokens <= n
+  const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+  const int64_t sb = static_cast<int64_t>(h) * c.CAP;
+  const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
+  const int32_t* segpos = c.segpos + static_cast<int64_t>(h) * (c.max_tokens + 1);
+  // read before the plan record arrives; meaningful only when w turns out to be a group
+  const int p0 = segpos[w], p1 = segpos[w + 1];
+  const int slot_g = c.segslot[tb + w];
+  const PlanRec pr = c.plan[h];
+  if (!pr.ok) return;
+  const int now = *c.now;
+  const __nv_bfloat16* kh = k_new + h * hs;
+  const __nv_bfloat16* vh = v_new + h * hs;
+
+  if (w < pr.n_seg) {
+    const int g = p1 - p0;
+    const int slot = slot_g;
+    const int page = pt_h[slot / c.PT];
+    const int m_old = c.count[sb + slot];
+    const int mine = (p0 + sl < p1) ? c.order[tb + p0 + sl] : 0x7fffffff;
+    const int64_t ro = (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D + sl * 8;
+    float acc[8];
+    {
+      const uint4 vo = *reinterpret_cast<const uint4*>(c.pool_v + ro);
+      unpack8(vo, acc);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] *= static_cast<float>(m_old);
+    }
+    int best_i;
+    if (g == 1) {
+      best_i = __shfl_sync(mask, mine, sub * LPR);
+      float f[8];
+      unpack8(*reinterpret_cast<const uint4*>(vh + best_i * ts + sl * 8), f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+    } else {
+      // Members in ascending token order (the scatter left them unordered): each round takes the smallest token
+      // index above the previous one.  Lanes hold the first LPR members, larger groups re-read the list.
+      int best_f = -1, last = -1;
+      float best_s = -INFINITY;
+      best_i = -1;
+      for (int r = 0; r < g; ++r) {
+        int cand = mine > last ? mine : 0x7fffffff;
+        for (int p = p0 + LPR + sl; p < p1; p += LPR) {
+          const int i2 = c.order[tb + p];
+          if (i2 > last && i2 < cand) cand = i2;
+        }
+#pragma unroll
+        for (int o = LPR / 2; o >= 1; o >>= 1) cand = min(cand, __shfl_xor_sync(mask, cand, o));
+        const int i = cand;
+        last = i;
+        float f[8];
+        unpack8(*reinterpret_cast<const uint4*>(vh + i * ts + sl * 8), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+        const int fr = i / frame_len;
+        const float s = c.sim[tb + i];
+        if (fr > best_f || (fr == best_f && s > best_s)) { best_f = fr; best_s = s; best_i = i; }
+      }
+    }
+    const uint4 krow = *reinterpret_cast<const uint4*>(kh + best_i * ts + sl * 8);
+    float rn = 0.f;
+    uint32_t code = 0;
+    if (sl == 0) {
+      rn = c.rnorm_new[tb + best_i];
+      code = c.code_new[tb + best_i];
+    }
+    const float inv = 1.f / static_cast<float>(m_old + g);
+    uint4 vout;
+    vout.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+    vout.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+    vout.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+    vout.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+    *reinterpret_cast<uint4*>(c.pool_v + ro) = vout;
+    *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
+    if (sl == 0) {
+      c.count[sb + slot] = m_old + g;
+      c.stamp[sb + slot] = now;
+      c.log2m[sb + slot] = log2f(static_cast<float>(m_old + g));
+      c.rnorm[sb + slot] = rn;
+      c.kcode[sb + slot] = code;
+    }
+  } else if (w - pr.n_seg < pr.n_unmatched) {
+    const int i = c.ulist[tb + (w - pr.n_seg)];
+    const int slot = c.dest[tb + i];
+    const uint4 krow = *reinterpret_cast<const uint4*>(kh + i * ts + sl * 8);
+    const uint4 vrow = *reinterpret_cast<const uint4*>(vh + i * ts + sl * 8);
+    float rn = 0.f;
+    uint32_t code = 0;
+    if (sl == 0) {
+      rn = c.rnorm_new[tb + i];
+      code = c.code_new[tb + i];
+    }
+    const int page = pt_h[slot / c.PT];
+    const int64_t ro = (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D + sl * 8;
+    *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
+    *reinterpret_cast<uint4*>(c.pool_v + ro) = vrow;
+    if (sl == 0) {
+      c.count[sb + slot] = 1;
+      c.stamp[sb + slot] = now;
+      c.log2m[sb + slot] = 0.f;
+      c.rnorm[sb + slot] = rn;
+      c.kcode[sb + slot] = code;
+    }
+  }
+}
+
+int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len, int64_t hs,
+                  int64_t ts, cudaStream_t st) {
+  if (n <= 0) return 0;
+  const int items_per_cta = 8 * (32 / (c.D / 8));
+  const dim3 grid((n + items_per_cta - 1) / items_per_cta, c.H);
+  if (c.D == 128) commit_kernel<128><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  else commit_kernel<64><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+}  // namespace fastar

@@ -2,7 +2,7 @@
 // shared-memory sorts and scans):
 //   S1  sign-random-projection codes (+ 1/|x|)               paper Section 5.1 (LSH)
 //   T2  threshold, T3 grouping plan, T4 compaction / append / eviction plan   Section 5.2
-//   T3/T4 commit: count-weighted value mean, last-key copy, append            Section 5.2, Lemma 1
+//   T3/T4 commit lives in commit_kernel.cu
 //   S2  per-block bucket histograms, S4 / C2 top-k with ties to the lower index   Sections 5.3, 5.4
 #include "common.h"
 #include "ptx.cuh"
@@ -415,118 +415,6 @@ int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_
   plan_kernel<<<c.H, 1024, 16384 * 8, st>>>(c, n);
   scatter_kernel<<<grid, 256, 0, st>>>(c, n);
   return cudaGetLastError() == cudaSuccess ? 3 : FASTAR_ERR_CUDA;
-}
-
-// ---------------------------------------------------------------------------------------------
-// T3/T4 commit: one warp per touched slot or per unmatched token.
-// ---------------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __nv_bfloat16* __restrict__ k_new,
-                                                     const __nv_bfloat16* __restrict__ v_new, int n, int frame_len, int64_t hs,
-                                                     int64_t ts) {
-  constexpr int EPL = D / 32;           // elements per lane (4 or 2), contiguous
-  const int h = blockIdx.y;
-  const int lane = threadIdx.x & 31;
-  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const PlanRec pr = c.plan[h];
-  if (!pr.ok) return;
-  const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
-  const int64_t sb = static_cast<int64_t>(h) * c.CAP;
-  const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
-  const int now = *c.now;
-  const __nv_bfloat16* kh = k_new + h * hs;
-  const __nv_bfloat16* vh = v_new + h * hs;
-
-  if (w < pr.n_seg) {
-    const int32_t* segpos = c.segpos + static_cast<int64_t>(h) * (c.max_tokens + 1);
-    const int p0 = segpos[w], p1 = segpos[w + 1];
-    const int g = p1 - p0;
-    const int slot = c.segslot[tb + w];
-    const int64_t ro = slot_row_offset(c, pt_h, slot);
-    const int m_old = c.count[sb + slot];
-    float acc[EPL];
-    {
-      const __nv_bfloat16* vr = c.pool_v + ro + lane * EPL;
-#pragma unroll
-      for (int e = 0; e < EPL; e += 2) {
-        const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(vr + e);
-        acc[e] = static_cast<float>(m_old) * __low2float(t);
-        acc[e + 1] = static_cast<float>(m_old) * __high2float(t);
-      }
-    }
-    // Walk the members in ascending token order (fixed summation order; the scatter left them unordered):
-    // each round takes the smallest token index above the previous one.  Lanes hold up to 32 members in a
-    // register, larger groups re-read the list.
-    const int mine = (p0 + lane < p1) ? c.order[tb + p0 + lane] : 0x7fffffff;
-    // representative: newest frame, then highest similarity, then lowest token index
-    int best_i = -1, best_f = -1, last = -1;
-    float best_s = -INFINITY;
-    for (int r = 0; r < g; ++r) {
-      int cand = mine > last ? mine : 0x7fffffff;
-      for (int p = p0 + 32 + lane; p < p1; p += 32) {
-        const int i2 = c.order[tb + p];
-        if (i2 > last && i2 < cand) cand = i2;
-      }
-#pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, o));
-      const int i = cand;
-      last = i;
-      const __nv_bfloat16* vr = vh + i * ts + lane * EPL;
-#pragma unroll
-      for (int e = 0; e < EPL; e += 2) {
-        const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(vr + e);
-        acc[e] += __low2float(t);
-        acc[e + 1] += __high2float(t);
-      }
-      const int f = i / frame_len;
-      const float s = c.sim[tb + i];
-      if (f > best_f || (f == best_f && s > best_s)) { best_f = f; best_s = s; best_i = i; }
-    }
-    const float inv = 1.f / static_cast<float>(m_old + g);
-    {
-      __nv_bfloat16* vw = c.pool_v + ro + lane * EPL;
-      const __nv_bfloat16* kr = kh + best_i * ts + lane * EPL;
-      __nv_bfloat16* kw = c.pool_k + ro + lane * EPL;
-#pragma unroll
-      for (int e = 0; e < EPL; e += 2) {
-        *reinterpret_cast<__nv_bfloat162*>(vw + e) = __floats2bfloat162_rn(acc[e] * inv, acc[e + 1] * inv);
-        *reinterpret_cast<__nv_bfloat162*>(kw + e) = *reinterpret_cast<const __nv_bfloat162*>(kr + e);
-      }
-    }
-    if (lane == 0) {
-      c.count[sb + slot] = m_old + g;
-      c.stamp[sb + slot] = now;
-      c.log2m[sb + slot] = log2f(static_cast<float>(m_old + g));
-      c.rnorm[sb + slot] = c.rnorm_new[tb + best_i];
-      c.kcode[sb + slot] = c.code_new[tb + best_i];
-    }
-  } else if (w - pr.n_seg < pr.n_unmatched) {
-    const int i = c.ulist[tb + (w - pr.n_seg)];
-    const int slot = c.dest[tb + i];
-    const int64_t ro = slot_row_offset(c, pt_h, slot);
-    const __nv_bfloat16* kr = kh + i * ts + lane * EPL;
-    const __nv_bfloat16* vr = vh + i * ts + lane * EPL;
-#pragma unroll
-    for (int e = 0; e < EPL; e += 2) {
-      *reinterpret_cast<__nv_bfloat162*>(c.pool_k + ro + lane * EPL + e) = *reinterpret_cast<const __nv_bfloat162*>(kr + e);
-      *reinterpret_cast<__nv_bfloat162*>(c.pool_v + ro + lane * EPL + e) = *reinterpret_cast<const __nv_bfloat162*>(vr + e);
-    }
-    if (lane == 0) {
-      c.count[sb + slot] = 1;
-      c.stamp[sb + slot] = now;
-      c.log2m[sb + slot] = 0.f;
-      c.rnorm[sb + slot] = c.rnorm_new[tb + i];
-      c.kcode[sb + slot] = c.code_new[tb + i];
-    }
-  }
-}
-int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len, int64_t hs,
-                  int64_t ts, cudaStream_t st) {
-  if (n <= 0) return 0;
-  const dim3 grid((n + 7) / 8, c.H);
-  if (c.D == 128) commit_kernel<128><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
-  else commit_kernel<64><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
-  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------
