@@ -16,8 +16,8 @@
 //   O_g += P_j V_j                  tcgen05.mma, V is the MN-major operand straight from its [key][d] page
 //   O = (O_0 2^(m_0-m) + O_1 2^(m_1-m)) / (l_0 2^(m_0-m) + l_1 2^(m_1-m))
 // O_g is rescaled lazily (only when a row maximum grew by more than 2^8).
-// TMEM columns: S[0], S[1], O_0, O_1 (4 x 128 at d = 128).  K and V tiles share one TMA ring filled in the
-// order the MMA warp consumes them: K0 K1 | K2 V0 | K3 V1 | ...
+// TMEM columns: S[0], S[1], O_0, O_1 (4 x 128 at d = 128).  K tiles and V tiles have a two-stage TMA ring each
+// (stages 0-1 and 2-3 of the ring memory); the MMA warp consumes K0 K1 | K2 V0 | K3 V1 | ...
 // Warp roles: warps 0-3 softmax group 0, warps 4-7 group 1, warp 8 producer (TMA or gather), warp 9 MMA issue.
 #include "common.h"
 #include "ptx.cuh"
@@ -154,7 +154,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const int idx = list[i];
         val = *reinterpret_cast<const uint4*>((which ? vp_h : kp_h) + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
       }
-      const uint32_t off = which * SM::kv_bytes + (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
+      const uint32_t off = which * 2 * SM::kv_bytes + (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
       asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_s + off), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w)
                    : "memory");
     }
@@ -162,15 +162,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     fence_proxy_async_smem();
     __syncthreads();
     if (threadIdx.x == 0) {
-      mbar_arrive(bar_r_full);                         // K0 -> stage 0
-      mbar_arrive(bar_r_full + 8);                     // V0 -> stage 1
+      mbar_arrive(bar_r_full);                         // K0 -> key stage 0
+      mbar_arrive(bar_r_full + 16);                    // V0 -> value stage 0 (ring stage 2)
       mbar_arrive(bar_b_full);
     }
     prefilled = true;
   }
 
-  // Ring order, identical in the producer and in the MMA warp:
-  //   K0, K1, then for j = 0, 1, ...: K_{j+2} (if any), V_j
+  // Tile j uses key stage j & 1 and value stage 2 + (j & 1), phase (j >> 1) & 1 of their barriers.
+  // The MMA warp consumes K0, K1, then for j = 0, 1, ...: K_{j+2} (if any), V_j.
   if (warp == kProducerWarp) {
     // ================================================================== producer
     if (lane == 0 && nt > 0) {
@@ -178,7 +178,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int kc = 0; kc < D / 64; ++kc) tma_load_3d(q_s + kc * kQChunk, &tm_q, bar_q_full, kc * 64, q0, h);
     }
     bool ok = true;
-    int it = 0;
     if (!GATHER) {
       // block ids and page ids of 32 tiles at a time, one coalesced load each; lane 0 issues the copies
       const int32_t* pt_h = c.page_table + static_cast<int64_t>(h) * c.CAPB;
@@ -191,11 +190,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           page = pt_h[blk];
         }
       };
+      // the stage of the tile is known to be free when this is called
       auto load_tile = [&](bool is_k, int j, int blk, int page) {
-        if (lane != 0 || !ok) return;
-        const int s = it % RS;
-        ok = mbar_wait(bar_r_empty + 8 * s, ((it / RS) & 1) ^ 1, abort_flag, c.status);
-        if (!ok) return;
+        if (lane != 0) return;
+        const int s = (is_k ? 0 : 2) + (j & 1);
+#ifdef FASTAR_PHASE_TIMING
+        reinterpret_cast<volatile long long*>(sgen + SM::bar_off + kBarBytes + 8)[s] = clock64();
+#endif
         mbar_arrive_expect_tx(bar_r_full + 8 * s, SM::kv_bytes);
         for (int kc = 0; kc < D / 64; ++kc)
           tma_load_3d(ring_s + s * SM::kv_bytes + kc * BKT * 128, is_k ? &tm_k : &tm_v, bar_r_full + 8 * s, kc * 64, 0, page);
@@ -204,30 +205,49 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           mbar_arrive_expect_tx(bar_b_full + 8 * b4, BKT * 4);
           bulk_load_1d(bias_s + b4 * BKT * 4, l2m_h + static_cast<int64_t>(blk) * BKT, BKT * 4, bar_b_full + 8 * b4);
         }
-        ++it;
       };
       if (nt > 0) {
-        // two windows of 32 tiles: the low one holds the value tile in turn, key tiles may already need the next
+        // Key and value tiles have a two-stage ring each and are issued independently, whichever stage frees first
+        // (a key stage frees as soon as its QK^T is done, a value stage only after its P.V): lane 0 polls both
+        // rings, the other lanes follow its decision for the lookups.  Key tiles stay ahead of value tiles.
+        // Two windows of 32 tiles: the low one holds the value tile in turn, key tiles may already need the next.
         fetch(0, blk_l, page_l);
         fetch(32, blk_n, page_n);
-        auto get = [&](int j, int& blk, int& page, int base) {   // base = first tile of the low window
-          const bool hi = j >= base + 32;
-          blk = __shfl_sync(0xffffffffu, hi ? blk_n : blk_l, j & 31);
-          page = __shfl_sync(0xffffffffu, hi ? page_n : page_l, j & 31);
-        };
-        int base = 0, blk, page;
-        get(0, blk, page, base);
-        load_tile(true, 0, blk, page);
-        if (nt > 1) { get(1, blk, page, base); load_tile(true, 1, blk, page); }
-        for (int j = 0; j < nt; ++j) {
-          if (j >= base + 32) {                                   // value tiles enter the next window
+        int base = 0, kj = 0, vj = 0;
+        while (true) {
+          int act = 0;                                            // 1: key tile kj, 2: value tile vj, 3: give up, 4: done
+          if (lane == 0) {
+            uint64_t t0 = 0;
+            for (uint32_t spin = 1;; ++spin) {
+              if (vj >= nt) { act = 4; break; }
+              if (kj < nt && mbar_test_wait(bar_r_empty + 8 * (kj & 1), ((kj >> 1) & 1) ^ 1)) { act = 1; break; }
+              if (mbar_test_wait(bar_r_empty + 8 * (2 + (vj & 1)), ((vj >> 1) & 1) ^ 1)) { act = 2; break; }
+              if ((spin & 255u) == 0) {                           // bounded like mbar_wait
+                if (*abort_flag) { act = 3; break; }
+                const uint64_t t = global_timer_ns();
+                if (t0 == 0) t0 = t;
+                else if (t - t0 > kWaitLimitNs) {
+                  *abort_flag = 1;
+                  record_status(c.status, kErrTimeout);
+                  act = 3;
+                  break;
+                }
+              }
+            }
+          }
+          act = __shfl_sync(0xffffffffu, act, 0);
+          if (act >= 3) { ok = act == 4; break; }
+          if (vj >= base + 32) {                                  // value tiles enter the next window
             base += 32;
             blk_l = blk_n; page_l = page_n;
             fetch(base + 32, blk_n, page_n);
           }
-          if (j + 2 < nt) { get(j + 2, blk, page, base); load_tile(true, j + 2, blk, page); }
-          get(j, blk, page, base);
-          load_tile(false, j, blk, page);
+          const int j = act == 1 ? kj : vj;
+          const bool hi = j >= base + 32;
+          const int blk = __shfl_sync(0xffffffffu, hi ? blk_n : blk_l, j & 31);
+          const int page = __shfl_sync(0xffffffffu, hi ? page_n : page_l, j & 31);
+          load_tile(act == 1, j, blk, page);
+          if (act == 1) ++kj; else ++vj;
         }
       }
     } else {
@@ -237,8 +257,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const __nv_bfloat16* vp_h = a.vp + static_cast<int64_t>(h) * a.p_head_stride;
       auto fill_tile = [&](bool is_k, int j) {
         if (!ok) return;
-        const int s = it % RS;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_r_empty + 8 * s, ((it / RS) & 1) ^ 1, abort_flag, c.status));
+        const int s = (is_k ? 0 : 2) + (j & 1);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_r_empty + 8 * s, ((j >> 1) & 1) ^ 1, abort_flag, c.status));
         if (!ok) return;
         const __nv_bfloat16* src_h = is_k ? kp_h : vp_h;
         const uint32_t dst = ring_s + s * SM::kv_bytes;
@@ -264,7 +284,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           mbar_arrive(bar_r_full + 8 * s);
           if (is_k) mbar_arrive(bar_b_full + 8 * b4);
         }
-        ++it;
       };
       if (nt > 0 && !prefilled) {
         fill_tile(true, 0);
@@ -281,11 +300,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, BKT, 0);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
       bool ok = mbar_wait(bar_q_full, 0, abort_flag, c.status);
-      int it = 0;                                       // position in the K/V ring (same order as the producer)
       PT_DECL
       auto issue_s = [&](int j) -> bool {
-        const int s = it % RS, g = j & 1, i = j >> 1;
-        if (!mbar_wait(bar_r_full + 8 * s, (it / RS) & 1, abort_flag, c.status)) return false;
+        const int s = j & 1, g = j & 1, i = j >> 1;      // key stage, softmax group, tile index inside the group
+        if (!mbar_wait(bar_r_full + 8 * s, i & 1, abort_flag, c.status)) return false;
+#ifdef FASTAR_PHASE_TIMING
+        if (clock64() - pt_t > 100) {     // the tile was late: time since its load was issued
+          pt_acc[6] += clock64() - reinterpret_cast<volatile long long*>(sgen + SM::bar_off + kBarBytes + 8)[s];
+          pt_acc[7] += 1000;          // printed value / 1000 = late tiles per iteration
+        }
+#endif
         PT_MARK(0)
         // S[g] is free once group g holds the logits of its previous tile (j - 2) in registers
         if (i > 0 && !mbar_wait(bar_s_empty + 8 * g, (i - 1) & 1, abort_flag, c.status)) return false;
@@ -300,7 +324,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         umma_commit(bar_r_empty + 8 * s);
         umma_commit(bar_s_full + 8 * g);
-        ++it;
         PT_MARK(2)
         return true;
       };
@@ -308,11 +331,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (ok && nt > 1) ok = issue_s(1);
       for (int j = 0; j < nt && ok; ++j) {
         if (j + 2 < nt) { ok = issue_s(j + 2); if (!ok) break; }
-        const int s = it % RS, g = j & 1, i = j >> 1;
+        const int s = 2 + (j & 1), g = j & 1, i = j >> 1;   // value stage, softmax group, tile index inside the group
         ok = mbar_wait(bar_p_full + 8 * g, i & 1, abort_flag, c.status);
         if (!ok) break;
         PT_MARK(3)
-        ok = mbar_wait(bar_r_full + 8 * s, (it / RS) & 1, abort_flag, c.status);
+        ok = mbar_wait(bar_r_full + 8 * s, i & 1, abort_flag, c.status);
         if (!ok) break;
         PT_MARK(4)
         tc_fence_after();
@@ -326,7 +349,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         umma_commit(bar_r_empty + 8 * s);
         umma_commit(bar_pv_done + 8 * g);
-        ++it;
         PT_MARK(5)
       }
       PT_FLUSH("attn mma (wait K, wait S buffer, issue QK, wait P, wait V, issue PV)", nt)
