@@ -129,12 +129,78 @@ def top1_cosine(K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.nda
     return j.astype(np.int64), c[np.arange(n), j]
 
 
+# ---------------------------------------------------------------------------------------------------
+# 8-bit quantised similarity search (Section 5.1 "quantised similarity search", 8 bits being the
+# paper's default, Section 6 / Appendix C bit-width ablation).  Reading taken here: a key is scaled
+# to unit length, multiplied by E4M3_SCALE and every component is rounded to an 8-bit float
+# (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448;
+# round to nearest even, saturating); the search score of two keys is the exact dot product of
+# their codes divided by E4M3_SCALE^2, an approximation of their cosine.
+# ---------------------------------------------------------------------------------------------------
+E4M3_SCALE = 16.0
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """float -> uint8 code of the nearest 8-bit float (ties to even, saturating at +-448)."""
+    x = np.asarray(x, np.float64)
+    sign = np.signbit(x).astype(np.uint8)
+    a = np.minimum(np.abs(x), 448.0)
+    # exponent of the binade (normal numbers start at 2^-6; below that the spacing stays 2^-9)
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -6))).astype(np.int64)
+    e = np.clip(e, -6, 8)
+    step = np.exp2(e - 3.0)
+    q = np.rint(a / step) * step                                   # np.rint rounds halves to even
+    q = np.minimum(q, 448.0)
+    # re-derive the fields from the rounded value (rounding may have moved it up one binade)
+    e2 = np.clip(np.floor(np.log2(np.maximum(q, 2.0 ** -6))).astype(np.int64), -6, 8)
+    normal = q >= 2.0 ** -6
+    mant = np.where(normal, np.rint(q / np.exp2(e2 - 3.0)) - 8, np.rint(q / 2.0 ** -9)).astype(np.int64)
+    expf = np.where(normal, e2 + 7, 0).astype(np.int64)
+    return ((sign.astype(np.int64) << 7) | (expf << 3) | mant).astype(np.uint8)
+
+
+def e4m3_decode(code: np.ndarray) -> np.ndarray:
+    """uint8 code -> value (the NaN codes 0x7f / 0xff never occur here and decode to nan)."""
+    c = np.asarray(code).astype(np.int64)
+    sign = np.where((c >> 7) & 1, -1.0, 1.0)
+    expf = (c >> 3) & 0xF
+    mant = c & 0x7
+    val = np.where(expf == 0, mant * 2.0 ** -9, (8 + mant) * np.exp2(expf - 7.0 - 3.0))
+    val = np.where((expf == 15) & (mant == 7), np.nan, val)
+    return sign * val
+
+
+def key_codes_e4m3(K: np.ndarray) -> np.ndarray:
+    """Search codes of keys [n][d] -> uint8 [n][d]; an all-zero key has an all-zero code."""
+    K = np.asarray(K, np.float64)
+    nrm = np.sqrt((K * K).sum(axis=1, keepdims=True))
+    unit = np.divide(K, nrm, out=np.zeros_like(K), where=nrm > 0)
+    return e4m3_encode(unit * E4M3_SCALE)
+
+
+def quantized_score_matrix(codes_a: np.ndarray, codes_b: np.ndarray) -> np.ndarray:
+    """Search scores of every pair of codes: dot product of the decoded codes / E4M3_SCALE^2."""
+    return (e4m3_decode(codes_a) @ e4m3_decode(codes_b).T) / (E4M3_SCALE * E4M3_SCALE)
+
+
+def top1_quantized(K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.ndarray]:
+    """top1_cosine with the 8-bit search score in place of the cosine."""
+    n = K_new.shape[0]
+    if cache.L == 0:
+        return np.full(n, -1, np.int64), np.zeros(n, np.float64)
+    s = quantized_score_matrix(key_codes_e4m3(K_new), key_codes_e4m3(cache.K[: cache.L]))
+    j = np.argmax(s, axis=1)
+    return j.astype(np.int64), s[np.arange(n), j]
+
+
 def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
-                     forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None) -> Dict[str, np.ndarray]:
+                     forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None,
+                     search_bits: int = 16) -> Dict[str, np.ndarray]:
     """One TempCache update of one head.
 
     forced = (j*, c*, matched) replaces steps 1-2 by decisions taken elsewhere
-    (staged parity: near-ties have several correct answers)."""
+    (staged parity: near-ties have several correct answers).  search_bits = 8 runs the
+    correspondence search on the 8-bit codes of the keys instead of the keys themselves."""
     K_new = np.asarray(K_new, np.float64)
     V_new = np.asarray(V_new, np.float64)
     n = K_new.shape[0]
@@ -142,7 +208,7 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
 
     # 1. top-1 correspondence against the pre-call cache; 2. threshold
     if forced is None:
-        jstar, cstar = top1_cosine(K_new, cache)
+        jstar, cstar = top1_quantized(K_new, cache) if search_bits == 8 else top1_cosine(K_new, cache)
         matched = (cstar >= tau) & (jstar >= 0)
     else:
         jstar, cstar, matched = (np.asarray(a) for a in forced)

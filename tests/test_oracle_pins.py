@@ -381,3 +381,59 @@ def test_c0_workload_behaves_as_designed():
     assert a["sel"].shape == (4, 4)
     rec = O.attention_recall(Q[0], c, a["sel"], cfg.block, cfg.block)
     assert rec > 0.5                                            # the selector finds the mass on clustered data
+
+
+# ----------------------------------------------------------------------------- 8-bit quantised search
+def test_e4m3_quantiser_against_the_format_definition_and_torch():
+    # hand values from the format: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits, subnormals of 2^-9, max 448
+    codes = np.array([0x00, 0x01, 0x07, 0x08, 0x38, 0x3C, 0x40, 0x7E, 0x80 | 0x38, 0x80 | 0x7E], np.uint8)
+    vals = np.array([0.0, 2.0 ** -9, 7 * 2.0 ** -9, 2.0 ** -6, 1.0, 1.5, 2.0, 448.0, -1.0, -448.0])
+    assert np.array_equal(O.e4m3_decode(codes), vals)
+    assert np.array_equal(O.e4m3_encode(vals), codes)
+    # ties go to the even mantissa: 1.0625 is halfway between 1.0 (mantissa 0) and 1.125 (mantissa 1)
+    assert O.e4m3_decode(O.e4m3_encode(np.array([1.0625, 1.1875, 17.0, 19.0]))).tolist() == [1.0, 1.25, 16.0, 20.0]
+    # saturation instead of infinities or NaN
+    assert O.e4m3_decode(O.e4m3_encode(np.array([1e9, -500.0, 464.0]))).tolist() == [448.0, -448.0, 448.0]
+    # every code round-trips, and the decoded value agrees with torch's view of the same byte
+    import torch
+    allc = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], np.uint8)
+    dec = O.e4m3_decode(allc)
+    assert np.array_equal(O.e4m3_encode(dec)[dec != 0], allc[dec != 0])
+    tv = torch.from_numpy(allc.copy()).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    assert np.array_equal(dec, tv)
+    # rounding of arbitrary values agrees with torch's float32 -> float8 cast inside the finite range
+    x = np.concatenate([_rng(30).standard_normal(20000) * 3.0, _rng(31).uniform(-440, 440, 5000),
+                        _rng(32).standard_normal(5000) * 0.01]).astype(np.float32)
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    assert np.array_equal(O.e4m3_decode(O.e4m3_encode(x.astype(np.float64))), want)
+
+
+def test_quantised_search_is_a_close_approximation_of_the_cosine_search():
+    rng = _rng(33)
+    d, L, n = 128, 600, 200
+    c = O.HeadCache(1024, d)
+    Kc = O.round_to_bf16(rng.standard_normal((L, d)))
+    c.load(Kc, rng.standard_normal((L, d)))
+    # new keys: near copies of cached keys (should be found) and unrelated keys
+    src = rng.integers(0, L, n // 2)
+    Kn = np.concatenate([Kc[src] * rng.uniform(0.5, 2.0, (n // 2, 1)) + 0.02 * rng.standard_normal((n // 2, d)),
+                         rng.standard_normal((n // 2, d))])
+    j8, s8 = O.top1_quantized(Kn, c)
+    j16, s16 = O.top1_cosine(Kn, c)
+    assert np.array_equal(j8[: n // 2], src) and np.array_equal(j16[: n // 2], src)       # scale-invariant, finds the copy
+    cos = O.cosine_matrix(Kn, Kc)
+    # the score is the cosine up to the quantisation error of 3 mantissa bits on 128 components
+    assert np.max(np.abs(O.quantized_score_matrix(O.key_codes_e4m3(Kn), O.key_codes_e4m3(Kc)) - cos)) < 0.02
+    assert np.max(np.abs(s8 - cos[np.arange(n), j8])) < 0.02
+    # codes of a key and of any positive multiple of it are identical; a zero key has a zero code
+    assert np.array_equal(O.key_codes_e4m3(Kc[:5]), O.key_codes_e4m3(Kc[:5] * 7.5))
+    assert not O.key_codes_e4m3(np.zeros((1, d))).any()
+    # brute force on a tiny case with Python loops
+    a, b = O.key_codes_e4m3(Kn[:3]), O.key_codes_e4m3(Kc[:4])
+    da, db = O.e4m3_decode(a), O.e4m3_decode(b)
+    brute = [[sum(float(da[i, k]) * float(db[j, k]) for k in range(d)) / 256.0 for j in range(4)] for i in range(3)]
+    assert np.allclose(O.quantized_score_matrix(a, b), brute, rtol=0, atol=1e-12)
+    # the update with search_bits = 8 uses these decisions
+    c2 = c.copy()
+    res = O.tempcache_update(c2, Kn, rng.standard_normal((n, d)), 100, 0.9, search_bits=8)
+    assert res["stats"]["matched"] >= n // 2 - 2 and res["stats"]["matched"] <= n // 2 + 2
