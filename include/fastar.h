@@ -68,6 +68,12 @@ typedef struct {
   int32_t max_frames;        /* largest number of frames per AnnCA call */
   int32_t dtype;             /* fastar_dtype_t of the tensors the caller passes */
   int32_t device;            /* CUDA device ordinal */
+  int32_t search_bits;       /* precision of TempCache's correspondence search: 16 (or 0) = the bf16 keys,
+                              * 8 = 8-bit quantised search (Section 5.1; the paper's default): every key is
+                              * reduced to x/|x|*16 in fp8 e4m3 (round to nearest even, saturating), kept in a
+                              * second paged pool of 128-byte rows, and the similarity of two keys is the
+                              * dot product of their codes / 256.  Top-1, ties and the threshold rule are
+                              * unchanged; the merge itself always uses the bf16 keys and values. */
 } fastar_cache_desc;
 
 typedef struct {
@@ -106,8 +112,16 @@ int fastar_cache_destroy(fastar_cache_t* cache);
 int fastar_cache_export(fastar_cache_t* cache, uint16_t* host_k, uint16_t* host_v, int32_t* count,
                         int32_t* stamp, uint32_t* code, int32_t* len, int32_t* now, void* stream);
 
+/* 8-bit search only (search_bits == 8, else FASTAR_ERR_UNSUPPORTED_SHAPE): copy the search codes to
+ * the host and synchronise the stream.  host_cache_codes: [H][CAP][128] bytes, the code row of every
+ * slot (d code bytes, zero padded to 128; fp8 e4m3 of x/|x|*16); host_new_codes: [H][n][128], the codes
+ * the most recent update computed for its n new keys.  Either pointer may be NULL.  (Section 5.1,
+ * quantised similarity search; used by the tests to check the quantiser and the search separately.) */
+int fastar_cache_export_search_codes(fastar_cache_t* cache, uint8_t* host_cache_codes, uint8_t* host_new_codes,
+                                     int32_t n, void* stream);
+
 /* Load a state (same layouts; count/stamp NULL = all ones / all zeros).  Slots >= len[h] are
- * cleared.  Derived per-slot data (1/|k|, log2 m, LSH codes, histograms) are recomputed on the
+ * cleared.  Derived per-slot data (1/|k|, log2 m, LSH codes, search codes, histograms) are recomputed on the
  * device.  `now` must exceed every stamp.  Synchronises the stream. */
 int fastar_cache_import(fastar_cache_t* cache, const uint16_t* host_k, const uint16_t* host_v,
                         const int32_t* count, const int32_t* stamp, const int32_t* len, int32_t now,

@@ -23,6 +23,18 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
   }
 }
 
+// Copy the 128-byte search code of new token `tok` into the code row of (page, row): LPR lanes, 128 / LPR bytes each.
+template <int LPR>
+__device__ __forceinline__ void copy_code_row(const CacheView& c, int h, int tok, int page, int row_in_page, int sl) {
+  const uint8_t* src = c.k8_new + (static_cast<int64_t>(h) * c.max_tokens + tok) * 128;
+  uint8_t* dst = c.pool_k8 + (static_cast<int64_t>(page) * c.PT + row_in_page) * 128;
+  if (LPR == 16) {
+    *reinterpret_cast<uint2*>(dst + sl * 8) = *reinterpret_cast<const uint2*>(src + sl * 8);
+  } else {
+    *reinterpret_cast<uint4*>(dst + sl * 16) = *reinterpret_cast<const uint4*>(src + sl * 16);
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __nv_bfloat16* __restrict__ k_new,
                                                      const __nv_bfloat16* __restrict__ v_new, int n, int frame_len, int64_t hs,
@@ -109,6 +121,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
     vout.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
     *reinterpret_cast<uint4*>(c.pool_v + ro) = vout;
     *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
+    if (c.pool_k8) copy_code_row<LPR>(c, h, best_i, page, slot % c.PT, sl);
     if (sl == 0) {
       c.count[sb + slot] = m_old + g;
       c.stamp[sb + slot] = now;
@@ -131,6 +144,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
     const int64_t ro = (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D + sl * 8;
     *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
     *reinterpret_cast<uint4*>(c.pool_v + ro) = vrow;
+    if (c.pool_k8) copy_code_row<LPR>(c, h, i, page, slot % c.PT, sl);
     if (sl == 0) {
       c.count[sb + slot] = 1;
       c.stamp[sb + slot] = now;

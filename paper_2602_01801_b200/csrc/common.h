@@ -69,6 +69,10 @@ struct CacheView {
   __nv_bfloat16* stage[6];         // k, v, q (AnnSA), kp, vp, q (AnnCA)  ([H][max_tokens][D] / [H][max_prompt][D])
   void* stage_out[2];              // [H][max_tokens][D] in the caller dtype
   void* stage_in_raw[5];           // raw caller-dtype copies for the host-tensor step (fp32 only)
+  // 8-bit quantised correspondence search (search_bits == 8; null otherwise)
+  int32_t search_bits;             // 16 or 8
+  uint8_t* pool_k8;                // [H*CAPB][PT][128]  fp8 e4m3 search codes of the cached keys, paged like pool_k
+  uint8_t* k8_new;                 // [H][max_tokens][128]  codes of the new keys of the update in flight
 };
 
 inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
@@ -86,6 +90,11 @@ int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUte
 int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,
                         int n_frames, cudaStream_t st);
 int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtensorMap& tm_hk, int nqb, cudaStream_t st);
+
+// search8_kernels.cu: fp8 search codes of bf16 rows (x / |x| * 16, 128-byte rows), and T1 on the codes
+int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, const float* rnorm,
+                         int64_t rn_stride, uint8_t* out, int64_t out_rows_per_head, cudaStream_t st);
+int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, cudaStream_t st);
 
 // attn_kernels.cu
 struct AttnArgs {

@@ -21,7 +21,7 @@ struct fastar_cache {
   std::vector<ProfRec> recs;
   fastar_cache_desc desc;
   CacheView v;
-  CUtensorMap tm_pool_k, tm_pool_k_half, tm_pool_v, tm_hq, tm_hk;
+  CUtensorMap tm_pool_k, tm_pool_k_half, tm_pool_v, tm_hq, tm_hk, tm_pool_k8;
   PFN_cuTensorMapEncodeTiled_v12000 encode;
   int64_t launches;
   size_t bytes;
@@ -59,6 +59,7 @@ bool desc_valid(const fastar_cache_desc* d) {
   if (d->max_tokens < 1 || d->max_tokens > 16384) return false;
   if (d->max_prompt_tokens < 1 || d->max_prompt_tokens > 1024 || d->max_frames < 1 || d->max_frames > 64) return false;
   if (d->dtype != FASTAR_BF16 && d->dtype != FASTAR_FP32) return false;
+  if (d->search_bits != 0 && d->search_bits != 16 && d->search_bits != 8) return false;
   return true;
 }
 
@@ -115,6 +116,9 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   for (int i = 0; i < 3; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
   for (int i = 3; i < 5; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MP * D * 2));
   t.stage[5] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
+  t.search_bits = d.search_bits == 8 ? 8 : 16;
+  t.pool_k8 = t.search_bits == 8 ? take(H * CAP * 128) : nullptr;
+  t.k8_new = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
   for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
   for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
   cur = (cur + 1023) & ~static_cast<size_t>(1023);
@@ -131,6 +135,20 @@ int make_map(fastar_cache* c, CUtensorMap* m, const void* ptr, uint64_t d0, uint
   const cuuint32_t box[3] = {64, box1, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+// 3-D byte tensor map of 128-byte search-code rows {128, d1, d2}, box {128, box1, 1}, 128-byte swizzle.
+int make_map_codes(fastar_cache* c, CUtensorMap* m, const void* ptr, uint64_t d1, uint64_t d2, uint64_t stride2_bytes,
+                   uint32_t box1) {
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (stride2_bytes & 15)) return FASTAR_ERR_INVALID_ARG;
+  const cuuint64_t dims[3] = {128, d1, d2};
+  const cuuint64_t strides[2] = {128, stride2_bytes};
+  const cuuint32_t box[3] = {128, box1, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? FASTAR_OK : FASTAR_ERR_CUDA;
@@ -227,6 +245,8 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
   if (r == FASTAR_OK)
     r = make_map(c, &c->tm_hk, v.hk, v.hist_cols, v.CAPB, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
                  static_cast<uint64_t>(v.CAPB) * v.hist_cols * 2, 128);
+  if (r == FASTAR_OK && v.search_bits == 8)
+    r = make_map_codes(c, &c->tm_pool_k8, v.pool_k8, PT, static_cast<uint64_t>(v.H) * v.CAPB, PT * 128, v.PT);
   if (r == FASTAR_OK &&
       (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -292,6 +312,24 @@ int fastar_cache_export(fastar_cache_t* c, uint16_t* host_k, uint16_t* host_v, i
   return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
 }
 
+int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_codes, uint8_t* host_new_codes, int32_t n,
+                                     void* stream) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  const CacheView& v = c->v;
+  if (v.search_bits != 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (host_new_codes && (n < 1 || n > v.max_tokens)) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool ok = true;
+  if (host_cache_codes)
+    ok &= cudaMemcpyAsync(host_cache_codes, v.pool_k8, static_cast<size_t>(v.H) * v.CAP * 128, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (host_new_codes)
+    ok &= cudaMemcpy2DAsync(host_new_codes, static_cast<size_t>(n) * 128, v.k8_new, static_cast<size_t>(v.max_tokens) * 128,
+                            static_cast<size_t>(n) * 128, v.H, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
 int fastar_cache_import(fastar_cache_t* c, const uint16_t* host_k, const uint16_t* host_v, const int32_t* count,
                         const int32_t* stamp, const int32_t* len, int32_t now, void* stream) {
   if (!c || !host_k || !host_v || !len || now < 0) return FASTAR_ERR_INVALID_ARG;
@@ -341,7 +379,16 @@ int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_
   // packed arg-max words and per-slot match counts start at zero (adjacent in the workspace: one memset)
   if (cudaMemsetAsync(v.best, 0, reinterpret_cast<uint8_t*>(v.cnt) - reinterpret_cast<uint8_t*>(v.best) + static_cast<size_t>(v.H) * v.CAP * 4, st) != cudaSuccess)
     return FASTAR_ERR_CUDA;
-  ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
+  if (v.search_bits == 8) {
+    // correspondence search on the 8-bit codes: quantise the new keys, then the fp8 contraction with the arg-max fused
+    CUtensorMap tm_a8;
+    r = make_map_codes(c, &tm_a8, v.k8_new, n, v.H, static_cast<uint64_t>(v.max_tokens) * 128, 128);
+    if (r != FASTAR_OK) return r;
+    ACCK(FASTAR_K_HASH, launch_quantize_keys(v, kb, n, khs, kts, v.rnorm_new, v.max_tokens, v.k8_new, v.max_tokens, st));
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(v, tm_a8, c->tm_pool_k8, n, st));
+  } else {
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
+  }
   ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
   ACCK(FASTAR_K_COMMIT, launch_commit(v, kb, vb, n, frame_len, khs, kts, st));
   ACCK(FASTAR_K_KEY_HIST, launch_finalize_hist(v, stats_out, 1, st));

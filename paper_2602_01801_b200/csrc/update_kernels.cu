@@ -557,6 +557,7 @@ int launch_reset(const CacheView& c, cudaStream_t st) {
   if (cudaMemsetAsync(c.pool_k, 0, pool, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   if (cudaMemsetAsync(c.pool_v, 0, pool, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   if (cudaMemsetAsync(c.hk, 0, static_cast<size_t>(c.H) * c.CAPB * c.hist_cols * 2, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (c.pool_k8 && cudaMemsetAsync(c.pool_k8, 0, static_cast<size_t>(c.H) * c.CAP * 128, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   reset_meta_kernel<<<296, 256, 0, st>>>(c);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
@@ -590,9 +591,14 @@ int launch_import_derive(const CacheView& c, cudaStream_t st) {
   if (c.D == 128) import_fix_kernel<128><<<grid, 256, 0, st>>>(c);
   else import_fix_kernel<64><<<grid, 256, 0, st>>>(c);
   if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+  int r3 = 0;
+  if (c.pool_k8) {                                   // search codes of every slot from the imported keys
+    r3 = launch_quantize_keys(c, c.pool_k, c.CAP, static_cast<int64_t>(c.CAP) * c.D, c.D, c.rnorm, c.CAP, c.pool_k8, c.CAP, st);
+    if (r3 < 0) return r3;
+  }
   int r2 = launch_finalize_hist(c, nullptr, -1, st);
   if (r2 < 0) return r2;
-  return r + 1 + r2;
+  return r + 1 + r2 + r3;
 }
 
 int launch_copy_outputs(const CacheView& c, int n, int32_t* match_out, float* sim_out, int32_t* dest_out, cudaStream_t st) {

@@ -25,7 +25,8 @@ class FastarError(RuntimeError):
 
 class CacheDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("num_heads", "head_dim", "capacity", "page_tokens", "n_sink", "lsh_tables",
-                                         "lsh_bits", "max_tokens", "max_prompt_tokens", "max_frames", "dtype", "device")]
+                                         "lsh_bits", "max_tokens", "max_prompt_tokens", "max_frames", "dtype", "device",
+                                         "search_bits")]
 
 
 class UpdateStats(C.Structure):
@@ -41,6 +42,7 @@ SIGNATURES = {
     "fastar_cache_reset": (C.c_int, [_vp, _vp]),
     "fastar_cache_destroy": (C.c_int, [_vp]),
     "fastar_cache_export": (C.c_int, [_vp] * 9),
+    "fastar_cache_export_search_codes": (C.c_int, [_vp, _vp, _vp, _i32, _vp]),
     "fastar_cache_import": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp]),
     "fastar_tempcache_update": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annsa_attention": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -98,7 +100,7 @@ class Cache:
 
     def __init__(self, num_heads: int, head_dim: int, capacity: int, page_tokens: int, lsh_proj: np.ndarray,
                  lsh_tables: int = 4, lsh_bits: int = 8, max_tokens: int = 4096, max_prompt_tokens: int = 512,
-                 max_frames: int = 8, n_sink: int = 0, fp32: bool = False, device: int = 0):
+                 max_frames: int = 8, n_sink: int = 0, fp32: bool = False, device: int = 0, search_bits: int = 16):
         import torch
         self.lib = load_library()
         self.torch = torch
@@ -107,7 +109,9 @@ class Cache:
         self.fp32 = fp32
         self.dtype = torch.float32 if fp32 else torch.bfloat16
         self.desc = CacheDesc(num_heads, head_dim, capacity, page_tokens, n_sink, lsh_tables, lsh_bits, max_tokens,
-                              max_prompt_tokens, max_frames, FP32 if fp32 else BF16, device)
+                              max_prompt_tokens, max_frames, FP32 if fp32 else BF16, device, search_bits)
+        self.search_bits = search_bits
+        self.max_tokens = max_tokens
         nbytes = self.lib.fastar_cache_workspace_bytes(C.byref(self.desc))
         if nbytes == 0:
             raise FastarError(ERR_INVALID_ARG, "fastar_cache_workspace_bytes")
@@ -160,6 +164,17 @@ class Cache:
                                             out["v"].ctypes.data if kv else None, out["count"].ctypes.data,
                                             out["stamp"].ctypes.data, out["code"].ctypes.data, out["len"].ctypes.data,
                                             out["now"].ctypes.data, _stream()), "fastar_cache_export")
+        return out
+
+    def export_search_codes(self, n_new: int = 0) -> Dict[str, np.ndarray]:
+        """8-bit search only: the code rows of every slot [H][CAP][128] and of the last update's n_new keys."""
+        out = dict(cache=np.empty((self.H, self.CAP, 128), np.uint8))
+        if n_new > 0:
+            out["new"] = np.empty((self.H, n_new, 128), np.uint8)
+        with self.torch.cuda.device(self.device):
+            _check(self.lib.fastar_cache_export_search_codes(self.handle, out["cache"].ctypes.data,
+                                                             out["new"].ctypes.data if n_new > 0 else None, n_new, _stream()),
+                   "fastar_cache_export_search_codes")
         return out
 
     def import_state(self, k_bits: np.ndarray, v_bits: np.ndarray, length: np.ndarray, count: Optional[np.ndarray] = None,

@@ -3,6 +3,7 @@ oracle.  This module imports only the oracle and numpy; it never touches the CUD
 two implementations stay independent.  Near-ties have several correct answers, hence the stages:
 
   T1  accept j iff cos_oracle(i, j) >= best_i - 1e-4                  (bit-equal wherever the margin is larger)
+      (8-bit search: the quantiser is checked byte by byte, then the scores of the codes produced, margin 5e-4)
   T2  matched flags agree wherever |best_i - tau| > 1e-4
   T3/T4  the decisions taken are fed to the oracle's merge -> dest, len, count, stamp, K rows bit-exact,
          V rows within one bf16 ulp
@@ -13,13 +14,14 @@ two implementations stay independent.  Near-ties have several correct answers, h
 """
 from __future__ import annotations
 
-from typing import Dict, List, Optional, Sequence
+from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
 
 from oracle import fastar_oracle as O
 
 MARGIN = 1e-4
+MARGIN_Q8 = 5e-4      # 8-bit search: the fp8 tensor-core accumulation is not bit-exact fp32
 ATT_MAX_ABS = 2e-2
 ATT_REL_L2 = 1e-2
 
@@ -43,27 +45,36 @@ def oracle_heads_from_export(state: Dict[str, np.ndarray], n_sink: int = 0) -> L
 
 def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float, match: np.ndarray,
                  sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
-                 rows: Optional[np.ndarray] = None) -> O.HeadCache:
+                 rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None) -> O.HeadCache:
     """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
-    exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases)."""
+    exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases).
+    `codes` = (codes of the new keys [n][128], codes of the pre-call cache [>= L][128]) as the GPU computed them
+    selects the 8-bit search: the scores are then the oracle's quantised scores of those codes (the quantiser
+    itself is checked by check_search_codes)."""
     n = K_new.shape[0]
     K64, V64 = K_new.astype(np.float64), V_new.astype(np.float64)
     matched = match >= 0
     idx = np.arange(n) if rows is None else rows
+    margin = MARGIN if codes is None else MARGIN_Q8
+    sim_tol = 2e-5 if codes is None else MARGIN_Q8
     if pre.L > 0:
-        cosm = O.cosine_matrix(K64[idx], pre.K[: pre.L])
+        if codes is None:
+            cosm = O.cosine_matrix(K64[idx], pre.K[: pre.L])
+        else:
+            d = K_new.shape[1]
+            cosm = O.quantized_score_matrix(codes[0][idx, :d], codes[1][: pre.L, :d])
         cbest = cosm.max(axis=1)
         # T1: the slot reported (for matched tokens) is within the margin of the best
         mi = np.flatnonzero(matched[idx])
         got = cosm[mi, match[idx][mi]]
-        assert np.all(got >= cbest[mi] - MARGIN), "T1: matched slot is not a (near-)best slot"
-        uniq = (cosm >= cbest[:, None] - MARGIN).sum(axis=1) == 1
+        assert np.all(got >= cbest[mi] - margin), "T1: matched slot is not a (near-)best slot"
+        uniq = (cosm >= cbest[:, None] - margin).sum(axis=1) == 1
         ui = mi[uniq[mi]]
         assert np.array_equal(match[idx][ui], np.argmax(cosm[ui], axis=1)), "T1: index differs outside the tie window"
         # the similarity reported is the cosine of the best slot
-        assert np.max(np.abs(sim[idx] - cbest)) <= 2e-5, "T1: similarity value"
+        assert np.max(np.abs(sim[idx] - cbest)) <= sim_tol, "T1: similarity value"
         # T2
-        far = np.abs(cbest - tau) > MARGIN
+        far = np.abs(cbest - tau) > margin
         assert np.array_equal(matched[idx][far], (cbest >= tau)[far]), "T2: threshold decision"
     else:
         assert not matched.any() and np.all(sim == 0)
@@ -83,6 +94,24 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
     assert (int(stats[0]), int(stats[1]), int(stats[2]), int(stats[3]), int(stats[4]), int(stats[5]), int(stats[6])) == (
         st["matched"], st["touched"], st["appended"], st["evicted_slots"], st["evicted_tokens"], st["length"], 1), "stats"
     return ref
+
+
+def check_search_codes(X: np.ndarray, got: np.ndarray, what: str) -> None:
+    """8-bit search codes of the rows of X ([n][d] float) as the GPU wrote them ([n][128] bytes) against the
+    oracle's quantiser.  The GPU scales in fp32, the oracle in fp64, so a component may land on the other side of a
+    rounding boundary when it sits on one: such a byte must be a neighbouring code and the exact scaled value must
+    lie at the midpoint of the two.  Bytes past d are zero."""
+    n, d = X.shape
+    assert got.shape == (n, 128) and not got[:, d:].any(), f"{what}: padding bytes"
+    want = O.key_codes_e4m3(X)
+    diff = got[:, :d] != want
+    assert diff.mean() < 1e-3, f"{what}: {diff.mean():.2e} of the code bytes differ"
+    if diff.any():
+        X64 = X.astype(np.float64)
+        nrm = np.sqrt((X64 * X64).sum(axis=1, keepdims=True))
+        y = np.divide(X64, nrm, out=np.zeros_like(X64), where=nrm > 0) * O.E4M3_SCALE
+        a, b = O.e4m3_decode(got[:, :d][diff]), O.e4m3_decode(want[diff])
+        assert np.all(np.abs(y[diff] - 0.5 * (a + b)) <= 2e-3 * np.abs(a - b) + 1e-9), f"{what}: code off a rounding boundary"
 
 
 def unpack_codes(packed: np.ndarray, tables: int) -> np.ndarray:

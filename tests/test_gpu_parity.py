@@ -16,23 +16,33 @@ def _gpu():
     return torch, fastar
 
 
-def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None):
+def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16):
     torch, fastar = _gpu()
     return fastar.Cache(cfg.num_heads, cfg.head_dim, capacity or cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables,
                         cfg.lsh_bits, max_tokens=max_tokens or cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64),
-                        max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32)
+                        max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32, search_bits=search_bits)
 
 
 def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False):
     """Runs one update on the GPU and checks it against the oracle heads `heads` (advanced in place)."""
     torch, fastar = _gpu()
+    q8 = cache.search_bits == 8
+    pre_codes = cache.export_search_codes()["cache"] if q8 else None      # codes of the cache the search will see
     res = cache.update(fastar.to_device(K, fp32), fastar.to_device(V, fp32), frame_len, tau)
     assert cache.status() == 0
     post = cache.export_state()
     match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
     synced = P.oracle_heads_from_export(post, heads[0].n_sink)
+    post_codes = cache.export_search_codes(K.shape[1]) if q8 else None
     for h in range(K.shape[0]):
-        ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h)
+        codes = None
+        if q8:
+            # the quantiser, byte by byte: codes of the new keys, and of every live slot after the update
+            P.check_search_codes(np.asarray(K[h], np.float64), post_codes["new"][h], f"new-key codes, head {h}")
+            Lh = int(post["len"][h])
+            P.check_search_codes(P.bits_to_f64(post["k"][h, :Lh]), post_codes["cache"][h, :Lh], f"cache codes, head {h}")
+            codes = (post_codes["new"][h], pre_codes[h])
+        ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes)
         # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
         # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
         synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
@@ -77,9 +87,9 @@ def gpu_annca_checked(cache, cfg, Q, Kp, Vp, keep, fp32=False):
     return res
 
 
-def full_step(cfg, fp32=False, tau=None, n_sink=0):
+def full_step(cfg, fp32=False, tau=None, n_sink=0, search_bits=16):
     w = synth.Workload(cfg)
-    cache = make_cache(cfg, w, fp32, n_sink)
+    cache = make_cache(cfg, w, fp32, n_sink, search_bits=search_bits)
     heads = [O.HeadCache(cfg.capacity, cfg.head_dim, n_sink) for _ in range(cfg.num_heads)]
     for ci in range(cfg.prior_chunks):                 # prior chunks enter un-merged (tau > 1): plain append
         _, K, V = w.chunk(ci)
@@ -128,6 +138,26 @@ def test_both_similarity_kernels(kernel, d, pt, monkeypatch):
     Q, K, V = w.chunk(cfg.prior_chunks + 1)
     post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
     assert post["count"].max() > 1
+
+
+@pytest.mark.parametrize("d,pt", [(128, 128), (64, 64), (128, 64)])
+def test_eight_bit_quantised_search(d, pt):
+    # TempCache's correspondence search on fp8 codes: quantiser checked byte by byte against the oracle's, top-1 /
+    # threshold decisions against the oracle's scores of those codes, then the usual teacher-forced merge; a second
+    # merging chunk runs against codes the commit copied, and the attention calls run on the resulting cache.
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    cache, w, heads, post, _, _ = full_step(cfg, search_bits=8)
+    Q, K, V = w.chunk(cfg.prior_chunks + 1)
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
+    assert post["count"].max() > 1
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+    # import rebuilds the codes from the keys
+    st = cache.export_state()
+    cache.import_state(st["k"], st["v"], st["len"], st["count"], st["stamp"], now=int(st["now"][0]))
+    codes = cache.export_search_codes()["cache"]
+    for h in range(cfg.num_heads):
+        Lh = int(st["len"][h])
+        P.check_search_codes(P.bits_to_f64(st["k"][h, :Lh]), codes[h, :Lh], f"codes after import, head {h}")
 
 
 def test_dense_mode_equals_eq1_on_uncompressed_cache():
