@@ -23,16 +23,27 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
   }
 }
 
-// Copy the 128-byte search code of new token `tok` into the code row of (page, row): LPR lanes, 128 / LPR bytes each.
+// The 128-byte search code of a new token goes to the code row of its slot: LPR lanes, 128 / LPR bytes each.  The
+// load is issued with the other row loads (it could alias the pools as far as the compiler knows, so it must not
+// sit behind their stores), the store with the other stores.
 template <int LPR>
-__device__ __forceinline__ void copy_code_row(const CacheView& c, int h, int tok, int page, int row_in_page, int sl) {
+__device__ __forceinline__ uint4 load_code_part(const CacheView& c, int h, int tok, int sl) {
   const uint8_t* src = c.k8_new + (static_cast<int64_t>(h) * c.max_tokens + tok) * 128;
-  uint8_t* dst = c.pool_k8 + (static_cast<int64_t>(page) * c.PT + row_in_page) * 128;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
   if (LPR == 16) {
-    *reinterpret_cast<uint2*>(dst + sl * 8) = *reinterpret_cast<const uint2*>(src + sl * 8);
+    const uint2 t = *reinterpret_cast<const uint2*>(src + sl * 8);
+    v.x = t.x;
+    v.y = t.y;
   } else {
-    *reinterpret_cast<uint4*>(dst + sl * 16) = *reinterpret_cast<const uint4*>(src + sl * 16);
+    v = *reinterpret_cast<const uint4*>(src + sl * 16);
   }
+  return v;
+}
+template <int LPR>
+__device__ __forceinline__ void store_code_part(const CacheView& c, int page, int row_in_page, int sl, const uint4& v) {
+  uint8_t* dst = c.pool_k8 + (static_cast<int64_t>(page) * c.PT + row_in_page) * 128;
+  if (LPR == 16) *reinterpret_cast<uint2*>(dst + sl * 8) = make_uint2(v.x, v.y);
+  else *reinterpret_cast<uint4*>(dst + sl * 16) = v;
 }
 
 template <int D>
@@ -107,6 +118,8 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
       }
     }
     const uint4 krow = *reinterpret_cast<const uint4*>(kh + best_i * ts + sl * 8);
+    uint4 code8 = make_uint4(0u, 0u, 0u, 0u);
+    if (c.pool_k8) code8 = load_code_part<LPR>(c, h, best_i, sl);
     float rn = 0.f;
     uint32_t code = 0;
     if (sl == 0) {
@@ -121,7 +134,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
     vout.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
     *reinterpret_cast<uint4*>(c.pool_v + ro) = vout;
     *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
-    if (c.pool_k8) copy_code_row<LPR>(c, h, best_i, page, slot % c.PT, sl);
+    if (c.pool_k8) store_code_part<LPR>(c, page, slot % c.PT, sl, code8);
     if (sl == 0) {
       c.count[sb + slot] = m_old + g;
       c.stamp[sb + slot] = now;
@@ -134,6 +147,8 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
     const int slot = c.dest[tb + i];
     const uint4 krow = *reinterpret_cast<const uint4*>(kh + i * ts + sl * 8);
     const uint4 vrow = *reinterpret_cast<const uint4*>(vh + i * ts + sl * 8);
+    uint4 code8 = make_uint4(0u, 0u, 0u, 0u);
+    if (c.pool_k8) code8 = load_code_part<LPR>(c, h, i, sl);
     float rn = 0.f;
     uint32_t code = 0;
     if (sl == 0) {
@@ -144,7 +159,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
     const int64_t ro = (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D + sl * 8;
     *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
     *reinterpret_cast<uint4*>(c.pool_v + ro) = vrow;
-    if (c.pool_k8) copy_code_row<LPR>(c, h, i, page, slot % c.PT, sl);
+    if (c.pool_k8) store_code_part<LPR>(c, page, slot % c.PT, sl, code8);
     if (sl == 0) {
       c.count[sb + slot] = 1;
       c.stamp[sb + slot] = now;
