@@ -23,6 +23,17 @@ __device__ __forceinline__ int block_sum(int v, int* red) {
   for (int w = 0; w < nw; ++w) t += red[w];
   return t;
 }
+__device__ __forceinline__ int block_max(int v, int* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  int t = red[0];
+  for (int w = 1; w < nw; ++w) t = max(t, red[w]);
+  return t;
+}
 // exclusive scan of one value per thread; *total receives the block sum
 __device__ __forceinline__ int block_exscan(int v, int* red, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -252,7 +263,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
   // groups: 16 consecutive slots per thread and pass (four 128-bit loads in flight; counts past the live length
   // are zero and the capacity is a multiple of 128, so whole vectors can be read up to the capacity).  The
   // numbers of groups and of members are scanned together, packed into one word (both stay below 2^16).
-  int seg_run = 0, mem_run = 0, touched_ns = 0;
+  int seg_run = 0, mem_run = 0;
   for (int j0 = 0; j0 < L; j0 += 16 * blockDim.x) {
     const int j = j0 + 16 * tid;
     int cn[16];
@@ -281,7 +292,6 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
         c.segslot[tb + seg] = j + u;
         c.segpos[gb + seg] = mem;
         c.cur[sb + j + u] = mem;
-        if (j + u >= c.n_sink) ++touched_ns;
         ++seg;
         mem += cn[u];
       }
@@ -290,7 +300,6 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
     mem_run += tot_mem;
   }
   const int n_seg = seg_run, M = mem_run;
-  touched_ns = block_sum(touched_ns, red);
   if (tid == 0) c.segpos[gb + n_seg] = M;
 
   // unmatched tokens in token order
@@ -311,43 +320,95 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
   const int A = min(U, c.CAP - L);
   const int E = U - A;
   int ok = 1;
+  // Eviction.  evictable = live, past the sink prefix, stamp < now, not touched by this update (cnt == 0); its key
+  // is its stamp, 0x7fffffff otherwise.  Every pass reads 16 consecutive slots per thread with 128-bit loads (eight
+  // of them in flight), so a pass over a 64k-slot cache is four round trips instead of sixty-four.
+  constexpr int kNever = 0x7fffffff;
+  auto evictable16 = [&](int j, int (&st)[16]) {
+    if (j < L) {                                   // j is a multiple of 16 and the capacity a multiple of 128
+      const int4* pc = reinterpret_cast<const int4*>(c.cnt + sb + j);
+      const int4* ps = reinterpret_cast<const int4*>(c.stamp + sb + j);
+      const int4 c0 = pc[0], c1 = pc[1], c2 = pc[2], c3 = pc[3];
+      const int4 s0 = ps[0], s1 = ps[1], s2 = ps[2], s3 = ps[3];
+      const int cn[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
+      const int sp[16] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w, s2.x, s2.y, s2.z, s2.w, s3.x, s3.y, s3.z, s3.w};
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        st[u] = (j + u < L && j + u >= c.n_sink && cn[u] == 0 && sp[u] < now) ? sp[u] : kNever;
+    } else {
+#pragma unroll
+      for (int u = 0; u < 16; ++u) st[u] = kNever;
+    }
+  };
+  int smin = kNever, smax = -1;
   if (E > 0) {
+    // one pass: how many evictable slots there are, and the range of their stamps
     int cand = 0;
-    for (int j = tid; j < L; j += blockDim.x) cand += (j >= c.n_sink && c.stamp[sb + j] < now) ? 1 : 0;
-    cand = block_sum(cand, red) - touched_ns;
+    for (int j0 = 0; j0 < L; j0 += 16 * blockDim.x) {
+      int st[16];
+      evictable16(j0 + 16 * tid, st);
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        if (st[u] != kNever) { ++cand; smin = min(smin, st[u]); smax = max(smax, st[u]); }
+    }
+    cand = block_sum(cand, red);
+    smin = -block_max(-smin, red);
+    smax = block_max(smax, red);
     if (cand < E) ok = 0;
   }
   int evicted_tokens = 0;
   if (ok && E > 0) {
-    // evictable = live, past the sink prefix, stamp < now, not touched by this update (cnt == 0).
     // smallest stamp value s* such that at least E evictable slots have stamp <= s*
-    auto evictable_stamp = [&](int j) -> int {
-      return (j < L && j >= c.n_sink && c.cnt[sb + j] == 0) ? c.stamp[sb + j] : 0x7fffffff;
-    };
-    int lo = 0, hi = now - 1;
+    int lo = smin, hi = smax;
     while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
+      const int mid = lo + ((hi - lo) >> 1);
       int cn = 0;
-      for (int j = tid; j < L; j += blockDim.x) cn += evictable_stamp(j) <= mid ? 1 : 0;
+      for (int j0 = 0; j0 < L; j0 += 16 * blockDim.x) {
+        int st[16];
+        evictable16(j0 + 16 * tid, st);
+#pragma unroll
+        for (int u = 0; u < 16; ++u) cn += st[u] <= mid ? 1 : 0;
+      }
       cn = block_sum(cn, red);
       if (cn >= E) hi = mid; else lo = mid + 1;
     }
     const int sstar = lo;
     int c_less = 0;
-    for (int j = tid; j < L; j += blockDim.x) c_less += evictable_stamp(j) < sstar ? 1 : 0;
+    for (int j0 = 0; j0 < L; j0 += 16 * blockDim.x) {
+      int st[16];
+      evictable16(j0 + 16 * tid, st);
+#pragma unroll
+      for (int u = 0; u < 16; ++u) c_less += st[u] < sstar ? 1 : 0;
+    }
     c_less = block_sum(c_less, red);
     const int need_eq = E - c_less;
+    // ordered compaction of the victims: all slots below s*, and the first need_eq slots at s*
     int eq_run = 0, out_run = 0;
-    for (int j0 = 0; j0 < L; j0 += blockDim.x) {
-      const int j = j0 + tid;
-      const int stp = evictable_stamp(j);
-      const int is_eq = stp == sstar ? 1 : 0;
+    for (int j0 = 0; j0 < L; j0 += 16 * blockDim.x) {
+      const int j = j0 + 16 * tid;
+      int st[16];
+      evictable16(j, st);
+      int my_eq = 0;
+#pragma unroll
+      for (int u = 0; u < 16; ++u) my_eq += st[u] == sstar ? 1 : 0;
       int tot_eq;
-      const int eq_rank = eq_run + block_exscan(is_eq, red, &tot_eq);
-      const int take = (stp < sstar || (is_eq && eq_rank < need_eq)) ? 1 : 0;
+      int eq_rank = eq_run + block_exscan(my_eq, red, &tot_eq);
+      int my_take = 0;
+      unsigned take_mask = 0;
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        const bool is_eq = st[u] == sstar;
+        const bool take = st[u] < sstar || (is_eq && eq_rank < need_eq);
+        eq_rank += is_eq ? 1 : 0;
+        take_mask |= (take ? 1u : 0u) << u;
+        my_take += take ? 1 : 0;
+      }
       int tot_take;
-      const int pos = out_run + block_exscan(take, red, &tot_take);
-      if (take) keys[pos] = (static_cast<unsigned long long>(static_cast<uint32_t>(stp)) << 32) | static_cast<uint32_t>(j);
+      int pos = out_run + block_exscan(my_take, red, &tot_take);
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        if ((take_mask >> u) & 1u)
+          keys[pos++] = (static_cast<unsigned long long>(static_cast<uint32_t>(st[u])) << 32) | static_cast<uint32_t>(j + u);
       eq_run += tot_eq;
       out_run += tot_take;
     }
