@@ -64,7 +64,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-
 // Non-blocking test (try_wait may suspend the thread for a while before it answers; a loop that watches two
 // barriers wants the answer at once).
 __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
