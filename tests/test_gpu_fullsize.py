@@ -115,3 +115,42 @@ def test_c2_style_rollout_invariants():
         assert bool(torch.isfinite(out.float()).all())
         lens.append(state["len"].copy())
     assert evicted.sum() > 0 and np.all(lens[-1] == cfg.capacity)
+
+
+def test_c1_full_size_update_with_eight_bit_search_sampled():
+    """The 8-bit quantised correspondence search at full c1 size: quantiser and top-1 on sampled tokens of three heads
+    (the oracle's scores of the GPU's codes), merge bookkeeping in full for those heads, invariants for all heads."""
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.CONFIGS["c1"]
+    w = synth.Workload(cfg)
+    H, n = cfg.num_heads, cfg.chunk_tokens
+    cache = fastar.Cache(H, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
+                         max_tokens=n, max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk, search_bits=8)
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, 2.0, outputs=False)
+    assert cache.status() == 0
+    pre = cache.export_state()
+    pre_codes = cache.export_search_codes()["cache"]
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    res = cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau)
+    assert cache.status() == 0
+    post = cache.export_state()
+    codes = cache.export_search_codes(n)
+    match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    rng = np.random.default_rng(1)
+    pre_heads = P.oracle_heads_from_export(pre)
+    for h in (0, 6, 11):
+        rows = np.sort(rng.choice(n, 96, replace=False))
+        P.check_search_codes(np.asarray(K[h][rows], np.float64), codes["new"][h][rows], f"new-key codes, head {h}")
+        Lh = int(post["len"][h])
+        samp = np.sort(rng.choice(Lh, 2048, replace=False))
+        P.check_search_codes(P.bits_to_f64(post["k"][h, samp]), codes["cache"][h, samp], f"cache codes, head {h}")
+        P.check_update(pre_heads[h], K[h], V[h], cfg.frame_len, cfg.tau, match[h], sim[h], dest[h], stats[h], post, h, rows=rows,
+                       codes=(codes["new"][h], pre_codes[h]))
+    for h in range(H):
+        L = int(post["len"][h])
+        assert L == int(pre["len"][h]) + int(stats[h, 2]) <= cfg.capacity
+        assert int(post["count"][h, :L].sum()) == (cfg.prior_chunks + 1) * n
+        assert int(stats[h, 0]) + int(stats[h, 2]) + int(stats[h, 3]) == n

@@ -160,6 +160,35 @@ def test_eight_bit_quantised_search(d, pt):
         P.check_search_codes(P.bits_to_f64(st["k"][h, :Lh]), codes[h, :Lh], f"codes after import, head {h}")
 
 
+def test_eight_bit_search_empty_cache_eviction_and_capacity_error():
+    # 8-bit search through the degenerate cases: first update into an empty cache (nothing to match), eviction at a
+    # small capacity (victims' code rows are overwritten with the new tokens' codes), and a rejected update.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(num_heads=2, capacity=1280, prior_chunks=0, resample=0.5)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, search_bits=8)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(5):                                     # 600 tokens per chunk, half of them new: fills 1280 and evicts
+        _, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
+    assert int(post["len"].max()) == cfg.capacity
+    # a chunk that cannot be placed: every slot was touched by ... nothing, so force it with a chunk larger than what
+    # is evictable: sink prefix covering the whole cache
+    cache2 = make_cache(cfg, w, n_sink=cfg.capacity, search_bits=8)
+    heads2 = [O.HeadCache(cfg.capacity, cfg.head_dim, cfg.capacity) for _ in range(cfg.num_heads)]
+    for ci in range(2):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache2, heads2, K, V, cfg.frame_len, 2.0)
+    before = cache2.export_state()
+    codes_before = cache2.export_search_codes()["cache"]
+    _, K, V = w.chunk(2)
+    res = cache2.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, 2.0)     # 1200 + 600 > 1280, nothing evictable
+    assert cache2.status() == fastar.ERR_CAPACITY
+    after = cache2.export_state()
+    assert all(np.array_equal(before[k], after[k]) for k in ("k", "v", "count", "stamp", "len"))
+    assert np.array_equal(codes_before, cache2.export_search_codes()["cache"])
+
+
 def test_dense_mode_equals_eq1_on_uncompressed_cache():
     cfg = synth.small_config(prior_chunks=2)
     w = synth.Workload(cfg)
