@@ -379,15 +379,29 @@ def prompt_relevance(Q: np.ndarray, K_p: np.ndarray, frame_len: int) -> np.ndarr
     return np.stack([s[f * frame_len: min((f + 1) * frame_len, nq)].max(axis=0) for f in range(F)])
 
 
+def prompt_relevance_quantized(Q: np.ndarray, K_p: np.ndarray, frame_len: int) -> np.ndarray:
+    """prompt_relevance with the 8-bit search score in place of the exact dot product:
+    <q, k> is replaced by |q| |k| * (dot product of the e4m3 codes of q/|q| and k/|k|) / E4M3_SCALE^2."""
+    Q = np.asarray(Q, np.float64)
+    K_p = np.asarray(K_p, np.float64)
+    nq, d = Q.shape
+    F = -(-nq // frame_len)
+    qn = np.sqrt((Q * Q).sum(axis=1))
+    kn = np.sqrt((K_p * K_p).sum(axis=1))
+    s = quantized_score_matrix(key_codes_e4m3(Q), key_codes_e4m3(K_p)) * qn[:, None] * kn[None, :] / np.sqrt(d)
+    return np.stack([s[f * frame_len: min((f + 1) * frame_len, nq)].max(axis=0) for f in range(F)])
+
+
 def annca(Q: np.ndarray, K_p: np.ndarray, V_p: np.ndarray, frame_len: int, keep: int,
-          sel: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+          sel: Optional[np.ndarray] = None, search_bits: int = 16) -> Dict[str, np.ndarray]:
     """AnnCA of one head: per frame keep the `keep` most relevant prompt tokens, then
-    o_i = softmax_{p in sel[f(i)]}(<q_i, k_p>/sqrt(d)) v_p."""
+    o_i = softmax_{p in sel[f(i)]}(<q_i, k_p>/sqrt(d)) v_p.  search_bits = 8 ranks the prompt tokens
+    by the 8-bit quantised relevance; the attention over the kept tokens is unchanged."""
     Q = np.asarray(Q, np.float64)
     K_p = np.asarray(K_p, np.float64)
     V_p = np.asarray(V_p, np.float64)
     nq, d = Q.shape
-    r = prompt_relevance(Q, K_p, frame_len)
+    r = prompt_relevance_quantized(Q, K_p, frame_len) if search_bits == 8 else prompt_relevance(Q, K_p, frame_len)
     if sel is None:
         sel = topk_lowest_index(r, keep)
     O = np.zeros((nq, d))

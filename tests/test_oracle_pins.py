@@ -437,3 +437,29 @@ def test_quantised_search_is_a_close_approximation_of_the_cosine_search():
     c2 = c.copy()
     res = O.tempcache_update(c2, Kn, rng.standard_normal((n, d)), 100, 0.9, search_bits=8)
     assert res["stats"]["matched"] >= n // 2 - 2 and res["stats"]["matched"] <= n // 2 + 2
+
+
+def test_quantised_prompt_relevance():
+    rng = _rng(34)
+    d, nq, npr, fl = 64, 90, 40, 30
+    Q = rng.standard_normal((nq, d)) * rng.uniform(0.5, 3.0, (nq, 1))
+    Kp = rng.standard_normal((npr, d)) * rng.uniform(0.5, 3.0, (npr, 1))
+    r8 = O.prompt_relevance_quantized(Q, Kp, fl)
+    r = O.prompt_relevance(Q, Kp, fl)
+    assert r8.shape == r.shape == (3, npr)
+    # close to the exact relevance on the scale |q||k|/sqrt(d) (cosine error of the codes < 0.02 at d = 64)
+    scale = np.sqrt((Q * Q).sum(1)).max() * np.sqrt((Kp * Kp).sum(1)) / np.sqrt(d)
+    assert np.all(np.abs(r8 - r) <= 0.03 * scale[None, :])
+    # homogeneous of degree one in q and in k (the codes only see directions)
+    assert np.allclose(O.prompt_relevance_quantized(2.5 * Q, Kp, fl), 2.5 * r8, rtol=1e-12)
+    assert np.allclose(O.prompt_relevance_quantized(Q, 0.5 * Kp, fl), 0.5 * r8, rtol=1e-12)
+    # brute force, Python loops, one frame
+    cq, ck = O.e4m3_decode(O.key_codes_e4m3(Q[:fl])), O.e4m3_decode(O.key_codes_e4m3(Kp[:5]))
+    for p in range(5):
+        best = max(float(np.linalg.norm(Q[i])) * float(np.linalg.norm(Kp[p])) *
+                   sum(float(cq[i, k]) * float(ck[p, k]) for k in range(d)) / 256.0 / np.sqrt(d) for i in range(fl))
+        assert abs(best - r8[0, p]) < 1e-10
+    # planted relevant tokens are still found
+    a = O.annca(Q, Kp, rng.standard_normal((npr, d)), fl, 8, search_bits=8)
+    b = O.annca(Q, Kp, rng.standard_normal((npr, d)), fl, 8)
+    assert all(len(set(a["sel"][f]) & set(b["sel"][f])) >= 6 for f in range(3))
