@@ -68,12 +68,16 @@ typedef struct {
   int32_t max_frames;        /* largest number of frames per AnnCA call */
   int32_t dtype;             /* fastar_dtype_t of the tensors the caller passes */
   int32_t device;            /* CUDA device ordinal */
-  int32_t search_bits;       /* precision of TempCache's correspondence search: 16 (or 0) = the bf16 keys,
+  int32_t search_bits;       /* precision of the similarity searches (TempCache's correspondence search and
+                              * AnnCA's prompt relevance): 16 (or 0) = the bf16 keys,
                               * 8 = 8-bit quantised search (Section 5.1; the paper's default): every key is
                               * reduced to x/|x|*16 in fp8 e4m3 (round to nearest even, saturating), kept in a
                               * second paged pool of 128-byte rows, and the similarity of two keys is the
                               * dot product of their codes / 256.  Top-1, ties and the threshold rule are
-                              * unchanged; the merge itself always uses the bf16 keys and values. */
+                              * unchanged; the merge itself always uses the bf16 keys and values.  AnnCA
+                              * then ranks prompt tokens by max_i code(q_i).code(k_p) |q_i| |k_p| / (256 sqrt d)
+                              * (codes of its queries and prompt keys are made per call); the attention over
+                              * the kept tokens uses the bf16 tensors. */
 } fastar_cache_desc;
 
 typedef struct {
@@ -119,6 +123,13 @@ int fastar_cache_export(fastar_cache_t* cache, uint16_t* host_k, uint16_t* host_
  * quantised similarity search; used by the tests to check the quantiser and the search separately.) */
 int fastar_cache_export_search_codes(fastar_cache_t* cache, uint8_t* host_cache_codes, uint8_t* host_new_codes,
                                      int32_t n, void* stream);
+
+/* 8-bit search only (else FASTAR_ERR_UNSUPPORTED_SHAPE): copy the search codes the most recent
+ * fastar_annca_attention call (one that selected, sel_in == NULL) computed for its nq queries,
+ * host_q_codes [H][nq][128], and its np prompt keys, host_prompt_codes [H][np][128], to the host and
+ * synchronise the stream.  Same code format as above; either pointer may be NULL.  (Sections 5.1, 5.3.) */
+int fastar_cache_export_annca_codes(fastar_cache_t* cache, uint8_t* host_q_codes, uint8_t* host_prompt_codes,
+                                    int32_t nq, int32_t np, void* stream);
 
 /* Load a state (same layouts; count/stamp NULL = all ones / all zeros).  Slots >= len[h] are
  * cleared.  Derived per-slot data (1/|k|, log2 m, LSH codes, search codes, histograms) are recomputed on the

@@ -379,16 +379,21 @@ def prompt_relevance(Q: np.ndarray, K_p: np.ndarray, frame_len: int) -> np.ndarr
     return np.stack([s[f * frame_len: min((f + 1) * frame_len, nq)].max(axis=0) for f in range(F)])
 
 
-def prompt_relevance_quantized(Q: np.ndarray, K_p: np.ndarray, frame_len: int) -> np.ndarray:
+def prompt_relevance_quantized(Q: np.ndarray, K_p: np.ndarray, frame_len: int, codes_q: Optional[np.ndarray] = None,
+                               codes_k: Optional[np.ndarray] = None) -> np.ndarray:
     """prompt_relevance with the 8-bit search score in place of the exact dot product:
-    <q, k> is replaced by |q| |k| * (dot product of the e4m3 codes of q/|q| and k/|k|) / E4M3_SCALE^2."""
+    <q, k> is replaced by |q| |k| * (dot product of the e4m3 codes of q/|q| and k/|k|) / E4M3_SCALE^2.
+    codes_q / codes_k, when given, replace the codes computed here (a test passes the codes another
+    implementation produced once it has checked them against key_codes_e4m3)."""
     Q = np.asarray(Q, np.float64)
     K_p = np.asarray(K_p, np.float64)
     nq, d = Q.shape
     F = -(-nq // frame_len)
     qn = np.sqrt((Q * Q).sum(axis=1))
     kn = np.sqrt((K_p * K_p).sum(axis=1))
-    s = quantized_score_matrix(key_codes_e4m3(Q), key_codes_e4m3(K_p)) * qn[:, None] * kn[None, :] / np.sqrt(d)
+    codes_q = key_codes_e4m3(Q) if codes_q is None else codes_q
+    codes_k = key_codes_e4m3(K_p) if codes_k is None else codes_k
+    s = quantized_score_matrix(codes_q, codes_k) * qn[:, None] * kn[None, :] / np.sqrt(d)
     return np.stack([s[f * frame_len: min((f + 1) * frame_len, nq)].max(axis=0) for f in range(F)])
 
 

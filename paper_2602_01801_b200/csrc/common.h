@@ -73,6 +73,11 @@ struct CacheView {
   int32_t search_bits;             // 16 or 8
   uint8_t* pool_k8;                // [H*CAPB][PT][128]  fp8 e4m3 search codes of the cached keys, paged like pool_k
   uint8_t* k8_new;                 // [H][max_tokens][128]  codes of the new keys of the update in flight
+  // AnnCA's own 8-bit scratch (an AnnCA call may run beside an update on another stream)
+  uint8_t* q8_ca;                  // [H][max_tokens][128]  codes of the queries
+  uint8_t* kp8_ca;                 // [H][max_prompt][128]  codes of the prompt keys
+  float* qn_ca;                    // [H][max_tokens]  |q|
+  float* kpn_ca;                   // [H][max_prompt]  |k_p|
 };
 
 inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
@@ -95,6 +100,10 @@ int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtenso
 int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, const float* rnorm,
                          int64_t rn_stride, uint8_t* out, int64_t out_rows_per_head, cudaStream_t st);
 int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, cudaStream_t st);
+int launch_quantize_rows(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint8_t* out,
+                         int64_t out_rows_per_head, float* norm_out, int64_t norm_stride, cudaStream_t st);
+int launch_c1_relevance_fp8(const CacheView& c, const CUtensorMap& tm_q8, const CUtensorMap& tm_kp8, const float* qn,
+                            const float* kn, int nq, int np, int frame_len, cudaStream_t st);
 
 // attn_kernels.cu
 struct AttnArgs {

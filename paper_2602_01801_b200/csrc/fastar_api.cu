@@ -119,6 +119,10 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.search_bits = d.search_bits == 8 ? 8 : 16;
   t.pool_k8 = t.search_bits == 8 ? take(H * CAP * 128) : nullptr;
   t.k8_new = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
+  t.q8_ca = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
+  t.kp8_ca = t.search_bits == 8 ? take(H * MP * 128) : nullptr;
+  t.qn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MT * 4)) : nullptr;
+  t.kpn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MP * 4)) : nullptr;
   for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
   for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
   cur = (cur + 1023) & ~static_cast<size_t>(1023);
@@ -330,6 +334,25 @@ int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_code
   return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
 }
 
+int fastar_cache_export_annca_codes(fastar_cache_t* c, uint8_t* host_q_codes, uint8_t* host_prompt_codes, int32_t nq, int32_t np,
+                                    void* stream) {
+  if (!c) return FASTAR_ERR_INVALID_ARG;
+  const CacheView& v = c->v;
+  if (v.search_bits != 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if ((host_q_codes && (nq < 1 || nq > v.max_tokens)) || (host_prompt_codes && (np < 1 || np > v.max_prompt))) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool ok = true;
+  if (host_q_codes)
+    ok &= cudaMemcpy2DAsync(host_q_codes, static_cast<size_t>(nq) * 128, v.q8_ca, static_cast<size_t>(v.max_tokens) * 128,
+                            static_cast<size_t>(nq) * 128, v.H, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (host_prompt_codes)
+    ok &= cudaMemcpy2DAsync(host_prompt_codes, static_cast<size_t>(np) * 128, v.kp8_ca, static_cast<size_t>(v.max_prompt) * 128,
+                            static_cast<size_t>(np) * 128, v.H, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
 int fastar_cache_import(fastar_cache_t* c, const uint16_t* host_k, const uint16_t* host_v, const int32_t* count,
                         const int32_t* stamp, const int32_t* len, int32_t now, void* stream) {
   if (!c || !host_k || !host_v || !len || now < 0) return FASTAR_ERR_INVALID_ARG;
@@ -506,10 +529,23 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
     a.sel_stride = keep_tokens;
     a.sel_head_stride = static_cast<int64_t>(F) * keep_tokens;
   } else {
-    r = make_map(c, &tm_kp, kpb, v.D, np, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
-    if (r != FASTAR_OK) return r;
     if (cudaMemsetAsync(v.rel, 0, static_cast<size_t>(v.H) * v.max_frames * v.max_prompt * 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-    ACCK(FASTAR_K_C1_RELEVANCE, launch_c1_relevance(v, tm_q, tm_kp, nq, np, frame_len, F, st));
+    float rel_scale = 1.0f / sqrtf(static_cast<float>(v.D));
+    if (v.search_bits == 8) {
+      // relevance on the 8-bit codes of the directions, scaled back by the norms (Section 5.1 quantised search)
+      CUtensorMap tm_q8, tm_kp8;
+      r = make_map_codes(c, &tm_q8, v.q8_ca, nq, v.H, static_cast<uint64_t>(v.max_tokens) * 128, 128);
+      if (r == FASTAR_OK) r = make_map_codes(c, &tm_kp8, v.kp8_ca, np, v.H, static_cast<uint64_t>(v.max_prompt) * 128, 128);
+      if (r != FASTAR_OK) return r;
+      ACCK(FASTAR_K_HASH, launch_quantize_rows(v, qb, nq, qhs, qts, v.q8_ca, v.max_tokens, v.qn_ca, v.max_tokens, st));
+      ACCK(FASTAR_K_HASH, launch_quantize_rows(v, kpb, np, khs, kts, v.kp8_ca, v.max_prompt, v.kpn_ca, v.max_prompt, st));
+      ACCK(FASTAR_K_C1_RELEVANCE, launch_c1_relevance_fp8(v, tm_q8, tm_kp8, v.qn_ca, v.kpn_ca, nq, np, frame_len, st));
+      rel_scale *= 1.0f / 256.0f;
+    } else {
+      r = make_map(c, &tm_kp, kpb, v.D, np, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
+      if (r != FASTAR_OK) return r;
+      ACCK(FASTAR_K_C1_RELEVANCE, launch_c1_relevance(v, tm_q, tm_kp, nq, np, frame_len, F, st));
+    }
     ACCK(FASTAR_K_TOPK_PROMPT, launch_topk_prompt(v, F, np, keep, st));
     a.sel = v.selp;
     a.sel_stride = v.max_prompt;
@@ -519,7 +555,7 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
       if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
       c->launches += 1;
     }
-    if (rel_out) ACC(launch_decode_rel(v, F, np, 1.0f / sqrtf(static_cast<float>(v.D)), rel_out, st));
+    if (rel_out) ACC(launch_decode_rel(v, F, np, rel_scale, rel_out, st));
   }
   ACCK(FASTAR_K_C3_ATTENTION, launch_attention_gather(v, tm_q, a, st));
   return FASTAR_OK;

@@ -8,8 +8,11 @@
 // accumulated in fp32 by tcgen05.mma kind::f8f6f4 (K = 32 per instruction, four instructions per 128 x 128 tile, a
 // quarter of the operand bytes of the bf16 search per score), divided by 256.
 //
-//   quantize_kernel : bf16 rows + 1/|x|  ->  codes
-//   t1_fp8_kernel   : codes of the new keys x codes of the cache, row arg-max fused (ties -> lowest slot)
+//   quantize_kernel      : bf16 rows + 1/|x|  ->  codes
+//   quantize_rows_kernel : bf16 rows  ->  codes and |x| (AnnCA's queries and prompt keys, Section 5.3)
+//   search8_kernel<false>: codes of the new keys x codes of the cache, row arg-max fused (ties -> lowest slot)
+//   search8_kernel<true> : codes of the queries x codes of the prompt keys, scaled back by |q| |k|, per-frame column
+//                          maximum fused (AnnCA's prompt relevance on the quantised scores)
 // Same CTA layout as the bf16 similarity kernel: 128 new keys per CTA (resident), key tiles streamed through a TMA
 // ring, two fp32 accumulators in TMEM, eight epilogue warps, 2 CTAs per SM.  Every wait is bounded.
 #include <cuda_fp8.h>
@@ -74,6 +77,56 @@ __device__ __forceinline__ void chunk_argmax_raw(const uint32_t (&acc)[32], int 
 
 }  // namespace
 
+// Half a warp per row: |x|, then the code of x / |x| * 16 (an all-zero row gets an all-zero code and norm 0).
+__global__ void __launch_bounds__(256) quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int H, int n, int D, int64_t hs,
+                                                            int64_t ts, uint8_t* __restrict__ out, int64_t out_rows_per_head,
+                                                            float* __restrict__ norm_out, int64_t norm_stride) {
+  const int64_t rows = static_cast<int64_t>(H) * n;
+  const unsigned hmask = 0xFFFFu << (threadIdx.x & 16);
+  for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; (q >> 4) < rows;
+       q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int e8 = static_cast<int>(q & 15);
+    const int64_t rowid = q >> 4;
+    const int h = static_cast<int>(rowid / n), i = static_cast<int>(rowid % n);
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = 0.f;
+    if (e8 * 8 < D) {
+      const uint4 v = *reinterpret_cast<const uint4*>(x + h * hs + i * ts + e8 * 8);
+      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 t = __bfloat1622float2(p[e]);
+        f[2 * e] = t.x;
+        f[2 * e + 1] = t.y;
+      }
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+#pragma unroll
+    for (int o = 8; o >= 1; o >>= 1) ss += __shfl_xor_sync(hmask, ss, o);
+    const float nrm = sqrtf(ss);
+    const float s = ss > 0.f ? kCodeScale / nrm : 0.f;
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      w[e] = __nv_cvt_float2_to_fp8x2(make_float2(f[2 * e] * s, f[2 * e + 1] * s), __NV_SATFINITE, __NV_E4M3);
+    *reinterpret_cast<uint2*>(out + (static_cast<int64_t>(h) * out_rows_per_head + i) * 128 + e8 * 8) =
+        make_uint2(w[0] | (w[1] << 16), w[2] | (w[3] << 16));
+    if (e8 == 0) norm_out[h * norm_stride + i] = nrm;
+  }
+}
+
+int launch_quantize_rows(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint8_t* out,
+                         int64_t out_rows_per_head, float* norm_out, int64_t norm_stride, cudaStream_t st) {
+  if (n <= 0) return 0;
+  const int64_t total = static_cast<int64_t>(c.H) * n * 16;
+  const int grid = static_cast<int>((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+  quantize_rows_kernel<<<grid, 256, 0, st>>>(x, c.H, n, c.D, hs, ts, out, out_rows_per_head, norm_out, norm_stride);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
 // One thread per 8 components of a 128-byte code row.
 __global__ void __launch_bounds__(256) quantize_kernel(const __nv_bfloat16* __restrict__ x, int H, int n, int D, int64_t hs,
                                                        int64_t ts, const float* __restrict__ rnorm, int64_t rn_stride,
@@ -111,8 +164,21 @@ int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int6
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
+// COLMAX = false: B = the paged code pool of the cache, row arg-max.  COLMAX = true: B = `cols_b` prompt-key codes
+// of head h (rows of a dense [H][rows][128] array), per-frame column maximum of score * |q| * |k|.
+struct Search8Args {
+  int rows_a;
+  int cols_b;              // COLMAX
+  int frame_len;           // COLMAX
+  const float* qn;         // COLMAX: |q|, [H][max_tokens]
+  const float* kn;         // COLMAX: |k_p|, [H][max_prompt]
+};
+
+template <bool COLMAX>
 __global__ void __launch_bounds__(kThreads, 2)
-t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c, int rows_a) {
+search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c,
+               const Search8Args g) {
+  const int rows_a = g.rows_a;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t sbase = smem_u32(smem_raw);
   uint8_t* sgen = smem_raw;
@@ -135,7 +201,7 @@ t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int h = blockIdx.y;
   const int m0 = blockIdx.x * 128;
-  const int L = c.len[h];
+  const int L = COLMAX ? g.cols_b : c.len[h];
   const int n_tiles = (L + 127) >> 7;
   const int per = (n_tiles + gridDim.z - 1) / gridDim.z;
   const int t0 = blockIdx.z * per;
@@ -181,7 +247,7 @@ t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
       int pg0 = 0, pg1 = 0;
       for (int tl = 0; tl < ntl; ++tl) {
         const int t = t0 + tl;
-        if ((tl & 31) == 0 && tl + lane < ntl) {                 // page ids of 32 tiles with one coalesced load
+        if (!COLMAX && (tl & 31) == 0 && tl + lane < ntl) {      // page ids of 32 tiles with one coalesced load
           pg0 = pt_h[(t + lane) * pages_per_tile];
           pg1 = pages_per_tile == 2 ? pt_h[(t + lane) * pages_per_tile + 1] : 0;
         }
@@ -193,8 +259,12 @@ t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
           if (ok) {
             const uint32_t b_s = ring_s + s * kTile;
             mbar_arrive_expect_tx(bar_full + 8 * s, kTile);
-            tma_load_3d(b_s, &tm_b, bar_full + 8 * s, 0, 0, page0);
-            if (pages_per_tile == 2) tma_load_3d(b_s + c.PT * 128, &tm_b, bar_full + 8 * s, 0, 0, page1);
+            if (COLMAX) {
+              tma_load_3d(b_s, &tm_b, bar_full + 8 * s, 0, t * 128, h);   // rows past cols_b arrive as zeros
+            } else {
+              tma_load_3d(b_s, &tm_b, bar_full + 8 * s, 0, 0, page0);
+              if (pages_per_tile == 2) tma_load_3d(b_s + c.PT * 128, &tm_b, bar_full + 8 * s, 0, 0, page1);
+            }
           }
         }
       }
@@ -232,10 +302,30 @@ t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
       float best = -INFINITY;
       int best_j = -1;
       bool ok = true;
+      // COLMAX: |q| of this thread's row and the range of frames the warp's 32 rows fall in
+      const bool rvalid = row < rows_a;
+      const float qn = (COLMAX && rvalid) ? g.qn[static_cast<int64_t>(h) * c.max_tokens + row] : 0.f;
+      const int f_r = (COLMAX && rvalid) ? row / g.frame_len : -1;
+      int f_lo = (COLMAX && rvalid) ? f_r : 0x7fffffff, f_hi = f_r;
+      if (COLMAX) {
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+          f_lo = min(f_lo, __shfl_xor_sync(0xffffffffu, f_lo, o));
+          f_hi = max(f_hi, __shfl_xor_sync(0xffffffffu, f_hi, o));
+        }
+      }
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
         const int buf = tl & 1;
         const int valid_cols = min(128, L - t * 128);
+        float kn[2] = {0.f, 0.f};
+        if (COLMAX) {
+#pragma unroll
+          for (int c2 = 0; c2 < 2; ++c2) {
+            const int col = t * 128 + (wg * 2 + c2) * 32 + lane;
+            kn[c2] = col < g.cols_b ? g.kn[static_cast<int64_t>(h) * c.max_prompt + col] : 0.f;
+          }
+        }
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
         tc_fence_after();
@@ -248,10 +338,33 @@ t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
-          chunk_argmax_raw(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+          if (!COLMAX) {
+            chunk_argmax_raw(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+          } else {
+            for (int f = f_lo; f <= f_hi; ++f) {       // empty when the warp has no valid row
+              float x[32];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) x[j] = (f_r == f) ? __uint_as_float(vv[c2][j]) * qn : -INFINITY;
+              // butterfly: after it, lane l holds the maximum of column l over the 32 rows
+#pragma unroll
+              for (int o = 16, w = 32; o >= 1; o >>= 1, w >>= 1) {
+                const bool up = (lane & o) != 0;
+#pragma unroll
+                for (int j = 0; j < w / 2; ++j) {
+                  const float send = up ? x[j] : x[j + w / 2];
+                  const float keep = up ? x[j + w / 2] : x[j];
+                  x[j] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, o));
+                }
+              }
+              const int col = t * 128 + cc * 32 + lane;
+              if (col < g.cols_b)
+                atomicMax(c.rel + (static_cast<int64_t>(h) * c.max_frames + f) * c.max_prompt + col,
+                          float_to_ordered(x[0] * kn[c2]));
+            }
+          }
         }
       }
-      if (ok && row < rows_a && best_j >= 0) {
+      if (!COLMAX && ok && row < rows_a && best_j >= 0) {
         const float sim = best * (1.f / (kCodeScale * kCodeScale));
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
                                        static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
@@ -268,31 +381,60 @@ t1_fp8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ 
   }
 }
 
-// Splits of the cache range fill whole waves of 2 CTAs per SM.
-int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, cudaStream_t st) {
+static int configure_search8() {
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(t1_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess)
+    if (cudaFuncSetAttribute(search8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess ||
+        cudaFuncSetAttribute(search8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess)
       return FASTAR_ERR_CUDA;
     configured = true;
   }
+  return FASTAR_OK;
+}
+
+// Splits of the B range that fill whole waves of 2 CTAs per SM.
+static int pick_splits8(int row_tiles, int H, int max_tiles) {
   int sm_count = 148;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
   const int slots = 2 * sm_count;
-  const int row_tiles = (n + 127) / 128;
-  const int max_tiles = c.CAP / 128;
   int splits = 1;
   double best_eff = 0.0;
   for (int s = 1; s <= 16 && s <= max_tiles; ++s) {
-    const int total = row_tiles * c.H * s;
+    const int total = row_tiles * H * s;
     const double eff = static_cast<double>(total) / (static_cast<double>((total + slots - 1) / slots) * slots);
     if (eff > best_eff + 1e-9) { best_eff = eff; splits = s; }
     if (eff >= 0.9) break;
   }
-  t1_fp8_kernel<<<dim3(row_tiles, c.H, splits), kThreads, Smem::total, st>>>(tm_a8, tm_pool_k8, c, n);
+  return splits;
+}
+
+int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, cudaStream_t st) {
+  if (configure_search8() != FASTAR_OK) return FASTAR_ERR_CUDA;
+  const int row_tiles = (n + 127) / 128;
+  Search8Args g{};
+  g.rows_a = n;
+  search8_kernel<false><<<dim3(row_tiles, c.H, pick_splits8(row_tiles, c.H, c.CAP / 128)), kThreads, Smem::total, st>>>(
+      tm_a8, tm_pool_k8, c, g);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
+// AnnCA prompt relevance on the 8-bit codes: c.rel (cleared by the caller) receives, as ordered integers,
+// max over the frame's queries of code(q) . code(k_p) * |q| * |k_p|; the caller decodes with 1 / (256 sqrt(d)).
+int launch_c1_relevance_fp8(const CacheView& c, const CUtensorMap& tm_q8, const CUtensorMap& tm_kp8, const float* qn,
+                            const float* kn, int nq, int np, int frame_len, cudaStream_t st) {
+  if (configure_search8() != FASTAR_OK) return FASTAR_ERR_CUDA;
+  const int row_tiles = (nq + 127) / 128;
+  Search8Args g{};
+  g.rows_a = nq;
+  g.cols_b = np;
+  g.frame_len = frame_len;
+  g.qn = qn;
+  g.kn = kn;
+  search8_kernel<true><<<dim3(row_tiles, c.H, pick_splits8(row_tiles, c.H, (np + 127) / 128)), kThreads, Smem::total, st>>>(
+      tm_q8, tm_kp8, c, g);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 

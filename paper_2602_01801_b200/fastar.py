@@ -43,6 +43,7 @@ SIGNATURES = {
     "fastar_cache_destroy": (C.c_int, [_vp]),
     "fastar_cache_export": (C.c_int, [_vp] * 9),
     "fastar_cache_export_search_codes": (C.c_int, [_vp, _vp, _vp, _i32, _vp]),
+    "fastar_cache_export_annca_codes": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _vp]),
     "fastar_cache_import": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp]),
     "fastar_tempcache_update": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annsa_attention": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -175,6 +176,14 @@ class Cache:
             _check(self.lib.fastar_cache_export_search_codes(self.handle, out["cache"].ctypes.data,
                                                              out["new"].ctypes.data if n_new > 0 else None, n_new, _stream()),
                    "fastar_cache_export_search_codes")
+        return out
+
+    def export_annca_codes(self, nq: int, n_prompt: int) -> Dict[str, np.ndarray]:
+        """8-bit search only: the code rows of the last selecting AnnCA call's queries and prompt keys."""
+        out = dict(q=np.empty((self.H, nq, 128), np.uint8), prompt=np.empty((self.H, n_prompt, 128), np.uint8))
+        with self.torch.cuda.device(self.device):
+            _check(self.lib.fastar_cache_export_annca_codes(self.handle, out["q"].ctypes.data, out["prompt"].ctypes.data, nq,
+                                                            n_prompt, _stream()), "fastar_cache_export_annca_codes")
         return out
 
     def import_state(self, k_bits: np.ndarray, v_bits: np.ndarray, length: np.ndarray, count: Optional[np.ndarray] = None,

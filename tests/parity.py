@@ -158,9 +158,14 @@ def check_attention(got: np.ndarray, want: np.ndarray, what: str) -> None:
 
 
 def check_prompt_selection(Q: np.ndarray, K_p: np.ndarray, frame_len: int, keep: int, sel: np.ndarray,
-                           rel: Optional[np.ndarray]) -> None:
-    """C1/C2: relevance values and the kept set, up to 1e-4 ties."""
-    r = O.prompt_relevance(Q.astype(np.float64), K_p.astype(np.float64), frame_len)
+                           rel: Optional[np.ndarray], codes=None) -> None:
+    """C1/C2: relevance values and the kept set, up to 1e-4 ties.  codes = (query codes, prompt codes) selects the
+    8-bit quantised relevance, evaluated by the oracle on those (already checked) codes."""
+    if codes is None:
+        r = O.prompt_relevance(Q.astype(np.float64), K_p.astype(np.float64), frame_len)
+    else:
+        r = O.prompt_relevance_quantized(Q.astype(np.float64), K_p.astype(np.float64), frame_len, codes_q=codes[0],
+                                         codes_k=codes[1])
     if rel is not None:
         assert np.max(np.abs(rel - r) / np.maximum(1.0, np.abs(r))) <= 2e-5, "C1: relevance values"
     k = min(keep, K_p.shape[0])

@@ -80,8 +80,14 @@ def gpu_annca_checked(cache, cfg, Q, Kp, Vp, keep, fp32=False):
     assert cache.status() == 0
     out = res["out"].float().cpu().numpy()
     sel, rel = res["sel"].cpu().numpy(), res["rel"].cpu().numpy()
+    q8 = cache.search_bits == 8
+    codes = cache.export_annca_codes(Q.shape[1], Kp.shape[1]) if q8 else None
     for h in range(Q.shape[0]):
-        P.check_prompt_selection(Q[h], Kp[h], cfg.frame_len, keep, sel[h], rel[h])
+        if q8:          # the quantiser byte by byte, then the relevance of the codes the GPU ranked with
+            P.check_search_codes(Q[h], codes["q"][h], f"AnnCA query codes, head {h}")
+            P.check_search_codes(Kp[h], codes["prompt"][h], f"AnnCA prompt codes, head {h}")
+        P.check_prompt_selection(Q[h], Kp[h], cfg.frame_len, keep, sel[h], rel[h],
+                                 codes=(codes["q"][h][:, : cfg.head_dim], codes["prompt"][h][:, : cfg.head_dim]) if q8 else None)
         want = O.annca(Q[h], Kp[h], Vp[h], cfg.frame_len, keep, sel=sel[h])["out"]
         P.check_attention(out[h], want, f"AnnCA head {h}")
     return res
