@@ -14,6 +14,10 @@ Paper passages followed
   * Eq. 1 (Section 3)            dense cached attention            -> dense_attention
   * Section 5.1                  attention over a candidate set    -> sparse_attention
   * Section 5.2 "Finding temporal correspondences"  top-1 key      -> top1_cosine
+  * Section 5.2 (same paragraph) query-probe form: highest attention
+                                 score of the token's query             -> top1_query_probe
+  * Section 5.1 "quantised similarity search"  8-bit codes         -> key_codes_e4m3, top1_quantized,
+                                                                      prompt_relevance_quantized
   * Section 5.2 / Appendix C     threshold merge, last-key representative,
                                  mean value, multiplicity m        -> tempcache_update
   * Lemma 1 (Section 5.2, Appendix A)  + log m bias                -> sparse_attention
@@ -193,14 +197,33 @@ def top1_quantized(K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.
     return j.astype(np.int64), s[np.arange(n), j]
 
 
+def top1_query_probe(Q_new: np.ndarray, K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.ndarray]:
+    """Correspondence read off the attention scores (Section 5.2, "Finding temporal correspondences"):
+    the token corresponding to query q_i is the live cached key with the highest score <q_i, k_j>
+    (softmax and the 1/sqrt(d) scale are monotone, so this is the highest attention weight; ties ->
+    smallest slot).  Returns (j*, cos(k_i, k_j*)): the similarity the merge threshold is applied to is
+    that of the keys (Appendix C, "key-similarity threshold").  j* = -1, c* = 0 on an empty cache."""
+    Q_new = np.asarray(Q_new, np.float64)
+    K_new = np.asarray(K_new, np.float64)
+    n = K_new.shape[0]
+    if cache.L == 0:
+        return np.full(n, -1, np.int64), np.zeros(n, np.float64)
+    Kc = cache.K[: cache.L]
+    j = np.argmax(Q_new @ Kc.T, axis=1).astype(np.int64)
+    num = np.sum(K_new * Kc[j], axis=1)
+    den = np.sqrt(np.sum(K_new * K_new, axis=1)) * np.sqrt(np.sum(Kc[j] * Kc[j], axis=1))
+    return j, np.where(den > 0, num / np.where(den > 0, den, 1.0), 0.0)
+
+
 def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
                      forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None,
-                     search_bits: int = 16) -> Dict[str, np.ndarray]:
+                     search_bits: int = 16, probe: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
     """One TempCache update of one head.
 
     forced = (j*, c*, matched) replaces steps 1-2 by decisions taken elsewhere
     (staged parity: near-ties have several correct answers).  search_bits = 8 runs the
-    correspondence search on the 8-bit codes of the keys instead of the keys themselves."""
+    correspondence search on the 8-bit codes of the keys instead of the keys themselves.
+    probe = the chunk's queries [n][d] selects the query-probe correspondence (top1_query_probe)."""
     K_new = np.asarray(K_new, np.float64)
     V_new = np.asarray(V_new, np.float64)
     n = K_new.shape[0]
@@ -208,7 +231,10 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
 
     # 1. top-1 correspondence against the pre-call cache; 2. threshold
     if forced is None:
-        jstar, cstar = top1_quantized(K_new, cache) if search_bits == 8 else top1_cosine(K_new, cache)
+        if probe is not None:
+            jstar, cstar = top1_query_probe(probe, K_new, cache)
+        else:
+            jstar, cstar = top1_quantized(K_new, cache) if search_bits == 8 else top1_cosine(K_new, cache)
         matched = (cstar >= tau) & (jstar >= 0)
     else:
         jstar, cstar, matched = (np.asarray(a) for a in forced)

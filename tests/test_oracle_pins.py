@@ -463,3 +463,44 @@ def test_quantised_prompt_relevance():
     a = O.annca(Q, Kp, rng.standard_normal((npr, d)), fl, 8, search_bits=8)
     b = O.annca(Q, Kp, rng.standard_normal((npr, d)), fl, 8)
     assert all(len(set(a["sel"][f]) & set(b["sel"][f])) >= 6 for f in range(3))
+
+
+def test_query_probe_correspondence():
+    rng = _rng(35)
+    d, L, n = 16, 40, 25
+    cache = O.HeadCache(64, d)
+    Kc = rng.standard_normal((L, d)) * rng.uniform(0.5, 2.0, (L, 1))
+    cache.load(Kc, rng.standard_normal((L, d)))
+    K = rng.standard_normal((n, d))
+    Q = rng.standard_normal((n, d))
+    j, c = O.top1_query_probe(Q, K, cache)
+    # brute force with Python loops: slot of the largest dot product with the query, cosine of the keys
+    for i in range(n):
+        dots = [sum(float(Q[i, k]) * float(Kc[s, k]) for k in range(d)) for s in range(L)]
+        jb = max(range(L), key=lambda s: (dots[s], -s))
+        assert j[i] == jb
+        cb = float(K[i] @ Kc[jb]) / (np.linalg.norm(K[i]) * np.linalg.norm(Kc[jb]))
+        assert abs(c[i] - cb) < 1e-12
+    # the winner is the slot of the largest softmax attention weight (what the paper names)
+    logits = (Q @ Kc.T) / np.sqrt(d)
+    w = np.exp(logits - logits.max(axis=1, keepdims=True))
+    assert np.array_equal(j, np.argmax(w / w.sum(axis=1, keepdims=True), axis=1))
+    # with unit-norm cached keys and the keys themselves as the probe it is the key -> key cosine search
+    cache1 = O.HeadCache(64, d)
+    cache1.load(Kc / np.linalg.norm(Kc, axis=1, keepdims=True), rng.standard_normal((L, d)))
+    j1, c1 = O.top1_query_probe(K, K, cache1)
+    j2, c2 = O.top1_cosine(K, cache1)
+    assert np.array_equal(j1, j2) and np.allclose(c1, c2, atol=1e-12)
+    # scaling the probe changes nothing; empty cache
+    j3, c3 = O.top1_query_probe(3.0 * Q, K, cache)
+    assert np.array_equal(j3, j) and np.allclose(c3, c)
+    je, ce = O.top1_query_probe(Q, K, O.HeadCache(64, d))
+    assert np.all(je == -1) and np.all(ce == 0)
+    # inside an update: a token merges only if its KEY is close to the slot its QUERY points at
+    cache2 = O.HeadCache(64, d)
+    cache2.load(Kc, np.zeros((L, d)))
+    Kn = np.stack([Kc[3] * 1.0, Kc[5] * 1.0])
+    Qn = np.stack([Kc[3] * 4.0, Kc[7] * 4.0])            # token 1's query points at slot 7, its key sits on slot 5
+    r = O.tempcache_update(cache2, Kn, np.ones((2, d)), 2, 0.9, probe=Qn)
+    assert r["jstar"].tolist() == [3, 7] and r["match"].tolist() == [3, -1]
+    assert r["stats"]["appended"] == 1 and cache2.m[3] == 2 and cache2.m[5] == 1
