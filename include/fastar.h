@@ -157,6 +157,20 @@ int fastar_tempcache_update(fastar_cache_t* cache, const void* k_new, const void
                             int32_t* match_out, float* sim_out, int32_t* dest_out,
                             fastar_update_stats* stats_out, void* stream);
 
+/* TempCache update with query-probe correspondence (Section 5.2, "Finding temporal correspondences":
+ * the corresponding token of a current-frame query is the cached key with the highest attention
+ * score).  As fastar_tempcache_update, except that the slot is chosen by the probe rows,
+ *   j*_i = argmax_j <q_i, K_j> over live slots (ties: lowest slot),
+ * and the merge decision is taken on the key similarity of that slot: matched iff
+ * cos(k_i, K_{j*_i}) >= tau.  sim_out receives that cosine (0 on an empty cache); the
+ * representative rule uses it.  q_probe: dev [H][n][d], same strides and dtype as k_new.
+ * search_bits == 8 caches return FASTAR_ERR_UNSUPPORTED_SHAPE (the probe ranks un-normalised
+ * dot products, which the direction-only 8-bit codes do not carry). */
+int fastar_tempcache_update_probe(fastar_cache_t* cache, const void* q_probe, const void* k_new, const void* v_new,
+                                  int32_t n, int32_t frame_len, int64_t head_stride, int64_t token_stride, float tau,
+                                  int32_t* match_out, float* sim_out, int32_t* dest_out,
+                                  fastar_update_stats* stats_out, void* stream);
+
 /* AnnSA (Sections 5.1 and 5.4 with the bias of Lemma 1).  Queries are cut into blocks of block_q
  * rows, the cache into blocks of page_tokens slots.  Each query and key gets T b-bit codes (signs
  * of the shared random projection); tile (a, b) scores the number of (query, key, table) triples

@@ -78,6 +78,9 @@ struct CacheView {
   uint8_t* kp8_ca;                 // [H][max_prompt][128]  codes of the prompt keys
   float* qn_ca;                    // [H][max_tokens]  |q|
   float* kpn_ca;                   // [H][max_prompt]  |k_p|
+  // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
+  // rank cached keys by the plain dot product with the probe rows instead of the cosine.
+  int raw_dot;
 };
 
 inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
@@ -131,6 +134,7 @@ int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const A
 int launch_convert_f32_to_bf16(const float* src, __nv_bfloat16* dst, int H, int n, int D, int64_t hs, int64_t ts, cudaStream_t st);
 int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
                       float* rnorm_out, cudaStream_t st);
+int launch_probe_cosine(const CacheView& c, const __nv_bfloat16* k_new, int n, int64_t hs, int64_t ts, cudaStream_t st);
 int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st);
 int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len,
                   int64_t hs, int64_t ts, cudaStream_t st);

@@ -380,23 +380,31 @@ int fastar_cache_import(fastar_cache_t* c, const uint16_t* host_k, const uint16_
   return cudaStreamSynchronize(st) == cudaSuccess ? FASTAR_OK : FASTAR_ERR_CUDA;
 }
 
-int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_new, int32_t n, int32_t frame_len,
-                            int64_t head_stride, int64_t token_stride, float tau, int32_t* match_out, float* sim_out,
-                            int32_t* dest_out, fastar_update_stats* stats_out, void* stream) {
+// One update; q_probe == nullptr is the key -> key cosine search, otherwise the cached keys are ranked by their dot
+// product with the probe rows and the threshold is applied to the key cosine of the winner.
+static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new, const void* v_new, int32_t n, int32_t frame_len,
+                       int64_t head_stride, int64_t token_stride, float tau, int32_t* match_out, float* sim_out,
+                       int32_t* dest_out, fastar_update_stats* stats_out, void* stream) {
   if (!c || !k_new || !v_new || n < 1 || frame_len < 1) return FASTAR_ERR_INVALID_ARG;
   if (n > c->v.max_tokens || n > 16384 || n > c->v.CAP) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (q_probe && c->v.search_bits == 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (token_stride < c->v.D || head_stride < 0) return FASTAR_ERR_INVALID_ARG;
   DeviceGuard guard(c->desc.device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const CacheView& v = c->v;
-  const __nv_bfloat16 *kb, *vb;
-  int64_t khs = head_stride, kts = token_stride, vhs = head_stride, vts = token_stride;
+  const __nv_bfloat16 *kb, *vb, *pb = nullptr;
+  int64_t khs = head_stride, kts = token_stride, vhs = head_stride, vts = token_stride, phs = head_stride, pts = token_stride;
   int r = as_bf16(c, k_new, n, &khs, &kts, 0, &kb, st);
   if (r != FASTAR_OK) return r;
   r = as_bf16(c, v_new, n, &vhs, &vts, 1, &vb, st);
   if (r != FASTAR_OK) return r;
+  if (q_probe) {
+    r = as_bf16(c, q_probe, n, &phs, &pts, 2, &pb, st);
+    if (r != FASTAR_OK) return r;
+  }
   CUtensorMap tm_a;
-  r = make_map(c, &tm_a, kb, v.D, n, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
+  r = q_probe ? make_map(c, &tm_a, pb, v.D, n, v.H, static_cast<uint64_t>(pts) * 2, static_cast<uint64_t>(phs) * 2, 128)
+              : make_map(c, &tm_a, kb, v.D, n, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, 128);
   if (r != FASTAR_OK) return r;
   ACCK(FASTAR_K_HASH, launch_prep_codes(v, kb, n, khs, kts, v.code_new, v.rnorm_new, st));
   // packed arg-max words and per-slot match counts start at zero (adjacent in the workspace: one memset)
@@ -409,6 +417,11 @@ int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_
     if (r != FASTAR_OK) return r;
     ACCK(FASTAR_K_HASH, launch_quantize_keys(v, kb, n, khs, kts, v.rnorm_new, v.max_tokens, v.k8_new, v.max_tokens, st));
     ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(v, tm_a8, c->tm_pool_k8, n, st));
+  } else if (q_probe) {
+    CacheView vr = v;
+    vr.raw_dot = 1;
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(vr, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
+    ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
   } else {
     ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
   }
@@ -417,6 +430,21 @@ int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_
   ACCK(FASTAR_K_KEY_HIST, launch_finalize_hist(v, stats_out, 1, st));
   ACC(launch_copy_outputs(v, n, match_out, sim_out, dest_out, st));
   return FASTAR_OK;
+}
+
+int fastar_tempcache_update(fastar_cache_t* c, const void* k_new, const void* v_new, int32_t n, int32_t frame_len,
+                            int64_t head_stride, int64_t token_stride, float tau, int32_t* match_out, float* sim_out,
+                            int32_t* dest_out, fastar_update_stats* stats_out, void* stream) {
+  return update_impl(c, nullptr, k_new, v_new, n, frame_len, head_stride, token_stride, tau, match_out, sim_out, dest_out, stats_out,
+                     stream);
+}
+
+int fastar_tempcache_update_probe(fastar_cache_t* c, const void* q_probe, const void* k_new, const void* v_new, int32_t n,
+                                  int32_t frame_len, int64_t head_stride, int64_t token_stride, float tau, int32_t* match_out,
+                                  float* sim_out, int32_t* dest_out, fastar_update_stats* stats_out, void* stream) {
+  if (!q_probe) return FASTAR_ERR_INVALID_ARG;
+  return update_impl(c, q_probe, k_new, v_new, n, frame_len, head_stride, token_stride, tau, match_out, sim_out, dest_out, stats_out,
+                     stream);
 }
 
 int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t nq, int64_t head_stride, int64_t token_stride,

@@ -213,10 +213,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         int valid_cols = 128;
         if (EPI == EPI_ARGMAX) {
           if (wg == 0) {
-            if (tl == 0) rn_next = (t * 128 + r < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r] : 0.f;
+            if (tl == 0) rn_next = (t * 128 + r < L) ? (c.raw_dot ? 1.f : c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r]) : 0.f;
             rn_s[buf * 128 + r] = rn_next;
             const int slot = (t + 1) * 128 + r;
-            rn_next = (tl + 1 < ntl && slot < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+            rn_next = (tl + 1 < ntl && slot < L) ? (c.raw_dot ? 1.f : c.rnorm[static_cast<int64_t>(h) * c.CAP + slot]) : 0.f;
           }
           valid_cols = min(128, L - t * 128);
           named_barrier_sync(1, 256);
@@ -283,7 +283,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       }
       if (threadIdx.x == 0) { PT_FLUSH("gemm epilogue (wait acc, tmem loads, compute, arrive)", ntl) }
       if (EPI == EPI_ARGMAX && ok && row < g.rows_a && best_j >= 0) {
-        const float sim = best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        const float sim = c.raw_dot ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
                                        static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
         atomicMax(c.best + static_cast<int64_t>(h) * c.max_tokens + row, key);
@@ -479,7 +479,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       // 1/|k| of the tile's cache keys goes through shared memory; the global load runs one tile ahead so that its
       // latency is not paid between two tiles
       const float* rn_h = c.rnorm + static_cast<int64_t>(h) * c.CAP;
-      float rn_next = (wg == 0 && t0 * 128 + r < L) ? rn_h[t0 * 128 + r] : 0.f;
+      float rn_next = (wg == 0 && t0 * 128 + r < L) ? (c.raw_dot ? 1.f : rn_h[t0 * 128 + r]) : 0.f;
       PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
@@ -487,7 +487,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (wg == 0) {
           rn_s[buf * 128 + r] = rn_next;
           const int slot = (t + 1) * 128 + r;
-          rn_next = (tl + 1 < ntl && slot < L) ? rn_h[slot] : 0.f;
+          rn_next = (tl + 1 < ntl && slot < L) ? (c.raw_dot ? 1.f : rn_h[slot]) : 0.f;
         }
         const int valid_cols = min(128, L - t * 128);
         named_barrier_sync(1, 256);
@@ -517,7 +517,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       if (threadIdx.x == 0 && rank == 0) { PT_FLUSH("t1 pair epilogue (wait acc, tmem loads, compute)", ntl) }
       if (ok && row < g.rows_a && best_j >= 0) {
-        const float sim = best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        const float sim = c.raw_dot ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
                                        static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
         atomicMax(c.best + static_cast<int64_t>(h) * c.max_tokens + row, key);

@@ -463,6 +463,54 @@ __global__ void __launch_bounds__(256) scatter_kernel(const CacheView c, int n) 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Query-probe correspondence (Section 5.2: the corresponding token of a query is the cached key with the highest
+// attention score): the similarity kernel ranked the cached keys by <q_i, k_j>; the merge decision is taken on the
+// key similarity, so the packed word of token i becomes (cos(k_i, k_j*), j*) with the cosine in the same fp32
+// form as the cosine search (dot * 1/|k_i| * 1/|k_j*|).  Half a warp per token, one 128-bit load per lane and row.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) probe_cosine_kernel(const CacheView c, const __nv_bfloat16* __restrict__ k_new, int n,
+                                                           int64_t hs, int64_t ts) {
+  const int64_t rows = static_cast<int64_t>(c.H) * n;
+  const unsigned hmask = 0xFFFFu << (threadIdx.x & 16);
+  for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; (q >> 4) < rows;
+       q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int e8 = static_cast<int>(q & 15);
+    const int64_t rowid = q >> 4;
+    const int h = static_cast<int>(rowid / n), i = static_cast<int>(rowid % n);
+    const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+    const unsigned long long b = c.best[tb + i];
+    if (b == 0ull) continue;                         // empty cache: nothing was ranked (same for all 16 lanes)
+    const int j = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull));
+    float dot = 0.f;
+    if (e8 * 8 < c.D) {
+      const uint4 a = *reinterpret_cast<const uint4*>(k_new + h * hs + i * ts + e8 * 8);
+      const uint4 kk = *reinterpret_cast<const uint4*>(c.pool_k + slot_row_offset(c, c.page_table + static_cast<int64_t>(h) * c.CAPB, j) + e8 * 8);
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* pk = reinterpret_cast<const __nv_bfloat162*>(&kk);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 fa = __bfloat1622float2(pa[e]), fk = __bfloat1622float2(pk[e]);
+        dot = fmaf(fa.x, fk.x, dot);
+        dot = fmaf(fa.y, fk.y, dot);
+      }
+    }
+#pragma unroll
+    for (int o = 8; o >= 1; o >>= 1) dot += __shfl_xor_sync(hmask, dot, o);
+    if (e8 == 0) {
+      const float cosv = dot * c.rnorm[static_cast<int64_t>(h) * c.CAP + j] * c.rnorm_new[tb + i];
+      c.best[tb + i] = (static_cast<unsigned long long>(float_to_ordered(cosv)) << 32) | (b & 0xFFFFFFFFull);
+    }
+  }
+}
+
+int launch_probe_cosine(const CacheView& c, const __nv_bfloat16* k_new, int n, int64_t hs, int64_t ts, cudaStream_t st) {
+  const int64_t total = static_cast<int64_t>(c.H) * n * 16;
+  const int grid = static_cast<int>((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+  probe_cosine_kernel<<<grid, 256, 0, st>>>(c, k_new, n, hs, ts);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
 int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st) {
   (void)frame_len;
   static bool configured = false;

@@ -46,6 +46,7 @@ SIGNATURES = {
     "fastar_cache_export_annca_codes": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _vp]),
     "fastar_cache_import": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp]),
     "fastar_tempcache_update": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
+    "fastar_tempcache_update_probe": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annsa_attention": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annca_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp,
                                          _vp, _vp]),
@@ -210,17 +211,24 @@ class Cache:
         assert t.dim() == 3 and t.stride(2) == 1 and t.dtype == self.dtype and t.is_cuda
         return t.stride(0), t.stride(1)
 
-    def update(self, k_new, v_new, frame_len: int, tau: float, outputs: bool = True) -> Dict[str, "object"]:
+    def update(self, k_new, v_new, frame_len: int, tau: float, outputs: bool = True, probe=None) -> Dict[str, "object"]:
+        """TempCache update; probe = the chunk's queries selects the query-probe correspondence."""
         torch = self.torch
         H, n, _ = k_new.shape
         hs, ts = self._strides(k_new)
-        assert self._strides(v_new) == (hs, ts)
+        assert self._strides(v_new) == (hs, ts) and (probe is None or self._strides(probe) == (hs, ts))
         res = {}
         if outputs:
             res = dict(match=torch.empty((H, n), dtype=torch.int32, device=self.device),
                        sim=torch.empty((H, n), dtype=torch.float32, device=self.device),
                        dest=torch.empty((H, n), dtype=torch.int32, device=self.device),
                        stats=torch.zeros((H, 8), dtype=torch.int32, device=self.device))
+        if probe is not None:
+            _check(self.lib.fastar_tempcache_update_probe(self.handle, probe.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n,
+                                                          frame_len, hs, ts, float(tau), _ptr(res.get("match")),
+                                                          _ptr(res.get("sim")), _ptr(res.get("dest")), _ptr(res.get("stats")),
+                                                          _stream()), "fastar_tempcache_update_probe")
+            return res
         _check(self.lib.fastar_tempcache_update(self.handle, k_new.data_ptr(), v_new.data_ptr(), n, frame_len, hs, ts,
                                                 float(tau), _ptr(res.get("match")), _ptr(res.get("sim")),
                                                 _ptr(res.get("dest")), _ptr(res.get("stats")), _stream()),

@@ -45,19 +45,43 @@ def oracle_heads_from_export(state: Dict[str, np.ndarray], n_sink: int = 0) -> L
 
 def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float, match: np.ndarray,
                  sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
-                 rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None) -> O.HeadCache:
+                 rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None,
+                 probe: Optional[np.ndarray] = None) -> O.HeadCache:
     """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
     exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases).
     `codes` = (codes of the new keys [n][128], codes of the pre-call cache [>= L][128]) as the GPU computed them
     selects the 8-bit search: the scores are then the oracle's quantised scores of those codes (the quantiser
-    itself is checked by check_search_codes)."""
+    itself is checked by check_search_codes).  `probe` = the chunk's queries selects the query-probe
+    correspondence: the slot maximises <q_i, k_j>, the similarity reported and thresholded is cos(k_i, k_j*)."""
     n = K_new.shape[0]
     K64, V64 = K_new.astype(np.float64), V_new.astype(np.float64)
     matched = match >= 0
     idx = np.arange(n) if rows is None else rows
     margin = MARGIN if codes is None else MARGIN_Q8
     sim_tol = 2e-5 if codes is None else MARGIN_Q8
-    if pre.L > 0:
+    if pre.L > 0 and probe is not None:
+        Kc = pre.K[: pre.L]
+        Q64 = probe.astype(np.float64)[idx]
+        s = Q64 @ Kc.T
+        sbest = s.max(axis=1)
+        # tie window on the scale of the dot products (fp32 accumulation of bf16 products)
+        win = MARGIN * np.linalg.norm(Q64, axis=1) * np.linalg.norm(Kc, axis=1).max()
+        near = s >= (sbest - win)[:, None]
+        cosm = O.cosine_matrix(K64[idx], Kc)
+        # the similarity reported is the key cosine of a (near-)best slot of the probe
+        assert np.all((near & (np.abs(cosm - sim[idx][:, None]) <= sim_tol)).any(axis=1)), "T1 probe: similarity value"
+        mi = np.flatnonzero(matched[idx])
+        assert np.all(near[mi, match[idx][mi]]), "T1 probe: matched slot is not a (near-)best slot"
+        assert np.max(np.abs(cosm[mi, match[idx][mi]] - sim[idx][mi]), initial=0.0) <= sim_tol, "T1 probe: cosine of the matched slot"
+        assert np.all(sim[idx][mi] >= tau - margin), "T2 probe: matched below the threshold"
+        uniq = near.sum(axis=1) == 1
+        ju = np.argmax(s, axis=1)
+        cu = cosm[np.arange(idx.size), ju]
+        far = uniq & (np.abs(cu - tau) > margin)
+        assert np.array_equal(matched[idx][far], (cu >= tau)[far]), "T2 probe: threshold decision"
+        fm = far & matched[idx]
+        assert np.array_equal(match[idx][fm], ju[fm]), "T1 probe: index differs outside the tie window"
+    elif pre.L > 0:
         if codes is None:
             cosm = O.cosine_matrix(K64[idx], pre.K[: pre.L])
         else:

@@ -23,12 +23,14 @@ def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, sea
                         max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32, search_bits=search_bits)
 
 
-def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False):
-    """Runs one update on the GPU and checks it against the oracle heads `heads` (advanced in place)."""
+def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=None):
+    """Runs one update on the GPU and checks it against the oracle heads `heads` (advanced in place).
+    probe = the chunk's queries [H][n][d] runs the query-probe correspondence."""
     torch, fastar = _gpu()
     q8 = cache.search_bits == 8
     pre_codes = cache.export_search_codes()["cache"] if q8 else None      # codes of the cache the search will see
-    res = cache.update(fastar.to_device(K, fp32), fastar.to_device(V, fp32), frame_len, tau)
+    res = cache.update(fastar.to_device(K, fp32), fastar.to_device(V, fp32), frame_len, tau,
+                       probe=None if probe is None else fastar.to_device(probe, fp32))
     assert cache.status() == 0
     post = cache.export_state()
     match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
@@ -42,7 +44,8 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False):
             Lh = int(post["len"][h])
             P.check_search_codes(P.bits_to_f64(post["k"][h, :Lh]), post_codes["cache"][h, :Lh], f"cache codes, head {h}")
             codes = (post_codes["new"][h], pre_codes[h])
-        ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes)
+        ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes,
+                             probe=None if probe is None else probe[h])
         # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
         # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
         synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
@@ -144,6 +147,38 @@ def test_both_similarity_kernels(kernel, d, pt, monkeypatch):
     Q, K, V = w.chunk(cfg.prior_chunks + 1)
     post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
     assert post["count"].max() > 1
+
+
+@pytest.mark.parametrize("d,pt,fp32,kernel", [(128, 128, False, "single"), (64, 64, True, "single"), (128, 128, False, "pair"),
+                                               (64, 64, False, "pair")])
+def test_query_probe_correspondence(d, pt, fp32, kernel, monkeypatch):
+    monkeypatch.setenv("FASTAR_T1_KERNEL", kernel)
+    # The slot is chosen by the token's QUERY (highest attention score over the cache), the merge decision by the key
+    # cosine of that slot.  Prior chunks enter un-merged; then two merging chunks, each probed with its own queries;
+    # AnnSA runs on the result.  An empty cache and the 8-bit refusal are covered too.
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, fp32)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    Q, K, V = w.chunk(0)
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, fp32, probe=Q)      # empty cache: all appended
+    assert int(post["len"][0]) == K.shape[1]
+    for ci in range(1, cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0, fp32)
+    matched = 0
+    for ci in (cfg.prior_chunks, cfg.prior_chunks + 1):
+        Q, K, V = w.chunk(ci)
+        before = [hc.L for hc in heads]
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, fp32, probe=Q)
+        matched += sum(K.shape[1] - (hc.L - b) for hc, b in zip(heads, before))
+    assert matched > 0.5 * 2 * cfg.num_heads * K.shape[1] and post["count"].max() > 1
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks, fp32)
+    if not fp32:
+        torch, fastar = _gpu()
+        c8 = make_cache(cfg, w, search_bits=8)
+        with pytest.raises(fastar.FastarError):
+            c8.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau, probe=fastar.to_device(Q))
 
 
 @pytest.mark.parametrize("d,pt", [(128, 128), (64, 64), (128, 64)])
