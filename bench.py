@@ -213,7 +213,7 @@ def run_ours(args, cfg):
         ca_stream.wait_stream(main)
         with torch.cuda.stream(ca_stream):
             cache.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt, out=out_ca)
-        cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)
+        cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq if args.probe else None)
         cache.annsa(dq, cfg.block, cfg.keep_blocks, out=out_sa)
         main.wait_stream(ca_stream)
 
@@ -266,7 +266,7 @@ def run_ours(args, cfg):
             cache.workspace.copy_(snap)
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-            cache.step_host(hk, hv, hq, hkp, hvp, ho1, ho2, cfg.frame_len, cfg.tau, cfg.block, cfg.keep_blocks, cfg.keep_prompt)
+            cache.step_host(hk, hv, hq, hkp, hvp, ho1, ho2, cfg.frame_len, cfg.tau, cfg.block, cfg.keep_blocks, cfg.keep_prompt, probe=args.probe)
             if i > 0:                            # first one is a warm-up of the copy path
                 e2e_s += time.perf_counter() - t0
         time.sleep(0.3)
@@ -288,7 +288,7 @@ def run_ours(args, cfg):
     prof_steps = max(3, min(args.steps, 10))
     for _ in range(prof_steps):                  # one stream here: a kernel timed beside another one is not its own time
         cache.workspace.copy_(snap)
-        cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)
+        cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq if args.probe else None)
         cache.annsa(dq, cfg.block, cfg.keep_blocks, out=out_sa)
         cache.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt, out=out_ca)
     torch.cuda.synchronize()
@@ -296,7 +296,7 @@ def run_ours(args, cfg):
     cache.profile(False)
     # algorithmic work of the two tensor-bound kernels
     cache.workspace.copy_(snap)
-    cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)
+    cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq if args.probe else None)
     dbg = cache.annsa(dq, cfg.block, cfg.keep_blocks, debug=True)
     len_after = cache.export_state(kv=False)["len"].astype(np.int64)
     t1_flops = float(np.sum(2.0 * n * len_before * D))
@@ -342,7 +342,7 @@ def run_ours(args, cfg):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": max_seconds / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if args.search_bits != 8 else "bf16 (correspondence search on fp8 e4m3 codes)", "data": "synthetic",
-            "config": {"workload": describe(cfg) + (" search=8bit" if args.search_bits == 8 else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
+            "config": {"workload": describe(cfg) + (" search=8bit" if args.search_bits == 8 else "") + (" correspondence=query-probe" if args.probe else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
                        f"({cache.workspace_bytes >> 20} MiB copy, untimed)", "parallelism": "replicas" if world > 1 else "1 GPU",
                        "cuda_graph": graph is not None},
             "e2e": {"value": e2e_units / e2e_max, "unit": "tok/s", "ms_per_step": e2e_max / args.steps * 1e3,
@@ -373,6 +373,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--search-bits", type=int, default=16, choices=[16, 8],
                     help="TempCache correspondence search on the bf16 keys (16, default) or on their 8-bit codes (8)")
+    ap.add_argument("--probe", action="store_true",
+                    help="query-probe correspondence: the update ranks cached keys by the dot product with the chunk's queries")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a captured CUDA graph")
     ap.add_argument("--mode", default="step", choices=["step", "rollout", "sweep"],
                     help="step = the one-line contract; rollout = c2 long rollout + dense baseline; sweep = c4 roofline sweep")

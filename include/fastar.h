@@ -210,12 +210,14 @@ int fastar_annca_attention(fastar_cache_t* cache, const void* q, const void* k_p
  * synchronises the stream.  Staging buffers live in the workspace.  The uploads of q and of the
  * prompt, AnnCA and the download of its output run on a second stream owned by the cache object,
  * beside the update; that stream starts after the work already queued on `stream` and is idle
- * again when the call returns. */
+ * again when the call returns.  flags: 0, or FASTAR_STEP_QUERY_PROBE to run the update as
+ * fastar_tempcache_update_probe with q as the probe. */
+#define FASTAR_STEP_QUERY_PROBE 1
 int fastar_attention_step_host(fastar_cache_t* cache, const void* k_new_host, const void* v_new_host,
                                const void* q_host, const void* k_prompt_host, const void* v_prompt_host,
                                void* out_sa_host, void* out_ca_host, int32_t n, int32_t frame_len, int32_t np,
                                float tau, int32_t block_q, int32_t keep_blocks, int32_t keep_tokens,
-                               void* stream);
+                               int32_t flags, void* stream);
 
 /* Synchronise the stream and return the device status word (FASTAR_OK or the first error a
  * kernel recorded since the last reset/clear); clears it. */

@@ -592,7 +592,7 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
 int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const void* v_new_host, const void* q_host,
                                const void* k_prompt_host, const void* v_prompt_host, void* out_sa_host, void* out_ca_host,
                                int32_t n, int32_t frame_len, int32_t np, float tau, int32_t block_q, int32_t keep_blocks,
-                               int32_t keep_tokens, void* stream) {
+                               int32_t keep_tokens, int32_t flags, void* stream) {
   if (!c || !k_new_host || !v_new_host || !q_host || !k_prompt_host || !v_prompt_host || !out_sa_host || !out_ca_host)
     return FASTAR_ERR_INVALID_ARG;
   if (n < 1 || n > c->v.max_tokens || np < 1 || np > c->v.max_prompt) return FASTAR_ERR_UNSUPPORTED_SHAPE;
@@ -620,8 +620,10 @@ int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const 
   bool copies_ok = upload(0, st) && upload(1, st) && upload(2, sd);
   copies_ok = copies_ok && cudaEventRecord(c->ev_q, sd) == cudaSuccess && upload(3, sd) && upload(4, sd);
   if (!copies_ok) r = FASTAR_ERR_CUDA;
+  const bool probe = (flags & FASTAR_STEP_QUERY_PROBE) != 0;
+  if (r == FASTAR_OK && probe && cudaStreamWaitEvent(st, c->ev_q, 0) != cudaSuccess) r = FASTAR_ERR_CUDA;   // the update reads q
   if (r == FASTAR_OK)
-    r = fastar_tempcache_update(c, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, st);
+    r = update_impl(c, probe ? dsrc[2] : nullptr, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, st);
   if (r == FASTAR_OK)
     r = fastar_annca_attention(c, dsrc[2], dsrc[3], dsrc[4], v.stage_out[1], n, frame_len, np, keep_tokens, hs, ts, phs, ts, nullptr,
                                nullptr, nullptr, sd);

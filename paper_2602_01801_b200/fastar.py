@@ -50,7 +50,7 @@ SIGNATURES = {
     "fastar_annsa_attention": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annca_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp,
                                          _vp, _vp]),
-    "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _vp]),
+    "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _i32, _vp]),
     "fastar_last_device_status": (C.c_int, [_vp, _vp]),
     "fastar_launch_count": (C.c_int64, [_vp]),
     "fastar_annca_select_noalloc": (C.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp]),
@@ -276,15 +276,16 @@ class Cache:
         return res
 
     def step_host(self, k_new, v_new, q, k_prompt, v_prompt, out_sa, out_ca, frame_len: int, tau: float, block_q: int,
-                  keep_blocks: int, keep_tokens: int) -> None:
-        """All tensors are contiguous HOST (ideally pinned) torch tensors of the cache dtype."""
+                  keep_blocks: int, keep_tokens: int, probe: bool = False) -> None:
+        """All tensors are contiguous HOST (ideally pinned) torch tensors of the cache dtype.
+        probe = True runs the update with the query-probe correspondence (q as the probe)."""
         for t in (k_new, v_new, q, k_prompt, v_prompt, out_sa, out_ca):
             assert not t.is_cuda and t.is_contiguous() and t.dtype == self.dtype
         n, np_ = k_new.shape[1], k_prompt.shape[1]
         _check(self.lib.fastar_attention_step_host(self.handle, k_new.data_ptr(), v_new.data_ptr(), q.data_ptr(),
                                                    k_prompt.data_ptr(), v_prompt.data_ptr(), out_sa.data_ptr(),
                                                    out_ca.data_ptr(), n, frame_len, np_, float(tau), block_q, keep_blocks,
-                                                   keep_tokens, _stream()), "fastar_attention_step_host")
+                                                   keep_tokens, 1 if probe else 0, _stream()), "fastar_attention_step_host")
 
 
 def annca_select_noalloc(q, k_prompt, frame_len: int, keep_tokens: int, sel_out=None):

@@ -335,7 +335,8 @@ def test_annca_keep_all_is_dense_cross_attention():
         P.check_attention(out[h], O.dense_attention(Q[h], Kp[h], Vp[h]), "AnnCA keep-all")
 
 
-def test_host_step_matches_device_calls():
+@pytest.mark.parametrize("probe", [False, True])
+def test_host_step_matches_device_calls(probe):
     torch, fastar = _gpu()
     cfg = synth.small_config()
     w = synth.Workload(cfg)
@@ -344,12 +345,13 @@ def test_host_step_matches_device_calls():
         Q, K, V = w.chunk(ci)
         Kp, Vp, _ = w.prompt(ci)
         dq, dk, dv, dkp, dvp = (fastar.to_device(x) for x in (Q, K, V, Kp, Vp))
-        ca.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)
+        ca.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq if probe else None)
         o1 = ca.annsa(dq, cfg.block, cfg.keep_blocks)["out"]
         o2 = ca.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt)["out"]
         hq, hk, hv, hkp, hvp = (t.cpu().pin_memory() for t in (dq, dk, dv, dkp, dvp))
         h1, h2 = torch.empty_like(hq).pin_memory(), torch.empty_like(hq).pin_memory()
-        cb.step_host(hk, hv, hq, hkp, hvp, h1, h2, cfg.frame_len, cfg.tau, cfg.block, cfg.keep_blocks, cfg.keep_prompt)
+        cb.step_host(hk, hv, hq, hkp, hvp, h1, h2, cfg.frame_len, cfg.tau, cfg.block, cfg.keep_blocks, cfg.keep_prompt,
+                     probe=probe)
         assert torch.equal(o1.cpu(), h1) and torch.equal(o2.cpu(), h2)
     assert ca.status() == 0 and cb.status() == 0
     assert ca.launch_count() > 0
