@@ -373,6 +373,36 @@ def sparse_attention(Q: np.ndarray, cache: HeadCache, sel: np.ndarray, block_q: 
     return (O, probs) if return_probs else O
 
 
+def sparse_attention_with_segment(Q: np.ndarray, cache: HeadCache, sel: np.ndarray, block_q: int, block_k: int,
+                                  K_seg: np.ndarray, V_seg: np.ndarray) -> np.ndarray:
+    """sparse_attention whose candidate set also holds every token of an un-cached segment (the keys and
+    values of the frames being generated: in Eq. 1 (Section 3) the attended set is the current frames'
+    keys and values concatenated with those of all earlier frames).  Segment tokens stand for
+    themselves (multiplicity 1, no bias); cached slots keep Lemma 1's ln m bias."""
+    Q = np.asarray(Q, np.float64)
+    K_seg = np.asarray(K_seg, np.float64)
+    V_seg = np.asarray(V_seg, np.float64)
+    nq, d = Q.shape
+    O = np.zeros((nq, d), dtype=np.float64)
+    scale = 1.0 / np.sqrt(d)
+    for a in range(-(-nq // block_q)):
+        rows = np.arange(a * block_q, min((a + 1) * block_q, nq))
+        blocks = sel[a] if cache.L else []
+        slots = np.concatenate([np.arange(b * block_k, min((b + 1) * block_k, cache.L)) for b in blocks]
+                               + [np.zeros(0, np.int64)]).astype(np.int64)
+        keys = np.concatenate([cache.K[slots], K_seg])
+        vals = np.concatenate([cache.V[slots], V_seg])
+        bias = np.concatenate([np.log(cache.m[slots].astype(np.float64)), np.zeros(K_seg.shape[0])])
+        if keys.shape[0] == 0:
+            continue
+        logits = (Q[rows] @ keys.T) * scale + bias[None, :]
+        logits -= logits.max(axis=1, keepdims=True)
+        p = np.exp(logits)
+        p /= p.sum(axis=1, keepdims=True)
+        O[rows] = p @ vals
+    return O
+
+
 def annsa(Q: np.ndarray, cache: HeadCache, R: np.ndarray, tables: int, bits: int, block_q: int, block_k: int,
           keep: int, qcodes: Optional[np.ndarray] = None, kcodes: Optional[np.ndarray] = None,
           sel: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:

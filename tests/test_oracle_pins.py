@@ -504,3 +504,39 @@ def test_query_probe_correspondence():
     r = O.tempcache_update(cache2, Kn, np.ones((2, d)), 2, 0.9, probe=Qn)
     assert r["jstar"].tolist() == [3, 7] and r["match"].tolist() == [3, -1]
     assert r["stats"]["appended"] == 1 and cache2.m[3] == 2 and cache2.m[5] == 1
+
+
+def test_attention_with_uncached_segment():
+    rng = _rng(36)
+    d, L, bq, bk, nq, ns = 8, 22, 4, 8, 10, 7
+    cache = O.HeadCache(32, d)
+    cache.load(rng.standard_normal((L, d)), rng.standard_normal((L, d)), m=rng.integers(1, 5, L))
+    Q = rng.standard_normal((nq, d))
+    Ks, Vs = rng.standard_normal((ns, d)), rng.standard_normal((ns, d))
+    sel = np.array([[0, 2], [1, 2], [0, 1]])
+    got = O.sparse_attention_with_segment(Q, cache, sel, bq, bk, Ks, Vs)
+    # (1) Lemma 1 written with weights instead of a bias, row by row, over [selected live slots, segment]
+    want = np.zeros_like(got)
+    for a in range(3):
+        rows = np.arange(a * bq, min((a + 1) * bq, nq))
+        slots = np.concatenate([np.arange(b * bk, min((b + 1) * bk, L)) for b in sel[a]])
+        keys = np.concatenate([cache.K[slots], Ks]); vals = np.concatenate([cache.V[slots], Vs])
+        w = np.concatenate([cache.m[slots].astype(float), np.ones(ns)])
+        for i in rows:
+            e = w * np.exp(keys @ Q[i] / np.sqrt(d))
+            want[i] = (e / e.sum()) @ vals
+    assert np.allclose(got, want, atol=1e-12)
+    # (2) empty segment: sparse_attention itself
+    assert np.allclose(O.sparse_attention_with_segment(Q, cache, sel, bq, bk, np.zeros((0, d)), np.zeros((0, d))),
+                       O.sparse_attention(Q, cache, sel, bq, bk), atol=1e-13)
+    # (3) empty cache: dense attention over the segment
+    assert np.allclose(O.sparse_attention_with_segment(Q, O.HeadCache(32, d), sel, bq, bk, Ks, Vs),
+                       O.dense_attention(Q, Ks, Vs), atol=1e-13)
+    # (4) Lemma 1 across the boundary: duplicate keys expanded into the segment give the same output as their
+    #     grouped form in the cache
+    c2 = O.HeadCache(32, d)
+    k0, v0a, v0b = rng.standard_normal(d), rng.standard_normal(d), rng.standard_normal(d)
+    c2.load(np.stack([k0]), np.stack([(v0a + v0b) / 2]), m=np.array([2]))
+    grouped = O.sparse_attention_with_segment(Q, c2, np.zeros((3, 1), np.int64), bq, bk, Ks, Vs)
+    expanded = O.dense_attention(Q, np.concatenate([np.stack([k0, k0]), Ks]), np.concatenate([np.stack([v0a, v0b]), Vs]))
+    assert np.allclose(grouped, expanded, atol=1e-12)
