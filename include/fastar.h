@@ -188,6 +188,22 @@ int fastar_annsa_attention(fastar_cache_t* cache, const void* q, void* out, int3
                            int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out, float* scores_out,
                            const int32_t* sel_in, const int32_t* nsel_in, void* stream);
 
+/* AnnSA over the cache and an un-cached segment (Eq. 1, Section 3: the attended set is the keys and
+ * values of the frames being generated concatenated with those of the earlier frames; the former
+ * enter the cache only when fastar_tempcache_update is called, so attention can run on every
+ * denoising step before that).  As fastar_annsa_attention, with the candidate set of every query
+ * extended by all ns tokens of k_seg / v_seg (dev [H][ns][d] with their own strides, cache dtype),
+ * each with multiplicity 1 (no bias):
+ *   o_i = softmax over {live slots of the kept blocks, bias ln m_j} U {segment tokens, bias 0}.
+ * The block selection is unchanged (it ranks cache blocks only); keep_blocks >= CAP/Bk gives dense
+ * attention over the whole cache plus the segment; an empty cache gives dense attention over the
+ * segment.  sel_in / nsel_in as above (may be NULL).  1 <= ns <= max_tokens. */
+int fastar_annsa_attention_segment(fastar_cache_t* cache, const void* q, const void* k_seg, const void* v_seg,
+                                   void* out, int32_t nq, int32_t ns, int64_t head_stride, int64_t token_stride,
+                                   int64_t seg_head_stride, int64_t seg_token_stride, int32_t block_q,
+                                   int32_t keep_blocks, const int32_t* sel_in, const int32_t* nsel_in,
+                                   void* stream);
+
 /* AnnCA (Section 5.3).  Per head and per frame f (queries [f*frame_len, (f+1)*frame_len)):
  *   r[f][p] = max_i q_i.k_p/sqrt(d); keep the min(keep_tokens, np) prompt tokens with the
  *   largest r (ties: lower p); o_i = softmax over the kept p of q_i.k_p/sqrt(d), times v_p.

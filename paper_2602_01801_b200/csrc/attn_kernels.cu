@@ -53,7 +53,8 @@ __device__ __forceinline__ void ld_shared_f32x2(uint32_t addr, float& a, float& 
 template <int D, int BKT, bool GATHER>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-            const __grid_constant__ CUtensorMap tm_v, const CacheView c, const AttnArgs a) {
+            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_sk,
+            const __grid_constant__ CUtensorMap tm_sv, const CacheView c, const AttnArgs a) {
   using SM = AttnSmem<D, BKT>;
   constexpr int RS = SM::RS, NB = SM::NB;
   constexpr int HD = D / 2;             // output columns written by one thread in the epilogue
@@ -89,18 +90,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
   // ---- which rows and which key tiles ---------------------------------------------------------
   int q0, valid_rows, nt;
+  int ntc = 0;                          // paged mode: tiles taken from the cache; tiles [ntc, nt) are segment tiles
   const int32_t* list;
   if (!GATHER) {
     const int qa = blockIdx.x;
     q0 = qa * a.block_q;
     valid_rows = min(a.block_q, a.nq - q0);
     if (a.sel == nullptr) {
-      nt = (L + BKT - 1) / BKT;
+      ntc = (L + BKT - 1) / BKT;
       list = nullptr;
     } else {
-      nt = a.nsel[h];
+      ntc = a.nsel[h];
       list = a.sel + static_cast<int64_t>(h) * a.sel_head_stride + static_cast<int64_t>(qa) * a.sel_stride;
     }
+    nt = ntc + a.seg_tiles;
   } else {
     const int f = blockIdx.z;
     q0 = f * a.rows_per_frame + blockIdx.x * 128;
@@ -127,6 +130,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if (warp == kProducerWarp && lane == 0) {
     tma_prefetch_desc(&tm_q);
     if (!GATHER) { tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); }
+    if (!GATHER && a.seg_tiles > 0) { tma_prefetch_desc(&tm_sk); tma_prefetch_desc(&tm_sv); }
   }
   __syncthreads();
   if (warp == kMmaWarp) {
@@ -185,9 +189,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       int blk_l = 0, page_l = 0;            // tiles [32w, 32w + 32) of the window in use
       int blk_n = 0, page_n = 0;            // the following window (key tiles run two ahead of value tiles)
       auto fetch = [&](int j0, int& blk, int& page) {
-        if (j0 + lane < nt) {
-          blk = list ? list[j0 + lane] : j0 + lane;
+        const int jj = j0 + lane;
+        if (jj < ntc) {
+          blk = list ? list[jj] : jj;
           page = pt_h[blk];
+        } else if (jj < nt) {               // tile of the un-cached segment: its index, no page
+          blk = jj - ntc;
+          page = -1;
         }
       };
       // the stage of the tile is known to be free when this is called
@@ -197,13 +205,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #ifdef FASTAR_PHASE_TIMING
         reinterpret_cast<volatile long long*>(sgen + SM::bar_off + kBarBytes + 8)[s] = clock64();
 #endif
+        const bool seg = page < 0;          // rows past the segment's end arrive as zeros and carry a -inf bias
+        const CUtensorMap* tm = seg ? (is_k ? &tm_sk : &tm_sv) : (is_k ? &tm_k : &tm_v);
         mbar_arrive_expect_tx(bar_r_full + 8 * s, SM::kv_bytes);
         for (int kc = 0; kc < D / 64; ++kc)
-          tma_load_3d(ring_s + s * SM::kv_bytes + kc * BKT * 128, is_k ? &tm_k : &tm_v, bar_r_full + 8 * s, kc * 64, 0, page);
+          tma_load_3d(ring_s + s * SM::kv_bytes + kc * BKT * 128, tm, bar_r_full + 8 * s, kc * 64, seg ? blk * BKT : 0,
+                      seg ? h : page);
         if (is_k) {
           const int b4 = j % NB;
+          const float* bias_src = seg ? a.seg_bias + static_cast<int64_t>(blk) * BKT : l2m_h + static_cast<int64_t>(blk) * BKT;
           mbar_arrive_expect_tx(bar_b_full + 8 * b4, BKT * 4);
-          bulk_load_1d(bias_s + b4 * BKT * 4, l2m_h + static_cast<int64_t>(blk) * BKT, BKT * 4, bar_b_full + 8 * b4);
+          bulk_load_1d(bias_s + b4 * BKT * 4, bias_src, BKT * 4, bar_b_full + 8 * b4);
         }
       };
       if (nt > 0) {
@@ -518,8 +530,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 }
 
 template <int D, int BKT, bool GATHER>
-static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CacheView& c,
-                       const AttnArgs& a, dim3 grid, cudaStream_t st) {
+static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tsk,
+                       const CUtensorMap& tsv, const CacheView& c, const AttnArgs& a, dim3 grid, cudaStream_t st) {
   using SM = AttnSmem<D, BKT>;
   auto kern = attn_kernel<D, BKT, GATHER>;
   static bool configured = false;
@@ -528,27 +540,32 @@ static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
       return FASTAR_ERR_CUDA;
     configured = true;
   }
-  kern<<<grid, kAttnThreads, SM::total, st>>>(tq, tk, tv, c, a);
+  kern<<<grid, kAttnThreads, SM::total, st>>>(tq, tk, tv, tsk, tsv, c, a);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
+// tm_seg_k / tm_seg_v: maps of the un-cached segment (box {64, page_tokens, 1}); nullptr when a.seg_tiles == 0.
 int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
-                           const CUtensorMap& tm_pool_v, const AttnArgs& a, cudaStream_t st) {
+                           const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
+                           const AttnArgs& a, cudaStream_t st) {
+  if (a.seg_tiles > 0 && (!tm_seg_k || !tm_seg_v || !a.seg_bias)) return FASTAR_ERR_INVALID_ARG;
+  const CUtensorMap& sk = a.seg_tiles > 0 ? *tm_seg_k : tm_q;      // never read without segment tiles
+  const CUtensorMap& sv = a.seg_tiles > 0 ? *tm_seg_v : tm_q;
   const dim3 grid((a.nq + a.block_q - 1) / a.block_q, c.H, 1);
-  if (c.D == 128 && c.PT == 128) return launch_attn<128, 128, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
-  if (c.D == 128 && c.PT == 64) return launch_attn<128, 64, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
-  if (c.D == 64 && c.PT == 128) return launch_attn<64, 128, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
-  if (c.D == 64 && c.PT == 64) return launch_attn<64, 64, false>(tm_q, tm_pool_k, tm_pool_v, c, a, grid, st);
+  if (c.D == 128 && c.PT == 128) return launch_attn<128, 128, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 128 && c.PT == 64) return launch_attn<128, 64, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 64 && c.PT == 128) return launch_attn<64, 128, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 64 && c.PT == 64) return launch_attn<64, 64, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
   return FASTAR_ERR_UNSUPPORTED_SHAPE;
 }
 
 int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st) {
   const dim3 grid((a.rows_per_frame + 127) / 128, c.H, a.n_frames);
   const bool small = a.keep <= 64;
-  if (c.D == 128 && !small) return launch_attn<128, 128, true>(tm_q, tm_q, tm_q, c, a, grid, st);
-  if (c.D == 128 && small) return launch_attn<128, 64, true>(tm_q, tm_q, tm_q, c, a, grid, st);
-  if (c.D == 64 && !small) return launch_attn<64, 128, true>(tm_q, tm_q, tm_q, c, a, grid, st);
-  if (c.D == 64 && small) return launch_attn<64, 64, true>(tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 128 && !small) return launch_attn<128, 128, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 128 && small) return launch_attn<128, 64, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 64 && !small) return launch_attn<64, 128, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 64 && small) return launch_attn<64, 64, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
   return FASTAR_ERR_UNSUPPORTED_SHAPE;
 }
 

@@ -81,6 +81,7 @@ struct CacheView {
   // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
+  float* seg_bias;                 // [max_tokens + 128]  bias of the rows of an un-cached attention segment
 };
 
 inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
@@ -125,9 +126,14 @@ struct AttnArgs {
   void* out;               // [H][nq][D] caller dtype
   int out_fp32;
   int64_t out_head_stride, out_token_stride;
+  // paged mode: tiles of an un-cached K/V segment attended after the cache tiles (0 = none), and the bias of its
+  // rows (0 for a token, -inf past its end), seg_tiles * page_tokens floats
+  int seg_tiles;
+  const float* seg_bias;
 };
 int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
-                           const CUtensorMap& tm_pool_v, const AttnArgs& a, cudaStream_t st);
+                           const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
+                           const AttnArgs& a, cudaStream_t st);
 int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st);
 
 // update_kernels.cu

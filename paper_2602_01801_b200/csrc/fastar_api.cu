@@ -123,6 +123,7 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.kp8_ca = t.search_bits == 8 ? take(H * MP * 128) : nullptr;
   t.qn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MT * 4)) : nullptr;
   t.kpn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MP * 4)) : nullptr;
+  t.seg_bias = reinterpret_cast<float*>(take((MT + 128) * 4));
   for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
   for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
   cur = (cur + 1023) & ~static_cast<size_t>(1023);
@@ -156,6 +157,10 @@ int make_map_codes(fastar_cache* c, CUtensorMap* m, const void* ptr, uint64_t d1
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+__global__ void seg_bias_kernel(float* __restrict__ bias, int ns, int total) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) bias[i] = i < ns ? 0.f : -INFINITY;
 }
 
 __global__ void copy_rows3_kernel(const int32_t* __restrict__ src, int64_t src_hs, int src_rs, int32_t* __restrict__ dst, int rows,
@@ -447,10 +452,14 @@ int fastar_tempcache_update_probe(fastar_cache_t* c, const void* q_probe, const 
                      stream);
 }
 
-int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t nq, int64_t head_stride, int64_t token_stride,
-                           int32_t block_q, int32_t keep_blocks, int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out,
-                           float* scores_out, const int32_t* sel_in, const int32_t* nsel_in, void* stream) {
+// AnnSA; k_seg != nullptr adds the ns tokens of an un-cached K/V segment to every query's candidate set.
+static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const void* v_seg, int32_t ns, int64_t seg_head_stride,
+                      int64_t seg_token_stride, void* out, int32_t nq, int64_t head_stride, int64_t token_stride, int32_t block_q,
+                      int32_t keep_blocks, int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out, float* scores_out,
+                      const int32_t* sel_in, const int32_t* nsel_in, void* stream) {
   if (!c || !q || !out || nq < 1 || keep_blocks < 1) return FASTAR_ERR_INVALID_ARG;
+  if (k_seg && (!v_seg || ns < 1 || seg_token_stride < c->v.D || seg_head_stride < 0)) return FASTAR_ERR_INVALID_ARG;
+  if (k_seg && ns > c->v.max_tokens) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (block_q != 64 && block_q != 128) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (nq > c->v.max_tokens) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (token_stride < c->v.D || head_stride < 0 || (sel_in && !nsel_in)) return FASTAR_ERR_INVALID_ARG;
@@ -508,8 +517,40 @@ int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t 
                                         cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return FASTAR_ERR_CUDA;
   }
-  ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, a, st));
+  CUtensorMap tm_sk, tm_sv;
+  if (k_seg) {
+    const __nv_bfloat16 *skb, *svb;
+    int64_t khs = seg_head_stride, kts = seg_token_stride, vhs = seg_head_stride, vts = seg_token_stride;
+    r = as_bf16(c, k_seg, ns, &khs, &kts, 0, &skb, st);          // the update's staging slots are free during an attention call
+    if (r == FASTAR_OK) r = as_bf16(c, v_seg, ns, &vhs, &vts, 1, &svb, st);
+    if (r == FASTAR_OK) r = make_map(c, &tm_sk, skb, v.D, ns, v.H, static_cast<uint64_t>(kts) * 2, static_cast<uint64_t>(khs) * 2, v.PT);
+    if (r == FASTAR_OK) r = make_map(c, &tm_sv, svb, v.D, ns, v.H, static_cast<uint64_t>(vts) * 2, static_cast<uint64_t>(vhs) * 2, v.PT);
+    if (r != FASTAR_OK) return r;
+    a.seg_tiles = (ns + v.PT - 1) / v.PT;
+    a.seg_bias = v.seg_bias;
+    seg_bias_kernel<<<(a.seg_tiles * v.PT + 255) / 256, 256, 0, st>>>(v.seg_bias, ns, a.seg_tiles * v.PT);
+    if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+    c->launches += 1;
+  }
+  ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, k_seg ? &tm_sk : nullptr,
+                                                     k_seg ? &tm_sv : nullptr, a, st));
   return FASTAR_OK;
+}
+
+int fastar_annsa_attention(fastar_cache_t* c, const void* q, void* out, int32_t nq, int64_t head_stride, int64_t token_stride,
+                           int32_t block_q, int32_t keep_blocks, int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out,
+                           float* scores_out, const int32_t* sel_in, const int32_t* nsel_in, void* stream) {
+  return annsa_impl(c, q, nullptr, nullptr, 0, 0, 0, out, nq, head_stride, token_stride, block_q, keep_blocks, sel_out, nsel_out,
+                    qcode_out, scores_out, sel_in, nsel_in, stream);
+}
+
+int fastar_annsa_attention_segment(fastar_cache_t* c, const void* q, const void* k_seg, const void* v_seg, void* out, int32_t nq,
+                                   int32_t ns, int64_t head_stride, int64_t token_stride, int64_t seg_head_stride,
+                                   int64_t seg_token_stride, int32_t block_q, int32_t keep_blocks, const int32_t* sel_in,
+                                   const int32_t* nsel_in, void* stream) {
+  if (!k_seg || !v_seg) return FASTAR_ERR_INVALID_ARG;
+  return annsa_impl(c, q, k_seg, v_seg, ns, seg_head_stride, seg_token_stride, out, nq, head_stride, token_stride, block_q,
+                    keep_blocks, nullptr, nullptr, nullptr, nullptr, sel_in, nsel_in, stream);
 }
 
 int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_prompt, const void* v_prompt, void* out, int32_t nq,

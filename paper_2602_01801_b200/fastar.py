@@ -48,6 +48,8 @@ SIGNATURES = {
     "fastar_tempcache_update": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
     "fastar_tempcache_update_probe": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annsa_attention": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "fastar_annsa_attention_segment": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _i64, _i64, _i32, _i32, _vp, _vp,
+                                                 _vp]),
     "fastar_annca_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp,
                                          _vp, _vp]),
     "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _i32, _vp]),
@@ -254,6 +256,20 @@ class Cache:
                                                _ptr(res.get("scores")), _ptr(sel_in), _ptr(nsel_in), _stream()),
                "fastar_annsa_attention")
         return res
+
+    def annsa_segment(self, q, k_seg, v_seg, block_q: int, keep_blocks: int, sel_in=None, nsel_in=None, out=None):
+        """AnnSA over the cache plus an un-cached K/V segment [H][ns][d] (every segment token is a candidate)."""
+        torch = self.torch
+        H, nq, _ = q.shape
+        hs, ts = self._strides(q)
+        shs, sts = self._strides(k_seg)
+        assert self._strides(v_seg) == (shs, sts)
+        if out is None:
+            out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=self.device)
+        _check(self.lib.fastar_annsa_attention_segment(self.handle, q.data_ptr(), k_seg.data_ptr(), v_seg.data_ptr(), out.data_ptr(),
+                                                       nq, k_seg.shape[1], hs, ts, shs, sts, block_q, keep_blocks, _ptr(sel_in),
+                                                       _ptr(nsel_in), _stream()), "fastar_annsa_attention_segment")
+        return dict(out=out)
 
     def annca(self, q, k_prompt, v_prompt, frame_len: int, keep_tokens: int, sel_in=None, debug: bool = False, out=None):
         torch = self.torch

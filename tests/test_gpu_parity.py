@@ -374,3 +374,45 @@ def test_argument_errors_are_rejected_on_the_host():
     with pytest.raises(fastar.FastarError) as e:
         cache.update(dq, dq, 0, 0.9)
     assert e.value.status == fastar.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("d,pt,fp32", [(128, 128, False), (64, 64, False), (128, 64, True), (64, 128, False)])
+def test_annsa_with_uncached_segment(d, pt, fp32):
+    # Attention over [kept cache blocks, bias ln m] U [every token of an un-cached K/V segment]: the chunk being
+    # generated attends to itself before it is merged into the cache.  Ragged segment lengths (several tiles and a
+    # tail, shorter than one tile), sparse and dense selection, an empty cache, selection bypass.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, fp32)
+    Q, K, V = w.chunk(cfg.prior_chunks + 1)
+    dq, dk, dv = (fastar.to_device(x, fp32) for x in (Q, K, V))
+    # empty cache: dense attention over the segment
+    out = cache.annsa_segment(dq, dk, dv, cfg.block, cfg.keep_blocks)["out"].float().cpu().numpy()
+    assert cache.status() == 0
+    for h in range(cfg.num_heads):
+        P.check_attention(out[h], O.dense_attention(Q[h], K[h], V[h]), f"segment only, head {h}")
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks + 1):
+        _, Kc, Vc = w.chunk(ci)
+        gpu_update_checked(cache, heads, Kc, Vc, cfg.frame_len, 2.0 if ci < cfg.prior_chunks else cfg.tau, fp32)
+    assert max(int(hc.m.max()) for hc in heads) > 1
+    res = cache.annsa(dq, cfg.block, cfg.keep_blocks, debug=True)
+    sel, nsel = res["sel"].cpu().numpy(), res["nsel"].cpu().numpy()
+    for ns in (K.shape[1], pt // 2 + 3):
+        ks, vs = dk[:, :ns].contiguous(), dv[:, :ns].contiguous()
+        a = cache.annsa_segment(dq, ks, vs, cfg.block, cfg.keep_blocks)["out"]
+        b = cache.annsa_segment(dq, ks, vs, cfg.block, cfg.keep_blocks, sel_in=res["sel"], nsel_in=res["nsel"])["out"]
+        assert cache.status() == 0 and torch.equal(a, b)
+        out = a.float().cpu().numpy()
+        for h, hc in enumerate(heads):
+            want = O.sparse_attention_with_segment(Q[h], hc, sel[h][:, : nsel[h]], cfg.block, cfg.block, K[h, :ns], V[h, :ns])
+            P.check_attention(out[h], want, f"cache + segment of {ns}, head {h}")
+    # strided segment (a slice of a longer tensor) and dense selection over the whole cache
+    ns = K.shape[1] - 7
+    out = cache.annsa_segment(dq, dk[:, :ns], dv[:, :ns], cfg.block, cache.CAP // cache.PT)["out"].float().cpu().numpy()
+    assert cache.status() == 0
+    for h, hc in enumerate(heads):
+        allb = np.tile(np.arange(-(-hc.L // cfg.block)), (-(-Q.shape[1] // cfg.block), 1))
+        want = O.sparse_attention_with_segment(Q[h], hc, allb, cfg.block, cfg.block, K[h, :ns], V[h, :ns])
+        P.check_attention(out[h], want, f"dense cache + segment, head {h}")
