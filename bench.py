@@ -333,6 +333,35 @@ def run_ours(args, cfg):
                 "peak_source": f"{peak_kind} bf16 burst" + (" x 2 (nominal fp8 : bf16 ratio)" if fp8_dominant else ""),
                 "kernels": kernels, "ms_per_step_by_kernel": others}
 
+    variants = None
+    if args.variants:
+        # the step's neighbours in a rollout, each timed alone with CUDA events on the launching stream:
+        # AnnSA over [kept cache blocks + the chunk's own un-cached K/V] and the query-probe update
+        def timed(fn, reps=10, restore=False):
+            ms = []
+            for _ in range(3 + reps):
+                if restore:
+                    cache.workspace.copy_(snap)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                ms.append(e0.elapsed_time(e1))
+            return float(np.median(ms[3:]))
+        cache.workspace.copy_(snap)
+        cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)
+        seg_ms = timed(lambda: cache.annsa_segment(dq, dk, dv, cfg.block, cfg.keep_blocks, out=out_sa))
+        plain_ms = timed(lambda: cache.annsa(dq, cfg.block, cfg.keep_blocks, out=out_sa))
+        seg_flops = s5_flops + 4.0 * H * n * n * D
+        variants = {"annsa_call_ms": plain_ms, "annsa_with_segment_call_ms": seg_ms, "segment_tokens": n,
+                    "annsa_with_segment_flops": seg_flops,
+                    "annsa_with_segment_tflops_whole_call": seg_flops / (seg_ms * 1e-3) / 1e12}
+        if args.search_bits != 8:
+            variants["update_call_ms"] = timed(lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False), restore=True)
+            variants["update_query_probe_call_ms"] = timed(
+                lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq), restore=True)
+
     total_units, max_seconds = aggregate(float(n * args.steps), seconds, world, dist, dev)
     e2e_units, e2e_max = aggregate(float(n * args.steps), e2e_s, world, dist, dev)
     esz = 2
@@ -349,6 +378,8 @@ def run_ours(args, cfg):
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches_per_timed, "clocks": clocks.summary(), "roofline": roofline,
             "cache": {"len_before": len_before.tolist(), "len_after": len_after.tolist(), "workspace_bytes": cache.workspace_bytes}}
+    if variants is not None:
+        line["variants"] = variants
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             heads = 2 if cfg.num_heads >= 2 else 1
@@ -375,6 +406,8 @@ def main():
                     help="TempCache correspondence search on the bf16 keys (16, default) or on their 8-bit codes (8)")
     ap.add_argument("--probe", action="store_true",
                     help="query-probe correspondence: the update ranks cached keys by the dot product with the chunk's queries")
+    ap.add_argument("--variants", action="store_true",
+                    help="also time AnnSA with the chunk's own un-cached K/V segment and the query-probe update, each alone")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a captured CUDA graph")
     ap.add_argument("--mode", default="step", choices=["step", "rollout", "sweep"],
                     help="step = the one-line contract; rollout = c2 long rollout + dense baseline; sweep = c4 roofline sweep")
