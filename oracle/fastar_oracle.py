@@ -480,6 +480,53 @@ def annca(Q: np.ndarray, K_p: np.ndarray, V_p: np.ndarray, frame_len: int, keep:
 # --------------------------------------------------------------------------- #
 # Eq. 1 and the diagnostics of Sections 4 / 6
 # --------------------------------------------------------------------------- #
+def prompt_bucket_selection(qcodes: np.ndarray, pcodes: np.ndarray, frame_len: int) -> List[np.ndarray]:
+    """AnnCA's bucket rule as Section 5.3 states it: prompt token p is kept for frame f iff, in at least one
+    table, some query of frame f falls into the bucket of k_p.  qcodes [nq][T], pcodes [np][T] are bucket ids
+    (lsh_codes).  Returns one ascending index array per frame (possibly empty)."""
+    nq = qcodes.shape[0]
+    F = -(-nq // frame_len)
+    out = []
+    for f in range(F):
+        qc = qcodes[f * frame_len: min((f + 1) * frame_len, nq)]
+        hit = np.zeros(pcodes.shape[0], bool)
+        for t in range(qcodes.shape[1]):
+            hit |= np.isin(pcodes[:, t], qc[:, t])
+        out.append(np.flatnonzero(hit).astype(np.int64))
+    return out
+
+
+def annca_lsh(Q: np.ndarray, K_p: np.ndarray, V_p: np.ndarray, R: np.ndarray, tables: int, bits: int, frame_len: int,
+              qcodes: Optional[np.ndarray] = None, pcodes: Optional[np.ndarray] = None,
+              sel: Optional[List[np.ndarray]] = None) -> Dict[str, object]:
+    """AnnCA with the LSH selector (Sections 5.1, 5.3): queries and prompt keys are hashed with the shared random
+    projection, prompt tokens that share no bucket with any query of the frame are dropped, and every query of the
+    frame attends to the rest: o_i = softmax_{p in sel[f(i)]}(<q_i, k_p>/sqrt(d)) v_p.  The kept set has no fixed
+    size; a frame that keeps nothing gets o_i = 0.  qcodes / pcodes / sel replace stages (staged parity)."""
+    Q = np.asarray(Q, np.float64)
+    K_p = np.asarray(K_p, np.float64)
+    V_p = np.asarray(V_p, np.float64)
+    nq, d = Q.shape
+    if qcodes is None:
+        qcodes = lsh_codes(Q, R, tables, bits)
+    if pcodes is None:
+        pcodes = lsh_codes(K_p, R, tables, bits)
+    if sel is None:
+        sel = prompt_bucket_selection(qcodes, pcodes, frame_len)
+    O = np.zeros((nq, d))
+    for f, P in enumerate(sel):
+        rows = np.arange(f * frame_len, min((f + 1) * frame_len, nq))
+        P = np.asarray(P, np.int64)
+        if P.size == 0:
+            continue
+        logits = (Q[rows] @ K_p[P].T) / np.sqrt(d)
+        logits -= logits.max(axis=1, keepdims=True)
+        p = np.exp(logits)
+        p /= p.sum(axis=1, keepdims=True)
+        O[rows] = p @ V_p[P]
+    return dict(out=O, sel=sel, qcodes=qcodes, pcodes=pcodes)
+
+
 def dense_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, return_probs: bool = False):
     """O = softmax(Q K^T / sqrt(d)) V   (Eq. 1)."""
     Q, K, V = (np.asarray(a, np.float64) for a in (Q, K, V))

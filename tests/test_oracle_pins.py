@@ -540,3 +540,39 @@ def test_attention_with_uncached_segment():
     grouped = O.sparse_attention_with_segment(Q, c2, np.zeros((3, 1), np.int64), bq, bk, Ks, Vs)
     expanded = O.dense_attention(Q, np.concatenate([np.stack([k0, k0]), Ks]), np.concatenate([np.stack([v0a, v0b]), Vs]))
     assert np.allclose(grouped, expanded, atol=1e-12)
+
+
+def test_annca_lsh_bucket_rule():
+    rng = _rng(37)
+    d, nq, npr, fl, T, b = 16, 24, 30, 8, 3, 4
+    R = rng.standard_normal((T * b, d))
+    Q = rng.standard_normal((nq, d))
+    Kp = rng.standard_normal((npr, d))
+    Vp = rng.standard_normal((npr, d))
+    Kp[4] = 2.5 * Q[1]                  # positive multiples hash alike: always kept for the query's frame
+    Kp[9] = 0.3 * Q[20]
+    r = O.annca_lsh(Q, Kp, Vp, R, T, b, fl)
+    qc, pc = r["qcodes"], r["pcodes"]
+    assert 4 in r["sel"][0] and 9 in r["sel"][2]
+    # brute force over (frame, token, query, table)
+    for f in range(3):
+        want = [p for p in range(npr)
+                if any(qc[i, t] == pc[p, t] for i in range(f * fl, (f + 1) * fl) for t in range(T))]
+        assert r["sel"][f].tolist() == want
+    # more tables can only add collisions; one table with one bit keeps a token iff a query lies on its side
+    r1 = O.annca_lsh(Q, Kp, Vp, R[:b], 1, b, fl)
+    assert all(set(r1["sel"][f]) <= set(r["sel"][f]) for f in range(3))
+    rb = O.annca_lsh(Q, Kp, Vp, R[:1], 1, 1, fl)
+    side_q = Q @ R[0] > 0
+    for f in range(3):
+        sides = set(side_q[f * fl:(f + 1) * fl].tolist())
+        assert rb["sel"][f].tolist() == [p for p in range(npr) if (Kp[p] @ R[0] > 0) in sides]
+    # the attention over the kept set is the dense cross-attention restricted to it; keeping all = Eq. 1
+    f = 1
+    rows = np.arange(fl, 2 * fl)
+    assert np.allclose(r["out"][rows], O.dense_attention(Q[rows], Kp[r["sel"][f]], Vp[r["sel"][f]]), atol=1e-13)
+    allsel = [np.arange(npr)] * 3
+    assert np.allclose(O.annca_lsh(Q, Kp, Vp, R, T, b, fl, sel=allsel)["out"], O.dense_attention(Q, Kp, Vp), atol=1e-13)
+    # a frame that keeps nothing produces zeros
+    none = O.annca_lsh(Q, Kp, Vp, R, T, b, fl, sel=[np.arange(npr), np.zeros(0, np.int64), np.arange(3)])
+    assert not none["out"][rows].any() and none["out"][:fl].any()
