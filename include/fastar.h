@@ -220,6 +220,20 @@ int fastar_annca_attention(fastar_cache_t* cache, const void* q, const void* k_p
                            int64_t prompt_head_stride, int64_t prompt_token_stride,
                            int32_t* sel_out, float* rel_out, const int32_t* sel_in, void* stream);
 
+/* AnnCA with the LSH selector (Sections 5.1 and 5.3): the queries and the prompt keys are hashed with
+ * the cache's shared random projection (T tables of b bits); prompt token p is kept for frame f iff,
+ * in at least one table, some query of frame f lies in the bucket of k_p; every query of the frame
+ * attends to the kept tokens, o_i = softmax over them of q_i.k_p/sqrt(d), times v_p.  The kept set has
+ * no fixed size; a frame that keeps nothing gets zeros.  Tensors, strides and limits as for
+ * fastar_annca_attention; same concurrency rule.  Optional dev outputs: sel_out [H][F][np] (the first
+ * nsel_out[h][f] entries of a row are the kept tokens, ascending; the rest is unspecified),
+ * nsel_out [H][F], qcode_out [H][nq] and pcode_out [H][np] (bucket ids, table t in byte t). */
+int fastar_annca_attention_lsh(fastar_cache_t* cache, const void* q, const void* k_prompt, const void* v_prompt,
+                               void* out, int32_t nq, int32_t frame_len, int32_t np, int64_t head_stride,
+                               int64_t token_stride, int64_t prompt_head_stride, int64_t prompt_token_stride,
+                               int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out, uint32_t* pcode_out,
+                               void* stream);
+
 /* One whole attention step with HOST tensors (contiguous [H][n][d] / [H][np][d], cache dtype):
  * copies the inputs to the device, runs update -> AnnSA -> AnnCA (same arguments as above, the
  * chunk's n tokens being both the new keys/values and the queries), copies both outputs back and

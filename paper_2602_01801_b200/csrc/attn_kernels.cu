@@ -91,6 +91,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // ---- which rows and which key tiles ---------------------------------------------------------
   int q0, valid_rows, nt;
   int ntc = 0;                          // paged mode: tiles taken from the cache; tiles [ntc, nt) are segment tiles
+  int keep_n = a.keep;                  // gather mode: kept prompt tokens of this CTA's frame
   const int32_t* list;
   if (!GATHER) {
     const int qa = blockIdx.x;
@@ -108,7 +109,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const int f = blockIdx.z;
     q0 = f * a.rows_per_frame + blockIdx.x * 128;
     valid_rows = min(128, min(a.rows_per_frame - static_cast<int>(blockIdx.x) * 128, a.nq - q0));
-    nt = (a.keep + BKT - 1) / BKT;
+    if (a.keep_frames) keep_n = a.keep_frames[static_cast<int64_t>(h) * a.keep_frames_stride + f];
+    nt = (keep_n + BKT - 1) / BKT;
     list = a.sel + static_cast<int64_t>(h) * a.sel_head_stride + static_cast<int64_t>(f) * a.sel_stride;
   }
   if (valid_rows <= 0) return;          // uniform for the CTA; nothing allocated yet
@@ -154,7 +156,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int which = q / (BKT * CPR), qq = q % (BKT * CPR);
       const int i = qq / CPR, ch = qq % CPR;
       uint4 val = make_uint4(0, 0, 0, 0);
-      if (i < a.keep) {
+      if (i < keep_n) {
         const int idx = list[i];
         val = *reinterpret_cast<const uint4*>((which ? vp_h : kp_h) + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
       }
@@ -162,7 +164,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_s + off), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w)
                    : "memory");
     }
-    for (int i = threadIdx.x; i < BKT; i += blockDim.x) bias_g[i] = (i < a.keep) ? 0.f : -INFINITY;
+    for (int i = threadIdx.x; i < BKT; i += blockDim.x) bias_g[i] = (i < keep_n) ? 0.f : -INFINITY;
     fence_proxy_async_smem();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -278,7 +280,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const int i = q / CPR, ch = q % CPR;
           const int tok = j * BKT + i;
           uint4 val = make_uint4(0, 0, 0, 0);
-          if (tok < a.keep) {
+          if (tok < keep_n) {
             const int idx = list[tok];
             val = *reinterpret_cast<const uint4*>(src_h + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
           }
@@ -289,7 +291,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         const int b4 = j % NB;
         if (is_k)
-          for (int i = lane; i < BKT; i += 32) bias_g[b4 * BKT + i] = (j * BKT + i < a.keep) ? 0.f : -INFINITY;
+          for (int i = lane; i < BKT; i += 32) bias_g[b4 * BKT + i] = (j * BKT + i < keep_n) ? 0.f : -INFINITY;
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {

@@ -82,6 +82,10 @@ struct CacheView {
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
   float* seg_bias;                 // [max_tokens + 128]  bias of the rows of an un-cached attention segment
+  // AnnCA with the LSH bucket rule: codes of the queries and of the prompt keys, kept tokens per frame
+  uint32_t* code_q_ca;             // [H][max_tokens]
+  uint32_t* code_p_ca;             // [H][max_prompt]
+  int32_t* nselp;                  // [H][max_frames]
 };
 
 inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
@@ -130,6 +134,9 @@ struct AttnArgs {
   // rows (0 for a token, -inf past its end), seg_tiles * page_tokens floats
   int seg_tiles;
   const float* seg_bias;
+  // gather mode: kept tokens of every frame, [H][keep_frames_stride] (nullptr: `keep` for all frames)
+  const int32_t* keep_frames;
+  int keep_frames_stride;
 };
 int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
                            const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
@@ -140,6 +147,9 @@ int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const A
 int launch_convert_f32_to_bf16(const float* src, __nv_bfloat16* dst, int H, int n, int D, int64_t hs, int64_t ts, cudaStream_t st);
 int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
                       float* rnorm_out, cudaStream_t st);
+int launch_prep_codes_strided(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
+                              int64_t out_stride, cudaStream_t st);
+int launch_bucket_select(const CacheView& c, int nq, int frame_len, int n_frames, int np, cudaStream_t st);
 int launch_probe_cosine(const CacheView& c, const __nv_bfloat16* k_new, int n, int64_t hs, int64_t ts, cudaStream_t st);
 int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st);
 int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len,

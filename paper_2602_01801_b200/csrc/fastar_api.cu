@@ -124,6 +124,9 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.qn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MT * 4)) : nullptr;
   t.kpn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MP * 4)) : nullptr;
   t.seg_bias = reinterpret_cast<float*>(take((MT + 128) * 4));
+  t.code_q_ca = reinterpret_cast<uint32_t*>(take(H * MT * 4));
+  t.code_p_ca = reinterpret_cast<uint32_t*>(take(H * MP * 4));
+  t.nselp = reinterpret_cast<int32_t*>(take(H * t.max_frames * 4));
   for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
   for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
   cur = (cur + 1023) & ~static_cast<size_t>(1023);
@@ -626,6 +629,72 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
     }
     if (rel_out) ACC(launch_decode_rel(v, F, np, rel_scale, rel_out, st));
   }
+  ACCK(FASTAR_K_C3_ATTENTION, launch_attention_gather(v, tm_q, a, st));
+  return FASTAR_OK;
+}
+
+int fastar_annca_attention_lsh(fastar_cache_t* c, const void* q, const void* k_prompt, const void* v_prompt, void* out, int32_t nq,
+                               int32_t frame_len, int32_t np, int64_t head_stride, int64_t token_stride, int64_t prompt_head_stride,
+                               int64_t prompt_token_stride, int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out,
+                               uint32_t* pcode_out, void* stream) {
+  if (!c || !q || !k_prompt || !v_prompt || !out || nq < 1 || frame_len < 1 || np < 1) return FASTAR_ERR_INVALID_ARG;
+  const int F = (nq + frame_len - 1) / frame_len;
+  if (nq > c->v.max_tokens || np > c->v.max_prompt || F > c->v.max_frames) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (token_stride < c->v.D || prompt_token_stride < c->v.D) return FASTAR_ERR_INVALID_ARG;
+  const size_t osz = c->desc.dtype == FASTAR_FP32 ? 4 : 2;
+  if ((reinterpret_cast<uintptr_t>(out) & 15) || ((head_stride * osz) & 15) || ((token_stride * osz) & 15)) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  const __nv_bfloat16 *qb, *kpb, *vpb;
+  int64_t qhs = head_stride, qts = token_stride, khs = prompt_head_stride, kts = prompt_token_stride, vhs = prompt_head_stride,
+          vts = prompt_token_stride;
+  int r = as_bf16(c, q, nq, &qhs, &qts, 5, &qb, st);
+  if (r == FASTAR_OK) r = as_bf16(c, k_prompt, np, &khs, &kts, 3, &kpb, st);
+  if (r == FASTAR_OK) r = as_bf16(c, v_prompt, np, &vhs, &vts, 4, &vpb, st);
+  if (r != FASTAR_OK) return r;
+  if ((reinterpret_cast<uintptr_t>(kpb) & 15) || (reinterpret_cast<uintptr_t>(vpb) & 15) || ((khs * 2) & 15) || ((kts * 2) & 15))
+    return FASTAR_ERR_INVALID_ARG;
+  CUtensorMap tm_q;
+  r = make_map(c, &tm_q, qb, v.D, nq, v.H, static_cast<uint64_t>(qts) * 2, static_cast<uint64_t>(qhs) * 2, 128);
+  if (r != FASTAR_OK) return r;
+  // hash queries and prompt keys with the shared projection, mark the frame's buckets, keep the colliding tokens
+  ACCK(FASTAR_K_HASH, launch_prep_codes_strided(v, qb, nq, qhs, qts, v.code_q_ca, v.max_tokens, st));
+  ACCK(FASTAR_K_HASH, launch_prep_codes_strided(v, kpb, np, khs, kts, v.code_p_ca, v.max_prompt, st));
+  ACCK(FASTAR_K_TOPK_PROMPT, launch_bucket_select(v, nq, frame_len, F, np, st));
+  AttnArgs a{};
+  a.nq = nq;
+  a.block_q = 128;
+  a.rows_per_frame = frame_len;
+  a.keep = np;                      // upper bound; the kept count of every frame comes from keep_frames
+  a.keep_frames = v.nselp;
+  a.keep_frames_stride = v.max_frames;
+  a.n_frames = F;
+  a.kp = kpb;
+  a.vp = vpb;
+  a.p_head_stride = khs;
+  a.p_token_stride = kts;
+  a.out = out;
+  a.out_fp32 = c->desc.dtype == FASTAR_FP32;
+  a.out_head_stride = head_stride;
+  a.out_token_stride = token_stride;
+  a.sel = v.selp;
+  a.sel_stride = v.max_prompt;
+  a.sel_head_stride = static_cast<int64_t>(v.max_frames) * v.max_prompt;
+  if (sel_out) {
+    copy_rows3_kernel<<<dim3((F * np + 255) / 256, v.H), 256, 0, st>>>(v.selp, a.sel_head_stride, v.max_prompt, sel_out, F, np);
+    if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+    c->launches += 1;
+  }
+  if (nsel_out && cudaMemcpy2DAsync(nsel_out, static_cast<size_t>(F) * 4, v.nselp, static_cast<size_t>(v.max_frames) * 4,
+                                    static_cast<size_t>(F) * 4, v.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return FASTAR_ERR_CUDA;
+  if (qcode_out && cudaMemcpy2DAsync(qcode_out, static_cast<size_t>(nq) * 4, v.code_q_ca, static_cast<size_t>(v.max_tokens) * 4,
+                                     static_cast<size_t>(nq) * 4, v.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return FASTAR_ERR_CUDA;
+  if (pcode_out && cudaMemcpy2DAsync(pcode_out, static_cast<size_t>(np) * 4, v.code_p_ca, static_cast<size_t>(v.max_prompt) * 4,
+                                     static_cast<size_t>(np) * 4, v.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return FASTAR_ERR_CUDA;
   ACCK(FASTAR_K_C3_ATTENTION, launch_attention_gather(v, tm_q, a, st));
   return FASTAR_OK;
 }

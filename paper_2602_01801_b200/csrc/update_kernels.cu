@@ -221,6 +221,10 @@ int launch_prep_codes(const CacheView& c, const __nv_bfloat16* x, int n, int64_t
                       float* rnorm_out, cudaStream_t st) {
   return launch_prep_generic(c, x, n, hs, ts, code_out, rnorm_out, c.max_tokens, st);
 }
+int launch_prep_codes_strided(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint32_t* code_out,
+                              int64_t out_stride, cudaStream_t st) {
+  return launch_prep_generic(c, x, n, hs, ts, code_out, nullptr, out_stride, st);
+}
 
 // ---------------------------------------------------------------------------------------------
 // T2-T4 planning in three small kernels (all work O(n + L), no sort):
@@ -636,6 +640,54 @@ int launch_topk_blocks(const CacheView& c, int nqb, int keep, cudaStream_t st) {
                                                             min(keep, c.CAPB), c.nsel);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
+// ---------------------------------------------------------------------------------------------
+// AnnCA with the LSH bucket rule (Section 5.3): a prompt token is kept for a frame iff, in at least one table, a
+// query of the frame falls into its bucket.  One CTA per (frame, head): the buckets the frame's queries occupy are
+// marked in a T x 256 bit map in shared memory, every prompt token tests its T buckets, and the kept tokens are
+// written in ascending order (block scan) with their count.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) bucket_select_kernel(const CacheView c, int nq, int frame_len, int np) {
+  __shared__ uint32_t marks[4 * 8];
+  __shared__ int red[32];
+  const int f = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+  if (tid < 32) marks[tid] = 0u;
+  __syncthreads();
+  const uint32_t* qc = c.code_q_ca + static_cast<int64_t>(h) * c.max_tokens;
+  const int i1 = min(nq, (f + 1) * frame_len);
+  for (int i = f * frame_len + tid; i < i1; i += blockDim.x) {
+    const uint32_t code = qc[i];
+    for (int t = 0; t < c.T; ++t) {
+      const uint32_t w = (code >> (8 * t)) & 0xFFu;
+      atomicOr(&marks[t * 8 + (w >> 5)], 1u << (w & 31u));
+    }
+  }
+  __syncthreads();
+  const uint32_t* pc = c.code_p_ca + static_cast<int64_t>(h) * c.max_prompt;
+  int32_t* out = c.selp + (static_cast<int64_t>(h) * c.max_frames + f) * c.max_prompt;
+  int run = 0;
+  for (int p0 = 0; p0 < np; p0 += blockDim.x) {
+    const int p = p0 + tid;
+    int take = 0;
+    if (p < np) {
+      const uint32_t code = pc[p];
+      for (int t = 0; t < c.T; ++t) {
+        const uint32_t w = (code >> (8 * t)) & 0xFFu;
+        take |= static_cast<int>((marks[t * 8 + (w >> 5)] >> (w & 31u)) & 1u);
+      }
+    }
+    int tot;
+    const int pos = run + block_exscan(take, red, &tot);
+    if (take) out[pos] = p;
+    run += tot;
+  }
+  if (tid == 0) c.nselp[static_cast<int64_t>(h) * c.max_frames + f] = run;
+}
+
+int launch_bucket_select(const CacheView& c, int nq, int frame_len, int n_frames, int np, cudaStream_t st) {
+  bucket_select_kernel<<<dim3(n_frames, c.H), 256, 0, st>>>(c, nq, frame_len, np);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
 int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st) {
   topk_kernel<true><<<dim3(n_frames, c.H), 256, np * 4, st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
                                                              c.max_prompt, nullptr, 1, np, keep, c.selp,

@@ -52,6 +52,8 @@ SIGNATURES = {
                                                  _vp]),
     "fastar_annca_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp,
                                          _vp, _vp]),
+    "fastar_annca_attention_lsh": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp,
+                                             _vp]),
     "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _i32, _vp]),
     "fastar_last_device_status": (C.c_int, [_vp, _vp]),
     "fastar_launch_count": (C.c_int64, [_vp]),
@@ -289,6 +291,31 @@ class Cache:
                                                out.data_ptr(), nq, frame_len, np_, keep_tokens, hs, ts, phs, pts,
                                                _ptr(res.get("sel")), _ptr(res.get("rel")), _ptr(sel_in), _stream()),
                "fastar_annca_attention")
+        return res
+
+    def annca_lsh(self, q, k_prompt, v_prompt, frame_len: int, debug: bool = False, out=None):
+        """AnnCA with the LSH bucket rule: a prompt token is kept for a frame iff it shares a bucket with one of the
+        frame's queries (variable-size kept set).  debug adds sel [H][F][np] (first nsel[h][f] entries valid), nsel,
+        qcode, pcode."""
+        torch = self.torch
+        H, nq, _ = q.shape
+        np_ = k_prompt.shape[1]
+        hs, ts = self._strides(q)
+        phs, pts = self._strides(k_prompt)
+        assert self._strides(v_prompt) == (phs, pts)
+        F = -(-nq // frame_len)
+        if out is None:
+            out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=self.device)
+        res = dict(out=out)
+        if debug:
+            res.update(sel=torch.full((H, F, np_), -1, dtype=torch.int32, device=self.device),
+                       nsel=torch.empty((H, F), dtype=torch.int32, device=self.device),
+                       qcode=torch.empty((H, nq), dtype=torch.int32, device=self.device),
+                       pcode=torch.empty((H, np_), dtype=torch.int32, device=self.device))
+        _check(self.lib.fastar_annca_attention_lsh(self.handle, q.data_ptr(), k_prompt.data_ptr(), v_prompt.data_ptr(),
+                                                   out.data_ptr(), nq, frame_len, np_, hs, ts, phs, pts, _ptr(res.get("sel")),
+                                                   _ptr(res.get("nsel")), _ptr(res.get("qcode")), _ptr(res.get("pcode")),
+                                                   _stream()), "fastar_annca_attention_lsh")
         return res
 
     def step_host(self, k_new, v_new, q, k_prompt, v_prompt, out_sa, out_ca, frame_len: int, tau: float, block_q: int,

@@ -416,3 +416,47 @@ def test_annsa_with_uncached_segment(d, pt, fp32):
         allb = np.tile(np.arange(-(-hc.L // cfg.block)), (-(-Q.shape[1] // cfg.block), 1))
         want = O.sparse_attention_with_segment(Q[h], hc, allb, cfg.block, cfg.block, K[h, :ns], V[h, :ns])
         P.check_attention(out[h], want, f"dense cache + segment, head {h}")
+
+
+@pytest.mark.parametrize("d,fp32,bits", [(128, False, 8), (64, True, 8), (128, False, 3)])
+def test_annca_lsh_bucket_rule(d, fp32, bits):
+    # AnnCA with the LSH selector: codes of queries and prompt keys (sign bits clear of zero must agree), the kept
+    # set of every frame exactly as the oracle derives it from those codes (variable size, ascending), attention
+    # over it.  A ragged last frame, a planted token that equals a query, and a frame that keeps nothing.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(head_dim=d, block=64, capacity=2048, keep_blocks=5, num_heads=3, lsh_bits=bits)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, fp32)
+    R = w.lsh_projection()
+    Q, _, _ = w.chunk(0)
+    Kp, Vp, _ = w.prompt(0)
+    Kp, Vp = Kp.copy(), Vp.copy()
+    Kp[:, 5] = Q[:, 7]                                     # shares every bucket with query 7 of frame 0
+    nq = Q.shape[1] - 11                                   # ragged last frame
+    Q = Q[:, :nq]
+    res = cache.annca_lsh(fastar.to_device(Q, fp32), fastar.to_device(Kp, fp32), fastar.to_device(Vp, fp32), cfg.frame_len,
+                          debug=True)
+    assert cache.status() == 0
+    out = res["out"].float().cpu().numpy()
+    sel, nsel = res["sel"].cpu().numpy(), res["nsel"].cpu().numpy()
+    F = -(-nq // cfg.frame_len)
+    sizes = set()
+    for h in range(cfg.num_heads):
+        qc = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, res["qcode"][h].cpu().numpy().view(np.uint32))
+        pc = P.check_codes(Kp[h], R, cfg.lsh_tables, cfg.lsh_bits, res["pcode"][h].cpu().numpy().view(np.uint32))
+        want_sel = O.prompt_bucket_selection(qc, pc, cfg.frame_len)
+        got_sel = [sel[h, f, : nsel[h, f]].astype(np.int64) for f in range(F)]
+        for f in range(F):
+            assert np.array_equal(got_sel[f], want_sel[f]), f"kept set of head {h}, frame {f}"
+            sizes.add(len(got_sel[f]))
+        assert 5 in got_sel[0]
+        want = O.annca_lsh(Q[h], Kp[h], Vp[h], R, cfg.lsh_tables, cfg.lsh_bits, cfg.frame_len, sel=got_sel)["out"]
+        P.check_attention(out[h], want, f"AnnCA-LSH head {h}")
+    assert max(sizes) <= Kp.shape[1] and (len(sizes) > 1 if bits == 8 else sizes == {Kp.shape[1]})   # 8 buckets: all collide
+    # no collision at all: prompt keys opposite to every query direction cannot share a full code when the queries
+    # of the frame all hash to one bucket per table (a single repeated query)
+    Q1 = np.repeat(Q[:, :1], nq, axis=1)
+    Kn = np.repeat(-Q[:, :1], Kp.shape[1], axis=1)
+    r2 = cache.annca_lsh(fastar.to_device(Q1, fp32), fastar.to_device(Kn, fp32), fastar.to_device(Vp, fp32), cfg.frame_len,
+                         debug=True)
+    assert cache.status() == 0 and int(r2["nsel"].max()) == 0 and not r2["out"].float().abs().max().item() > 0
