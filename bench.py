@@ -357,6 +357,11 @@ def run_ours(args, cfg):
         variants = {"annsa_call_ms": plain_ms, "annsa_with_segment_call_ms": seg_ms, "segment_tokens": n,
                     "annsa_with_segment_flops": seg_flops,
                     "annsa_with_segment_tflops_whole_call": seg_flops / (seg_ms * 1e-3) / 1e12}
+        variants["annca_call_ms"] = timed(lambda: cache.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt, out=out_ca))
+        variants["annca_lsh_call_ms"] = timed(lambda: cache.annca_lsh(dq, dkp, dvp, cfg.frame_len, out=out_ca))
+        kept = cache.annca_lsh(dq, dkp, dvp, cfg.frame_len, debug=True)["nsel"].cpu().numpy()
+        variants["annca_lsh_kept_tokens"] = {"min": int(kept.min()), "mean": float(kept.mean()), "max": int(kept.max()),
+                                             "of": cfg.prompt_tokens}
         if args.search_bits != 8:
             variants["update_call_ms"] = timed(lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False), restore=True)
             variants["update_query_probe_call_ms"] = timed(
