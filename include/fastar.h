@@ -21,7 +21,7 @@
  *     void* (0 = the legacy default stream).  All work is enqueued on that stream and the
  *     call returns without synchronising unless stated otherwise.
  *   - Ownership: the caller owns every tensor and the workspace buffer; the library owns only
- *     the small host object behind fastar_cache_t (with a CUDA stream and three events created and
+ *     the small host object behind fastar_cache_t (with two CUDA streams and five events created and
  *     destroyed with it).  Nothing here allocates device memory.
  *   - Tensors are [head][token][channel] with element strides `head_stride`, `token_stride`
  *     (channel stride 1).  Strides in bytes must be multiples of 16 and base pointers 16-byte
@@ -239,8 +239,10 @@ int fastar_annca_attention_lsh(fastar_cache_t* cache, const void* q, const void*
  * chunk's n tokens being both the new keys/values and the queries), copies both outputs back and
  * synchronises the stream.  Staging buffers live in the workspace.  The uploads of q and of the
  * prompt, AnnCA and the download of its output run on a second stream owned by the cache object,
- * beside the update; that stream starts after the work already queued on `stream` and is idle
- * again when the call returns.  flags: 0, or FASTAR_STEP_QUERY_PROBE to run the update as
+ * beside the update, and the new values are uploaded last, on a third stream, while the
+ * correspondence search (which reads only the keys) already runs; those streams start after the
+ * work already queued on `stream` and are idle again when the call returns.
+ * flags: 0, or FASTAR_STEP_QUERY_PROBE to run the update as
  * fastar_tempcache_update_probe with q as the probe. */
 #define FASTAR_STEP_QUERY_PROBE 1
 int fastar_attention_step_host(fastar_cache_t* cache, const void* k_new_host, const void* v_new_host,

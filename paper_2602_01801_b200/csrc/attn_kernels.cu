@@ -50,7 +50,8 @@ __device__ __forceinline__ void ld_shared_f32x2(uint32_t addr, float& a, float& 
   asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
 }
 
-template <int D, int BKT, bool GATHER>
+// SEG (paged mode only): tiles of an un-cached K/V segment follow the cache tiles.
+template <int D, int BKT, bool GATHER, bool SEG>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_sk,
@@ -104,7 +105,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       ntc = a.nsel[h];
       list = a.sel + static_cast<int64_t>(h) * a.sel_head_stride + static_cast<int64_t>(qa) * a.sel_stride;
     }
-    nt = ntc + a.seg_tiles;
+    nt = ntc + (SEG ? a.seg_tiles : 0);
   } else {
     const int f = blockIdx.z;
     q0 = f * a.rows_per_frame + blockIdx.x * 128;
@@ -132,7 +133,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if (warp == kProducerWarp && lane == 0) {
     tma_prefetch_desc(&tm_q);
     if (!GATHER) { tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); }
-    if (!GATHER && a.seg_tiles > 0) { tma_prefetch_desc(&tm_sk); tma_prefetch_desc(&tm_sv); }
+    if (SEG) { tma_prefetch_desc(&tm_sk); tma_prefetch_desc(&tm_sv); }
   }
   __syncthreads();
   if (warp == kMmaWarp) {
@@ -195,7 +196,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (jj < ntc) {
           blk = list ? list[jj] : jj;
           page = pt_h[blk];
-        } else if (jj < nt) {               // tile of the un-cached segment: its index, no page
+        } else if (SEG && jj < nt) {        // tile of the un-cached segment: its index, no page
           blk = jj - ntc;
           page = -1;
         }
@@ -207,7 +208,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #ifdef FASTAR_PHASE_TIMING
         reinterpret_cast<volatile long long*>(sgen + SM::bar_off + kBarBytes + 8)[s] = clock64();
 #endif
-        const bool seg = page < 0;          // rows past the segment's end arrive as zeros and carry a -inf bias
+        const bool seg = SEG && page < 0;   // rows past the segment's end arrive as zeros and carry a -inf bias
         const CUtensorMap* tm = seg ? (is_k ? &tm_sk : &tm_sv) : (is_k ? &tm_k : &tm_v);
         mbar_arrive_expect_tx(bar_r_full + 8 * s, SM::kv_bytes);
         for (int kc = 0; kc < D / 64; ++kc)
@@ -531,11 +532,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int D, int BKT, bool GATHER>
+template <int D, int BKT, bool GATHER, bool SEG>
 static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tsk,
                        const CUtensorMap& tsv, const CacheView& c, const AttnArgs& a, dim3 grid, cudaStream_t st) {
   using SM = AttnSmem<D, BKT>;
-  auto kern = attn_kernel<D, BKT, GATHER>;
+  auto kern = attn_kernel<D, BKT, GATHER, SEG>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
@@ -554,20 +555,24 @@ int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CU
   const CUtensorMap& sk = a.seg_tiles > 0 ? *tm_seg_k : tm_q;      // never read without segment tiles
   const CUtensorMap& sv = a.seg_tiles > 0 ? *tm_seg_v : tm_q;
   const dim3 grid((a.nq + a.block_q - 1) / a.block_q, c.H, 1);
-  if (c.D == 128 && c.PT == 128) return launch_attn<128, 128, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
-  if (c.D == 128 && c.PT == 64) return launch_attn<128, 64, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
-  if (c.D == 64 && c.PT == 128) return launch_attn<64, 128, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
-  if (c.D == 64 && c.PT == 64) return launch_attn<64, 64, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 128 && c.PT == 128) return a.seg_tiles > 0 ? launch_attn<128, 128, false, true>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st)
+                                                          : launch_attn<128, 128, false, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 128 && c.PT == 64) return a.seg_tiles > 0 ? launch_attn<128, 64, false, true>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st)
+                                                          : launch_attn<128, 64, false, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 64 && c.PT == 128) return a.seg_tiles > 0 ? launch_attn<64, 128, false, true>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st)
+                                                          : launch_attn<64, 128, false, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
+  if (c.D == 64 && c.PT == 64) return a.seg_tiles > 0 ? launch_attn<64, 64, false, true>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st)
+                                                          : launch_attn<64, 64, false, false>(tm_q, tm_pool_k, tm_pool_v, sk, sv, c, a, grid, st);
   return FASTAR_ERR_UNSUPPORTED_SHAPE;
 }
 
 int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st) {
   const dim3 grid((a.rows_per_frame + 127) / 128, c.H, a.n_frames);
   const bool small = a.keep <= 64;
-  if (c.D == 128 && !small) return launch_attn<128, 128, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
-  if (c.D == 128 && small) return launch_attn<128, 64, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
-  if (c.D == 64 && !small) return launch_attn<64, 128, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
-  if (c.D == 64 && small) return launch_attn<64, 64, true>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 128 && !small) return launch_attn<128, 128, true, false>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 128 && small) return launch_attn<128, 64, true, false>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 64 && !small) return launch_attn<64, 128, true, false>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
+  if (c.D == 64 && small) return launch_attn<64, 64, true, false>(tm_q, tm_q, tm_q, tm_q, tm_q, c, a, grid, st);
   return FASTAR_ERR_UNSUPPORTED_SHAPE;
 }
 

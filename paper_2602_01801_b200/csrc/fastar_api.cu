@@ -26,13 +26,16 @@ struct fastar_cache {
   int64_t launches;
   size_t bytes;
   // second stream of the host-tensor step (uploads of q and the prompt, AnnCA, its download) and its fork/join events
-  cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_q = nullptr, ev_join = nullptr;
+  cudaStream_t side = nullptr, copy = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_q = nullptr, ev_join = nullptr, ev_p = nullptr, ev_v = nullptr;
   ~fastar_cache() {
     if (ev_fork) cudaEventDestroy(ev_fork);
     if (ev_q) cudaEventDestroy(ev_q);
     if (ev_join) cudaEventDestroy(ev_join);
+    if (ev_p) cudaEventDestroy(ev_p);
+    if (ev_v) cudaEventDestroy(ev_v);
     if (side) cudaStreamDestroy(side);
+    if (copy) cudaStreamDestroy(copy);
   }
 };
 
@@ -261,6 +264,9 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
     r = make_map_codes(c, &c->tm_pool_k8, v.pool_k8, PT, static_cast<uint64_t>(v.H) * v.CAPB, PT * 128, v.PT);
   if (r == FASTAR_OK &&
       (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+       cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
+       cudaEventCreateWithFlags(&c->ev_p, cudaEventDisableTiming) != cudaSuccess ||
+       cudaEventCreateWithFlags(&c->ev_v, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_q, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
@@ -390,9 +396,11 @@ int fastar_cache_import(fastar_cache_t* c, const uint16_t* host_k, const uint16_
 
 // One update; q_probe == nullptr is the key -> key cosine search, otherwise the cached keys are ranked by their dot
 // product with the probe rows and the threshold is applied to the key cosine of the winner.
+// v_ready (may be null): an event after which v_new may be read; the search and the planning, which read only the
+// keys, are queued before the wait.
 static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new, const void* v_new, int32_t n, int32_t frame_len,
                        int64_t head_stride, int64_t token_stride, float tau, int32_t* match_out, float* sim_out,
-                       int32_t* dest_out, fastar_update_stats* stats_out, void* stream) {
+                       int32_t* dest_out, fastar_update_stats* stats_out, void* stream, cudaEvent_t v_ready = nullptr) {
   if (!c || !k_new || !v_new || n < 1 || frame_len < 1) return FASTAR_ERR_INVALID_ARG;
   if (n > c->v.max_tokens || n > 16384 || n > c->v.CAP) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (q_probe && c->v.search_bits == 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
@@ -404,6 +412,8 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
   int64_t khs = head_stride, kts = token_stride, vhs = head_stride, vts = token_stride, phs = head_stride, pts = token_stride;
   int r = as_bf16(c, k_new, n, &khs, &kts, 0, &kb, st);
   if (r != FASTAR_OK) return r;
+  const bool v_converted = c->desc.dtype != FASTAR_BF16;      // the entry conversion already reads v_new
+  if (v_ready && v_converted && cudaStreamWaitEvent(st, v_ready, 0) != cudaSuccess) return FASTAR_ERR_CUDA;
   r = as_bf16(c, v_new, n, &vhs, &vts, 1, &vb, st);
   if (r != FASTAR_OK) return r;
   if (q_probe) {
@@ -434,6 +444,7 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
     ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
   }
   ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
+  if (v_ready && !v_converted && cudaStreamWaitEvent(st, v_ready, 0) != cudaSuccess) return FASTAR_ERR_CUDA;
   ACCK(FASTAR_K_COMMIT, launch_commit(v, kb, vb, n, frame_len, khs, kts, st));
   ACCK(FASTAR_K_KEY_HIST, launch_finalize_hist(v, stats_out, 1, st));
   ACC(launch_copy_outputs(v, n, match_out, sim_out, dest_out, st));
@@ -718,22 +729,30 @@ int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const 
     const size_t bytes = static_cast<size_t>(v.H) * (i < 3 ? n : np) * v.D * esz;
     return cudaMemcpyAsync(dsrc[i], hsrc[i], bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
   };
-  // Two streams, so that the copies and the two attentions overlap the cache update instead of queueing behind it:
-  //   caller's stream : upload K, V -> update -> (q uploaded) AnnSA -> download its output
+  // Three streams, so that the copies and the two attentions overlap the cache update instead of queueing behind it.
+  // The host link is the bottleneck of this call, so the uploads are ordered by when their consumer can start:
+  // K first (the correspondence search and the planning read only the keys), then q and the prompt (AnnCA), V last
+  // (read by the merge at the end of the update).
+  //   caller's stream : upload K -> update [search, plan | wait V | merge] -> (q uploaded) AnnSA -> download its output
   //   side stream     : upload q, prompt K/V -> AnnCA (reads no cache state) -> download its output
-  // The side stream starts after everything already queued on the caller's stream and is joined before returning.
-  cudaStream_t sd = c->side;
+  //   copy stream     : (prompt uploaded) upload V
+  // The owned streams start after everything already queued on the caller's stream and are joined before returning.
+  cudaStream_t sd = c->side, sc = c->copy;
   const int64_t hs = static_cast<int64_t>(n) * v.D, ts = v.D, phs = static_cast<int64_t>(np) * v.D;
   const size_t obytes = static_cast<size_t>(v.H) * n * v.D * esz;
   if (cudaEventRecord(c->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(sd, c->ev_fork, 0) != cudaSuccess) return FASTAR_ERR_CUDA;
   int r = FASTAR_OK;
-  bool copies_ok = upload(0, st) && upload(1, st) && upload(2, sd);
-  copies_ok = copies_ok && cudaEventRecord(c->ev_q, sd) == cudaSuccess && upload(3, sd) && upload(4, sd);
+  bool copies_ok = upload(0, st) && upload(2, sd);
+  copies_ok = copies_ok && cudaEventRecord(c->ev_q, sd) == cudaSuccess && upload(3, sd) && upload(4, sd) &&
+              cudaEventRecord(c->ev_p, sd) == cudaSuccess && cudaStreamWaitEvent(sc, c->ev_p, 0) == cudaSuccess && upload(1, sc);
+  // recorded even after a failed copy: the update below waits on it
+  copies_ok = (cudaEventRecord(c->ev_v, sc) == cudaSuccess) && copies_ok;
   if (!copies_ok) r = FASTAR_ERR_CUDA;
   const bool probe = (flags & FASTAR_STEP_QUERY_PROBE) != 0;
   if (r == FASTAR_OK && probe && cudaStreamWaitEvent(st, c->ev_q, 0) != cudaSuccess) r = FASTAR_ERR_CUDA;   // the update reads q
   if (r == FASTAR_OK)
-    r = update_impl(c, probe ? dsrc[2] : nullptr, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, st);
+    r = update_impl(c, probe ? dsrc[2] : nullptr, dsrc[0], dsrc[1], n, frame_len, hs, ts, tau, nullptr, nullptr, nullptr, nullptr, st,
+                    c->ev_v);
   if (r == FASTAR_OK)
     r = fastar_annca_attention(c, dsrc[2], dsrc[3], dsrc[4], v.stage_out[1], n, frame_len, np, keep_tokens, hs, ts, phs, ts, nullptr,
                                nullptr, nullptr, sd);
@@ -743,11 +762,12 @@ int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const 
     r = fastar_annsa_attention(c, dsrc[2], v.stage_out[0], n, hs, ts, block_q, keep_blocks, nullptr, nullptr, nullptr, nullptr, nullptr,
                                nullptr, st);
   if (r == FASTAR_OK && cudaMemcpyAsync(out_sa_host, v.stage_out[0], obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) r = FASTAR_ERR_CUDA;
-  // always join: the side stream must be idle when this call returns, whatever happened above
+  // always join: the owned streams must be idle when this call returns, whatever happened above
   const bool joined = cudaEventRecord(c->ev_join, sd) == cudaSuccess && cudaStreamWaitEvent(st, c->ev_join, 0) == cudaSuccess &&
-                      cudaStreamSynchronize(st) == cudaSuccess;
+                      cudaStreamWaitEvent(st, c->ev_v, 0) == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
   if (!joined) {
     cudaStreamSynchronize(sd);
+    cudaStreamSynchronize(sc);
     return r != FASTAR_OK ? r : FASTAR_ERR_CUDA;
   }
   return r;
