@@ -41,7 +41,9 @@ struct GemmSmem {
   static constexpr int total = bar_off + 256;
 };
 
-template <int EPI, bool A_RES, int NST>
+// A_TMEM (with A_RES): the resident A tile is moved from shared memory into tensor memory once, so that an MMA
+// reads only its B operand from shared memory; the CTA then owns all 512 TMEM columns (one CTA per SM).
+template <int EPI, bool A_RES, int NST, bool A_TMEM = false>
 __global__ void __launch_bounds__(kGemmThreads, A_RES ? 2 : 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c,
             const GemmArgs g) {
@@ -65,6 +67,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   const uint32_t bar_afull = bar_tempty + 16;        // [1]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + SM::bar_off + 16 * NST + 40);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + SM::bar_off + 16 * NST + 44);
+  const uint32_t bar_atm = bar_s + 16 * NST + 48;    // [1] A copied into tensor memory (A_TMEM)
+  static_assert(16 * NST + 56 <= 256, "barrier area");
+  constexpr int kCols = kTmemCols;                   // A_TMEM: one accumulator (128 columns) + A (64 columns)
+  constexpr int kAcol = 128;                         // first TMEM column of A (A_TMEM)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int h = blockIdx.y;
@@ -91,6 +97,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       mbar_init(bar_tempty + 8 * b, 8);          // one arrival per epilogue warp
     }
     mbar_init(bar_afull, 1);
+    mbar_init(bar_atm, 4);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -100,7 +107,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   }
   __syncthreads();
   if (warp == kGemmMmaWarp) {
-    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_alloc(smem_u32(tmem_slot), kCols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -163,11 +170,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         constexpr uint32_t idesc = make_idesc_bf16(128, 128, 0);
         bool ok = true;
         if (A_RES) ok = mbar_wait(bar_afull, 0, abort_flag, c.status);
+        if (A_TMEM && ok) ok = mbar_wait(bar_atm, 0, abort_flag, c.status);
         int it = 0;
         PT_DECL
         for (int tl = 0; tl < ntl && ok; ++tl) {
-          const int buf = tl & 1;
-          ok = mbar_wait(bar_tempty + 8 * buf, ((tl >> 1) & 1) ^ 1, abort_flag, c.status);
+          const int buf = A_TMEM ? 0 : (tl & 1), bph = A_TMEM ? (tl & 1) : ((tl >> 1) & 1);
+          ok = mbar_wait(bar_tempty + 8 * buf, bph ^ 1, abort_flag, c.status);
           if (!ok) break;
           PT_MARK(0)
           tc_fence_after();
@@ -185,7 +193,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             for (int k4 = 0; k4 < 4; ++k4) {
               const uint64_t ad = make_smem_desc(a_c + k4 * 32, 16, 1024);
               const uint64_t bd = make_smem_desc(b_c + k4 * 32, 16, 1024);
-              umma_ss(d_t, ad, bd, idesc, (kc | k4) != 0);
+              if (A_TMEM) umma_ts(d_t, tmem + kAcol + kc * 32 + k4 * 8, bd, idesc, (kc | k4) != 0);
+              else umma_ss(d_t, ad, bd, idesc, (kc | k4) != 0);
             }
             umma_commit(bar_empty + 8 * s);
             PT_MARK(2)
@@ -206,22 +215,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       int best_j = -1;
       float rn_next = 0.f;                           // 1/|k| of the next tile's keys, loaded one tile ahead
       bool ok = true;
+      if (A_TMEM && wg == 0) {
+        // shared memory (128-byte swizzle) -> registers -> tensor memory: thread r moves row r, 64 elements
+        // (32 columns) per store
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_afull, 0, abort_flag, c.status));
+        if (ok) {
+          for (int kc = 0; kc < nkc; ++kc) {
+            uint32_t regs[32];
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+              const uint32_t addr = a_s + kc * kChunkBytes + r * 128 + ((ch ^ (r & 7)) << 4);
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                           : "=r"(regs[4 * ch]), "=r"(regs[4 * ch + 1]), "=r"(regs[4 * ch + 2]), "=r"(regs[4 * ch + 3])
+                           : "r"(addr));
+            }
+            tmem_st32(tmem + lane_addr + kAcol + kc * 32, regs);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive_warp(bar_atm);
+        }
+      }
       PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
-        const int buf = tl & 1;
+        const int buf = A_TMEM ? 0 : (tl & 1), bph = A_TMEM ? (tl & 1) : ((tl >> 1) & 1), rbuf = tl & 1;
         int valid_cols = 128;
         if (EPI == EPI_ARGMAX) {
           if (wg == 0) {
             if (tl == 0) rn_next = (t * 128 + r < L) ? (c.raw_dot ? 1.f : c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r]) : 0.f;
-            rn_s[buf * 128 + r] = rn_next;
+            rn_s[rbuf * 128 + r] = rn_next;
             const int slot = (t + 1) * 128 + r;
             rn_next = (tl + 1 < ntl && slot < L) ? (c.raw_dot ? 1.f : c.rnorm[static_cast<int64_t>(h) * c.CAP + slot]) : 0.f;
           }
           valid_cols = min(128, L - t * 128);
           named_barrier_sync(1, 256);
         }
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bph, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
         PT_MARK(0)
         tc_fence_after();
@@ -239,7 +269,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           if (EPI == EPI_ARGMAX) {
             // Scores of the chunk, then a tree maximum (no serial compare/select chain); the index is
             // searched only when the chunk holds a new strict maximum, which is rare after the first tiles.
-            chunk_argmax(v, reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
+            chunk_argmax(v, reinterpret_cast<const float4*>(rn_s + rbuf * 128 + cc * 32), valid_cols - cc * 32,
                          t * 128 + cc * 32, best, best_j);
           } else if (EPI == EPI_COLMAX) {
             const bool rvalid = row < g.rows_a;
@@ -295,15 +325,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   __syncthreads();
   if (warp == kGemmMmaWarp) {
     tc_fence_after();
-    tmem_dealloc(tmem, kTmemCols);
+    tmem_dealloc(tmem, kCols);
   }
 }
 
-template <int EPI, bool A_RES, int NST>
+template <int EPI, bool A_RES, int NST, bool A_TMEM = false>
 static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const CacheView& c, const GemmArgs& g, dim3 grid,
                        cudaStream_t st) {
   using SM = GemmSmem<EPI, A_RES, NST>;
-  auto kern = gemm_kernel<EPI, A_RES, NST>;
+  auto kern = gemm_kernel<EPI, A_RES, NST, A_TMEM>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
@@ -592,6 +622,13 @@ int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUte
   if (const char* force = std::getenv("FASTAR_T1_KERNEL")) {
     if (std::strcmp(force, "pair") == 0) use_pair = true;
     else if (std::strcmp(force, "single") == 0) use_pair = false;
+  }
+  if (const char* force = std::getenv("FASTAR_T1_KERNEL")) {
+    if (std::strcmp(force, "ts") == 0) {
+      double eff = 0.0;
+      const int splits = pick_splits(tiles_single * c.H, slots, max_tiles, &eff);
+      return launch_gemm<EPI_ARGMAX, true, 4, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits), st);
+    }
   }
   if (use_pair) return launch_t1_pair(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st);
   return launch_gemm<EPI_ARGMAX, true, 4>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st);

@@ -136,11 +136,12 @@ def test_other_tile_shapes(d, pt):
     full_step(cfg)
 
 
-@pytest.mark.parametrize("kernel", ["single", "pair"])
+@pytest.mark.parametrize("kernel", ["single", "pair", "ts"])
 @pytest.mark.parametrize("d,pt", [(128, 128), (64, 64)])
 def test_both_similarity_kernels(kernel, d, pt, monkeypatch):
     # The launcher picks the single-CTA or the CTA-pair similarity kernel from the grid's wave efficiency; force each
     # one in turn so that both are checked against the oracle (ragged row tiles, ragged cache lengths, two updates).
+    # "ts" is the single-CTA kernel with the new keys held in tensor memory (A operand from TMEM), an option.
     monkeypatch.setenv("FASTAR_T1_KERNEL", kernel)
     cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
     cache, w, heads, post, _, _ = full_step(cfg)
