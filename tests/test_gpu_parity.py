@@ -461,3 +461,26 @@ def test_annca_lsh_bucket_rule(d, fp32, bits):
     r2 = cache.annca_lsh(fastar.to_device(Q1, fp32), fastar.to_device(Kn, fp32), fastar.to_device(Vp, fp32), cfg.frame_len,
                          debug=True)
     assert cache.status() == 0 and int(r2["nsel"].max()) == 0 and not r2["out"].float().abs().max().item() > 0
+
+
+def test_frame_sequential_updates_and_per_call_dense_switch():
+    # A chunk fed to the cache one frame per call (a later frame can then merge into slots an earlier frame of the
+    # same chunk created or refreshed), and attention switched between dense and sparse from one call to the next
+    # on the same cache, as a schedule that keeps the first denoising steps dense would do.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(num_heads=2)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0)
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    fl = cfg.frame_len
+    post = None
+    for f in range(K.shape[1] // fl):
+        post = gpu_update_checked(cache, heads, K[:, f * fl:(f + 1) * fl], V[:, f * fl:(f + 1) * fl], fl, cfg.tau)
+    assert int(post["now"][0]) == cfg.prior_chunks + K.shape[1] // fl
+    capb = cache.CAP // cache.PT
+    for keep in (capb, cfg.keep_blocks, capb, cfg.keep_blocks):
+        gpu_annsa_checked(cache, cfg, w, Q, post, keep)
