@@ -417,6 +417,8 @@ def main():
     ap.add_argument("--mode", default="step", choices=["step", "rollout", "sweep"],
                     help="step = the one-line contract; rollout = c2 long rollout + dense baseline; sweep = c4 roofline sweep")
     ap.add_argument("--chunks", type=int, default=120)
+    ap.add_argument("--denoise-steps", type=int, default=0,
+                    help="rollout mode: denoising steps per chunk, each attending to the cache plus the chunk's own un-cached K/V")
     ap.add_argument("--out", default=None)
     ap.add_argument("--no-dense", action="store_true")
     args = ap.parse_args()

@@ -58,9 +58,18 @@ def run_rollout(args):
         Kp, Vp, _ = w.prompt(ci)
         dq, dk, dv, dkp, dvp = (fastar.to_device(x) for x in (Q, K, V, Kp, Vp))
         flush.zero_()
-        ev = [_timed(lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False)),
+        den_ms = None
+        if args.denoise_steps > 0:
+            # the order of a real rollout: every denoising step of the chunk attends to [cache + the chunk's own,
+            # still un-cached keys and values] and to the prompt; the chunk enters the cache once, afterwards
+            den = [(_timed(lambda: cache.annsa_segment(dq, dk, dv, cfg.block, cfg.keep_blocks)),
+                    _timed(lambda: cache.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt))) for _ in range(args.denoise_steps)]
+        ev = [_timed(lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq if args.probe else None)),
               _timed(lambda: cache.annsa(dq, cfg.block, cfg.keep_blocks)),
               _timed(lambda: cache.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt))]
+        if args.denoise_steps > 0:
+            torch.cuda.synchronize()
+            den_ms = [(a[0].elapsed_time(a[1]), b[0].elapsed_time(b[1])) for a, b in den]
         dense_ms = dense_upd = None
         if dense is not None:
             e0 = _timed(lambda: dense.update(dk, dv, cfg.frame_len, 2.0, outputs=False))
@@ -74,6 +83,8 @@ def run_rollout(args):
         assert cache.status() == 0
         rows.append(dict(chunk=ci, update_ms=ms[0], annsa_ms=ms[1], annca_ms=ms[2], step_ms=sum(ms),
                          len_min=int(lens.min()), len_max=int(lens.max()), live_kv_bytes=int(lens.sum()) * D * 2 * 2,
+                         denoise_annsa_segment_ms=None if den_ms is None else [x[0] for x in den_ms],
+                         denoise_annca_ms=None if den_ms is None else [x[1] for x in den_ms],
                          dense_keys=(ci + 1) * n, dense_attn_ms=dense_ms, dense_update_ms=dense_upd,
                          dense_kv_bytes=(ci + 1) * n * H * D * 2 * 2,
                          dense_tflops=None if dense_ms is None else 4.0 * n * (ci + 1) * n * D * H / (dense_ms * 1e-3) / 1e12))
@@ -86,6 +97,16 @@ def run_rollout(args):
         json.dump(report, f)
     print(f"{'chunk':>5} {'len':>13} {'upd ms':>7} {'sa ms':>7} {'ca ms':>7} {'step ms':>8} {'tok/s':>10} {'live MB':>8} | "
           f"{'dense keys':>10} {'dense ms':>9} {'TF/s':>6} {'dense MB':>9}")
+    if args.denoise_steps > 0:
+        print(f"denoising order, {args.denoise_steps} steps per chunk"
+              f"{', query-probe update' if args.probe else ''}: per chunk  [AnnSA over cache + own chunk, AnnCA] x steps, then update")
+        print(f"{'chunk':>5} {'len':>13} {'sa+seg ms':>10} {'ca ms':>7} {'upd ms':>7} {'chunk ms':>9} {'frames/s':>9}")
+        for r in rows:
+            if r["chunk"] < 3 or r["chunk"] % 10 == 9 or r["chunk"] >= chunks - 3:
+                sa, ca = float(np.mean(r["denoise_annsa_segment_ms"])), float(np.mean(r["denoise_annca_ms"]))
+                tot = sum(r["denoise_annsa_segment_ms"]) + sum(r["denoise_annca_ms"]) + r["update_ms"]
+                print(f"{r['chunk']:>5} {r['len_min']:>6}-{r['len_max']:<6} {sa:>10.3f} {ca:>7.3f} {r['update_ms']:>7.3f} {tot:>9.3f} "
+                      f"{cfg.frames_per_chunk / (tot * 1e-3):>9.0f}")
     for r in rows:
         if r["chunk"] < 3 or r["chunk"] % 10 == 9 or r["chunk"] >= chunks - 3:
             d_ms = "-" if r["dense_attn_ms"] is None else f"{r['dense_attn_ms']:.3f}"
