@@ -217,9 +217,12 @@ def top1_query_probe(Q_new: np.ndarray, K_new: np.ndarray, cache: HeadCache) -> 
 
 def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
                      forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None,
-                     search_bits: int = 16, probe: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+                     search_bits: int = 16, probe: Optional[np.ndarray] = None,
+                     representative: str = "last") -> Dict[str, np.ndarray]:
     """One TempCache update of one head.
 
+    representative = "last" keeps the newest matching key in a merged slot (the paper's choice), "mean" the
+    count-weighted mean key (m_j k_j + sum_{i in G_j} k_i)/(m_j + |G_j|), rounded like the mean value.
     forced = (j*, c*, matched) replaces steps 1-2 by decisions taken elsewhere
     (staged parity: near-ties have several correct answers).  search_bits = 8 runs the
     correspondence search on the 8-bit codes of the keys instead of the keys themselves.
@@ -272,8 +275,15 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
             acc = acc + V_new[i]
         vbar = acc / (cache.m[j] + g)
         cache.V[j] = round_to_bf16(vbar) if cache.store_bf16 else vbar
-        rep = min(G, key=lambda i: (-frame_of[i], -cstar[i], i))
-        cache.K[j] = K_new[rep]
+        if representative == "mean":                           # Appendix C ablation: mean key of the group
+            kacc = cache.m[j] * cache.K[j]
+            for i in G:
+                kacc = kacc + K_new[i]
+            kbar = kacc / (cache.m[j] + g)
+            cache.K[j] = round_to_bf16(kbar) if cache.store_bf16 else kbar
+        else:                                                  # the paper's choice: the most recent key
+            rep = min(G, key=lambda i: (-frame_of[i], -cstar[i], i))
+            cache.K[j] = K_new[rep]
         cache.m[j] += g
         cache.stamp[j] = now
         dest[G] = j

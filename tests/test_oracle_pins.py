@@ -576,3 +576,42 @@ def test_annca_lsh_bucket_rule():
     # a frame that keeps nothing produces zeros
     none = O.annca_lsh(Q, Kp, Vp, R, T, b, fl, sel=[np.arange(npr), np.zeros(0, np.int64), np.arange(3)])
     assert not none["out"][rows].any() and none["out"][:fl].any()
+
+
+def test_mean_key_representative():
+    rng = _rng(38)
+    d = 8
+    a = rng.standard_normal(d)
+    a /= np.linalg.norm(a)
+    def cache_with(m):
+        c = O.HeadCache(16, d, store_bf16=False)
+        c.load(np.stack([a, -a]), np.zeros((2, d)), m=np.array([m, 1]))
+        return c
+    # closed form: slot 0 holds 3 tokens with key a, two close tokens b, c merge into it
+    b, cc = a + 0.01 * rng.standard_normal(d), a + 0.01 * rng.standard_normal(d)
+    c1 = cache_with(3)
+    r = O.tempcache_update(c1, np.stack([b, cc]), np.ones((2, d)), 2, 0.5, representative="mean")
+    assert r["match"].tolist() == [0, 0] and c1.m[0] == 5
+    assert np.allclose(c1.K[0], (3 * a + b + cc) / 5, atol=1e-15)
+    assert np.allclose(c1.K[1], -a)                                   # untouched slot
+    # the paper's default keeps a member's key instead
+    c2 = cache_with(3)
+    O.tempcache_update(c2, np.stack([b, cc]), np.ones((2, d)), 2, 0.5)
+    assert any(np.array_equal(c2.K[0], x) for x in (b, cc))
+    # exact duplicates leave the key where it is
+    c3 = cache_with(2)
+    O.tempcache_update(c3, np.stack([a, a, a]), np.ones((3, d)), 3, 0.5, representative="mean")
+    assert np.allclose(c3.K[0], a, atol=1e-15) and c3.m[0] == 5
+    # one token per update or all at once: the count-weighted mean does not depend on the grouping
+    toks = a + 0.01 * rng.standard_normal((4, d))
+    ca, cb = cache_with(1), cache_with(1)
+    O.tempcache_update(ca, toks, np.ones((4, d)), 4, 0.5, representative="mean")
+    for t in toks:
+        O.tempcache_update(cb, t[None], np.ones((1, d)), 1, 0.5, representative="mean")
+    assert np.allclose(ca.K[0], cb.K[0], atol=1e-14) and ca.m[0] == cb.m[0] == 5
+    # stored in the cache dtype: one rounding of the mean
+    cd = O.HeadCache(16, d)
+    cd.load(O.round_to_bf16(np.stack([a])), np.zeros((1, d)), m=np.array([3]))
+    bb = O.round_to_bf16(b)
+    O.tempcache_update(cd, bb[None], np.ones((1, d)), 1, 0.5, representative="mean")
+    assert np.array_equal(cd.K[0], O.round_to_bf16((3 * O.round_to_bf16(a) + bb) / 4))
