@@ -78,7 +78,16 @@ typedef struct {
                               * then ranks prompt tokens by max_i code(q_i).code(k_p) |q_i| |k_p| / (256 sqrt d)
                               * (codes of its queries and prompt keys are made per call); the attention over
                               * the kept tokens uses the bf16 tensors. */
+  int32_t representative;    /* key a merged slot keeps (Appendix C, "Representative selection"):
+                              * FASTAR_REP_LAST_KEY (0, the paper's choice) = the key of its newest matching
+                              * token; FASTAR_REP_MEAN_KEY (1, the ablation's alternative) = the count-weighted
+                              * mean (m_j K_j + sum k_i)/(m_j + g), summed in fp32 in ascending token order and
+                              * rounded to bf16 once, like the value; 1/|k|, the LSH code and the search code of
+                              * the slot are then those of the rounded mean. */
 } fastar_cache_desc;
+
+#define FASTAR_REP_LAST_KEY 0
+#define FASTAR_REP_MEAN_KEY 1
 
 typedef struct {
   int32_t matched;           /* new tokens merged into an existing slot */

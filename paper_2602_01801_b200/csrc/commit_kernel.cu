@@ -8,6 +8,12 @@
 // so what it needs is many items in flight and no lookup that waits for one it does not depend on: the group
 // tables are read before the plan record is known, and a group of one member (the usual case) fetches its
 // value row, key row and metadata together.
+//
+// MEANK (the mean-key representative of the paper's Appendix C ablation): the slot keeps the count-weighted mean of
+// the keys, formed exactly like the mean value; its derived data (1/|k|, LSH code, 8-bit search code) are then
+// recomputed from the rounded mean inside this kernel instead of being copied from the representative token.
+#include <cuda_fp8.h>
+
 #include "common.h"
 #include "ptx.cuh"
 
@@ -46,7 +52,7 @@ __device__ __forceinline__ void store_code_part(const CacheView& c, int page, in
   else *reinterpret_cast<uint4*>(dst + sl * 16) = v;
 }
 
-template <int D>
+template <int D, bool MEANK>
 __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __nv_bfloat16* __restrict__ k_new,
                                                      const __nv_bfloat16* __restrict__ v_new, int n, int frame_len, int64_t hs,
                                                      int64_t ts) {
@@ -85,6 +91,12 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] *= static_cast<float>(m_old);
     }
+    float kacc[8];
+    if (MEANK) {
+      unpack8(*reinterpret_cast<const uint4*>(c.pool_k + ro), kacc);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) kacc[e] *= static_cast<float>(m_old);
+    }
     int best_i;
     if (g == 1) {
       best_i = __shfl_sync(mask, mine, sub * LPR);
@@ -92,6 +104,11 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
       unpack8(*reinterpret_cast<const uint4*>(vh + best_i * ts + sl * 8), f);
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      if (MEANK) {
+        unpack8(*reinterpret_cast<const uint4*>(kh + best_i * ts + sl * 8), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) kacc[e] += f[e];
+      }
     } else {
       // Members in ascending token order (the scatter left them unordered): each round takes the smallest token
       // index above the previous one.  Lanes hold the first LPR members, larger groups re-read the list.
@@ -112,21 +129,70 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
         unpack8(*reinterpret_cast<const uint4*>(vh + i * ts + sl * 8), f);
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] += f[e];
+        if (MEANK) {
+          unpack8(*reinterpret_cast<const uint4*>(kh + i * ts + sl * 8), f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) kacc[e] += f[e];
+        }
         const int fr = i / frame_len;
         const float s = c.sim[tb + i];
         if (fr > best_f || (fr == best_f && s > best_s)) { best_f = fr; best_s = s; best_i = i; }
       }
     }
-    const uint4 krow = *reinterpret_cast<const uint4*>(kh + best_i * ts + sl * 8);
+    const float inv = 1.f / static_cast<float>(m_old + g);
+    uint4 krow;
     uint4 code8 = make_uint4(0u, 0u, 0u, 0u);
-    if (c.pool_k8) code8 = load_code_part<LPR>(c, h, best_i, sl);
     float rn = 0.f;
     uint32_t code = 0;
-    if (sl == 0) {
-      rn = c.rnorm_new[tb + best_i];
-      code = c.code_new[tb + best_i];
+    if (!MEANK) {
+      krow = *reinterpret_cast<const uint4*>(kh + best_i * ts + sl * 8);
+      if (c.pool_k8) code8 = load_code_part<LPR>(c, h, best_i, sl);
+      if (sl == 0) {
+        rn = c.rnorm_new[tb + best_i];
+        code = c.code_new[tb + best_i];
+      }
+    } else {
+      krow.x = pack_bf16x2(kacc[0] * inv, kacc[1] * inv);
+      krow.y = pack_bf16x2(kacc[2] * inv, kacc[3] * inv);
+      krow.z = pack_bf16x2(kacc[4] * inv, kacc[5] * inv);
+      krow.w = pack_bf16x2(kacc[6] * inv, kacc[7] * inv);
+      float f[8];
+      unpack8(krow, f);                      // everything below is derived from the stored (rounded) key
+      float ss = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+#pragma unroll
+      for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(mask, ss, o);
+      rn = ss > 0.f ? 1.f / sqrtf(ss) : 0.f;
+      // sign-random-projection code: bit u of table t = [<k, R[t*B + u]> > 0]
+      for (int col = 0; col < c.T * c.B; ++col) {
+        float r8[8];
+        unpack8(*reinterpret_cast<const uint4*>(c.lsh + col * D + sl * 8), r8);
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot = fmaf(f[e], r8[e], dot);
+#pragma unroll
+        for (int o = LPR / 2; o >= 1; o >>= 1) dot += __shfl_xor_sync(mask, dot, o);
+        if (dot > 0.f) code |= 1u << (8 * (col / c.B) + (col % c.B));
+      }
+      if (c.pool_k8) {
+        const float sc = rn * 16.f;
+        uint32_t w8[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          w8[e] = __nv_cvt_float2_to_fp8x2(make_float2(f[2 * e] * sc, f[2 * e + 1] * sc), __NV_SATFINITE, __NV_E4M3);
+        const uint32_t lo = w8[0] | (w8[1] << 16), hi = w8[2] | (w8[3] << 16);   // code bytes of elements 8 sl .. 8 sl + 7
+        if (LPR == 16) {
+          code8.x = lo;
+          code8.y = hi;
+        } else {                             // 16 bytes per lane: the bytes of lanes 2 sl and 2 sl + 1; zero padding past d
+          const int src = sub * LPR + ((2 * sl) % LPR);
+          const uint32_t a0 = __shfl_sync(mask, lo, src), a1 = __shfl_sync(mask, hi, src);
+          const uint32_t b0 = __shfl_sync(mask, lo, src + 1), b1 = __shfl_sync(mask, hi, src + 1);
+          if (2 * sl < LPR) code8 = make_uint4(a0, a1, b0, b1);
+        }
+      }
     }
-    const float inv = 1.f / static_cast<float>(m_old + g);
     uint4 vout;
     vout.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
     vout.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
@@ -175,8 +241,10 @@ int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfl
   if (n <= 0) return 0;
   const int items_per_cta = 8 * (32 / (c.D / 8));
   const dim3 grid((n + items_per_cta - 1) / items_per_cta, c.H);
-  if (c.D == 128) commit_kernel<128><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
-  else commit_kernel<64><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  if (c.D == 128 && !c.rep_mean) commit_kernel<128, false><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  else if (c.D == 128) commit_kernel<128, true><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  else if (!c.rep_mean) commit_kernel<64, false><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
+  else commit_kernel<64, true><<<grid, 256, 0, st>>>(c, k_new, v_new, n, frame_len, hs, ts);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 

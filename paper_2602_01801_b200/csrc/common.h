@@ -81,6 +81,7 @@ struct CacheView {
   // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
+  int rep_mean;                    // representative key of a merged slot: 0 = newest key, 1 = count-weighted mean key
   float* seg_bias;                 // [max_tokens + 128]  bias of the rows of an un-cached attention segment
   // AnnCA with the LSH bucket rule: codes of the queries and of the prompt keys, kept tokens per frame
   uint32_t* code_q_ca;             // [H][max_tokens]

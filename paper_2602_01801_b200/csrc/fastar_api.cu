@@ -63,6 +63,7 @@ bool desc_valid(const fastar_cache_desc* d) {
   if (d->max_prompt_tokens < 1 || d->max_prompt_tokens > 1024 || d->max_frames < 1 || d->max_frames > 64) return false;
   if (d->dtype != FASTAR_BF16 && d->dtype != FASTAR_FP32) return false;
   if (d->search_bits != 0 && d->search_bits != 16 && d->search_bits != 8) return false;
+  if (d->representative != FASTAR_REP_LAST_KEY && d->representative != FASTAR_REP_MEAN_KEY) return false;
   return true;
 }
 
@@ -120,6 +121,7 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   for (int i = 3; i < 5; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MP * D * 2));
   t.stage[5] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
   t.search_bits = d.search_bits == 8 ? 8 : 16;
+  t.rep_mean = d.representative == FASTAR_REP_MEAN_KEY ? 1 : 0;
   t.pool_k8 = t.search_bits == 8 ? take(H * CAP * 128) : nullptr;
   t.k8_new = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
   t.q8_ca = t.search_bits == 8 ? take(H * MT * 128) : nullptr;

@@ -26,7 +26,7 @@ class FastarError(RuntimeError):
 class CacheDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("num_heads", "head_dim", "capacity", "page_tokens", "n_sink", "lsh_tables",
                                          "lsh_bits", "max_tokens", "max_prompt_tokens", "max_frames", "dtype", "device",
-                                         "search_bits")]
+                                         "search_bits", "representative")]
 
 
 class UpdateStats(C.Structure):
@@ -106,7 +106,8 @@ class Cache:
 
     def __init__(self, num_heads: int, head_dim: int, capacity: int, page_tokens: int, lsh_proj: np.ndarray,
                  lsh_tables: int = 4, lsh_bits: int = 8, max_tokens: int = 4096, max_prompt_tokens: int = 512,
-                 max_frames: int = 8, n_sink: int = 0, fp32: bool = False, device: int = 0, search_bits: int = 16):
+                 max_frames: int = 8, n_sink: int = 0, fp32: bool = False, device: int = 0, search_bits: int = 16,
+                 representative: str = "last"):
         import torch
         self.lib = load_library()
         self.torch = torch
@@ -115,8 +116,10 @@ class Cache:
         self.fp32 = fp32
         self.dtype = torch.float32 if fp32 else torch.bfloat16
         self.desc = CacheDesc(num_heads, head_dim, capacity, page_tokens, n_sink, lsh_tables, lsh_bits, max_tokens,
-                              max_prompt_tokens, max_frames, FP32 if fp32 else BF16, device, search_bits)
+                              max_prompt_tokens, max_frames, FP32 if fp32 else BF16, device, search_bits,
+                              {"last": 0, "mean": 1}[representative])
         self.search_bits = search_bits
+        self.representative = representative
         self.max_tokens = max_tokens
         nbytes = self.lib.fastar_cache_workspace_bytes(C.byref(self.desc))
         if nbytes == 0:

@@ -46,7 +46,7 @@ def oracle_heads_from_export(state: Dict[str, np.ndarray], n_sink: int = 0) -> L
 def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float, match: np.ndarray,
                  sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
                  rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None,
-                 probe: Optional[np.ndarray] = None) -> O.HeadCache:
+                 probe: Optional[np.ndarray] = None, representative: str = "last") -> O.HeadCache:
     """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
     exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases).
     `codes` = (codes of the new keys [n][128], codes of the pre-call cache [>= L][128]) as the GPU computed them
@@ -104,14 +104,23 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
         assert not matched.any() and np.all(sim == 0)
     # T3/T4: teacher-forced merge
     ref = pre.copy()
-    res = O.tempcache_update(ref, K64, V64, frame_len, tau, forced=(np.where(matched, match, 0), sim.astype(np.float64), matched))
+    res = O.tempcache_update(ref, K64, V64, frame_len, tau, forced=(np.where(matched, match, 0), sim.astype(np.float64), matched),
+                             representative=representative)
     st = res["stats"]
     assert np.array_equal(dest, res["dest"]), "T3/T4: destination slots"
     assert int(post["len"][h]) == ref.L == st["length"], "T4: length"
     L = ref.L
     assert np.array_equal(post["count"][h, :L], ref.m[:L]), "T3: multiplicities"
     assert np.array_equal(post["stamp"][h, :L], ref.stamp[:L]), "T3/T4: stamps"
-    assert np.array_equal(bits_to_f64(post["k"][h, :L]), ref.K[:L]), "T3/T4: keys are bit copies"
+    k_got = bits_to_f64(post["k"][h, :L])
+    if representative == "last":
+        assert np.array_equal(k_got, ref.K[:L]), "T3/T4: keys are bit copies"
+    else:     # mean keys are fp32 sums rounded once: within one bf16 ulp of the oracle's fp64 mean, bit copies elsewhere
+        kulp = np.maximum(np.abs(ref.K[:L]), 2.0 ** -126) * 2.0 ** -7
+        assert np.all(np.abs(k_got - ref.K[:L]) <= kulp + 1e-6), "T3: mean keys beyond one bf16 ulp"
+        untouched = np.ones(L, bool)
+        untouched[np.unique(match[matched])] = False
+        assert np.array_equal(k_got[untouched], ref.K[:L][untouched]), "T4: keys of untouched / new slots are bit copies"
     v_got = bits_to_f64(post["v"][h, :L])
     ulp = np.maximum(np.abs(ref.V[:L]), 2.0 ** -126) * 2.0 ** -7
     assert np.all(np.abs(v_got - ref.V[:L]) <= ulp + 1e-6), "T3: merged values beyond one bf16 ulp"

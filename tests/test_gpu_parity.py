@@ -16,11 +16,12 @@ def _gpu():
     return torch, fastar
 
 
-def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16):
+def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16, representative="last"):
     torch, fastar = _gpu()
     return fastar.Cache(cfg.num_heads, cfg.head_dim, capacity or cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables,
                         cfg.lsh_bits, max_tokens=max_tokens or cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64),
-                        max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32, search_bits=search_bits)
+                        max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32, search_bits=search_bits,
+                        representative=representative)
 
 
 def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=None):
@@ -45,7 +46,7 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
             P.check_search_codes(P.bits_to_f64(post["k"][h, :Lh]), post_codes["cache"][h, :Lh], f"cache codes, head {h}")
             codes = (post_codes["new"][h], pre_codes[h])
         ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes,
-                             probe=None if probe is None else probe[h])
+                             probe=None if probe is None else probe[h], representative=cache.representative)
         # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
         # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
         synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
@@ -484,3 +485,23 @@ def test_frame_sequential_updates_and_per_call_dense_switch():
     capb = cache.CAP // cache.PT
     for keep in (capb, cfg.keep_blocks, capb, cfg.keep_blocks):
         gpu_annsa_checked(cache, cfg, w, Q, post, keep)
+
+
+@pytest.mark.parametrize("d,pt,bits", [(128, 128, 16), (64, 64, 16), (128, 64, 8), (64, 128, 8)])
+def test_mean_key_representative(d, pt, bits):
+    # The ablation's representative: a merged slot keeps the count-weighted mean key.  Its 1/|k|, LSH code and 8-bit
+    # search code are recomputed inside the commit: the next update searches against them (similarity values and
+    # codes are checked there), and AnnSA hashes and attends with them.
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, search_bits=bits, representative="mean")
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0)
+    post = None
+    for ci in range(cfg.prior_chunks, cfg.prior_chunks + 3):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
+    assert post["count"].max() > 2
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
