@@ -356,6 +356,21 @@ def topk_lowest_index(scores: np.ndarray, keep: int) -> np.ndarray:
     return out
 
 
+def select_blocks(scores: np.ndarray, keep: int, force_sink: int = 0, force_recent: int = 0) -> np.ndarray:
+    """AnnSA's block selection with forced blocks (a selector option; the paper's rule has none): the first
+    `force_sink` and the last `force_recent` live key blocks of every row are kept before any other block, the
+    rest of the budget goes to the highest collision scores as in topk_lowest_index.  If the forced blocks alone
+    exceed the budget, those with the highest score (ties -> lower block) are kept.  scores: [rows][live blocks]."""
+    scores = np.asarray(scores, dtype=np.int64)
+    ncol = scores.shape[1]
+    forced = np.zeros(ncol, dtype=bool)
+    forced[: min(force_sink, ncol)] = True
+    if force_recent > 0:
+        forced[max(0, ncol - force_recent):] = True
+    big = int(scores.max(initial=0)) + 1
+    return topk_lowest_index(scores + big * forced[None, :].astype(np.int64), keep)
+
+
 def sparse_attention(Q: np.ndarray, cache: HeadCache, sel: np.ndarray, block_q: int, block_k: int,
                      return_probs: bool = False):
     """o_i = sum_j softmax_j(<q_i, k_j>/sqrt(d) + ln m_j) V_j over the live slots j of the key

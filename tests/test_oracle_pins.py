@@ -615,3 +615,25 @@ def test_mean_key_representative():
     bb = O.round_to_bf16(b)
     O.tempcache_update(cd, bb[None], np.ones((1, d)), 1, 0.5, representative="mean")
     assert np.array_equal(cd.K[0], O.round_to_bf16((3 * O.round_to_bf16(a) + bb) / 4))
+
+
+def test_forced_blocks_in_selection():
+    rng = _rng(39)
+    S = rng.integers(0, 50, size=(5, 12))
+    # nothing forced: the plain rule
+    assert np.array_equal(O.select_blocks(S, 4), O.topk_lowest_index(S, 4))
+    got = O.select_blocks(S, 6, force_sink=1, force_recent=2)
+    for r in range(5):
+        row = got[r].tolist()
+        assert row == sorted(row) and len(row) == 6 and {0, 10, 11} <= set(row)
+        rest = [c for c in row if c not in (0, 10, 11)]
+        # brute force: the other three are the best of the unforced blocks, ties to the lower block
+        cand = sorted((c for c in range(12) if c not in (0, 10, 11)), key=lambda c: (-S[r, c], c))[:3]
+        assert sorted(rest) == sorted(cand)
+    # more forced blocks than budget: the forced ones compete by score
+    tight = O.select_blocks(S, 2, force_sink=2, force_recent=2)
+    for r in range(5):
+        cand = sorted((0, 1, 10, 11), key=lambda c: (-S[r, c], c))[:2]
+        assert tight[r].tolist() == sorted(cand)
+    # budget beyond the row: everything
+    assert np.array_equal(O.select_blocks(S, 99, 1, 1), np.tile(np.arange(12), (5, 1)))
