@@ -197,6 +197,14 @@ int fastar_annsa_attention(fastar_cache_t* cache, const void* q, void* out, int3
                            int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out, float* scores_out,
                            const int32_t* sel_in, const int32_t* nsel_in, void* stream);
 
+/* AnnSA selector option (host-side setting, takes effect from the next AnnSA call; default 0, 0 = the
+ * plain rule): the first `sink_blocks` and the last `recent_blocks` live key blocks of every head are
+ * kept by every query block before any other block; the rest of keep_blocks goes to the highest
+ * collision scores.  If the forced blocks alone exceed keep_blocks, those with the highest score (ties:
+ * lower block) are kept.  The paper's rule has no forced blocks; attention sinks and the newest
+ * frames are what streaming caches usually pin. */
+int fastar_cache_set_forced_blocks(fastar_cache_t* cache, int32_t sink_blocks, int32_t recent_blocks);
+
 /* AnnSA over the cache and an un-cached segment (Eq. 1, Section 3: the attended set is the keys and
  * values of the frames being generated concatenated with those of the earlier frames; the former
  * enter the cache only when fastar_tempcache_update is called, so attention can run on every

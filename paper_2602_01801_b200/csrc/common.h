@@ -157,7 +157,7 @@ int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfl
                   int64_t hs, int64_t ts, cudaStream_t st);
 int launch_finalize_hist(const CacheView& c, fastar_update_stats* stats_out, int advance_clock, cudaStream_t st);
 int launch_query_hist(const CacheView& c, int nq, int block_q, cudaStream_t st);
-int launch_topk_blocks(const CacheView& c, int nqb, int keep, cudaStream_t st);
+int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, int force_recent, cudaStream_t st);
 int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st);
 int launch_reset(const CacheView& c, cudaStream_t st);
 int launch_import_derive(const CacheView& c, cudaStream_t st);

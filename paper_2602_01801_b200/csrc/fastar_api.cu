@@ -26,6 +26,7 @@ struct fastar_cache {
   int64_t launches;
   size_t bytes;
   // second stream of the host-tensor step (uploads of q and the prompt, AnnCA, its download) and its fork/join events
+  int force_sink_blocks = 0, force_recent_blocks = 0;    // AnnSA selector option (fastar_cache_set_forced_blocks)
   cudaStream_t side = nullptr, copy = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_q = nullptr, ev_join = nullptr, ev_p = nullptr, ev_v = nullptr;
   ~fastar_cache() {
@@ -332,6 +333,13 @@ int fastar_cache_export(fastar_cache_t* c, uint16_t* host_k, uint16_t* host_v, i
   return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
 }
 
+int fastar_cache_set_forced_blocks(fastar_cache_t* c, int32_t sink_blocks, int32_t recent_blocks) {
+  if (!c || sink_blocks < 0 || recent_blocks < 0) return FASTAR_ERR_INVALID_ARG;
+  c->force_sink_blocks = sink_blocks;
+  c->force_recent_blocks = recent_blocks;
+  return FASTAR_OK;
+}
+
 int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_codes, uint8_t* host_new_codes, int32_t n,
                                      void* stream) {
   if (!c) return FASTAR_ERR_INVALID_ARG;
@@ -512,7 +520,7 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     ACCK(FASTAR_K_HASH, launch_prep_codes(v, qb, nq, qhs, qts, v.code_new, nullptr, st));
     ACCK(FASTAR_K_QUERY_HIST, launch_query_hist(v, nq, block_q, st));
     ACCK(FASTAR_K_S3_SCORES, launch_s3_scores(v, c->tm_hq, c->tm_hk, nqb, st));
-    ACCK(FASTAR_K_TOPK_BLOCKS, launch_topk_blocks(v, nqb, keep, st));
+    ACCK(FASTAR_K_TOPK_BLOCKS, launch_topk_blocks(v, nqb, keep, c->force_sink_blocks, c->force_recent_blocks, st));
     a.sel = v.sel;
     a.nsel = v.nsel;
     a.sel_stride = v.CAPB;

@@ -602,15 +602,20 @@ template <bool ORDERED_UINT>
 __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src, int64_t src_head_stride, int src_row_stride,
                                                    const int32_t* __restrict__ len, int len_div, int n_fixed, int keep,
                                                    int32_t* __restrict__ out, int64_t out_head_stride, int out_row_stride,
-                                                   int out_fill, int32_t* __restrict__ nsel) {
+                                                   int out_fill, int32_t* __restrict__ nsel, int force_first, int force_last) {
   extern __shared__ float vals[];
   __shared__ int red[32];
   const int row = blockIdx.x, h = blockIdx.y;
   const int n = len ? (len[h] + len_div - 1) / len_div : n_fixed;
   const int k = min(keep, n);
   const int64_t so = static_cast<int64_t>(h) * src_head_stride + static_cast<int64_t>(row) * src_row_stride;
-  for (int i = threadIdx.x; i < n; i += blockDim.x)
-    vals[i] = ORDERED_UINT ? ordered_to_float(static_cast<const uint32_t*>(src)[so + i]) : static_cast<const float*>(src)[so + i];
+  // Forced entries (the first force_first and the last force_last of the row) rank before all others: their scores
+  // are integer counts below 2^23, so adding 2^23 is exact in fp32 and keeps their order among themselves.
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    float v = ORDERED_UINT ? ordered_to_float(static_cast<const uint32_t*>(src)[so + i]) : static_cast<const float*>(src)[so + i];
+    if (!ORDERED_UINT && (i < force_first || i >= n - force_last)) v += 8388608.f;
+    vals[i] = v;
+  }
   __syncthreads();
   int32_t* orow = out + static_cast<int64_t>(h) * out_head_stride + static_cast<int64_t>(row) * out_row_stride;
   int run = 0;
@@ -634,10 +639,10 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
   for (int i = k + threadIdx.x; i < out_fill; i += blockDim.x) orow[i] = -1;
   if (nsel && row == 0 && threadIdx.x == 0) nsel[h] = k;
 }
-int launch_topk_blocks(const CacheView& c, int nqb, int keep, cudaStream_t st) {
+int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, int force_recent, cudaStream_t st) {
   topk_kernel<false><<<dim3(nqb, c.H), 256, c.CAPB * 4, st>>>(c.scores, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB, c.len,
                                                             c.PT, 0, keep, c.sel, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB,
-                                                            min(keep, c.CAPB), c.nsel);
+                                                            min(keep, c.CAPB), c.nsel, force_sink, force_recent);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 // ---------------------------------------------------------------------------------------------
@@ -692,7 +697,7 @@ int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaS
   topk_kernel<true><<<dim3(n_frames, c.H), 256, np * 4, st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
                                                              c.max_prompt, nullptr, 1, np, keep, c.selp,
                                                              static_cast<int64_t>(c.max_frames) * c.max_prompt, c.max_prompt,
-                                                             min(keep, np), nullptr);
+                                                             min(keep, np), nullptr, 0, 0);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 

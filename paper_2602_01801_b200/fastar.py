@@ -42,6 +42,7 @@ SIGNATURES = {
     "fastar_cache_reset": (C.c_int, [_vp, _vp]),
     "fastar_cache_destroy": (C.c_int, [_vp]),
     "fastar_cache_export": (C.c_int, [_vp] * 9),
+    "fastar_cache_set_forced_blocks": (C.c_int, [_vp, _i32, _i32]),
     "fastar_cache_export_search_codes": (C.c_int, [_vp, _vp, _vp, _i32, _vp]),
     "fastar_cache_export_annca_codes": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _vp]),
     "fastar_cache_import": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp]),
@@ -174,6 +175,10 @@ class Cache:
                                             out["stamp"].ctypes.data, out["code"].ctypes.data, out["len"].ctypes.data,
                                             out["now"].ctypes.data, _stream()), "fastar_cache_export")
         return out
+
+    def set_forced_blocks(self, sink_blocks: int = 0, recent_blocks: int = 0) -> None:
+        """AnnSA selector option: always keep the first / the last live key blocks of every head (within the budget)."""
+        _check(self.lib.fastar_cache_set_forced_blocks(self.handle, sink_blocks, recent_blocks), "fastar_cache_set_forced_blocks")
 
     def export_search_codes(self, n_new: int = 0) -> Dict[str, np.ndarray]:
         """8-bit search only: the code rows of every slot [H][CAP][128] and of the last update's n_new keys."""

@@ -505,3 +505,33 @@ def test_mean_key_representative(d, pt, bits):
         post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
     assert post["count"].max() > 2
     gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+
+
+@pytest.mark.parametrize("sink,recent,keep", [(1, 2, 6), (2, 3, 3), (0, 1, 4)])
+def test_forced_sink_and_recent_blocks(sink, recent, keep):
+    # AnnSA selector option: the first / last live key blocks of every head are kept before the collision ranking
+    # (ragged head lengths, so "last" differs per head); with more forced blocks than budget they compete by score.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(block=64, capacity=2048, num_heads=3)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks + 1):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0 if ci < cfg.prior_chunks else cfg.tau)
+    cache.set_forced_blocks(sink, recent)
+    res = cache.annsa(fastar.to_device(Q), cfg.block, keep, debug=True)
+    assert cache.status() == 0
+    out = res["out"].float().cpu().numpy()
+    for h, hc in enumerate(heads):
+        nkb = -(-hc.L // cfg.block)
+        S = res["scores"][h].cpu().numpy()[:, :nkb].astype(np.int64)
+        want = O.select_blocks(S, keep, sink, recent)
+        nsel = int(res["nsel"][h])
+        assert nsel == want.shape[1] and np.array_equal(res["sel"][h].cpu().numpy()[:, :nsel], want)
+        if keep >= sink + recent:
+            forced = set(range(sink)) | set(range(nkb - recent, nkb))
+            assert all(forced <= set(row.tolist()) for row in want)
+        P.check_attention(out[h], O.sparse_attention(Q[h].astype(np.float64), hc, want, cfg.block, cfg.block), f"forced blocks, head {h}")
+    cache.set_forced_blocks(0, 0)
+    gpu_annsa_checked(cache, cfg, w, Q, post, keep)          # back to the plain rule
