@@ -197,19 +197,31 @@ def top1_quantized(K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.
     return j.astype(np.int64), s[np.arange(n), j]
 
 
-def top1_query_probe(Q_new: np.ndarray, K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.ndarray]:
+def probe_scores_quantized(codes_q: np.ndarray, codes_k: np.ndarray, K_cache: np.ndarray) -> np.ndarray:
+    """8-bit form of the probe's ranking score <q_i, k_j>: the codes carry directions only, so the dot product of
+    the codes (an estimate of cos(q_i, k_j)) is scaled back by |k_j|; |q_i| is the same for every j and is left out."""
+    kn = np.sqrt(np.sum(np.asarray(K_cache, np.float64) ** 2, axis=1))
+    return quantized_score_matrix(codes_q, codes_k) * kn[None, :]
+
+
+def top1_query_probe(Q_new: np.ndarray, K_new: np.ndarray, cache: HeadCache, search_bits: int = 16) -> Tuple[np.ndarray, np.ndarray]:
     """Correspondence read off the attention scores (Section 5.2, "Finding temporal correspondences"):
     the token corresponding to query q_i is the live cached key with the highest score <q_i, k_j>
     (softmax and the 1/sqrt(d) scale are monotone, so this is the highest attention weight; ties ->
     smallest slot).  Returns (j*, cos(k_i, k_j*)): the similarity the merge threshold is applied to is
-    that of the keys (Appendix C, "key-similarity threshold").  j* = -1, c* = 0 on an empty cache."""
+    that of the keys (Appendix C, "key-similarity threshold").  j* = -1, c* = 0 on an empty cache.
+    search_bits = 8 ranks with probe_scores_quantized instead of the exact dot products; the cosine of the
+    winner is always exact."""
     Q_new = np.asarray(Q_new, np.float64)
     K_new = np.asarray(K_new, np.float64)
     n = K_new.shape[0]
     if cache.L == 0:
         return np.full(n, -1, np.int64), np.zeros(n, np.float64)
     Kc = cache.K[: cache.L]
-    j = np.argmax(Q_new @ Kc.T, axis=1).astype(np.int64)
+    if search_bits == 8:
+        j = np.argmax(probe_scores_quantized(key_codes_e4m3(Q_new), key_codes_e4m3(Kc), Kc), axis=1).astype(np.int64)
+    else:
+        j = np.argmax(Q_new @ Kc.T, axis=1).astype(np.int64)
     num = np.sum(K_new * Kc[j], axis=1)
     den = np.sqrt(np.sum(K_new * K_new, axis=1)) * np.sqrt(np.sum(Kc[j] * Kc[j], axis=1))
     return j, np.where(den > 0, num / np.where(den > 0, den, 1.0), 0.0)
@@ -235,7 +247,7 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
     # 1. top-1 correspondence against the pre-call cache; 2. threshold
     if forced is None:
         if probe is not None:
-            jstar, cstar = top1_query_probe(probe, K_new, cache)
+            jstar, cstar = top1_query_probe(probe, K_new, cache, search_bits)
         else:
             jstar, cstar = top1_quantized(K_new, cache) if search_bits == 8 else top1_cosine(K_new, cache)
         matched = (cstar >= tau) & (jstar >= 0)

@@ -637,3 +637,34 @@ def test_forced_blocks_in_selection():
         assert tight[r].tolist() == sorted(cand)
     # budget beyond the row: everything
     assert np.array_equal(O.select_blocks(S, 99, 1, 1), np.tile(np.arange(12), (5, 1)))
+
+
+def test_query_probe_on_eight_bit_codes():
+    rng = _rng(40)
+    d, L, n = 32, 30, 20
+    cache = O.HeadCache(64, d)
+    Kc = rng.standard_normal((L, d)) * rng.uniform(0.5, 2.0, (L, 1))
+    cache.load(Kc, rng.standard_normal((L, d)))
+    K = rng.standard_normal((n, d))
+    Q = rng.standard_normal((n, d))
+    j8, c8 = O.top1_query_probe(Q, K, cache, search_bits=8)
+    # brute force: decoded codes, Python loops
+    cq, ck = O.e4m3_decode(O.key_codes_e4m3(Q)), O.e4m3_decode(O.key_codes_e4m3(Kc))
+    for i in range(n):
+        sc = [sum(float(cq[i, k]) * float(ck[s, k]) for k in range(d)) / 256.0 * float(np.linalg.norm(Kc[s])) for s in range(L)]
+        jb = max(range(L), key=lambda s: (sc[s], -s))
+        assert j8[i] == jb
+        assert abs(c8[i] - float(K[i] @ Kc[jb]) / (np.linalg.norm(K[i]) * np.linalg.norm(Kc[jb]))) < 1e-12
+    # the quantised ranking score approximates <q, k> / |q| within the code error
+    exact = (Q @ Kc.T) / np.linalg.norm(Q, axis=1, keepdims=True)
+    approx = O.probe_scores_quantized(O.key_codes_e4m3(Q), O.key_codes_e4m3(Kc), Kc)
+    assert np.max(np.abs(approx - exact)) <= 0.04 * np.linalg.norm(Kc, axis=1).max()
+    # and mostly agrees with the exact probe
+    j16, _ = O.top1_query_probe(Q, K, cache)
+    assert np.mean(j8 == j16) >= 0.7
+    # scaling a cached key up makes it win where it was close: the norm is part of the score
+    cache2 = O.HeadCache(64, d)
+    Kc2 = Kc.copy()
+    Kc2[4] = 50.0 * Q[3] / np.linalg.norm(Q[3])
+    cache2.load(Kc2, np.zeros((L, d)))
+    assert O.top1_query_probe(Q, K, cache2, search_bits=8)[0][3] == 4
