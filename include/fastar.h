@@ -133,6 +133,11 @@ int fastar_cache_export(fastar_cache_t* cache, uint16_t* host_k, uint16_t* host_
 int fastar_cache_export_search_codes(fastar_cache_t* cache, uint8_t* host_cache_codes, uint8_t* host_new_codes,
                                      int32_t n, void* stream);
 
+/* 8-bit search only (else FASTAR_ERR_UNSUPPORTED_SHAPE): copy the codes of the probe rows of the most
+ * recent fastar_tempcache_update_probe call, host_probe_codes [H][n][128], to the host and synchronise
+ * the stream.  (Sections 5.1, 5.2.) */
+int fastar_cache_export_probe_codes(fastar_cache_t* cache, uint8_t* host_probe_codes, int32_t n, void* stream);
+
 /* 8-bit search only (else FASTAR_ERR_UNSUPPORTED_SHAPE): copy the search codes the most recent
  * fastar_annca_attention call (one that selected, sel_in == NULL) computed for its nq queries,
  * host_q_codes [H][nq][128], and its np prompt keys, host_prompt_codes [H][np][128], to the host and
@@ -173,8 +178,9 @@ int fastar_tempcache_update(fastar_cache_t* cache, const void* k_new, const void
  * and the merge decision is taken on the key similarity of that slot: matched iff
  * cos(k_i, K_{j*_i}) >= tau.  sim_out receives that cosine (0 on an empty cache); the
  * representative rule uses it.  q_probe: dev [H][n][d], same strides and dtype as k_new.
- * search_bits == 8 caches return FASTAR_ERR_UNSUPPORTED_SHAPE (the probe ranks un-normalised
- * dot products, which the direction-only 8-bit codes do not carry). */
+ * With search_bits == 8 the ranking uses the 8-bit codes: the codes carry directions only, so the
+ * score of slot j is code(q_i).code(K_j) |K_j| / 256 (|q_i| does not change the arg-max); the cosine
+ * of the winner is exact as before. */
 int fastar_tempcache_update_probe(fastar_cache_t* cache, const void* q_probe, const void* k_new, const void* v_new,
                                   int32_t n, int32_t frame_len, int64_t head_stride, int64_t token_stride, float tau,
                                   int32_t* match_out, float* sim_out, int32_t* dest_out,

@@ -78,6 +78,8 @@ struct CacheView {
   uint8_t* kp8_ca;                 // [H][max_prompt][128]  codes of the prompt keys
   float* qn_ca;                    // [H][max_tokens]  |q|
   float* kpn_ca;                   // [H][max_prompt]  |k_p|
+  uint8_t* q8_probe;               // [H][max_tokens][128]  codes of the probe rows of a query-probe update
+  float* qn_probe;                 // [H][max_tokens]  their norms (written by the quantiser, not used)
   // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
@@ -108,7 +110,8 @@ int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtenso
 // search8_kernels.cu: fp8 search codes of bf16 rows (x / |x| * 16, 128-byte rows), and T1 on the codes
 int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, const float* rnorm,
                          int64_t rn_stride, uint8_t* out, int64_t out_rows_per_head, cudaStream_t st);
-int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, cudaStream_t st);
+int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, bool col_norm,
+                             cudaStream_t st);
 int launch_quantize_rows(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint8_t* out,
                          int64_t out_rows_per_head, float* norm_out, int64_t norm_stride, cudaStream_t st);
 int launch_c1_relevance_fp8(const CacheView& c, const CUtensorMap& tm_q8, const CUtensorMap& tm_kp8, const float* qn,

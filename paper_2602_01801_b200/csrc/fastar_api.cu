@@ -129,6 +129,8 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.kp8_ca = t.search_bits == 8 ? take(H * MP * 128) : nullptr;
   t.qn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MT * 4)) : nullptr;
   t.kpn_ca = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MP * 4)) : nullptr;
+  t.q8_probe = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
+  t.qn_probe = t.search_bits == 8 ? reinterpret_cast<float*>(take(H * MT * 4)) : nullptr;
   t.seg_bias = reinterpret_cast<float*>(take((MT + 128) * 4));
   t.code_q_ca = reinterpret_cast<uint32_t*>(take(H * MT * 4));
   t.code_p_ca = reinterpret_cast<uint32_t*>(take(H * MP * 4));
@@ -358,6 +360,19 @@ int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_code
   return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
 }
 
+int fastar_cache_export_probe_codes(fastar_cache_t* c, uint8_t* host_probe_codes, int32_t n, void* stream) {
+  if (!c || !host_probe_codes) return FASTAR_ERR_INVALID_ARG;
+  const CacheView& v = c->v;
+  if (v.search_bits != 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (n < 1 || n > v.max_tokens) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool ok = cudaMemcpy2DAsync(host_probe_codes, static_cast<size_t>(n) * 128, v.q8_probe, static_cast<size_t>(v.max_tokens) * 128,
+                              static_cast<size_t>(n) * 128, v.H, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
 int fastar_cache_export_annca_codes(fastar_cache_t* c, uint8_t* host_q_codes, uint8_t* host_prompt_codes, int32_t nq, int32_t np,
                                     void* stream) {
   if (!c) return FASTAR_ERR_INVALID_ARG;
@@ -413,7 +428,6 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
                        int32_t* dest_out, fastar_update_stats* stats_out, void* stream, cudaEvent_t v_ready = nullptr) {
   if (!c || !k_new || !v_new || n < 1 || frame_len < 1) return FASTAR_ERR_INVALID_ARG;
   if (n > c->v.max_tokens || n > 16384 || n > c->v.CAP) return FASTAR_ERR_UNSUPPORTED_SHAPE;
-  if (q_probe && c->v.search_bits == 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (token_stride < c->v.D || head_stride < 0) return FASTAR_ERR_INVALID_ARG;
   DeviceGuard guard(c->desc.device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -441,10 +455,14 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
   if (v.search_bits == 8) {
     // correspondence search on the 8-bit codes: quantise the new keys, then the fp8 contraction with the arg-max fused
     CUtensorMap tm_a8;
-    r = make_map_codes(c, &tm_a8, v.k8_new, n, v.H, static_cast<uint64_t>(v.max_tokens) * 128, 128);
+    // key -> key: the rows are the codes of the new keys; query-probe: the codes of the probe rows, and the scores are
+    // scaled by |k_j| before the arg-max (the codes carry directions only)
+    r = make_map_codes(c, &tm_a8, q_probe ? v.q8_probe : v.k8_new, n, v.H, static_cast<uint64_t>(v.max_tokens) * 128, 128);
     if (r != FASTAR_OK) return r;
     ACCK(FASTAR_K_HASH, launch_quantize_keys(v, kb, n, khs, kts, v.rnorm_new, v.max_tokens, v.k8_new, v.max_tokens, st));
-    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(v, tm_a8, c->tm_pool_k8, n, st));
+    if (q_probe) ACCK(FASTAR_K_HASH, launch_quantize_rows(v, pb, n, phs, pts, v.q8_probe, v.max_tokens, v.qn_probe, v.max_tokens, st));
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(v, tm_a8, c->tm_pool_k8, n, q_probe != nullptr, st));
+    if (q_probe) ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
   } else if (q_probe) {
     CacheView vr = v;
     vr.raw_dot = 1;

@@ -75,6 +75,34 @@ __device__ __forceinline__ void chunk_argmax_raw(const uint32_t (&acc)[32], int 
   }
 }
 
+// The same on scores scaled by the norm of their column's key (query-probe ranking: the codes carry directions, the
+// attention score also depends on |k_j|).  rn = 1/|k_j| of the 32 columns, 0 for an all-zero key.
+__device__ __forceinline__ void chunk_argmax_scaled(const uint32_t (&acc)[32], const float4* __restrict__ rn, int valid, int jbase,
+                                                    float& best, int& best_j) {
+  float x[32];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const float4 r4 = __ldg(rn + q);
+    x[4 * q] = r4.x > 0.f ? __uint_as_float(acc[4 * q]) / r4.x : 0.f;
+    x[4 * q + 1] = r4.y > 0.f ? __uint_as_float(acc[4 * q + 1]) / r4.y : 0.f;
+    x[4 * q + 2] = r4.z > 0.f ? __uint_as_float(acc[4 * q + 2]) / r4.z : 0.f;
+    x[4 * q + 3] = r4.w > 0.f ? __uint_as_float(acc[4 * q + 3]) / r4.w : 0.f;
+  }
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j >= valid) x[j] = -INFINITY;
+  float cm = x[0];
+#pragma unroll
+  for (int j = 1; j < 32; ++j) cm = fmaxf(cm, x[j]);
+  if (cm > best) {
+    best = cm;
+    int idx = 31;
+#pragma unroll
+    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;
+    best_j = jbase + idx;
+  }
+}
+
 }  // namespace
 
 // Half a warp per row: |x|, then the code of x / |x| * 16 (an all-zero row gets an all-zero code and norm 0).
@@ -168,6 +196,7 @@ int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int6
 // of head h (rows of a dense [H][rows][128] array), per-frame column maximum of score * |q| * |k|.
 struct Search8Args {
   int rows_a;
+  int col_norm;            // arg-max: scores are multiplied by |k_j| before the maximum (query-probe ranking)
   int cols_b;              // COLMAX
   int frame_len;           // COLMAX
   const float* qn;         // COLMAX: |q|, [H][max_tokens]
@@ -339,7 +368,11 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
           if (!COLMAX) {
-            chunk_argmax_raw(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+            if (g.col_norm)
+              chunk_argmax_scaled(vv[c2], reinterpret_cast<const float4*>(c.rnorm + static_cast<int64_t>(h) * c.CAP + t * 128 + cc * 32),
+                                  valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+            else
+              chunk_argmax_raw(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
           } else {
             for (int f = f_lo; f <= f_hi; ++f) {       // empty when the warp has no valid row
               float x[32];
@@ -411,11 +444,13 @@ static int pick_splits8(int row_tiles, int H, int max_tiles) {
   return splits;
 }
 
-int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, cudaStream_t st) {
+int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, bool col_norm,
+                             cudaStream_t st) {
   if (configure_search8() != FASTAR_OK) return FASTAR_ERR_CUDA;
   const int row_tiles = (n + 127) / 128;
   Search8Args g{};
   g.rows_a = n;
+  g.col_norm = col_norm ? 1 : 0;
   search8_kernel<false><<<dim3(row_tiles, c.H, pick_splits8(row_tiles, c.H, c.CAP / 128)), kThreads, Smem::total, st>>>(
       tm_a8, tm_pool_k8, c, g);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;

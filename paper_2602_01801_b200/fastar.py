@@ -44,6 +44,7 @@ SIGNATURES = {
     "fastar_cache_export": (C.c_int, [_vp] * 9),
     "fastar_cache_set_forced_blocks": (C.c_int, [_vp, _i32, _i32]),
     "fastar_cache_export_search_codes": (C.c_int, [_vp, _vp, _vp, _i32, _vp]),
+    "fastar_cache_export_probe_codes": (C.c_int, [_vp, _vp, _i32, _vp]),
     "fastar_cache_export_annca_codes": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _vp]),
     "fastar_cache_import": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp]),
     "fastar_tempcache_update": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
@@ -189,6 +190,14 @@ class Cache:
             _check(self.lib.fastar_cache_export_search_codes(self.handle, out["cache"].ctypes.data,
                                                              out["new"].ctypes.data if n_new > 0 else None, n_new, _stream()),
                    "fastar_cache_export_search_codes")
+        return out
+
+    def export_probe_codes(self, n: int) -> np.ndarray:
+        """8-bit search only: the code rows of the probe rows of the last query-probe update, [H][n][128]."""
+        out = np.empty((self.H, n, 128), np.uint8)
+        with self.torch.cuda.device(self.device):
+            _check(self.lib.fastar_cache_export_probe_codes(self.handle, out.ctypes.data, n, _stream()),
+                   "fastar_cache_export_probe_codes")
         return out
 
     def export_annca_codes(self, nq: int, n_prompt: int) -> Dict[str, np.ndarray]:

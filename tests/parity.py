@@ -46,7 +46,8 @@ def oracle_heads_from_export(state: Dict[str, np.ndarray], n_sink: int = 0) -> L
 def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float, match: np.ndarray,
                  sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
                  rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None,
-                 probe: Optional[np.ndarray] = None, representative: str = "last") -> O.HeadCache:
+                 probe: Optional[np.ndarray] = None, representative: str = "last",
+                 probe_codes: Optional[np.ndarray] = None) -> O.HeadCache:
     """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
     exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases).
     `codes` = (codes of the new keys [n][128], codes of the pre-call cache [>= L][128]) as the GPU computed them
@@ -62,10 +63,16 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
     if pre.L > 0 and probe is not None:
         Kc = pre.K[: pre.L]
         Q64 = probe.astype(np.float64)[idx]
-        s = Q64 @ Kc.T
+        if codes is None:
+            s = Q64 @ Kc.T
+            # tie window on the scale of the dot products (fp32 accumulation of bf16 products)
+            win = MARGIN * np.linalg.norm(Q64, axis=1) * np.linalg.norm(Kc, axis=1).max()
+        else:     # 8-bit ranking: code dot products (of the codes the GPU used) scaled by the cached keys' norms
+            d = K_new.shape[1]
+            s = O.probe_scores_quantized(probe_codes[idx, :d], codes[1][: pre.L, :d], Kc)
+            win = np.full(idx.size, MARGIN_Q8 * np.linalg.norm(Kc, axis=1).max())
         sbest = s.max(axis=1)
-        # tie window on the scale of the dot products (fp32 accumulation of bf16 products)
-        win = MARGIN * np.linalg.norm(Q64, axis=1) * np.linalg.norm(Kc, axis=1).max()
+        margin, sim_tol = MARGIN, 2e-5            # the cosine of the winner is exact in both modes
         near = s >= (sbest - win)[:, None]
         cosm = O.cosine_matrix(K64[idx], Kc)
         # the similarity reported is the key cosine of a (near-)best slot of the probe

@@ -37,8 +37,11 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
     match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
     synced = P.oracle_heads_from_export(post, heads[0].n_sink)
     post_codes = cache.export_search_codes(K.shape[1]) if q8 else None
+    probe_codes = cache.export_probe_codes(K.shape[1]) if (q8 and probe is not None) else None
     for h in range(K.shape[0]):
         codes = None
+        if q8 and probe is not None:
+            P.check_search_codes(np.asarray(probe[h], np.float64), probe_codes[h], f"probe codes, head {h}")
         if q8:
             # the quantiser, byte by byte: codes of the new keys, and of every live slot after the update
             P.check_search_codes(np.asarray(K[h], np.float64), post_codes["new"][h], f"new-key codes, head {h}")
@@ -46,7 +49,8 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
             P.check_search_codes(P.bits_to_f64(post["k"][h, :Lh]), post_codes["cache"][h, :Lh], f"cache codes, head {h}")
             codes = (post_codes["new"][h], pre_codes[h])
         ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes,
-                             probe=None if probe is None else probe[h], representative=cache.representative)
+                             probe=None if probe is None else probe[h], representative=cache.representative,
+                             probe_codes=probe_codes[h] if (q8 and probe is not None) else None)
         # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
         # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
         synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
@@ -176,11 +180,29 @@ def test_query_probe_correspondence(d, pt, fp32, kernel, monkeypatch):
         matched += sum(K.shape[1] - (hc.L - b) for hc, b in zip(heads, before))
     assert matched > 0.5 * 2 * cfg.num_heads * K.shape[1] and post["count"].max() > 1
     gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks, fp32)
-    if not fp32:
-        torch, fastar = _gpu()
-        c8 = make_cache(cfg, w, search_bits=8)
-        with pytest.raises(fastar.FastarError):
-            c8.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau, probe=fastar.to_device(Q))
+
+
+@pytest.mark.parametrize("d,pt", [(128, 128), (64, 64)])
+def test_query_probe_on_eight_bit_codes(d, pt):
+    # The paper's default bit width with the paper's literal correspondence rule: slots ranked by the dot product of
+    # the 8-bit codes of query and cached key times the cached key's norm, threshold on the exact key cosine.
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, search_bits=8)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    Q, K, V = w.chunk(0)
+    gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, probe=Q)                     # empty cache
+    for ci in range(1, cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0)
+    matched = 0
+    for ci in (cfg.prior_chunks, cfg.prior_chunks + 1):
+        Q, K, V = w.chunk(ci)
+        before = [hc.L for hc in heads]
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, probe=Q)
+        matched += sum(K.shape[1] - (hc.L - b) for hc, b in zip(heads, before))
+    assert matched > 0.5 * 2 * cfg.num_heads * K.shape[1] and post["count"].max() > 1
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
 
 
 @pytest.mark.parametrize("d,pt", [(128, 128), (64, 64), (128, 64)])
