@@ -34,7 +34,8 @@ constexpr float kCodeScale = 16.f;
 struct Smem {
   static constexpr int ring_off = kTile;                        // A (128 new keys) first
   static constexpr int bar_off = ring_off + kStages * kTile;
-  static constexpr int total = bar_off + 256;
+  static constexpr int kn_off = bar_off + 256;                  // 2 x 128 floats: |k_j| of a tile's keys (query-probe ranking)
+  static constexpr int total = kn_off + 2 * 128 * 4;
 };
 
 // Instruction descriptor of kind::f8f6f4 with e4m3 A and B (format 0), fp32 accumulation, K-major operands.
@@ -76,24 +77,29 @@ __device__ __forceinline__ void chunk_argmax_raw(const uint32_t (&acc)[32], int 
 }
 
 // The same on scores scaled by the norm of their column's key (query-probe ranking: the codes carry directions, the
-// attention score also depends on |k_j|).  rn = 1/|k_j| of the 32 columns, 0 for an all-zero key.
-__device__ __forceinline__ void chunk_argmax_scaled(const uint32_t (&acc)[32], const float4* __restrict__ rn, int valid, int jbase,
+// attention score also depends on |k_j|).  kn = |k_j| of the 32 columns (shared memory, the same for every lane).
+__device__ __forceinline__ void chunk_argmax_scaled(const uint32_t (&acc)[32], const float4* __restrict__ kn, int valid, int jbase,
                                                     float& best, int& best_j) {
   float x[32];
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
-    const float4 r4 = __ldg(rn + q);
-    x[4 * q] = r4.x > 0.f ? __uint_as_float(acc[4 * q]) / r4.x : 0.f;
-    x[4 * q + 1] = r4.y > 0.f ? __uint_as_float(acc[4 * q + 1]) / r4.y : 0.f;
-    x[4 * q + 2] = r4.z > 0.f ? __uint_as_float(acc[4 * q + 2]) / r4.z : 0.f;
-    x[4 * q + 3] = r4.w > 0.f ? __uint_as_float(acc[4 * q + 3]) / r4.w : 0.f;
+    const float4 k4 = kn[q];
+    x[4 * q] = __uint_as_float(acc[4 * q]) * k4.x;
+    x[4 * q + 1] = __uint_as_float(acc[4 * q + 1]) * k4.y;
+    x[4 * q + 2] = __uint_as_float(acc[4 * q + 2]) * k4.z;
+    x[4 * q + 3] = __uint_as_float(acc[4 * q + 3]) * k4.w;
   }
+  if (valid < 32) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j)
-    if (j >= valid) x[j] = -INFINITY;
-  float cm = x[0];
+    for (int j = 0; j < 32; ++j)
+      if (j >= valid) x[j] = -INFINITY;
+  }
+  float m[11];
 #pragma unroll
-  for (int j = 1; j < 32; ++j) cm = fmaxf(cm, x[j]);
+  for (int j = 0; j < 10; ++j) m[j] = fmax3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
+  m[10] = fmaxf(x[30], x[31]);
+  const float a0 = fmax3(m[0], m[1], m[2]), a1 = fmax3(m[3], m[4], m[5]), a2 = fmax3(m[6], m[7], m[8]);
+  const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
   if (cm > best) {
     best = cm;
     int idx = 31;
@@ -225,6 +231,7 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const uint32_t bar_afull = bar_tempty + 16;            // [1]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sgen + Smem::bar_off + 16 * kStages + 40);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + Smem::bar_off + 16 * kStages + 44);
+  float* kn_s = reinterpret_cast<float*>(sgen + Smem::kn_off);
   static_assert(16 * kStages + 48 <= 256, "barrier area");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -330,6 +337,7 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
       float best = -INFINITY;
       int best_j = -1;
+      float rn_next = 0.f;
       bool ok = true;
       // COLMAX: |q| of this thread's row and the range of frames the warp's 32 rows fall in
       const bool rvalid = row < rows_a;
@@ -347,6 +355,16 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int t = t0 + tl;
         const int buf = tl & 1;
         const int valid_cols = min(128, L - t * 128);
+        if (!COLMAX && g.col_norm) {
+          // |k_j| of the tile's keys through shared memory: one reciprocal per key, then broadcast reads
+          if (wg == 0) {                 // the global load runs one tile ahead of its use
+            if (tl == 0) rn_next = (t * 128 + r < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r] : 0.f;
+            kn_s[buf * 128 + r] = rn_next > 0.f ? 1.f / rn_next : 0.f;
+            const int slot = (t + 1) * 128 + r;
+            rn_next = (tl + 1 < ntl && slot < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+          }
+          named_barrier_sync(1, 256);
+        }
         float kn[2] = {0.f, 0.f};
         if (COLMAX) {
 #pragma unroll
@@ -369,8 +387,8 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const int cc = wg * 2 + c2;
           if (!COLMAX) {
             if (g.col_norm)
-              chunk_argmax_scaled(vv[c2], reinterpret_cast<const float4*>(c.rnorm + static_cast<int64_t>(h) * c.CAP + t * 128 + cc * 32),
-                                  valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+              chunk_argmax_scaled(vv[c2], reinterpret_cast<const float4*>(kn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
+                                  t * 128 + cc * 32, best, best_j);
             else
               chunk_argmax_raw(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
           } else {
