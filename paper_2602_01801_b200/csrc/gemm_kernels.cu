@@ -242,14 +242,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         const int buf = A_TMEM ? 0 : (tl & 1), bph = A_TMEM ? (tl & 1) : ((tl >> 1) & 1), rbuf = tl & 1;
         int valid_cols = 128;
         if (EPI == EPI_ARGMAX) {
-          if (wg == 0) {
-            if (tl == 0) rn_next = (t * 128 + r < L) ? (c.raw_dot ? 1.f : c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r]) : 0.f;
-            rn_s[rbuf * 128 + r] = rn_next;
-            const int slot = (t + 1) * 128 + r;
-            rn_next = (tl + 1 < ntl && slot < L) ? (c.raw_dot ? 1.f : c.rnorm[static_cast<int64_t>(h) * c.CAP + slot]) : 0.f;
-          }
           valid_cols = min(128, L - t * 128);
-          named_barrier_sync(1, 256);
+          if (!c.raw_dot) {                            // plain dot products need no per-column factor, staging or barrier
+            if (wg == 0) {
+              if (tl == 0) rn_next = (t * 128 + r < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r] : 0.f;
+              rn_s[rbuf * 128 + r] = rn_next;
+              const int slot = (t + 1) * 128 + r;
+              rn_next = (tl + 1 < ntl && slot < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + slot] : 0.f;
+            }
+            named_barrier_sync(1, 256);
+          }
         }
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bph, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
@@ -269,8 +271,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           if (EPI == EPI_ARGMAX) {
             // Scores of the chunk, then a tree maximum (no serial compare/select chain); the index is
             // searched only when the chunk holds a new strict maximum, which is rare after the first tiles.
-            chunk_argmax(v, reinterpret_cast<const float4*>(rn_s + rbuf * 128 + cc * 32), valid_cols - cc * 32,
-                         t * 128 + cc * 32, best, best_j);
+            if (c.raw_dot) chunk_argmax_plain(v, valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+            else chunk_argmax(v, reinterpret_cast<const float4*>(rn_s + rbuf * 128 + cc * 32), valid_cols - cc * 32,
+                              t * 128 + cc * 32, best, best_j);
           } else if (EPI == EPI_COLMAX) {
             const bool rvalid = row < g.rows_a;
             const int f_r = rvalid ? row / g.frame_len : -1;
@@ -509,18 +512,20 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       // 1/|k| of the tile's cache keys goes through shared memory; the global load runs one tile ahead so that its
       // latency is not paid between two tiles
       const float* rn_h = c.rnorm + static_cast<int64_t>(h) * c.CAP;
-      float rn_next = (wg == 0 && t0 * 128 + r < L) ? (c.raw_dot ? 1.f : rn_h[t0 * 128 + r]) : 0.f;
+      float rn_next = (wg == 0 && !c.raw_dot && t0 * 128 + r < L) ? rn_h[t0 * 128 + r] : 0.f;
       PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
         const int buf = tl & 1;
-        if (wg == 0) {
-          rn_s[buf * 128 + r] = rn_next;
-          const int slot = (t + 1) * 128 + r;
-          rn_next = (tl + 1 < ntl && slot < L) ? (c.raw_dot ? 1.f : rn_h[slot]) : 0.f;
+        if (!c.raw_dot) {                              // plain dot products need no per-column factor, staging or barrier
+          if (wg == 0) {
+            rn_s[buf * 128 + r] = rn_next;
+            const int slot = (t + 1) * 128 + r;
+            rn_next = (tl + 1 < ntl && slot < L) ? rn_h[slot] : 0.f;
+          }
+          named_barrier_sync(1, 256);
         }
         const int valid_cols = min(128, L - t * 128);
-        named_barrier_sync(1, 256);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
         PT_MARK(0)
@@ -540,8 +545,9 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
-          chunk_argmax(vv[c2], reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
-                       t * 128 + cc * 32, best, best_j);
+          if (c.raw_dot) chunk_argmax_plain(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+          else chunk_argmax(vv[c2], reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
+                            t * 128 + cc * 32, best, best_j);
         }
         PT_MARK(2)
       }

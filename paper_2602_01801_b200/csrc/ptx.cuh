@@ -375,6 +375,31 @@ __device__ __forceinline__ void chunk_argmax(const uint32_t (&acc)[32], const fl
   }
 }
 
+// The same without the per-column factor (scores ranked as they are).
+__device__ __forceinline__ void chunk_argmax_plain(const uint32_t (&acc)[32], int valid, int jbase, float& best, int& best_j) {
+  float x[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(acc[j]);
+  if (valid < 32) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j >= valid) x[j] = -INFINITY;
+  }
+  float m[11];
+#pragma unroll
+  for (int j = 0; j < 10; ++j) m[j] = fmax3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
+  m[10] = fmaxf(x[30], x[31]);
+  const float a0 = fmax3(m[0], m[1], m[2]), a1 = fmax3(m[3], m[4], m[5]), a2 = fmax3(m[6], m[7], m[8]);
+  const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
+  if (cm > best) {
+    best = cm;
+    int idx = 31;
+#pragma unroll
+    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;
+    best_j = jbase + idx;
+  }
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
