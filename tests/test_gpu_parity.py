@@ -557,3 +557,75 @@ def test_forced_sink_and_recent_blocks(sink, recent, keep):
         P.check_attention(out[h], O.sparse_attention(Q[h].astype(np.float64), hc, want, cfg.block, cfg.block), f"forced blocks, head {h}")
     cache.set_forced_blocks(0, 0)
     gpu_annsa_checked(cache, cfg, w, Q, post, keep)          # back to the plain rule
+
+
+def _random_case(seed):
+    rng = np.random.default_rng(seed)
+    d = int(rng.choice([64, 128]))
+    pt = int(rng.choice([64, 128]))
+    gh, gw, fpc = int(rng.integers(3, 15)), int(rng.integers(5, 31)), int(rng.integers(1, 4))
+    chunk = gh * gw * fpc
+    prior = int(rng.integers(1, 4))
+    # capacity: sometimes roomy, sometimes so tight that the later updates evict
+    cap = (prior + 3) * chunk if rng.random() < 0.6 else (prior + 1) * chunk + chunk // 3
+    cap = max(-(-cap // 128) * 128, 256)
+    cfg = synth.small_config(num_heads=int(rng.integers(1, 4)), head_dim=d, grid_h=gh, grid_w=gw, frames_per_chunk=fpc,
+                             clusters=int(rng.integers(4, 40)), resample=float(rng.choice([0.0, 0.1, 0.4])),
+                             prompt_tokens=int(rng.integers(17, 200)), relevant=int(rng.integers(1, 6)), capacity=cap, block=pt,
+                             keep_blocks=int(rng.integers(1, 9)), keep_prompt=int(rng.integers(1, 40)), prior_chunks=prior,
+                             lsh_tables=int(rng.integers(1, 5)), lsh_bits=int(rng.integers(2, 9)),
+                             tau=float(rng.choice([0.5, 0.9, 0.99])), seed=int(rng.integers(1, 10 ** 6)))
+    opts = dict(fp32=bool(rng.random() < 0.3), search_bits=int(rng.choice([16, 8])), probe=bool(rng.random() < 0.4),
+                representative=str(rng.choice(["last", "mean"])), block_q=int(rng.choice([64, 128])),
+                n_sink=int(rng.integers(0, 3)) * 16)
+    return cfg, opts
+
+
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_shapes_and_options(seed):
+    # Seeded random cases over head dim, page size, frame shape (row counts that are no multiple of anything), cache
+    # capacity (some evict), LSH shape, budgets, threshold, input dtype, search width, correspondence rule and
+    # representative: a whole step plus two more updates, every stage checked against the oracle.
+    cfg, o = _random_case(1000 + seed)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, o["fp32"], o["n_sink"], search_bits=o["search_bits"], representative=o["representative"])
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim, o["n_sink"]) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0, o["fp32"])
+    post = None
+    for ci in range(cfg.prior_chunks, cfg.prior_chunks + 3):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, o["fp32"], probe=Q if o["probe"] else None)
+    res = gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks, o["fp32"], block_q=o["block_q"])
+    Kp, Vp, _ = w.prompt(cfg.prior_chunks)
+    gpu_annca_checked(cache, cfg, Q, Kp, Vp, cfg.keep_prompt, o["fp32"])
+    # the same selection with an un-cached segment of random length on top
+    torch, fastar = _gpu()
+    ns = int(np.random.default_rng(seed).integers(1, K.shape[1] + 1))
+    _, K2, V2 = w.chunk(cfg.prior_chunks + 3)
+    out = cache.annsa_segment(fastar.to_device(Q, o["fp32"]), fastar.to_device(K2[:, :ns], o["fp32"]),
+                              fastar.to_device(V2[:, :ns], o["fp32"]), o["block_q"], cfg.keep_blocks)["out"].float().cpu().numpy()
+    assert cache.status() == 0
+    for h, hc in enumerate(P.oracle_heads_from_export(post)):
+        nqb = -(-Q.shape[1] // o["block_q"])
+        if "sel" in res:
+            sel = res["sel"][h].cpu().numpy()[:, : int(res["nsel"][h])]
+        else:
+            sel = np.tile(np.arange(-(-hc.L // cfg.block)), (nqb, 1))
+        want = O.sparse_attention_with_segment(Q[h], hc, sel, o["block_q"], cfg.block, K2[h, :ns], V2[h, :ns])
+        P.check_attention(out[h], want, f"segment of {ns}, head {h}")
+    # AnnCA with the bucket rule
+    r2 = cache.annca_lsh(fastar.to_device(Q, o["fp32"]), fastar.to_device(Kp, o["fp32"]), fastar.to_device(Vp, o["fp32"]),
+                         cfg.frame_len, debug=True)
+    assert cache.status() == 0
+    R = w.lsh_projection()
+    for h in range(cfg.num_heads):
+        qc = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, r2["qcode"][h].cpu().numpy().view(np.uint32))
+        pc = P.check_codes(Kp[h], R, cfg.lsh_tables, cfg.lsh_bits, r2["pcode"][h].cpu().numpy().view(np.uint32))
+        want_sel = O.prompt_bucket_selection(qc, pc, cfg.frame_len)
+        nsel = r2["nsel"][h].cpu().numpy()
+        got_sel = [r2["sel"][h, f, : nsel[f]].cpu().numpy().astype(np.int64) for f in range(len(want_sel))]
+        assert all(np.array_equal(a, b) for a, b in zip(got_sel, want_sel)), f"bucket rule, head {h}"
+        want = O.annca_lsh(Q[h], Kp[h], Vp[h], R, cfg.lsh_tables, cfg.lsh_bits, cfg.frame_len, sel=got_sel)["out"]
+        P.check_attention(r2["out"][h].float().cpu().numpy(), want, f"AnnCA-LSH head {h}")
