@@ -154,3 +154,62 @@ def test_c1_full_size_update_with_eight_bit_search_sampled():
         assert L == int(pre["len"][h]) + int(stats[h, 2]) <= cfg.capacity
         assert int(post["count"][h, :L].sum()) == (cfg.prior_chunks + 1) * n
         assert int(stats[h, 0]) + int(stats[h, 2]) + int(stats[h, 3]) == n
+    # AnnCA's prompt relevance on 8-bit codes at full size (two heads; the matrix is only 4680 x 512 per head)
+    Kp, Vp, _ = w.prompt(cfg.prior_chunks)
+    c = cache.annca(fastar.to_device(Q), fastar.to_device(Kp), fastar.to_device(Vp), cfg.frame_len, cfg.keep_prompt, debug=True)
+    assert cache.status() == 0
+    ac = cache.export_annca_codes(n, cfg.prompt_tokens)
+    oc = c["out"].float().cpu().numpy()
+    for h in (0, 11):
+        P.check_search_codes(Q[h], ac["q"][h], f"AnnCA query codes, head {h}")
+        P.check_search_codes(Kp[h], ac["prompt"][h], f"AnnCA prompt codes, head {h}")
+        selp = c["sel"][h].cpu().numpy()
+        P.check_prompt_selection(Q[h], Kp[h], cfg.frame_len, cfg.keep_prompt, selp, c["rel"][h].cpu().numpy(),
+                                 codes=(ac["q"][h][:, : cfg.head_dim], ac["prompt"][h][:, : cfg.head_dim]))
+        P.check_attention(oc[h], O.annca(Q[h], Kp[h], Vp[h], cfg.frame_len, cfg.keep_prompt, sel=selp)["out"], f"AnnCA 8-bit c1 head {h}")
+
+
+def test_c1_full_size_probe_update_and_segment_attention_sampled():
+    """The neighbouring calls of the step at full c1 size: the query-probe update (top-1 and cosine on sampled tokens,
+    merge bookkeeping in full for two heads) and AnnSA over the cache plus the chunk's own 4680 un-cached keys and
+    values (sampled query blocks, incl. the ragged last one)."""
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.CONFIGS["c1"]
+    w = synth.Workload(cfg)
+    H, n = cfg.num_heads, cfg.chunk_tokens
+    cache = fastar.Cache(H, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
+                         max_tokens=n, max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk)
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, 2.0, outputs=False)
+    assert cache.status() == 0
+    pre = cache.export_state()
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    dq, dk, dv = fastar.to_device(Q), fastar.to_device(K), fastar.to_device(V)
+    # attention of the chunk before it is cached: kept cache blocks + its own keys and values
+    a = cache.annsa(dq, cfg.block, cfg.keep_blocks, debug=True)
+    seg = cache.annsa_segment(dq, dk, dv, cfg.block, cfg.keep_blocks)["out"].float().cpu().numpy()
+    assert cache.status() == 0
+    pre_heads = P.oracle_heads_from_export(pre)
+    nqb = -(-n // cfg.block)
+    for h in (0, 11):
+        sel = a["sel"][h].cpu().numpy()[:, : int(a["nsel"][h])]
+        for blk in (0, nqb // 2, nqb - 1):
+            rows = slice(blk * cfg.block, min((blk + 1) * cfg.block, n))
+            want = O.sparse_attention_with_segment(Q[h][rows], pre_heads[h], sel[blk: blk + 1], cfg.block, cfg.block, K[h], V[h])
+            P.check_attention(seg[h][rows], want, f"segment attention c1 head {h} block {blk}")
+    # then the chunk enters the cache through the query-probe update
+    res = cache.update(dk, dv, cfg.frame_len, cfg.tau, probe=dq)
+    assert cache.status() == 0
+    post = cache.export_state()
+    match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    rng = np.random.default_rng(2)
+    for h in (0, 11):
+        rows = np.sort(rng.choice(n, 96, replace=False))
+        P.check_update(pre_heads[h], K[h], V[h], cfg.frame_len, cfg.tau, match[h], sim[h], dest[h], stats[h], post, h, rows=rows,
+                       probe=Q[h])
+    for h in range(H):
+        L = int(post["len"][h])
+        assert L == int(pre["len"][h]) + int(stats[h, 2]) <= cfg.capacity
+        assert int(post["count"][h, :L].sum()) == (cfg.prior_chunks + 1) * n
