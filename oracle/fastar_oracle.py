@@ -26,12 +26,21 @@ Paper passages followed
                                                                       block_scores, topk_lowest_index
   * Section 5.3 (AnnCA)          prompt token kept iff a current-frame query
                                  is its neighbour                  -> prompt_relevance, annca
+  * Section 5.3, LSH flavour     kept iff it shares a bucket with a query
+                                 of the frame                      -> prompt_bucket_selection, annca_lsh
+  * Eq. 1 (Section 3)            attended set = current frames' K/V joined
+                                 with the cache                    -> sparse_attention_with_segment
+  * Appendix C "Representative selection"  mean key (ablation)     -> tempcache_update(representative="mean")
+  * selector option (no passage) forced sink / recent blocks       -> select_blocks
   * Section 4 / Section 6 "Metrics"  recall, density              -> attention_recall, density
 
 Pinned by tests/test_oracle_pins.py: Lemma exactness, brute-force nearest
 neighbour, cache invariants, reduction to dense attention (checked against
 torch's scaled_dot_product_attention), brute-force collision counts, hand-made
-eviction and top-k cases, closed-form fixtures under tests/golden/.
+eviction and top-k cases, closed-form fixtures under tests/golden/; the 8-bit
+format against torch's float8_e4m3fn, brute-force quantised scores, the probe
+against the soft-max arg-max, the segment against Lemma 1 written with weights,
+the bucket rule and the forced blocks by brute force, the mean key in closed form.
 Parity unpinned: the paper's recall/density/speed-up values (they need the
 paper's models and prompts) — nothing here reproduces them.
 
