@@ -398,6 +398,25 @@ def test_argument_errors_are_rejected_on_the_host():
     with pytest.raises(fastar.FastarError) as e:
         cache.update(dq, dq, 0, 0.9)
     assert e.value.status == fastar.ERR_INVALID_ARG
+    # the later entry points
+    with pytest.raises(fastar.FastarError) as e:
+        cache.annsa_segment(dq, big, big, cfg.block, 4)                 # segment longer than max_tokens
+    assert e.value.status == fastar.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fastar.FastarError) as e:
+        cache.annca_lsh(dq, dq[:, :64], dq[:, :64], 1)                   # more frames than max_frames
+    assert e.value.status == fastar.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fastar.FastarError) as e:
+        cache.set_forced_blocks(-1, 0)
+    assert e.value.status == fastar.ERR_INVALID_ARG
+    with pytest.raises(fastar.FastarError) as e:
+        cache.export_probe_codes(16)                                    # not an 8-bit cache
+    assert e.value.status == fastar.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fastar.FastarError) as e:
+        cache.export_annca_codes(16, 16)
+    assert e.value.status == fastar.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fastar.FastarError):
+        fastar.Cache(cfg.num_heads, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), search_bits=4)
+    assert cache.status() == 0                                          # nothing was launched by the rejected calls
 
 
 @pytest.mark.parametrize("d,pt,fp32", [(128, 128, False), (64, 64, False), (128, 64, True), (64, 128, False)])
