@@ -164,17 +164,40 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
 #pragma unroll
       for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(mask, ss, o);
       rn = ss > 0.f ? 1.f / sqrtf(ss) : 0.f;
-      // sign-random-projection code: bit u of table t = [<k, R[t*B + u]> > 0]
-      for (int col = 0; col < c.T * c.B; ++col) {
-        float r8[8];
-        unpack8(*reinterpret_cast<const uint4*>(c.lsh + col * D + sl * 8), r8);
+      // sign-random-projection code: bit u of table t = [<k, R[t*B + u]> > 0].  Every lane forms its part of all 32
+      // projections, then a reduce-scatter over the row's lanes (each step halves the values a lane keeps) leaves
+      // 32 / LPR complete sums per lane: 30 shuffles instead of 128.
+      float pd[32];
+      const int ncol = c.T * c.B;
+#pragma unroll
+      for (int col = 0; col < 32; ++col) {
         float dot = 0.f;
+        if (col < ncol) {
+          float r8[8];
+          unpack8(*reinterpret_cast<const uint4*>(c.lsh + col * D + sl * 8), r8);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) dot = fmaf(f[e], r8[e], dot);
-#pragma unroll
-        for (int o = LPR / 2; o >= 1; o >>= 1) dot += __shfl_xor_sync(mask, dot, o);
-        if (dot > 0.f) code |= 1u << (8 * (col / c.B) + (col % c.B));
+          for (int e = 0; e < 8; ++e) dot = fmaf(f[e], r8[e], dot);
+        }
+        pd[col] = dot;
       }
+#pragma unroll
+      for (int o = LPR / 2, half = 16; o >= 1; o >>= 1, half >>= 1) {
+        const bool upper = (sl & o) != 0;
+#pragma unroll
+        for (int j = 0; j < half; ++j) {
+          const float send = upper ? pd[j] : pd[j + half];
+          const float keep = upper ? pd[j + half] : pd[j];
+          pd[j] = keep + __shfl_xor_sync(mask, send, o);
+        }
+      }
+      constexpr int NV = 32 / LPR;                 // complete sums per lane: columns NV * sl ... NV * sl + NV - 1
+#pragma unroll
+      for (int j = 0; j < NV; ++j) {
+        const int col = NV * sl + j;
+        if (col < ncol && pd[j] > 0.f) code |= 1u << (8 * (col / c.B) + (col % c.B));
+      }
+#pragma unroll
+      for (int o = LPR / 2; o >= 1; o >>= 1) code |= __shfl_xor_sync(mask, code, o);
       if (c.pool_k8) {
         const float sc = rn * 16.f;
         uint32_t w8[4];
