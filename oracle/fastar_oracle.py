@@ -236,10 +236,41 @@ def top1_query_probe(Q_new: np.ndarray, K_new: np.ndarray, cache: HeadCache, sea
     return j, np.where(den > 0, num / np.where(den > 0, den, 1.0), 0.0)
 
 
+def hamming_distances(codes_a: np.ndarray, codes_b: np.ndarray, bits: int) -> np.ndarray:
+    """Number of differing sign bits between every pair of LSH codes.  codes: [n][T] bucket ids of `bits` bits."""
+    x = np.asarray(codes_a, np.int64)[:, None, :] ^ np.asarray(codes_b, np.int64)[None, :, :]
+    d = np.zeros(x.shape[:2], dtype=np.int64)
+    for u in range(bits):
+        d += ((x >> u) & 1).sum(axis=2)
+    return d
+
+
+def top1_hamming(K_new: np.ndarray, cache: HeadCache, R: np.ndarray, tables: int, bits: int,
+                 codes_new: Optional[np.ndarray] = None, codes_cache: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """The LSH flavour of the correspondence search (Section 5.1 "LSH", Section 5.2): keys are compared through the
+    T*b sign bits of the shared random projection; the corresponding token of a new key is the live cached key at
+    the smallest Hamming distance (ties -> smallest slot).  Returns (j*, cos(k_i, k_j*)): the merge threshold is
+    applied to the exact cosine of that key.  codes_*: bucket ids computed elsewhere (staged parity)."""
+    K_new = np.asarray(K_new, np.float64)
+    n = K_new.shape[0]
+    if cache.L == 0:
+        return np.full(n, -1, np.int64), np.zeros(n, np.float64)
+    Kc = cache.K[: cache.L]
+    if codes_new is None:
+        codes_new = lsh_codes(K_new, R, tables, bits)
+    if codes_cache is None:
+        codes_cache = lsh_codes(Kc, R, tables, bits)
+    j = np.argmin(hamming_distances(codes_new, codes_cache, bits), axis=1).astype(np.int64)
+    num = np.sum(K_new * Kc[j], axis=1)
+    den = np.sqrt(np.sum(K_new * K_new, axis=1)) * np.sqrt(np.sum(Kc[j] * Kc[j], axis=1))
+    return j, np.where(den > 0, num / np.where(den > 0, den, 1.0), 0.0)
+
+
 def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
                      forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None,
                      search_bits: int = 16, probe: Optional[np.ndarray] = None,
-                     representative: str = "last") -> Dict[str, np.ndarray]:
+                     representative: str = "last",
+                     lsh: Optional[Tuple[np.ndarray, int, int]] = None) -> Dict[str, np.ndarray]:
     """One TempCache update of one head.
 
     representative = "last" keeps the newest matching key in a merged slot (the paper's choice), "mean" the
@@ -247,7 +278,8 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
     forced = (j*, c*, matched) replaces steps 1-2 by decisions taken elsewhere
     (staged parity: near-ties have several correct answers).  search_bits = 8 runs the
     correspondence search on the 8-bit codes of the keys instead of the keys themselves.
-    probe = the chunk's queries [n][d] selects the query-probe correspondence (top1_query_probe)."""
+    probe = the chunk's queries [n][d] selects the query-probe correspondence (top1_query_probe).
+    search_bits = 1 with lsh = (R, tables, bits) searches by Hamming distance of the LSH sign bits (top1_hamming)."""
     K_new = np.asarray(K_new, np.float64)
     V_new = np.asarray(V_new, np.float64)
     n = K_new.shape[0]
@@ -255,7 +287,9 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
 
     # 1. top-1 correspondence against the pre-call cache; 2. threshold
     if forced is None:
-        if probe is not None:
+        if search_bits == 1:
+            jstar, cstar = top1_hamming(K_new, cache, lsh[0], lsh[1], lsh[2])
+        elif probe is not None:
             jstar, cstar = top1_query_probe(probe, K_new, cache, search_bits)
         else:
             jstar, cstar = top1_quantized(K_new, cache) if search_bits == 8 else top1_cosine(K_new, cache)

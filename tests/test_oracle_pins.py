@@ -668,3 +668,38 @@ def test_query_probe_on_eight_bit_codes():
     Kc2[4] = 50.0 * Q[3] / np.linalg.norm(Q[3])
     cache2.load(Kc2, np.zeros((L, d)))
     assert O.top1_query_probe(Q, K, cache2, search_bits=8)[0][3] == 4
+
+
+def test_hamming_correspondence():
+    rng = _rng(41)
+    d, L, n, T, b = 16, 35, 20, 3, 5
+    R = rng.standard_normal((T * b, d))
+    cache = O.HeadCache(64, d)
+    Kc = rng.standard_normal((L, d))
+    cache.load(Kc, rng.standard_normal((L, d)))
+    K = rng.standard_normal((n, d))
+    K[2] = 3.0 * Kc[17]                                   # same direction: distance 0, found whatever the ties
+    K[3] = -Kc[5]                                         # opposite direction: every bit differs from slot 5
+    j, c = O.top1_hamming(K, cache, R, T, b)
+    # brute force on the sign bits themselves, Python loops
+    sb = lambda x: [int(v > 0) for v in (R @ x)]
+    bits_c = [sb(Kc[s]) for s in range(L)]
+    for i in range(n):
+        bi = sb(K[i])
+        dist = [sum(p != q for p, q in zip(bi, bits_c[s])) for s in range(L)]
+        jb = min(range(L), key=lambda s: (dist[s], s))
+        assert j[i] == jb
+        assert abs(c[i] - float(K[i] @ Kc[jb]) / (np.linalg.norm(K[i]) * np.linalg.norm(Kc[jb]))) < 1e-12
+    assert j[2] <= 17 and O.hamming_distances(O.lsh_codes(K[2:3], R, T, b), O.lsh_codes(Kc[j[2]:j[2] + 1], R, T, b), b)[0, 0] == 0
+    assert O.hamming_distances(O.lsh_codes(K[3:4], R, T, b), O.lsh_codes(Kc[5:6], R, T, b), b)[0, 0] == T * b
+    # distance = (T*b - <s_a, s_b>) / 2 for the +-1 sign vectors
+    ca, cb = O.lsh_codes(K, R, T, b), O.lsh_codes(Kc, R, T, b)
+    sa = np.where((R @ K.T).T > 0, 1.0, -1.0)
+    sc = np.where((R @ Kc.T).T > 0, 1.0, -1.0)
+    assert np.array_equal(O.hamming_distances(ca, cb, b), ((T * b - sa @ sc.T) / 2).astype(np.int64))
+    # inside an update: the threshold applies to the exact cosine of the Hamming winner
+    c2 = cache.copy()
+    r = O.tempcache_update(c2, K[:4], np.ones((4, d)), 4, 0.9, search_bits=1, lsh=(R, T, b))
+    assert r["matched"][2] and not r["matched"][3] and r["jstar"][2] == j[2]
+    je, ce = O.top1_hamming(K, O.HeadCache(64, d), R, T, b)
+    assert np.all(je == -1) and np.all(ce == 0)
