@@ -322,14 +322,14 @@ def run_ours(args, cfg):
         ms = prof[name]["ms"] / max(prof[name]["launches"], 1)
         ach = fl / (ms * 1e-3) / 1e12 if ms > 0 else 0.0
         # the 8-bit search runs on fp8 operands: its peak is the measured bf16 figure times the nominal 2:1 ratio
-        pk = peak_tf * 2.0 if (name == "t1_similarity" and args.search_bits == 8) else peak_tf
+        pk = peak_tf * 2.0 if (name == "t1_similarity" and args.search_bits in (8, 1)) else peak_tf
         kernels[name] = {"ms": ms, "flops": fl, "achieved": ach, "frac": ach / pk, "peak": pk}
     others = {k: v["ms"] / max(v["launches"], 1) * (v["launches"] / prof_steps) for k, v in prof.items() if v["launches"]}
     dominant = max(("t1_similarity", "s5_attention"), key=lambda k: kernels[k]["ms"])
-    fp8_dominant = dominant == "t1_similarity" and args.search_bits == 8
+    fp8_dominant = dominant == "t1_similarity" and args.search_bits in (8, 1)
     roofline = {"kernel": dominant, "bound": "tensor", "achieved": kernels[dominant]["achieved"], "peak": kernels[dominant]["peak"],
                 "unit": "TFLOP/s", "frac": kernels[dominant]["frac"],
-                "traffic": None if args.search_bits == 8 else traffic.get(f"{cfg.name}.{dominant}"),
+                "traffic": None if args.search_bits in (8, 1) else traffic.get(f"{cfg.name}.{dominant}"),
                 "peak_source": f"{peak_kind} bf16 burst" + (" x 2 (nominal fp8 : bf16 ratio)" if fp8_dominant else ""),
                 "kernels": kernels, "ms_per_step_by_kernel": others}
 
@@ -362,7 +362,7 @@ def run_ours(args, cfg):
         kept = cache.annca_lsh(dq, dkp, dvp, cfg.frame_len, debug=True)["nsel"].cpu().numpy()
         variants["annca_lsh_kept_tokens"] = {"min": int(kept.min()), "mean": float(kept.mean()), "max": int(kept.max()),
                                              "of": cfg.prompt_tokens}
-        if args.search_bits != 8:
+        if args.search_bits == 16:
             variants["update_call_ms"] = timed(lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False), restore=True)
             variants["update_query_probe_call_ms"] = timed(
                 lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq), restore=True)
@@ -375,8 +375,9 @@ def run_ours(args, cfg):
     line = {"metric": "query_tokens_per_s", "value": total_units / max_seconds, "unit": "tok/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": max_seconds / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if args.search_bits != 8 else "bf16 (correspondence search on fp8 e4m3 codes)", "data": "synthetic",
-            "config": {"workload": describe(cfg) + (" search=8bit" if args.search_bits == 8 else "") + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
+            "dtype": {16: "bf16", 8: "bf16 (correspondence search on fp8 e4m3 codes)",
+                      1: "bf16 (correspondence search on LSH sign bits as fp8 +-1)"}[args.search_bits], "data": "synthetic",
+            "config": {"workload": describe(cfg) + ({16: "", 8: " search=8bit", 1: " search=hamming"}[args.search_bits]) + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
                        f"({cache.workspace_bytes >> 20} MiB copy, untimed)", "parallelism": "replicas" if world > 1 else "1 GPU",
                        "cuda_graph": graph is not None},
             "e2e": {"value": e2e_units / e2e_max, "unit": "tok/s", "ms_per_step": e2e_max / args.steps * 1e3,
@@ -407,7 +408,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1", choices=["c1", "c3", "c0", "small"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--search-bits", type=int, default=16, choices=[16, 8],
+    ap.add_argument("--search-bits", type=int, default=16, choices=[16, 8, 1],
                     help="TempCache correspondence search on the bf16 keys (16, default) or on their 8-bit codes (8)")
     ap.add_argument("--representative", default="last", choices=["last", "mean"],
                     help="key a merged slot keeps: the newest key (the paper's choice) or the mean key of its ablation")

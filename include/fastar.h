@@ -77,7 +77,12 @@ typedef struct {
                               * unchanged; the merge itself always uses the bf16 keys and values.  AnnCA
                               * then ranks prompt tokens by max_i code(q_i).code(k_p) |q_i| |k_p| / (256 sqrt d)
                               * (codes of its queries and prompt keys are made per call); the attention over
-                              * the kept tokens uses the bf16 tensors. */
+                              * the kept tokens uses the bf16 tensors.
+                              * 1 = the LSH flavour (Section 5.1, "LSH"): the code row of a key holds the T*b sign
+                              * bits of the shared projection as +1 / -1; TempCache's correspondence is the live
+                              * slot at the smallest Hamming distance (ties: lowest slot) and the threshold is
+                              * applied to the exact cosine of that slot.  AnnCA is not affected (use
+                              * fastar_annca_attention_lsh for its LSH flavour); the probe update is refused. */
   int32_t representative;    /* key a merged slot keeps (Appendix C, "Representative selection"):
                               * FASTAR_REP_LAST_KEY (0, the paper's choice) = the key of its newest matching
                               * token; FASTAR_REP_MEAN_KEY (1, the ablation's alternative) = the count-weighted

@@ -199,12 +199,25 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
 #pragma unroll
       for (int o = LPR / 2; o >= 1; o >>= 1) code |= __shfl_xor_sync(mask, code, o);
       if (c.pool_k8) {
-        const float sc = rn * 16.f;
-        uint32_t w8[4];
+        uint32_t lo, hi;                         // code bytes 8 sl .. 8 sl + 7 of the row
+        if (c.sign_codes) {                      // the LSH sign bits of the mean key as +1 / -1 in e4m3
+          uint32_t w2[2] = {0u, 0u};
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          w8[e] = __nv_cvt_float2_to_fp8x2(make_float2(f[2 * e] * sc, f[2 * e + 1] * sc), __NV_SATFINITE, __NV_E4M3);
-        const uint32_t lo = w8[0] | (w8[1] << 16), hi = w8[2] | (w8[3] << 16);   // code bytes of elements 8 sl .. 8 sl + 7
+          for (int e = 0; e < 8; ++e) {
+            const int idx = sl * 8 + e;
+            if (idx < ncol) w2[e >> 2] |= (((code >> (8 * (idx / c.B) + (idx % c.B))) & 1u) ? 0x38u : 0xB8u) << (8 * (e & 3));
+          }
+          lo = w2[0];
+          hi = w2[1];
+        } else {
+          const float sc = rn * 16.f;
+          uint32_t w8[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            w8[e] = __nv_cvt_float2_to_fp8x2(make_float2(f[2 * e] * sc, f[2 * e + 1] * sc), __NV_SATFINITE, __NV_E4M3);
+          lo = w8[0] | (w8[1] << 16);
+          hi = w8[2] | (w8[3] << 16);
+        }
         if (LPR == 16) {
           code8.x = lo;
           code8.y = hi;

@@ -83,6 +83,7 @@ struct CacheView {
   // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
+  int sign_codes;                  // the search code rows hold LSH sign bits as +-1 (Hamming search) instead of fp8 directions
   int rep_mean;                    // representative key of a merged slot: 0 = newest key, 1 = count-weighted mean key
   float* seg_bias;                 // [max_tokens + 128]  bias of the rows of an un-cached attention segment
   // AnnCA with the LSH bucket rule: codes of the queries and of the prompt keys, kept tokens per frame
@@ -112,6 +113,8 @@ int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int6
                          int64_t rn_stride, uint8_t* out, int64_t out_rows_per_head, cudaStream_t st);
 int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const CUtensorMap& tm_pool_k8, int n, bool col_norm,
                              cudaStream_t st);
+int launch_sign_rows(const CacheView& c, const uint32_t* codes, int n, int64_t code_stride, uint8_t* out, int64_t out_rows_per_head,
+                     cudaStream_t st);
 int launch_quantize_rows(const CacheView& c, const __nv_bfloat16* x, int n, int64_t hs, int64_t ts, uint8_t* out,
                          int64_t out_rows_per_head, float* norm_out, int64_t norm_stride, cudaStream_t st);
 int launch_c1_relevance_fp8(const CacheView& c, const CUtensorMap& tm_q8, const CUtensorMap& tm_kp8, const float* qn,

@@ -63,7 +63,7 @@ bool desc_valid(const fastar_cache_desc* d) {
   if (d->max_tokens < 1 || d->max_tokens > 16384) return false;
   if (d->max_prompt_tokens < 1 || d->max_prompt_tokens > 1024 || d->max_frames < 1 || d->max_frames > 64) return false;
   if (d->dtype != FASTAR_BF16 && d->dtype != FASTAR_FP32) return false;
-  if (d->search_bits != 0 && d->search_bits != 16 && d->search_bits != 8) return false;
+  if (d->search_bits != 0 && d->search_bits != 16 && d->search_bits != 8 && d->search_bits != 1) return false;
   if (d->representative != FASTAR_REP_LAST_KEY && d->representative != FASTAR_REP_MEAN_KEY) return false;
   return true;
 }
@@ -121,7 +121,8 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   for (int i = 0; i < 3; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
   for (int i = 3; i < 5; ++i) t.stage[i] = reinterpret_cast<__nv_bfloat16*>(take(H * MP * D * 2));
   t.stage[5] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
-  t.search_bits = d.search_bits == 8 ? 8 : 16;
+  t.search_bits = (d.search_bits == 8 || d.search_bits == 1) ? 8 : 16;     // both keep a pool of 128-byte code rows
+  t.sign_codes = d.search_bits == 1 ? 1 : 0;
   t.rep_mean = d.representative == FASTAR_REP_MEAN_KEY ? 1 : 0;
   t.pool_k8 = t.search_bits == 8 ? take(H * CAP * 128) : nullptr;
   t.k8_new = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
@@ -363,7 +364,7 @@ int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_code
 int fastar_cache_export_probe_codes(fastar_cache_t* c, uint8_t* host_probe_codes, int32_t n, void* stream) {
   if (!c || !host_probe_codes) return FASTAR_ERR_INVALID_ARG;
   const CacheView& v = c->v;
-  if (v.search_bits != 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (v.search_bits != 8 || v.sign_codes) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (n < 1 || n > v.max_tokens) return FASTAR_ERR_INVALID_ARG;
   DeviceGuard guard(c->desc.device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -377,7 +378,7 @@ int fastar_cache_export_annca_codes(fastar_cache_t* c, uint8_t* host_q_codes, ui
                                     void* stream) {
   if (!c) return FASTAR_ERR_INVALID_ARG;
   const CacheView& v = c->v;
-  if (v.search_bits != 8) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (v.search_bits != 8 || v.sign_codes) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if ((host_q_codes && (nq < 1 || nq > v.max_tokens)) || (host_prompt_codes && (np < 1 || np > v.max_prompt))) return FASTAR_ERR_INVALID_ARG;
   DeviceGuard guard(c->desc.device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -429,6 +430,7 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
   if (!c || !k_new || !v_new || n < 1 || frame_len < 1) return FASTAR_ERR_INVALID_ARG;
   if (n > c->v.max_tokens || n > 16384 || n > c->v.CAP) return FASTAR_ERR_UNSUPPORTED_SHAPE;
   if (token_stride < c->v.D || head_stride < 0) return FASTAR_ERR_INVALID_ARG;
+  if (q_probe && c->v.sign_codes) return FASTAR_ERR_UNSUPPORTED_SHAPE;      // the Hamming search compares keys with keys
   DeviceGuard guard(c->desc.device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const CacheView& v = c->v;
@@ -459,10 +461,12 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
     // scaled by |k_j| before the arg-max (the codes carry directions only)
     r = make_map_codes(c, &tm_a8, q_probe ? v.q8_probe : v.k8_new, n, v.H, static_cast<uint64_t>(v.max_tokens) * 128, 128);
     if (r != FASTAR_OK) return r;
-    ACCK(FASTAR_K_HASH, launch_quantize_keys(v, kb, n, khs, kts, v.rnorm_new, v.max_tokens, v.k8_new, v.max_tokens, st));
+    if (v.sign_codes) ACCK(FASTAR_K_HASH, launch_sign_rows(v, v.code_new, n, v.max_tokens, v.k8_new, v.max_tokens, st));
+    else ACCK(FASTAR_K_HASH, launch_quantize_keys(v, kb, n, khs, kts, v.rnorm_new, v.max_tokens, v.k8_new, v.max_tokens, st));
     if (q_probe) ACCK(FASTAR_K_HASH, launch_quantize_rows(v, pb, n, phs, pts, v.q8_probe, v.max_tokens, v.qn_probe, v.max_tokens, st));
     ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(v, tm_a8, c->tm_pool_k8, n, q_probe != nullptr, st));
-    if (q_probe) ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
+    // query-probe and Hamming rankings are not similarities: the threshold is applied to the exact key cosine of the winner
+    if (q_probe || v.sign_codes) ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
   } else if (q_probe) {
     CacheView vr = v;
     vr.raw_dot = 1;
@@ -642,7 +646,7 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
   } else {
     if (cudaMemsetAsync(v.rel, 0, static_cast<size_t>(v.H) * v.max_frames * v.max_prompt * 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
     float rel_scale = 1.0f / sqrtf(static_cast<float>(v.D));
-    if (v.search_bits == 8) {
+    if (v.search_bits == 8 && !v.sign_codes) {
       // relevance on the 8-bit codes of the directions, scaled back by the norms (Section 5.1 quantised search)
       CUtensorMap tm_q8, tm_kp8;
       r = make_map_codes(c, &tm_q8, v.q8_ca, nq, v.H, static_cast<uint64_t>(v.max_tokens) * 128, 128);

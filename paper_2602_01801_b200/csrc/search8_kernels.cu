@@ -161,6 +161,41 @@ int launch_quantize_rows(const CacheView& c, const __nv_bfloat16* x, int n, int6
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
+// LSH flavour of the search (Section 5.1): the code row of a key holds its T*b sign bits as +1 / -1 in e4m3 (0x38 /
+// 0xB8), zero padded to 128 bytes, so that the dot product of two rows is T*b - 2 * (Hamming distance) and the
+// arg-max of the search kernel is the key at the smallest Hamming distance (ties -> lowest slot).  One thread per 8
+// bytes; bit u of table t sits at bit 8*t + u of the packed code.
+__global__ void __launch_bounds__(256) sign_rows_kernel(const uint32_t* __restrict__ codes, int H, int n, int64_t code_stride, int T,
+                                                        int B, uint8_t* __restrict__ out, int64_t out_rows_per_head) {
+  const int64_t total = static_cast<int64_t>(H) * n * 16;
+  for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; q < total;
+       q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int e8 = static_cast<int>(q & 15);
+    const int64_t rowid = q >> 4;
+    const int h = static_cast<int>(rowid / n), i = static_cast<int>(rowid % n);
+    const uint32_t code = codes[h * code_stride + i];
+    uint32_t w[2] = {0u, 0u};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = e8 * 8 + e;
+      if (idx < T * B) {
+        const uint32_t bit = (code >> (8 * (idx / B) + (idx % B))) & 1u;
+        w[e >> 2] |= (bit ? 0x38u : 0xB8u) << (8 * (e & 3));
+      }
+    }
+    *reinterpret_cast<uint2*>(out + (static_cast<int64_t>(h) * out_rows_per_head + i) * 128 + e8 * 8) = make_uint2(w[0], w[1]);
+  }
+}
+
+int launch_sign_rows(const CacheView& c, const uint32_t* codes, int n, int64_t code_stride, uint8_t* out, int64_t out_rows_per_head,
+                     cudaStream_t st) {
+  if (n <= 0) return 0;
+  const int64_t total = static_cast<int64_t>(c.H) * n * 16;
+  const int grid = static_cast<int>((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+  sign_rows_kernel<<<grid, 256, 0, st>>>(codes, c.H, n, code_stride, c.T, c.B, out, out_rows_per_head);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
+}
+
 // One thread per 8 components of a 128-byte code row.
 __global__ void __launch_bounds__(256) quantize_kernel(const __nv_bfloat16* __restrict__ x, int H, int n, int D, int64_t hs,
                                                        int64_t ts, const float* __restrict__ rnorm, int64_t rn_stride,

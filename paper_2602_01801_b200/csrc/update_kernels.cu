@@ -759,7 +759,9 @@ int launch_import_derive(const CacheView& c, cudaStream_t st) {
   if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
   int r3 = 0;
   if (c.pool_k8) {                                   // search codes of every slot from the imported keys
-    r3 = launch_quantize_keys(c, c.pool_k, c.CAP, static_cast<int64_t>(c.CAP) * c.D, c.D, c.rnorm, c.CAP, c.pool_k8, c.CAP, st);
+    r3 = c.sign_codes ? launch_sign_rows(c, c.kcode, c.CAP, c.CAP, c.pool_k8, c.CAP, st)
+                      : launch_quantize_keys(c, c.pool_k, c.CAP, static_cast<int64_t>(c.CAP) * c.D, c.D, c.rnorm, c.CAP, c.pool_k8,
+                                             c.CAP, st);
     if (r3 < 0) return r3;
   }
   int r2 = launch_finalize_hist(c, nullptr, -1, st);

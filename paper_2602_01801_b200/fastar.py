@@ -120,7 +120,7 @@ class Cache:
         self.desc = CacheDesc(num_heads, head_dim, capacity, page_tokens, n_sink, lsh_tables, lsh_bits, max_tokens,
                               max_prompt_tokens, max_frames, FP32 if fp32 else BF16, device, search_bits,
                               {"last": 0, "mean": 1}[representative])
-        self.search_bits = search_bits
+        self.search_bits = search_bits           # 16 = bf16 keys, 8 = fp8 direction codes, 1 = LSH sign bits (Hamming)
         self.representative = representative
         self.max_tokens = max_tokens
         nbytes = self.lib.fastar_cache_workspace_bytes(C.byref(self.desc))

@@ -47,7 +47,7 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
                  sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
                  rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None,
                  probe: Optional[np.ndarray] = None, representative: str = "last",
-                 probe_codes: Optional[np.ndarray] = None) -> O.HeadCache:
+                 probe_codes: Optional[np.ndarray] = None, hamming=None) -> O.HeadCache:
     """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
     exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases).
     `codes` = (codes of the new keys [n][128], codes of the pre-call cache [>= L][128]) as the GPU computed them
@@ -60,7 +60,18 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
     idx = np.arange(n) if rows is None else rows
     margin = MARGIN if codes is None else MARGIN_Q8
     sim_tol = 2e-5 if codes is None else MARGIN_Q8
-    if pre.L > 0 and probe is not None:
+    if pre.L > 0 and hamming is not None:
+        # integer ranking: the slot is the arg-min of the Hamming distance of the GPU's own sign bits, exactly
+        codes_new, codes_cache, bits = hamming
+        dist = O.hamming_distances(codes_new[idx], codes_cache[: pre.L], bits)
+        jb = np.argmin(dist, axis=1)
+        cos_b = O.cosine_matrix(K64[idx], pre.K[: pre.L])[np.arange(idx.size), jb]
+        assert np.max(np.abs(sim[idx] - cos_b)) <= 2e-5, "T1 Hamming: cosine of the nearest slot"
+        mi = np.flatnonzero(matched[idx])
+        assert np.array_equal(match[idx][mi], jb[mi]), "T1 Hamming: matched slot is not the nearest"
+        far = np.abs(cos_b - tau) > MARGIN
+        assert np.array_equal(matched[idx][far], (cos_b >= tau)[far]), "T2 Hamming: threshold decision"
+    elif pre.L > 0 and probe is not None:
         Kc = pre.K[: pre.L]
         Q64 = probe.astype(np.float64)[idx]
         if codes is None:
@@ -134,6 +145,18 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
     assert (int(stats[0]), int(stats[1]), int(stats[2]), int(stats[3]), int(stats[4]), int(stats[5]), int(stats[6])) == (
         st["matched"], st["touched"], st["appended"], st["evicted_slots"], st["evicted_tokens"], st["length"], 1), "stats"
     return ref
+
+
+def sign_rows_to_packed(rows: np.ndarray, tables: int, bits: int, what: str) -> np.ndarray:
+    """Code rows of the Hamming search ([n][128] bytes: +1 = 0x38 / -1 = 0xB8 for each of the T*b sign bits, zero
+    padding) -> packed LSH codes (uint32, table t in byte t).  Any other byte fails."""
+    nb = tables * bits
+    body, pad = rows[:, :nb], rows[:, nb:]
+    assert not pad.any(), f"{what}: padding bytes"
+    assert np.all((body == 0x38) | (body == 0xB8)), f"{what}: a byte is neither +1 nor -1"
+    b = (body == 0x38).astype(np.uint32).reshape(rows.shape[0], tables, bits)
+    per_table = (b << np.arange(bits, dtype=np.uint32)).sum(axis=2).astype(np.uint32)
+    return (per_table << (8 * np.arange(tables, dtype=np.uint32))).sum(axis=1).astype(np.uint32)
 
 
 def check_search_codes(X: np.ndarray, got: np.ndarray, what: str) -> None:

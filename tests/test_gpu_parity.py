@@ -24,22 +24,36 @@ def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, sea
                         representative=representative)
 
 
-def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=None):
+def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=None, lsh=None):
     """Runs one update on the GPU and checks it against the oracle heads `heads` (advanced in place).
-    probe = the chunk's queries [H][n][d] runs the query-probe correspondence."""
+    probe = the chunk's queries [H][n][d] runs the query-probe correspondence.  lsh = (R, tables, bits) is needed
+    for a cache that searches by Hamming distance (search_bits = 1)."""
     torch, fastar = _gpu()
     q8 = cache.search_bits == 8
-    pre_codes = cache.export_search_codes()["cache"] if q8 else None      # codes of the cache the search will see
+    sign = cache.search_bits == 1
+    pre_codes = cache.export_search_codes()["cache"] if (q8 or sign) else None      # codes of the cache the search will see
     res = cache.update(fastar.to_device(K, fp32), fastar.to_device(V, fp32), frame_len, tau,
                        probe=None if probe is None else fastar.to_device(probe, fp32))
     assert cache.status() == 0
     post = cache.export_state()
     match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
     synced = P.oracle_heads_from_export(post, heads[0].n_sink)
-    post_codes = cache.export_search_codes(K.shape[1]) if q8 else None
+    post_codes = cache.export_search_codes(K.shape[1]) if (q8 or sign) else None
     probe_codes = cache.export_probe_codes(K.shape[1]) if (q8 and probe is not None) else None
     for h in range(K.shape[0]):
         codes = None
+        hamming = None
+        if sign:
+            # the code rows hold the sign bits the GPU hashed: every byte is +1 / -1, bits clear of zero agree with the
+            # oracle's projections, and after the update every live slot's row matches its exported LSH code
+            R, T, b = lsh
+            new_packed = P.sign_rows_to_packed(post_codes["new"][h], T, b, f"new-key sign rows, head {h}")
+            codes_new = P.check_codes(np.asarray(K[h], np.float64), R, T, b, new_packed)
+            Lh = int(post["len"][h])
+            assert np.array_equal(P.sign_rows_to_packed(post_codes["cache"][h, :Lh], T, b, f"cache sign rows, head {h}"),
+                                  post["code"][h, :Lh].astype(np.uint32))
+            pre_packed = P.sign_rows_to_packed(pre_codes[h][: heads[h].L], T, b, f"pre-call sign rows, head {h}")
+            hamming = (codes_new, P.unpack_codes(pre_packed, T), b)
         if q8 and probe is not None:
             P.check_search_codes(np.asarray(probe[h], np.float64), probe_codes[h], f"probe codes, head {h}")
         if q8:
@@ -50,7 +64,7 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
             codes = (post_codes["new"][h], pre_codes[h])
         ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes,
                              probe=None if probe is None else probe[h], representative=cache.representative,
-                             probe_codes=probe_codes[h] if (q8 and probe is not None) else None)
+                             probe_codes=probe_codes[h] if (q8 and probe is not None) else None, hamming=hamming)
         # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
         # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
         synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
@@ -648,3 +662,38 @@ def test_random_shapes_and_options(seed):
         assert all(np.array_equal(a, b) for a, b in zip(got_sel, want_sel)), f"bucket rule, head {h}"
         want = O.annca_lsh(Q[h], Kp[h], Vp[h], R, cfg.lsh_tables, cfg.lsh_bits, cfg.frame_len, sel=got_sel)["out"]
         P.check_attention(r2["out"][h].float().cpu().numpy(), want, f"AnnCA-LSH head {h}")
+
+
+@pytest.mark.parametrize("d,pt,tables,bits,rep", [(128, 128, 4, 8, "last"), (64, 64, 3, 5, "last"), (128, 64, 4, 8, "mean")])
+def test_hamming_search_on_lsh_sign_bits(d, pt, tables, bits, rep):
+    # The LSH flavour of the correspondence search: code rows of +1 / -1 sign bits, the tensor-core arg-max is the
+    # arg-min of the Hamming distance (checked exactly on the GPU's own bits, ties -> lowest slot), the threshold is
+    # applied to the exact cosine of that slot.  Rows of merged slots are copied (last key) or rebuilt (mean key);
+    # an import rebuilds all of them; the probe form is refused.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3, lsh_tables=tables, lsh_bits=bits)
+    w = synth.Workload(cfg)
+    lsh = (w.lsh_projection(), tables, bits)
+    cache = make_cache(cfg, w, search_bits=1, representative=rep)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0, lsh=lsh)
+    matched = 0
+    for ci in range(cfg.prior_chunks, cfg.prior_chunks + 3):
+        Q, K, V = w.chunk(ci)
+        before = [hc.L for hc in heads]
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, lsh=lsh)
+        matched += sum(K.shape[1] - (hc.L - b) for hc, b in zip(heads, before))
+    assert matched > 0 and post["count"].max() > 1
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+    st = cache.export_state()
+    cache.import_state(st["k"], st["v"], st["len"], st["count"], st["stamp"], now=int(st["now"][0]))
+    rows = cache.export_search_codes()["cache"]
+    st2 = cache.export_state()
+    for h in range(cfg.num_heads):
+        Lh = int(st["len"][h])
+        assert np.array_equal(P.sign_rows_to_packed(rows[h, :Lh], tables, bits, f"rows after import, head {h}"),
+                              st2["code"][h, :Lh].astype(np.uint32))
+    with pytest.raises(fastar.FastarError):
+        cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau, probe=fastar.to_device(Q))
