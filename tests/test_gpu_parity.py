@@ -608,7 +608,7 @@ def _random_case(seed):
                              keep_blocks=int(rng.integers(1, 9)), keep_prompt=int(rng.integers(1, 40)), prior_chunks=prior,
                              lsh_tables=int(rng.integers(1, 5)), lsh_bits=int(rng.integers(2, 9)),
                              tau=float(rng.choice([0.5, 0.9, 0.99])), seed=int(rng.integers(1, 10 ** 6)))
-    opts = dict(fp32=bool(rng.random() < 0.3), search_bits=int(rng.choice([16, 8])), probe=bool(rng.random() < 0.4),
+    opts = dict(fp32=bool(rng.random() < 0.3), search_bits=int(rng.choice([16, 8, 1])), probe=bool(rng.random() < 0.4),
                 representative=str(rng.choice(["last", "mean"])), block_q=int(rng.choice([64, 128])),
                 n_sink=int(rng.integers(0, 3)) * 16)
     return cfg, opts
@@ -620,16 +620,19 @@ def test_random_shapes_and_options(seed):
     # capacity (some evict), LSH shape, budgets, threshold, input dtype, search width, correspondence rule and
     # representative: a whole step plus two more updates, every stage checked against the oracle.
     cfg, o = _random_case(1000 + seed)
+    if o["search_bits"] == 1:
+        o["probe"] = False                       # the Hamming search compares keys with keys
     w = synth.Workload(cfg)
+    lsh = (w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits)
     cache = make_cache(cfg, w, o["fp32"], o["n_sink"], search_bits=o["search_bits"], representative=o["representative"])
     heads = [O.HeadCache(cfg.capacity, cfg.head_dim, o["n_sink"]) for _ in range(cfg.num_heads)]
     for ci in range(cfg.prior_chunks):
         _, K, V = w.chunk(ci)
-        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0, o["fp32"])
+        gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0, o["fp32"], lsh=lsh)
     post = None
     for ci in range(cfg.prior_chunks, cfg.prior_chunks + 3):
         Q, K, V = w.chunk(ci)
-        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, o["fp32"], probe=Q if o["probe"] else None)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, o["fp32"], probe=Q if o["probe"] else None, lsh=lsh)
     res = gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks, o["fp32"], block_q=o["block_q"])
     Kp, Vp, _ = w.prompt(cfg.prior_chunks)
     gpu_annca_checked(cache, cfg, Q, Kp, Vp, cfg.keep_prompt, o["fp32"])
