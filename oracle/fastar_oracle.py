@@ -380,15 +380,22 @@ def lsh_codes(X: np.ndarray, R: np.ndarray, tables: int, bits: int) -> np.ndarra
     return (sign << np.arange(bits, dtype=np.int64)).sum(axis=2)
 
 
-def block_histograms(codes: np.ndarray, n_live: int, block: int, bits: int) -> np.ndarray:
-    """H[blk][t][w] = number of rows r < n_live of block blk with code_t = w."""
+HIST_WEIGHT_MAX = 65535                       # weighted histogram entries saturate here (two 8-bit digits)
+
+
+def block_histograms(codes: np.ndarray, n_live: int, block: int, bits: int, weights: Optional[np.ndarray] = None) -> np.ndarray:
+    """H[blk][t][w] = number of rows r < n_live of block blk with code_t = w.
+    weights (the multiplicities m of the cached keys, a selector option): every row counts m_r times, so that the
+    score of a key block is what the block would score with its merged tokens still in place (Lemma 1: a slot
+    stands for m_r identical keys); an entry saturates at HIST_WEIGHT_MAX."""
     tables = codes.shape[1]
     nblk = -(-n_live // block) if n_live > 0 else 0
     H = np.zeros((nblk, tables, 1 << bits), dtype=np.int64)
     rows = np.arange(n_live)
+    w = 1 if weights is None else np.asarray(weights, np.int64)[:n_live]
     for t in range(tables):
-        np.add.at(H, (rows // block, t, codes[:n_live, t]), 1)
-    return H
+        np.add.at(H, (rows // block, t, codes[:n_live, t]), w)
+    return np.minimum(H, HIST_WEIGHT_MAX) if weights is not None else H
 
 
 def block_scores(HQ: np.ndarray, HK: np.ndarray) -> np.ndarray:
@@ -485,16 +492,16 @@ def sparse_attention_with_segment(Q: np.ndarray, cache: HeadCache, sel: np.ndarr
 
 def annsa(Q: np.ndarray, cache: HeadCache, R: np.ndarray, tables: int, bits: int, block_q: int, block_k: int,
           keep: int, qcodes: Optional[np.ndarray] = None, kcodes: Optional[np.ndarray] = None,
-          sel: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+          sel: Optional[np.ndarray] = None, weighted: bool = False) -> Dict[str, np.ndarray]:
     """AnnSA of one head.  qcodes/kcodes/sel, when given, replace the corresponding
-    stage by decisions taken elsewhere (staged parity)."""
+    stage by decisions taken elsewhere (staged parity).  weighted: key histograms count every slot m times."""
     nq = Q.shape[0]
     if qcodes is None:
         qcodes = lsh_codes(Q, R, tables, bits)
     if kcodes is None:
         kcodes = lsh_codes(cache.K[: cache.L], R, tables, bits) if cache.L else np.zeros((0, tables), np.int64)
     HQ = block_histograms(qcodes, nq, block_q, bits)
-    HK = block_histograms(kcodes, cache.L, block_k, bits)
+    HK = block_histograms(kcodes, cache.L, block_k, bits, weights=cache.m if weighted else None)
     S = block_scores(HQ, HK) if cache.L else np.zeros((HQ.shape[0], 0), np.int64)
     if sel is None:
         sel = topk_lowest_index(S, keep) if cache.L else np.zeros((HQ.shape[0], 0), np.int64)

@@ -703,3 +703,35 @@ def test_hamming_correspondence():
     assert r["matched"][2] and not r["matched"][3] and r["jstar"][2] == j[2]
     je, ce = O.top1_hamming(K, O.HeadCache(64, d), R, T, b)
     assert np.all(je == -1) and np.all(ce == 0)
+
+
+def test_multiplicity_weighted_block_scores():
+    rng = _rng(42)
+    d, L, nq, T, b, bq, bk = 12, 40, 18, 2, 3, 6, 8
+    R = rng.standard_normal((T * b, d))
+    Kc = rng.standard_normal((L, d))
+    m = rng.integers(1, 6, L)
+    Q = rng.standard_normal((nq, d))
+    cache = O.HeadCache(64, d)
+    cache.load(Kc, rng.standard_normal((L, d)), m=m)
+    kc, qc = O.lsh_codes(Kc, R, T, b), O.lsh_codes(Q, R, T, b)
+    HKw = O.block_histograms(kc, L, bk, b, weights=m)
+    # (1) a weighted histogram is the plain histogram of the cache with every slot written out m times ...
+    for blk in range(HKw.shape[0]):
+        rows = np.arange(blk * bk, min((blk + 1) * bk, L))
+        rep = np.repeat(kc[rows], m[rows], axis=0)
+        assert np.array_equal(HKw[blk], O.block_histograms(rep, rep.shape[0], 10 ** 6, b)[0])
+    # (2) ... so the block score counts same-bucket (query, token, table) triples of the uncompressed stream: brute force
+    S = O.block_scores(O.block_histograms(qc, nq, bq, b), HKw)
+    for a in range(S.shape[0]):
+        for blk in range(S.shape[1]):
+            want = sum(int(m[j]) for i in range(a * bq, min((a + 1) * bq, nq)) for j in range(blk * bk, min((blk + 1) * bk, L))
+                       for t in range(T) if qc[i, t] == kc[j, t])
+            assert S[a, blk] == want
+    # (3) all multiplicities one: the plain rule; saturation at the two-digit limit
+    assert np.array_equal(O.block_histograms(kc, L, bk, b, weights=np.ones(L, np.int64)), O.block_histograms(kc, L, bk, b))
+    big = O.block_histograms(kc[:1], 1, bk, b, weights=np.array([10 ** 6]))
+    assert big.max() == O.HIST_WEIGHT_MAX
+    # (4) inside annsa: the selection follows the weighted scores
+    r = O.annsa(Q, cache, R, T, b, bq, bk, 2, weighted=True)
+    assert np.array_equal(r["scores"], S) and np.array_equal(r["sel"], O.topk_lowest_index(S, 2))
