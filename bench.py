@@ -187,7 +187,8 @@ def run_ours(args, cfg):
     H, D, n = cfg.num_heads, cfg.head_dim, cfg.chunk_tokens
     cache = fastar.Cache(H, D, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
                          max_prompt_tokens=cfg.prompt_tokens, max_frames=max(cfg.frames_per_chunk, 1), device=local,
-                         search_bits=args.search_bits, representative=args.representative)
+                         search_bits=args.search_bits, representative=args.representative,
+                         weighted_histograms=args.weighted_histograms)
     for ci in range(cfg.prior_chunks):
         _, K, V = w.chunk(ci)
         cache.update(fastar.to_device(K, device=local), fastar.to_device(V, device=local), cfg.frame_len, 2.0, outputs=False)
@@ -377,7 +378,7 @@ def run_ours(args, cfg):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {16: "bf16", 8: "bf16 (correspondence search on fp8 e4m3 codes)",
                       1: "bf16 (correspondence search on LSH sign bits as fp8 +-1)"}[args.search_bits], "data": "synthetic",
-            "config": {"workload": describe(cfg) + ({16: "", 8: " search=8bit", 1: " search=hamming"}[args.search_bits]) + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
+            "config": {"workload": describe(cfg) + ({16: "", 8: " search=8bit", 1: " search=hamming"}[args.search_bits]) + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else "") + (" weighted-histograms" if args.weighted_histograms else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
                        f"({cache.workspace_bytes >> 20} MiB copy, untimed)", "parallelism": "replicas" if world > 1 else "1 GPU",
                        "cuda_graph": graph is not None},
             "e2e": {"value": e2e_units / e2e_max, "unit": "tok/s", "ms_per_step": e2e_max / args.steps * 1e3,
@@ -410,6 +411,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--search-bits", type=int, default=16, choices=[16, 8, 1],
                     help="TempCache correspondence search on the bf16 keys (16, default) or on their 8-bit codes (8)")
+    ap.add_argument("--weighted-histograms", action="store_true",
+                    help="AnnSA selector option: a cached slot counts m times in its block's bucket histogram")
     ap.add_argument("--representative", default="last", choices=["last", "mean"],
                     help="key a merged slot keeps: the newest key (the paper's choice) or the mean key of its ablation")
     ap.add_argument("--probe", action="store_true",

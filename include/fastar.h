@@ -89,6 +89,11 @@ typedef struct {
                               * mean (m_j K_j + sum k_i)/(m_j + g), summed in fp32 in ascending token order and
                               * rounded to bf16 once, like the value; 1/|k|, the LSH code and the search code of
                               * the slot are then those of the rounded mean. */
+  int32_t weighted_histograms; /* AnnSA selector option, 0 (the paper's rule: every cached key counts once) or 1:
+                              * a slot counts m times in its block's bucket histogram, so that a key block scores
+                              * what it would score with its merged tokens still in place (Lemma 1: a slot stands
+                              * for m identical keys).  A histogram entry saturates at 65535; block scores stay
+                              * exact integers (two 8-bit digits contracted separately). */
 } fastar_cache_desc;
 
 #define FASTAR_REP_LAST_KEY 0

@@ -83,6 +83,9 @@ struct CacheView {
   // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
+  int hist_weighted;               // key histograms count a slot m times (selector option); high digits in hk_hi / scores_hi
+  __nv_bfloat16* hk_hi;            // [H][CAPB][hist_cols]  entry >> 8 (entry & 255 is in hk)
+  float* scores_hi;                // [H][max_qb][CAPB]  HQ . HK_hi^T
   int sign_codes;                  // the search code rows hold LSH sign bits as +-1 (Hamming search) instead of fp8 directions
   int rep_mean;                    // representative key of a merged slot: 0 = newest key, 1 = count-weighted mean key
   float* seg_bias;                 // [max_tokens + 128]  bias of the rows of an un-cached attention segment

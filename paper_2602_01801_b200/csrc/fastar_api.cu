@@ -21,7 +21,7 @@ struct fastar_cache {
   std::vector<ProfRec> recs;
   fastar_cache_desc desc;
   CacheView v;
-  CUtensorMap tm_pool_k, tm_pool_k_half, tm_pool_v, tm_hq, tm_hk, tm_pool_k8;
+  CUtensorMap tm_pool_k, tm_pool_k_half, tm_pool_v, tm_hq, tm_hk, tm_hk_hi, tm_pool_k8;
   PFN_cuTensorMapEncodeTiled_v12000 encode;
   int64_t launches;
   size_t bytes;
@@ -65,6 +65,7 @@ bool desc_valid(const fastar_cache_desc* d) {
   if (d->dtype != FASTAR_BF16 && d->dtype != FASTAR_FP32) return false;
   if (d->search_bits != 0 && d->search_bits != 16 && d->search_bits != 8 && d->search_bits != 1) return false;
   if (d->representative != FASTAR_REP_LAST_KEY && d->representative != FASTAR_REP_MEAN_KEY) return false;
+  if (d->weighted_histograms != 0 && d->weighted_histograms != 1) return false;
   return true;
 }
 
@@ -124,6 +125,9 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.search_bits = (d.search_bits == 8 || d.search_bits == 1) ? 8 : 16;     // both keep a pool of 128-byte code rows
   t.sign_codes = d.search_bits == 1 ? 1 : 0;
   t.rep_mean = d.representative == FASTAR_REP_MEAN_KEY ? 1 : 0;
+  t.hist_weighted = d.weighted_histograms ? 1 : 0;
+  t.hk_hi = t.hist_weighted ? reinterpret_cast<__nv_bfloat16*>(take(H * t.CAPB * t.hist_cols * 2)) : nullptr;
+  t.scores_hi = t.hist_weighted ? reinterpret_cast<float*>(take(H * t.max_qb * t.CAPB * 4)) : nullptr;
   t.pool_k8 = t.search_bits == 8 ? take(H * CAP * 128) : nullptr;
   t.k8_new = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
   t.q8_ca = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
@@ -169,6 +173,14 @@ int make_map_codes(fastar_cache* c, CUtensorMap* m, const void* ptr, uint64_t d1
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+// Block scores of weighted histograms as one number: lo + 256 * hi (exact in fp32 below 2^24).
+__global__ void combine_scores_kernel(const float* __restrict__ lo, const float* __restrict__ hi, int64_t head_stride,
+                                      float* __restrict__ out, int per_head) {
+  const int h = blockIdx.y;
+  for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < per_head; q += gridDim.x * blockDim.x)
+    out[static_cast<int64_t>(h) * per_head + q] = lo[h * head_stride + q] + 256.f * hi[h * head_stride + q];
 }
 
 __global__ void seg_bias_kernel(float* __restrict__ bias, int ns, int total) {
@@ -265,6 +277,9 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
                  static_cast<uint64_t>(v.max_qb) * v.hist_cols * 2, 128);
   if (r == FASTAR_OK)
     r = make_map(c, &c->tm_hk, v.hk, v.hist_cols, v.CAPB, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
+                 static_cast<uint64_t>(v.CAPB) * v.hist_cols * 2, 128);
+  if (r == FASTAR_OK && v.hist_weighted)
+    r = make_map(c, &c->tm_hk_hi, v.hk_hi, v.hist_cols, v.CAPB, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
                  static_cast<uint64_t>(v.CAPB) * v.hist_cols * 2, 128);
   if (r == FASTAR_OK && v.search_bits == 8)
     r = make_map_codes(c, &c->tm_pool_k8, v.pool_k8, PT, static_cast<uint64_t>(v.H) * v.CAPB, PT * 128, v.PT);
@@ -542,6 +557,11 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     ACCK(FASTAR_K_HASH, launch_prep_codes(v, qb, nq, qhs, qts, v.code_new, nullptr, st));
     ACCK(FASTAR_K_QUERY_HIST, launch_query_hist(v, nq, block_q, st));
     ACCK(FASTAR_K_S3_SCORES, launch_s3_scores(v, c->tm_hq, c->tm_hk, nqb, st));
+    if (v.hist_weighted) {                   // the high digits of the weighted histograms, into their own score array
+      CacheView vh = v;
+      vh.scores = v.scores_hi;
+      ACCK(FASTAR_K_S3_SCORES, launch_s3_scores(vh, c->tm_hq, c->tm_hk_hi, nqb, st));
+    }
     ACCK(FASTAR_K_TOPK_BLOCKS, launch_topk_blocks(v, nqb, keep, c->force_sink_blocks, c->force_recent_blocks, st));
     a.sel = v.sel;
     a.nsel = v.nsel;
@@ -558,10 +578,16 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     if (qcode_out && cudaMemcpy2DAsync(qcode_out, static_cast<size_t>(nq) * 4, v.code_new, static_cast<size_t>(v.max_tokens) * 4,
                                        static_cast<size_t>(nq) * 4, v.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return FASTAR_ERR_CUDA;
-    if (scores_out && cudaMemcpy2DAsync(scores_out, static_cast<size_t>(nqb) * v.CAPB * 4, v.scores,
-                                        static_cast<size_t>(v.max_qb) * v.CAPB * 4, static_cast<size_t>(nqb) * v.CAPB * 4, v.H,
-                                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    if (scores_out && v.hist_weighted) {
+      combine_scores_kernel<<<dim3((nqb * v.CAPB + 255) / 256, v.H), 256, 0, st>>>(v.scores, v.scores_hi, static_cast<int64_t>(v.max_qb) * v.CAPB,
+                                                                               scores_out, nqb * v.CAPB);
+      if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
+      c->launches += 1;
+    } else if (scores_out && cudaMemcpy2DAsync(scores_out, static_cast<size_t>(nqb) * v.CAPB * 4, v.scores,
+                                               static_cast<size_t>(v.max_qb) * v.CAPB * 4, static_cast<size_t>(nqb) * v.CAPB * 4, v.H,
+                                               cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
       return FASTAR_ERR_CUDA;
+    }
   }
   CUtensorMap tm_sk, tm_sv;
   if (k_seg) {

@@ -542,13 +542,24 @@ __global__ void __launch_bounds__(256) key_hist_kernel(const CacheView c, int us
   __syncthreads();
   const int s0 = b * c.PT, s1 = min(L, s0 + c.PT);
   const int nb = 1 << c.B;
+  // weighted histograms (a selector option): a slot counts m times, as its merged tokens would; an entry saturates
+  // at 65535 and is stored as two 8-bit digits, each exact in bf16, that S3 contracts separately
   for (int s = s0 + threadIdx.x; s < s1; s += blockDim.x) {
     const uint32_t code = c.kcode[static_cast<int64_t>(h) * c.CAP + s];
-    for (int t = 0; t < c.T; ++t) atomicAdd(&hist[t * nb + ((code >> (8 * t)) & 0xFFu)], 1);
+    const int wgt = c.hist_weighted ? min(c.count[static_cast<int64_t>(h) * c.CAP + s], 65535) : 1;
+    for (int t = 0; t < c.T; ++t) atomicAdd(&hist[t * nb + ((code >> (8 * t)) & 0xFFu)], wgt);
   }
   __syncthreads();
-  __nv_bfloat16* dst = c.hk + (static_cast<int64_t>(h) * c.CAPB + b) * c.hist_cols;
-  for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) dst[q] = __float2bfloat16(static_cast<float>(hist[q]));
+  const int64_t ho = (static_cast<int64_t>(h) * c.CAPB + b) * c.hist_cols;
+  for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) {
+    if (c.hist_weighted) {
+      const int v = min(max(hist[q], 0), 65535);       // max: a sum of saturated weights could wrap
+      c.hk[ho + q] = __float2bfloat16(static_cast<float>(v & 255));
+      c.hk_hi[ho + q] = __float2bfloat16(static_cast<float>(v >> 8));
+    } else {
+      c.hk[ho + q] = __float2bfloat16(static_cast<float>(hist[q]));
+    }
+  }
   if (b == 0 && threadIdx.x == 0 && use_plan) {
     const PlanRec pr = c.plan[h];
     c.len[h] = pr.len_new;
@@ -602,18 +613,27 @@ template <bool ORDERED_UINT>
 __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src, int64_t src_head_stride, int src_row_stride,
                                                    const int32_t* __restrict__ len, int len_div, int n_fixed, int keep,
                                                    int32_t* __restrict__ out, int64_t out_head_stride, int out_row_stride,
-                                                   int out_fill, int32_t* __restrict__ nsel, int force_first, int force_last) {
-  extern __shared__ float vals[];
+                                                   int out_fill, int32_t* __restrict__ nsel, int force_first, int force_last,
+                                                   const float* __restrict__ src_hi) {
+  extern __shared__ uint32_t vals[];     // ranking keys: larger key = better entry
   __shared__ int red[32];
   const int row = blockIdx.x, h = blockIdx.y;
   const int n = len ? (len[h] + len_div - 1) / len_div : n_fixed;
   const int k = min(keep, n);
   const int64_t so = static_cast<int64_t>(h) * src_head_stride + static_cast<int64_t>(row) * src_row_stride;
-  // Forced entries (the first force_first and the last force_last of the row) rank before all others: their scores
-  // are integer counts below 2^23, so adding 2^23 is exact in fp32 and keeps their order among themselves.
+  // Keys are unsigned integers: the order-preserving image of a float (prompt relevance), or a block's collision
+  // count, lo + 256 * hi when the histograms are weighted (both parts are exact integers in fp32, their sum below
+  // 2^26).  Forced entries (the first force_first and the last force_last of the row) get bit 30 and so rank before
+  // all others, in their own score order.
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    float v = ORDERED_UINT ? ordered_to_float(static_cast<const uint32_t*>(src)[so + i]) : static_cast<const float*>(src)[so + i];
-    if (!ORDERED_UINT && (i < force_first || i >= n - force_last)) v += 8388608.f;
+    uint32_t v;
+    if (ORDERED_UINT) {
+      v = static_cast<const uint32_t*>(src)[so + i];
+    } else {
+      v = static_cast<uint32_t>(static_cast<const float*>(src)[so + i]);
+      if (src_hi) v += 256u * static_cast<uint32_t>(src_hi[so + i]);
+      if (i < force_first || i >= n - force_last) v |= 1u << 30;
+    }
     vals[i] = v;
   }
   __syncthreads();
@@ -623,10 +643,10 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
     const int i = i0 + threadIdx.x;
     int take = 0;
     if (i < n) {
-      const float v = vals[i];
+      const uint32_t v = vals[i];
       int rank = 0;
       for (int j = 0; j < n; ++j) {
-        const float u = vals[j];
+        const uint32_t u = vals[j];
         rank += (u > v || (u == v && j < i)) ? 1 : 0;
       }
       take = rank < k ? 1 : 0;
@@ -642,7 +662,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
 int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, int force_recent, cudaStream_t st) {
   topk_kernel<false><<<dim3(nqb, c.H), 256, c.CAPB * 4, st>>>(c.scores, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB, c.len,
                                                             c.PT, 0, keep, c.sel, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB,
-                                                            min(keep, c.CAPB), c.nsel, force_sink, force_recent);
+                                                            min(keep, c.CAPB), c.nsel, force_sink, force_recent,
+                                                            c.hist_weighted ? c.scores_hi : nullptr);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 // ---------------------------------------------------------------------------------------------
@@ -697,7 +718,7 @@ int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaS
   topk_kernel<true><<<dim3(n_frames, c.H), 256, np * 4, st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
                                                              c.max_prompt, nullptr, 1, np, keep, c.selp,
                                                              static_cast<int64_t>(c.max_frames) * c.max_prompt, c.max_prompt,
-                                                             min(keep, np), nullptr, 0, 0);
+                                                             min(keep, np), nullptr, 0, 0, nullptr);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 

@@ -198,10 +198,11 @@ def check_codes(X: np.ndarray, R: np.ndarray, tables: int, bits: int, packed: np
 
 
 def check_selection(qcodes: np.ndarray, kcodes: np.ndarray, nq: int, L: int, block_q: int, block_k: int, bits: int, keep: int,
-                    scores: Optional[np.ndarray], sel: np.ndarray, nsel: int) -> np.ndarray:
-    """S2-S4 from the codes produced elsewhere: integer domain, bit-exact."""
+                    scores: Optional[np.ndarray], sel: np.ndarray, nsel: int, weights: Optional[np.ndarray] = None) -> np.ndarray:
+    """S2-S4 from the codes produced elsewhere: integer domain, bit-exact.  weights = the slots' multiplicities when
+    the cache uses weighted histograms."""
     HQ = O.block_histograms(qcodes, nq, block_q, bits)
-    HK = O.block_histograms(kcodes, L, block_k, bits)
+    HK = O.block_histograms(kcodes, L, block_k, bits, weights=weights)
     S = O.block_scores(HQ, HK) if L else np.zeros((HQ.shape[0], 0), np.int64)
     nkb = S.shape[1]
     if scores is not None:

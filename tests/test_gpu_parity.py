@@ -87,7 +87,8 @@ def gpu_annsa_checked(cache, cfg, w, Q, post, keep, fp32=False, block_q=None):
             qcodes = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, res["qcode"][h].cpu().numpy().view(np.uint32))
             kcodes = P.check_codes(P.bits_to_f64(post["k"][h, : hc.L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][h, : hc.L])
             sel = P.check_selection(qcodes, kcodes, nq, hc.L, block_q, cfg.block, cfg.lsh_bits, keep,
-                                    res["scores"][h].cpu().numpy(), res["sel"][h].cpu().numpy(), int(res["nsel"][h]))
+                                    res["scores"][h].cpu().numpy(), res["sel"][h].cpu().numpy(), int(res["nsel"][h]),
+                                    weights=hc.m if getattr(cache, "weighted_histograms", False) else None)
         else:
             sel = np.tile(np.arange(-(-hc.L // cfg.block)), (-(-nq // block_q), 1))
         want = O.sparse_attention(Q[h].astype(np.float64), hc, sel, block_q, cfg.block)
@@ -700,3 +701,36 @@ def test_hamming_search_on_lsh_sign_bits(d, pt, tables, bits, rep):
                               st2["code"][h, :Lh].astype(np.uint32))
     with pytest.raises(fastar.FastarError):
         cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau, probe=fastar.to_device(Q))
+
+
+@pytest.mark.parametrize("d,pt,big", [(128, 128, False), (64, 64, False), (128, 64, True)])
+def test_multiplicity_weighted_histograms(d, pt, big):
+    # Selector option: a slot counts m times in its block's bucket histogram.  Scores and selections stay bit-exact
+    # (two 8-bit digits contracted separately); with `big`, imported multiplicities of a few thousand push entries past
+    # 255 and one of them past the 65535 saturation.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
+    w = synth.Workload(cfg)
+    cache = fastar.Cache(cfg.num_heads, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
+                         max_tokens=cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64), max_frames=4,
+                         weighted_histograms=True)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(cfg.prior_chunks + 2):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0 if ci < cfg.prior_chunks else cfg.tau)
+    assert post["count"].max() > 1
+    if big:
+        rng = np.random.default_rng(5)
+        cnt = post["count"].copy()
+        for h in range(cfg.num_heads):
+            Lh = int(post["len"][h])
+            cnt[h, :Lh] = rng.integers(1, 3000, Lh)
+            cnt[h, 0] = 70000                                   # past the saturation on its own
+        cache.import_state(post["k"], post["v"], post["len"], cnt, post["stamp"], now=int(post["now"][0]))
+        post = cache.export_state()
+    res = gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+    # the weights matter: the plain rule on the same state selects differently somewhere
+    plain = make_cache(cfg, w)
+    plain.import_state(post["k"], post["v"], post["len"], post["count"], post["stamp"], now=int(post["now"][0]))
+    r2 = plain.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks, debug=True)
+    assert not torch.equal(res["scores"], r2["scores"])
