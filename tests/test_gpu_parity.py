@@ -16,12 +16,13 @@ def _gpu():
     return torch, fastar
 
 
-def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16, representative="last"):
+def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16, representative="last",
+               weighted_histograms=False):
     torch, fastar = _gpu()
     return fastar.Cache(cfg.num_heads, cfg.head_dim, capacity or cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables,
                         cfg.lsh_bits, max_tokens=max_tokens or cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64),
                         max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32, search_bits=search_bits,
-                        representative=representative)
+                        representative=representative, weighted_histograms=weighted_histograms)
 
 
 def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=None, lsh=None):
@@ -611,7 +612,7 @@ def _random_case(seed):
                              tau=float(rng.choice([0.5, 0.9, 0.99])), seed=int(rng.integers(1, 10 ** 6)))
     opts = dict(fp32=bool(rng.random() < 0.3), search_bits=int(rng.choice([16, 8, 1])), probe=bool(rng.random() < 0.4),
                 representative=str(rng.choice(["last", "mean"])), block_q=int(rng.choice([64, 128])),
-                n_sink=int(rng.integers(0, 3)) * 16)
+                n_sink=int(rng.integers(0, 3)) * 16, weighted=bool(rng.random() < 0.3))
     return cfg, opts
 
 
@@ -625,7 +626,8 @@ def test_random_shapes_and_options(seed):
         o["probe"] = False                       # the Hamming search compares keys with keys
     w = synth.Workload(cfg)
     lsh = (w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits)
-    cache = make_cache(cfg, w, o["fp32"], o["n_sink"], search_bits=o["search_bits"], representative=o["representative"])
+    cache = make_cache(cfg, w, o["fp32"], o["n_sink"], search_bits=o["search_bits"], representative=o["representative"],
+                       weighted_histograms=o["weighted"])
     heads = [O.HeadCache(cfg.capacity, cfg.head_dim, o["n_sink"]) for _ in range(cfg.num_heads)]
     for ci in range(cfg.prior_chunks):
         _, K, V = w.chunk(ci)
