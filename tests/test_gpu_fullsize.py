@@ -213,3 +213,56 @@ def test_c1_full_size_probe_update_and_segment_attention_sampled():
         L = int(post["len"][h])
         assert L == int(pre["len"][h]) + int(stats[h, 2]) <= cfg.capacity
         assert int(post["count"][h, :L].sum()) == (cfg.prior_chunks + 1) * n
+
+
+def test_c3_full_size_step_sampled():
+    """The world-model-scale configuration (40 heads, 3 x 3600-token chunk, 64 800 cached keys, capacity 65 536): the
+    CTA-pair similarity kernel and the eviction path at full size.  Two heads are checked: top-1 on sampled tokens,
+    merge bookkeeping and eviction victims in full, block scores and selections in full, attention on sampled
+    query blocks; invariants for all heads."""
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.CONFIGS["c3"]
+    w = synth.Workload(cfg)
+    H, n = cfg.num_heads, cfg.chunk_tokens
+    cache = fastar.Cache(H, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
+                         max_tokens=n, max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk)
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, 2.0, outputs=False)
+    assert cache.status() == 0
+    pre = cache.export_state()
+    assert np.all(pre["len"] == cfg.prior_chunks * n)
+    Q, K, V = w.chunk(cfg.prior_chunks)
+    res = cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau)
+    assert cache.status() == 0
+    post = cache.export_state()
+    match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    rng = np.random.default_rng(3)
+    heads_checked = [0, H - 1]
+    pre_heads = P.oracle_heads_from_export(pre)
+    for h in heads_checked:
+        rows = np.sort(rng.choice(n, 64, replace=False))
+        P.check_update(pre_heads[h], K[h], V[h], cfg.frame_len, cfg.tau, match[h], sim[h], dest[h], stats[h], post, h, rows=rows)
+    assert int(stats[:, 3].sum()) > 0, "the step was meant to evict"
+    for h in range(H):
+        L = int(post["len"][h])
+        assert L == int(pre["len"][h]) + int(stats[h, 2]) <= cfg.capacity
+        assert int(stats[h, 0]) + int(stats[h, 2]) + int(stats[h, 3]) == n
+        assert int(post["count"][h, :L].sum()) == (cfg.prior_chunks + 1) * n - int(stats[h, 4])
+    a = cache.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks, debug=True)
+    assert cache.status() == 0
+    out = a["out"].float().cpu().numpy()
+    R = w.lsh_projection()
+    post_heads = P.oracle_heads_from_export(post)
+    nqb = -(-n // cfg.block)
+    for h in heads_checked:
+        hc = post_heads[h]
+        qcodes = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, a["qcode"][h].cpu().numpy().view(np.uint32))
+        kcodes = P.check_codes(P.bits_to_f64(post["k"][h, : hc.L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][h, : hc.L])
+        sel = P.check_selection(qcodes, kcodes, n, hc.L, cfg.block, cfg.block, cfg.lsh_bits, cfg.keep_blocks,
+                                a["scores"][h].cpu().numpy(), a["sel"][h].cpu().numpy(), int(a["nsel"][h]))
+        want = _oracle_blocks(Q[h], hc, sel, [0, nqb // 2, nqb - 1], cfg.block, cfg.block)
+        for blk, wnt in want.items():
+            rows = slice(blk * cfg.block, min((blk + 1) * cfg.block, n))
+            P.check_attention(out[h][rows], wnt, f"AnnSA c3 head {h} block {blk}")
