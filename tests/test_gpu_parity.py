@@ -736,3 +736,31 @@ def test_multiplicity_weighted_histograms(d, pt, big):
     plain.import_state(post["k"], post["v"], post["len"], post["count"], post["stamp"], now=int(post["now"][0]))
     r2 = plain.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks, debug=True)
     assert not torch.equal(res["scores"], r2["scores"])
+
+
+@pytest.mark.parametrize("d,pt", [(128, 64), (64, 128)])
+def test_long_selection_lists(d, pt):
+    # More than 64 key tiles per query block: the attention producer looks block and page ids up in windows of 32
+    # tiles, two windows at a time, so lists of 70-130 tiles roll the windows over several times (sparse, dense and
+    # with a segment on top).  The similarity kernel scans the same long cache through its own 32-tile windows.
+    torch, fastar = _gpu()
+    prior = 14 if pt == 64 else 28
+    cfg = synth.small_config(head_dim=d, block=pt, capacity=-(-(prior * 600 + 1024) // 128) * 128, keep_blocks=100 if pt == 64 else 70, num_heads=2,
+                             prior_chunks=prior)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w)
+    heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
+    for ci in range(prior + 1):
+        Q, K, V = w.chunk(ci)
+        post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, 2.0 if ci < prior else cfg.tau)
+    nkb = -(-int(post["len"][0]) // pt)
+    assert nkb > cfg.keep_blocks > 64
+    res = gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)                 # sparse: keep_blocks tiles
+    gpu_annsa_checked(cache, cfg, w, Q, post, cache.CAP // cache.PT)                 # dense: every live block
+    dq, dk, dv = (fastar.to_device(x) for x in (Q, K, V))
+    out = cache.annsa_segment(dq, dk, dv, cfg.block, cfg.keep_blocks)["out"].float().cpu().numpy()
+    assert cache.status() == 0
+    for h, hc in enumerate(P.oracle_heads_from_export(post)):
+        sel = res["sel"][h].cpu().numpy()[:, : int(res["nsel"][h])]
+        P.check_attention(out[h], O.sparse_attention_with_segment(Q[h], hc, sel, cfg.block, cfg.block, K[h], V[h]),
+                          f"long list + segment, head {h}")
