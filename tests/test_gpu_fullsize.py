@@ -266,3 +266,49 @@ def test_c3_full_size_step_sampled():
         for blk, wnt in want.items():
             rows = slice(blk * cfg.block, min((blk + 1) * cfg.block, n))
             P.check_attention(out[h][rows], wnt, f"AnnSA c3 head {h} block {blk}")
+
+
+def test_maximum_chunk_and_prompt_sizes():
+    """The size limits of the entry points: an update and an AnnSA call of n = 16 384 tokens (the update's maximum) and an
+    AnnCA call over np = 1024 prompt tokens keeping 1000 of them (eight key tiles gathered per query block).  One head;
+    top-1 on sampled tokens, bookkeeping in full, attention on sampled query blocks."""
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.small_config(num_heads=1, head_dim=64, grid_h=128, grid_w=128, frames_per_chunk=1, clusters=128, capacity=40960,
+                             block=128, keep_blocks=16, prompt_tokens=1024, relevant=8, keep_prompt=1000, prior_chunks=1)
+    w = synth.Workload(cfg)
+    n = cfg.chunk_tokens
+    assert n == 16384
+    cache = fastar.Cache(1, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
+                         max_prompt_tokens=1024, max_frames=1)
+    _, K0, V0 = w.chunk(0)
+    cache.update(fastar.to_device(K0), fastar.to_device(V0), cfg.frame_len, 2.0, outputs=False)
+    pre = cache.export_state()
+    Q, K, V = w.chunk(1)
+    res = cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau)
+    assert cache.status() == 0
+    post = cache.export_state()
+    match, sim, dest, stats = (res[k].cpu().numpy() for k in ("match", "sim", "dest", "stats"))
+    rows = np.sort(np.random.default_rng(4).choice(n, 128, replace=False))
+    pre_heads = P.oracle_heads_from_export(pre)
+    P.check_update(pre_heads[0], K[0], V[0], cfg.frame_len, cfg.tau, match[0], sim[0], dest[0], stats[0], post, 0, rows=rows)
+    assert int(stats[0, 0]) > n // 2
+    a = cache.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks, debug=True)
+    assert cache.status() == 0
+    hc = P.oracle_heads_from_export(post)[0]
+    R = w.lsh_projection()
+    qcodes = P.check_codes(Q[0], R, cfg.lsh_tables, cfg.lsh_bits, a["qcode"][0].cpu().numpy().view(np.uint32))
+    kcodes = P.check_codes(P.bits_to_f64(post["k"][0, : hc.L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][0, : hc.L])
+    sel = P.check_selection(qcodes, kcodes, n, hc.L, cfg.block, cfg.block, cfg.lsh_bits, cfg.keep_blocks,
+                            a["scores"][0].cpu().numpy(), a["sel"][0].cpu().numpy(), int(a["nsel"][0]))
+    out = a["out"].float().cpu().numpy()
+    for blk, wnt in _oracle_blocks(Q[0], hc, sel, [0, 63, 127], cfg.block, cfg.block).items():
+        P.check_attention(out[0][blk * 128:(blk + 1) * 128], wnt, f"AnnSA n=16384 block {blk}")
+    Kp, Vp, _ = w.prompt(1)
+    c = cache.annca(fastar.to_device(Q), fastar.to_device(Kp), fastar.to_device(Vp), cfg.frame_len, cfg.keep_prompt, debug=True)
+    assert cache.status() == 0
+    selp = c["sel"][0].cpu().numpy()
+    P.check_prompt_selection(Q[0], Kp[0], cfg.frame_len, cfg.keep_prompt, selp, c["rel"][0].cpu().numpy())
+    samp = np.sort(np.random.default_rng(5).choice(n, 512, replace=False))
+    want = O.dense_attention(Q[0][samp], Kp[0][selp[0]], Vp[0][selp[0]])
+    P.check_attention(c["out"][0].float().cpu().numpy()[samp], want, "AnnCA np=1024 keep=1000")
