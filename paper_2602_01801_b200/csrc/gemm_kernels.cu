@@ -43,7 +43,9 @@ struct GemmSmem {
 
 // A_TMEM (with A_RES): the resident A tile is moved from shared memory into tensor memory once, so that an MMA
 // reads only its B operand from shared memory; the CTA then owns all 512 TMEM columns (one CTA per SM).
-template <int EPI, bool A_RES, int NST, bool A_TMEM = false>
+// RAW (arg-max epilogue): scores are ranked as plain dot products (query-probe correspondence); a template parameter,
+// not a run-time flag, so that the cosine search compiles to exactly the loop it always had.
+template <int EPI, bool A_RES, int NST, bool A_TMEM = false, bool RAW = false>
 __global__ void __launch_bounds__(kGemmThreads, A_RES ? 2 : 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c,
             const GemmArgs g) {
@@ -243,7 +245,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         int valid_cols = 128;
         if (EPI == EPI_ARGMAX) {
           valid_cols = min(128, L - t * 128);
-          if (!c.raw_dot) {                            // plain dot products need no per-column factor, staging or barrier
+          if (!RAW) {                                  // plain dot products need no per-column factor, staging or barrier
             if (wg == 0) {
               if (tl == 0) rn_next = (t * 128 + r < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r] : 0.f;
               rn_s[rbuf * 128 + r] = rn_next;
@@ -271,7 +273,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           if (EPI == EPI_ARGMAX) {
             // Scores of the chunk, then a tree maximum (no serial compare/select chain); the index is
             // searched only when the chunk holds a new strict maximum, which is rare after the first tiles.
-            if (c.raw_dot) chunk_argmax_plain(v, valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+            if (RAW) chunk_argmax_plain(v, valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
             else chunk_argmax(v, reinterpret_cast<const float4*>(rn_s + rbuf * 128 + cc * 32), valid_cols - cc * 32,
                               t * 128 + cc * 32, best, best_j);
           } else if (EPI == EPI_COLMAX) {
@@ -316,7 +318,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       }
       if (threadIdx.x == 0) { PT_FLUSH("gemm epilogue (wait acc, tmem loads, compute, arrive)", ntl) }
       if (EPI == EPI_ARGMAX && ok && row < g.rows_a && best_j >= 0) {
-        const float sim = c.raw_dot ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        const float sim = RAW ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
                                        static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
         atomicMax(c.best + static_cast<int64_t>(h) * c.max_tokens + row, key);
@@ -332,11 +334,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   }
 }
 
-template <int EPI, bool A_RES, int NST, bool A_TMEM = false>
+template <int EPI, bool A_RES, int NST, bool A_TMEM = false, bool RAW = false>
 static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const CacheView& c, const GemmArgs& g, dim3 grid,
                        cudaStream_t st) {
   using SM = GemmSmem<EPI, A_RES, NST>;
-  auto kern = gemm_kernel<EPI, A_RES, NST, A_TMEM>;
+  auto kern = gemm_kernel<EPI, A_RES, NST, A_TMEM, RAW>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
@@ -368,6 +370,7 @@ struct PairSmem {
   static constexpr int total = bar_off + 256;
 };
 
+template <bool RAW>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 2)
 t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b_half, const CacheView c,
                const GemmArgs g) {
@@ -512,12 +515,12 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       // 1/|k| of the tile's cache keys goes through shared memory; the global load runs one tile ahead so that its
       // latency is not paid between two tiles
       const float* rn_h = c.rnorm + static_cast<int64_t>(h) * c.CAP;
-      float rn_next = (wg == 0 && !c.raw_dot && t0 * 128 + r < L) ? rn_h[t0 * 128 + r] : 0.f;
+      float rn_next = (wg == 0 && !RAW && t0 * 128 + r < L) ? rn_h[t0 * 128 + r] : 0.f;
       PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
         const int buf = tl & 1;
-        if (!c.raw_dot) {                              // plain dot products need no per-column factor, staging or barrier
+        if (!RAW) {                                    // plain dot products need no per-column factor, staging or barrier
           if (wg == 0) {
             rn_s[buf * 128 + r] = rn_next;
             const int slot = (t + 1) * 128 + r;
@@ -545,7 +548,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
-          if (c.raw_dot) chunk_argmax_plain(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
+          if (RAW) chunk_argmax_plain(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
           else chunk_argmax(vv[c2], reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
                             t * 128 + cc * 32, best, best_j);
         }
@@ -553,7 +556,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       if (threadIdx.x == 0 && rank == 0) { PT_FLUSH("t1 pair epilogue (wait acc, tmem loads, compute)", ntl) }
       if (ok && row < g.rows_a && best_j >= 0) {
-        const float sim = c.raw_dot ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        const float sim = RAW ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
                                        static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(best_j));
         atomicMax(c.best + static_cast<int64_t>(h) * c.max_tokens + row, key);
@@ -573,9 +576,10 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   }
 }
 
+template <bool RAW>
 static int launch_t1_pair(const CUtensorMap& tm_a, const CUtensorMap& tm_b_half, const CacheView& c, const GemmArgs& g,
                           dim3 grid, cudaStream_t st) {
-  auto kern = t1_pair_kernel;
+  auto kern = t1_pair_kernel<RAW>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::total) != cudaSuccess)
@@ -633,11 +637,15 @@ int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUte
     if (std::strcmp(force, "ts") == 0) {
       double eff = 0.0;
       const int splits = pick_splits(tiles_single * c.H, slots, max_tiles, &eff);
-      return launch_gemm<EPI_ARGMAX, true, 4, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits), st);
+      return c.raw_dot ? launch_gemm<EPI_ARGMAX, true, 4, true, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits), st)
+                       : launch_gemm<EPI_ARGMAX, true, 4, true, false>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits), st);
     }
   }
-  if (use_pair) return launch_t1_pair(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st);
-  return launch_gemm<EPI_ARGMAX, true, 4>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st);
+  if (use_pair)
+    return c.raw_dot ? launch_t1_pair<true>(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st)
+                     : launch_t1_pair<false>(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st);
+  return c.raw_dot ? launch_gemm<EPI_ARGMAX, true, 4, false, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st)
+                   : launch_gemm<EPI_ARGMAX, true, 4, false, false>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st);
 }
 
 int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,

@@ -237,14 +237,15 @@ int launch_quantize_keys(const CacheView& c, const __nv_bfloat16* x, int n, int6
 // of head h (rows of a dense [H][rows][128] array), per-frame column maximum of score * |q| * |k|.
 struct Search8Args {
   int rows_a;
-  int col_norm;            // arg-max: scores are multiplied by |k_j| before the maximum (query-probe ranking)
   int cols_b;              // COLMAX
   int frame_len;           // COLMAX
   const float* qn;         // COLMAX: |q|, [H][max_tokens]
   const float* kn;         // COLMAX: |k_p|, [H][max_prompt]
 };
 
-template <bool COLMAX>
+// COLNORM (arg-max only): scores are multiplied by |k_j| before the maximum (query-probe ranking).  A template
+// parameter, so that the plain search keeps its short epilogue.
+template <bool COLMAX, bool COLNORM = false>
 __global__ void __launch_bounds__(kThreads, 2)
 search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const CacheView c,
                const Search8Args g) {
@@ -390,7 +391,7 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int t = t0 + tl;
         const int buf = tl & 1;
         const int valid_cols = min(128, L - t * 128);
-        if (!COLMAX && g.col_norm) {
+        if (!COLMAX && COLNORM) {
           // |k_j| of the tile's keys through shared memory: one reciprocal per key, then broadcast reads
           if (wg == 0) {                 // the global load runs one tile ahead of its use
             if (tl == 0) rn_next = (t * 128 + r < L) ? c.rnorm[static_cast<int64_t>(h) * c.CAP + t * 128 + r] : 0.f;
@@ -421,7 +422,7 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
           if (!COLMAX) {
-            if (g.col_norm)
+            if (COLNORM)
               chunk_argmax_scaled(vv[c2], reinterpret_cast<const float4*>(kn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
                                   t * 128 + cc * 32, best, best_j);
             else
@@ -471,6 +472,7 @@ static int configure_search8() {
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(search8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess ||
+        cudaFuncSetAttribute(search8_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess ||
         cudaFuncSetAttribute(search8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess)
       return FASTAR_ERR_CUDA;
     configured = true;
@@ -503,9 +505,9 @@ int launch_t1_similarity_fp8(const CacheView& c, const CUtensorMap& tm_a8, const
   const int row_tiles = (n + 127) / 128;
   Search8Args g{};
   g.rows_a = n;
-  g.col_norm = col_norm ? 1 : 0;
-  search8_kernel<false><<<dim3(row_tiles, c.H, pick_splits8(row_tiles, c.H, c.CAP / 128)), kThreads, Smem::total, st>>>(
-      tm_a8, tm_pool_k8, c, g);
+  const dim3 grid(row_tiles, c.H, pick_splits8(row_tiles, c.H, c.CAP / 128));
+  if (col_norm) search8_kernel<false, true><<<grid, kThreads, Smem::total, st>>>(tm_a8, tm_pool_k8, c, g);
+  else search8_kernel<false, false><<<grid, kThreads, Smem::total, st>>>(tm_a8, tm_pool_k8, c, g);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
