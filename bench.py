@@ -168,6 +168,23 @@ def aggregate(total_units: float, seconds: float, world: int, dist=None, device=
     return total_units, seconds
 
 
+class HeadSlice:
+    """The heads [h0, h1) of a synthetic workload (same data as the full workload's, sliced)."""
+
+    def __init__(self, w, h0, h1):
+        self.w, self.sl = w, slice(h0, h1)
+
+    def chunk(self, ci):
+        return tuple(np.ascontiguousarray(x[self.sl]) for x in self.w.chunk(ci))
+
+    def prompt(self, ci):
+        kp, vp, pos = self.w.prompt(ci)
+        return np.ascontiguousarray(kp[self.sl]), np.ascontiguousarray(vp[self.sl]), pos
+
+    def lsh_projection(self):
+        return self.w.lsh_projection()
+
+
 def run_ours(args, cfg):
     import torch
     from paper_2602_01801_b200 import fastar
@@ -185,6 +202,13 @@ def run_ours(args, cfg):
 
     w = synth.Workload(cfg)
     H, D, n = cfg.num_heads, cfg.head_dim, cfg.chunk_tokens
+    head_lo, head_hi = 0, H
+    if args.shard == "heads" and world > 1:
+        # heads are independent: each rank owns a contiguous range of them, cache and all; no exchange between ranks
+        head_lo, head_hi = fastar.head_shard(H, world, rank)
+        assert head_hi > head_lo, "more ranks than heads"
+        w = HeadSlice(w, head_lo, head_hi)
+        H = head_hi - head_lo
     cache = fastar.Cache(H, D, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
                          max_prompt_tokens=cfg.prompt_tokens, max_frames=max(cfg.frames_per_chunk, 1), device=local,
                          search_bits=args.search_bits, representative=args.representative,
@@ -368,18 +392,22 @@ def run_ours(args, cfg):
             variants["update_query_probe_call_ms"] = timed(
                 lambda: cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq), restore=True)
 
-    total_units, max_seconds = aggregate(float(n * args.steps), seconds, world, dist, dev)
-    e2e_units, e2e_max = aggregate(float(n * args.steps), e2e_s, world, dist, dev)
+    sharded = head_hi - head_lo != cfg.num_heads
+    # replicas: every rank processes n query tokens per step; head shards: its share H_local/H of each of the n tokens
+    rank_units = float(n * args.steps) * (H / cfg.num_heads if sharded else 1.0)
+    total_units, max_seconds = aggregate(rank_units, seconds, world, dist, dev)
+    e2e_units, e2e_max = aggregate(rank_units, e2e_s, world, dist, dev)
     esz = 2
     h2d = (3 * H * n * D + 2 * H * cfg.prompt_tokens * D) * esz
     d2h = 2 * H * n * D * esz
     line = {"metric": "query_tokens_per_s", "value": total_units / max_seconds, "unit": "tok/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": max_seconds / args.steps * 1e3,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": {16: "bf16", 8: "bf16 (correspondence search on fp8 e4m3 codes)",
                       1: "bf16 (correspondence search on LSH sign bits as fp8 +-1)"}[args.search_bits], "data": "synthetic",
             "config": {"workload": describe(cfg) + ({16: "", 8: " search=8bit", 1: " search=hamming"}[args.search_bits]) + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else "") + (" weighted-histograms" if args.weighted_histograms else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
-                       f"({cache.workspace_bytes >> 20} MiB copy, untimed)", "parallelism": "replicas" if world > 1 else "1 GPU",
+                       f"({cache.workspace_bytes >> 20} MiB copy, untimed)", "parallelism": (f"heads sharded over {world} ranks (rank 0: heads {head_lo}..{head_hi - 1})" if sharded
+                                       else "replicas" if world > 1 else "1 GPU"),
                        "cuda_graph": graph is not None},
             "e2e": {"value": e2e_units / e2e_max, "unit": "tok/s", "ms_per_step": e2e_max / args.steps * 1e3,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -419,6 +447,8 @@ def main():
                     help="query-probe correspondence: the update ranks cached keys by the dot product with the chunk's queries")
     ap.add_argument("--variants", action="store_true",
                     help="also time AnnSA with the chunk's own un-cached K/V segment and the query-probe update, each alone")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: independent replicas of the workload (default, weak scaling) or its heads split over the ranks")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a captured CUDA graph")
     ap.add_argument("--mode", default="step", choices=["step", "rollout", "sweep"],
                     help="step = the one-line contract; rollout = c2 long rollout + dense baseline; sweep = c4 roofline sweep")

@@ -608,7 +608,7 @@ static int pick_splits(int ctas_per_split, int slots, int max_splits, double* ef
 // T1.  Two kernels: single CTAs of 128 rows, and CTA pairs (256 rows, half the operand traffic per SM).  The pair
 // kernel is the faster one when both fill their waves equally well (about 10 % at 16k new keys against a 130k-key
 // cache); with few row tiles the padding to an even tile count and the coarser grid can cost more than it gains, so
-// the launcher compares the wave efficiencies.  FASTAR_T1_KERNEL=single|pair in the environment forces one (tests).
+// the launcher compares the wave efficiencies.  FASTAR_T1_KERNEL=single|pair|ts in the environment forces one (tests).
 int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k,
                          const CUtensorMap& tm_pool_k_half, int n, cudaStream_t st) {
   GemmArgs g{};
@@ -628,20 +628,17 @@ int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUte
   const int splits_pair = pick_splits(tiles_pair * c.H, slots, max_tiles, &eff_pair);
   // useful fraction of the pair grid: padded tiles do no useful work
   eff_pair *= static_cast<double>(tiles_single) / tiles_pair;
-  bool use_pair = eff_pair >= 0.96 * eff_single;
+  // ts = the single-CTA kernel with the new keys held in tensor memory (A operand from TMEM)
+  enum { SINGLE, PAIR, TS } kind = eff_pair >= 0.96 * eff_single ? PAIR : SINGLE;
   if (const char* force = std::getenv("FASTAR_T1_KERNEL")) {
-    if (std::strcmp(force, "pair") == 0) use_pair = true;
-    else if (std::strcmp(force, "single") == 0) use_pair = false;
+    if (std::strcmp(force, "pair") == 0) kind = PAIR;
+    else if (std::strcmp(force, "single") == 0) kind = SINGLE;
+    else if (std::strcmp(force, "ts") == 0) kind = TS;
   }
-  if (const char* force = std::getenv("FASTAR_T1_KERNEL")) {
-    if (std::strcmp(force, "ts") == 0) {
-      double eff = 0.0;
-      const int splits = pick_splits(tiles_single * c.H, slots, max_tiles, &eff);
-      return c.raw_dot ? launch_gemm<EPI_ARGMAX, true, 4, true, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits), st)
-                       : launch_gemm<EPI_ARGMAX, true, 4, true, false>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits), st);
-    }
-  }
-  if (use_pair)
+  if (kind == TS)
+    return c.raw_dot ? launch_gemm<EPI_ARGMAX, true, 4, true, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st)
+                     : launch_gemm<EPI_ARGMAX, true, 4, true, false>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st);
+  if (kind == PAIR)
     return c.raw_dot ? launch_t1_pair<true>(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st)
                      : launch_t1_pair<false>(tm_a, tm_pool_k_half, c, g, dim3(tiles_pair, c.H, splits_pair), st);
   return c.raw_dot ? launch_gemm<EPI_ARGMAX, true, 4, false, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st)

@@ -371,6 +371,17 @@ def annca_select_noalloc(q, k_prompt, frame_len: int, keep_tokens: int, sel_out=
 
 
 # ---- helpers for moving synthetic numpy data (bf16-exact float32) onto the device ---------------
+def head_shard(num_heads: int, world: int, rank: int):
+    """Heads [h0, h1) of rank `rank` when `num_heads` independent heads are split over `world` ranks: contiguous ranges,
+    the first `num_heads % world` ranks hold one head more.  Every head's cache, update and attention are independent of
+    the other heads (Eq. 1 is per head), so a head-sharded run needs no exchange between the ranks."""
+    if world < 1 or not 0 <= rank < world or num_heads < 0:
+        raise ValueError("head_shard: need world >= 1, 0 <= rank < world, num_heads >= 0")
+    base, extra = divmod(num_heads, world)
+    h0 = rank * base + min(rank, extra)
+    return h0, h0 + base + (1 if rank < extra else 0)
+
+
 def to_device(x_f32: np.ndarray, fp32: bool = False, device: int = 0):
     import torch
     t = torch.from_numpy(np.ascontiguousarray(x_f32, dtype=np.float32)).to(torch.device("cuda", device))
