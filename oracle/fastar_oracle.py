@@ -40,7 +40,8 @@ torch's scaled_dot_product_attention), brute-force collision counts, hand-made
 eviction and top-k cases, closed-form fixtures under tests/golden/; the 8-bit
 format against torch's float8_e4m3fn, brute-force quantised scores, the probe
 against the soft-max arg-max, the segment against Lemma 1 written with weights,
-the bucket rule and the forced blocks by brute force, the mean key in closed form.
+the bucket rule and the forced blocks by brute force, the mean key in closed form,
+the shared page pool by a hand-made case, conservation, and a smaller cache.
 Parity unpinned: the paper's recall/density/speed-up values (they need the
 paper's models and prompts) — nothing here reproduces them.
 
@@ -51,7 +52,8 @@ lowest token index; unmatched tokens appended in token order; at capacity the
 least-recently-touched slots (smallest (stamp, slot)) are overwritten; sign
 random projections with T tables of b bits; tile score = number of same-bucket
 (query, key, table) triples; fixed budgets with ties to the lower index; AnnCA
-relevance = max over the frame's queries of the scaled dot product.
+relevance = max over the frame's queries of the scaled dot product; a shared
+page pool grants pages in head order and never takes them back (page_grants).
 """
 from __future__ import annotations
 
@@ -266,11 +268,30 @@ def top1_hamming(K_new: np.ndarray, cache: HeadCache, R: np.ndarray, tables: int
     return j, np.where(den > 0, num / np.where(den > 0, den, 1.0), 0.0)
 
 
+def page_grants(lengths, unmatched, free_pages: int, page: int, capacity: int) -> Tuple[List[int], List[int]]:
+    """Shared page pool of a multi-head cache (a memory bound of this implementation, not of the paper: Section 4.1
+    lets the cache grow; heads merge at different rates, so their lengths are ragged and a pool smaller than
+    heads x capacity serves them).  A head holds ceil(L_h / page) pages.  Before an update places its unmatched tokens
+    the heads ask, in head order, for the pages their appends need, ceil(min(capacity, L_h + U_h) / page) minus what they
+    hold, and get min(asked, pages left); pages are never returned.  Returns (pages granted per head, slot limit per
+    head): a head appends up to its limit and replaces its own least recently used slots beyond it."""
+    grants, limits = [], []
+    for L, U in zip(lengths, unmatched):
+        held = -(-int(L) // page)
+        asked = -(-min(capacity, int(L) + int(U)) // page) - held
+        g = min(asked, free_pages)
+        free_pages -= g
+        grants.append(g)
+        limits.append(min(capacity, (held + g) * page))
+    return grants, limits
+
+
 def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_len: int, tau: float,
                      forced: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None,
                      search_bits: int = 16, probe: Optional[np.ndarray] = None,
                      representative: str = "last",
-                     lsh: Optional[Tuple[np.ndarray, int, int]] = None) -> Dict[str, np.ndarray]:
+                     lsh: Optional[Tuple[np.ndarray, int, int]] = None,
+                     slot_limit: Optional[int] = None) -> Dict[str, np.ndarray]:
     """One TempCache update of one head.
 
     representative = "last" keeps the newest matching key in a merged slot (the paper's choice), "mean" the
@@ -279,11 +300,15 @@ def tempcache_update(cache: HeadCache, K_new: np.ndarray, V_new: np.ndarray, fra
     (staged parity: near-ties have several correct answers).  search_bits = 8 runs the
     correspondence search on the 8-bit codes of the keys instead of the keys themselves.
     probe = the chunk's queries [n][d] selects the query-probe correspondence (top1_query_probe).
-    search_bits = 1 with lsh = (R, tables, bits) searches by Hamming distance of the LSH sign bits (top1_hamming)."""
+    search_bits = 1 with lsh = (R, tables, bits) searches by Hamming distance of the LSH sign bits (top1_hamming).
+    slot_limit (page_grants) bounds the slots this call may use below the cache's capacity."""
     K_new = np.asarray(K_new, np.float64)
     V_new = np.asarray(V_new, np.float64)
     n = K_new.shape[0]
     L, CAP, now = cache.L, cache.capacity, cache.now
+    if slot_limit is not None:
+        assert L <= slot_limit <= CAP
+        CAP = slot_limit
 
     # 1. top-1 correspondence against the pre-call cache; 2. threshold
     if forced is None:

@@ -735,3 +735,53 @@ def test_multiplicity_weighted_block_scores():
     # (4) inside annsa: the selection follows the weighted scores
     r = O.annsa(Q, cache, R, T, b, bq, bk, 2, weighted=True)
     assert np.array_equal(r["scores"], S) and np.array_equal(r["sel"], O.topk_lowest_index(S, 2))
+
+
+def test_shared_page_pool_grants():
+    # Hand-made case, page = 4 slots, capacity 16 slots per head, 5 free pages.
+    #   head 0: L = 3 (holds 1 page), U = 6 -> needs ceil(9/4) = 3 pages, asks 2, gets 2, limit 12
+    #   head 1: L = 8 (2 pages),      U = 0 -> asks 0,                               limit 8
+    #   head 2: L = 4 (1 page),       U = 30 -> min(16, 34) = 16 -> 4 pages, asks 3, gets 3, limit 16
+    #   head 3: L = 0 (0 pages),      U = 5 -> asks 2, none left,                    limit 0
+    grants, limits = O.page_grants([3, 8, 4, 0], [6, 0, 30, 5], 5, 4, 16)
+    assert grants == [2, 0, 3, 0] and limits == [12, 8, 16, 0]
+    # enough pages for everyone: every head may grow to min(capacity, L + U) rounded up to whole pages
+    grants, limits = O.page_grants([3, 8, 4, 0], [6, 0, 30, 5], 100, 4, 16)
+    assert grants == [2, 0, 3, 2] and limits == [12, 8, 16, 8]
+    # properties on random inputs: never more than the free pages, nobody above the capacity, a grant never exceeds the
+    # request, and a head behind an unserved request gets nothing (head order is the priority)
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        H, page, cap = int(rng.integers(1, 9)), int(rng.choice([2, 4, 8])), 32
+        L = rng.integers(0, cap + 1, H)
+        U = rng.integers(0, 40, H)
+        free = int(rng.integers(0, 20))
+        grants, limits = O.page_grants(L, U, free, page, cap)
+        asked = [-(-min(cap, int(l) + int(u)) // page) - -(-int(l) // page) for l, u in zip(L, U)]
+        assert sum(grants) <= free and all(0 <= g <= a for g, a in zip(grants, asked))
+        assert all(int(l) <= lim <= cap and lim % page == 0 or lim == cap for l, lim in zip(L, limits))
+        short = [h for h in range(H) if grants[h] < asked[h]]
+        if short:
+            assert sum(grants[: short[0] + 1]) == free and all(g == 0 for g in grants[short[0] + 1:])
+        else:
+            assert limits == [min(cap, -(-(int(l) + int(u)) // page) * page) for l, u in zip(L, U)]
+
+
+def test_slot_limit_is_a_smaller_cache():
+    # An update under a slot limit is the update of a cache whose capacity is that limit (same appends, same victims).
+    rng = np.random.default_rng(11)
+    d, n = 8, 10
+    for limit in (10, 14, 16):
+        K0, V0 = rng.standard_normal((10, d)), rng.standard_normal((10, d))
+        stamps = rng.integers(0, 3, 10)
+        big, small = O.HeadCache(16, d), O.HeadCache(limit, d)
+        for c in (big, small):
+            c.load(O.round_to_bf16(K0), O.round_to_bf16(V0), stamp=stamps, now=3)
+        K = O.round_to_bf16(np.concatenate([K0[:4] * 1.5, rng.standard_normal((n - 4, d))]))
+        V = O.round_to_bf16(rng.standard_normal((n, d)))
+        a = O.tempcache_update(big, K, V, 6, 0.9, slot_limit=limit)
+        b = O.tempcache_update(small, K, V, 6, 0.9)
+        assert np.array_equal(a["dest"], b["dest"]) and a["stats"] == b["stats"] and big.L == small.L
+        for name in ("K", "V", "m", "stamp"):
+            assert np.array_equal(getattr(big, name)[:limit], getattr(small, name))
+        assert a["stats"]["matched"] == 4 and a["stats"]["evicted_slots"] == max(0, 6 - (limit - 10))
