@@ -94,6 +94,16 @@ typedef struct {
                               * what it would score with its merged tokens still in place (Lemma 1: a slot stands
                               * for m identical keys).  A histogram entry saturates at 65535; block scores stay
                               * exact integers (two 8-bit digits contracted separately). */
+  int32_t pool_pages;        /* pages (of page_tokens slots) in the K and V pools, shared by all heads; 0 = one full
+                              * set per head, num_heads * capacity / page_tokens.  A smaller pool serves heads of
+                              * ragged lengths (heads merge at different rates, Section 4.1): a head holds
+                              * ceil(length / page_tokens) pages; an update hands the free pages out in head order,
+                              * each head asking for what its unmatched tokens need up to `capacity`, and never takes
+                              * them back (only a reset does).  A head that got fewer pages than it asked for appends
+                              * up to the end of its pages and replaces its own least recently touched slots beyond
+                              * that; with no slot to replace its update is rejected (FASTAR_ERR_CAPACITY).
+                              * 1 <= pool_pages <= num_heads * capacity / page_tokens.  fastar_cache_import is not
+                              * available on a cache with a shared pool (FASTAR_ERR_UNSUPPORTED_SHAPE). */
 } fastar_cache_desc;
 
 #define FASTAR_REP_LAST_KEY 0

@@ -21,7 +21,8 @@ struct PlanRec {          // per head, written by the planning kernel of an upda
   int32_t len_old;
   int32_t len_new;
   int32_t evicted_tokens;
-  int32_t pad[3];
+  int32_t pages_granted;  // shared page pool: pages this head took from the pool in this update
+  int32_t pad[2];
 };
 
 struct CacheView {
@@ -31,9 +32,13 @@ struct CacheView {
   int32_t max_tokens, max_prompt, max_frames, max_qb;
   int32_t hist_cols;               // T * 2^B rounded up to a multiple of 64
   // persistent state
-  __nv_bfloat16* pool_k;           // [H*CAPB][PT][D]
+  __nv_bfloat16* pool_k;           // [pool_pages][PT][D]
   __nv_bfloat16* pool_v;
   int32_t* page_table;             // [H][CAPB]
+  int32_t pool_pages;              // pages in each pool; H * CAPB = one full set per head (identity page table)
+  int32_t pool_shared;             // 1 = fewer pages than H * CAPB: heads take pages from the pool as they grow
+  int32_t* next_free;              // [1]  shared pool: pages handed out so far (pages are never returned)
+  int32_t* n_match;                // [H]  per-call scratch: tokens of the update matched to a slot
   int32_t* count;                  // [H][CAP]   multiplicity m (0 = dead)
   int32_t* stamp;                  // [H][CAP]
   float* log2m;                    // [H][CAP]   log2(m), -inf for dead slots
@@ -71,7 +76,7 @@ struct CacheView {
   void* stage_in_raw[5];           // raw caller-dtype copies for the host-tensor step (fp32 only)
   // 8-bit quantised correspondence search (search_bits == 8; null otherwise)
   int32_t search_bits;             // 16 or 8
-  uint8_t* pool_k8;                // [H*CAPB][PT][128]  fp8 e4m3 search codes of the cached keys, paged like pool_k
+  uint8_t* pool_k8;                // [pool_pages][PT][128]  fp8 e4m3 search codes of the cached keys, paged like pool_k
   uint8_t* k8_new;                 // [H][max_tokens][128]  codes of the new keys of the update in flight
   // AnnCA's own 8-bit scratch (an AnnCA call may run beside an update on another stream)
   uint8_t* q8_ca;                  // [H][max_tokens][128]  codes of the queries

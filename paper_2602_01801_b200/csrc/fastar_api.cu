@@ -66,6 +66,7 @@ bool desc_valid(const fastar_cache_desc* d) {
   if (d->search_bits != 0 && d->search_bits != 16 && d->search_bits != 8 && d->search_bits != 1) return false;
   if (d->representative != FASTAR_REP_LAST_KEY && d->representative != FASTAR_REP_MEAN_KEY) return false;
   if (d->weighted_histograms != 0 && d->weighted_histograms != 1) return false;
+  if (d->pool_pages < 0 || static_cast<int64_t>(d->pool_pages) > static_cast<int64_t>(d->num_heads) * (d->capacity / d->page_tokens)) return false;
   return true;
 }
 
@@ -86,9 +87,13 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.hist_cols = ((d.lsh_tables << d.lsh_bits) + 63) / 64 * 64;
   const size_t H = t.H, CAP = t.CAP, D = t.D, MT = t.max_tokens, MP = t.max_prompt;
   const size_t esz = d.dtype == FASTAR_FP32 ? 4 : 2;
-  t.pool_k = reinterpret_cast<__nv_bfloat16*>(take(H * CAP * D * 2));
-  t.pool_v = reinterpret_cast<__nv_bfloat16*>(take(H * CAP * D * 2));
+  t.pool_pages = d.pool_pages > 0 ? d.pool_pages : t.H * t.CAPB;
+  t.pool_shared = t.pool_pages < t.H * t.CAPB ? 1 : 0;
+  const size_t pool_rows = static_cast<size_t>(t.pool_pages) * t.PT;
+  t.pool_k = reinterpret_cast<__nv_bfloat16*>(take(pool_rows * D * 2));
+  t.pool_v = reinterpret_cast<__nv_bfloat16*>(take(pool_rows * D * 2));
   t.page_table = reinterpret_cast<int32_t*>(take(H * t.CAPB * 4));
+  t.next_free = reinterpret_cast<int32_t*>(take(4));
   t.count = reinterpret_cast<int32_t*>(take(H * CAP * 4));
   t.stamp = reinterpret_cast<int32_t*>(take(H * CAP * 4));
   t.log2m = reinterpret_cast<float*>(take(H * CAP * 4));
@@ -100,7 +105,8 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.status = reinterpret_cast<int32_t*>(take(4));
   t.lsh = reinterpret_cast<__nv_bfloat16*>(take(32 * D * 2));
   t.best = reinterpret_cast<unsigned long long*>(take(H * MT * 8));
-  t.cnt = reinterpret_cast<int32_t*>(take(H * CAP * 4));            // directly after `best`: one memset clears both
+  t.n_match = reinterpret_cast<int32_t*>(take(H * 4));              // between `best` and `cnt`: one memset clears all three
+  t.cnt = reinterpret_cast<int32_t*>(take(H * CAP * 4));
   t.cur = reinterpret_cast<int32_t*>(take(H * CAP * 4));
   t.segslot = reinterpret_cast<int32_t*>(take(H * MT * 4));
   t.ulist = reinterpret_cast<int32_t*>(take(H * MT * 4));
@@ -128,7 +134,7 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.hist_weighted = d.weighted_histograms ? 1 : 0;
   t.hk_hi = t.hist_weighted ? reinterpret_cast<__nv_bfloat16*>(take(H * t.CAPB * t.hist_cols * 2)) : nullptr;
   t.scores_hi = t.hist_weighted ? reinterpret_cast<float*>(take(H * t.max_qb * t.CAPB * 4)) : nullptr;
-  t.pool_k8 = t.search_bits == 8 ? take(H * CAP * 128) : nullptr;
+  t.pool_k8 = t.search_bits == 8 ? take(pool_rows * 128) : nullptr;
   t.k8_new = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
   t.q8_ca = t.search_bits == 8 ? take(H * MT * 128) : nullptr;
   t.kp8_ca = t.search_bits == 8 ? take(H * MP * 128) : nullptr;
@@ -269,9 +275,9 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
   c->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
   const CacheView& v = c->v;
   const uint64_t D = v.D, PT = v.PT;
-  int r = make_map(c, &c->tm_pool_k, v.pool_k, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, v.PT);
-  if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_k_half, v.pool_k, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, 64);
-  if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_v, v.pool_v, D, PT, static_cast<uint64_t>(v.H) * v.CAPB, D * 2, PT * D * 2, v.PT);
+  int r = make_map(c, &c->tm_pool_k, v.pool_k, D, PT, static_cast<uint64_t>(v.pool_pages), D * 2, PT * D * 2, v.PT);
+  if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_k_half, v.pool_k, D, PT, static_cast<uint64_t>(v.pool_pages), D * 2, PT * D * 2, 64);
+  if (r == FASTAR_OK) r = make_map(c, &c->tm_pool_v, v.pool_v, D, PT, static_cast<uint64_t>(v.pool_pages), D * 2, PT * D * 2, v.PT);
   if (r == FASTAR_OK)
     r = make_map(c, &c->tm_hq, v.hq, v.hist_cols, v.max_qb, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
                  static_cast<uint64_t>(v.max_qb) * v.hist_cols * 2, 128);
@@ -282,7 +288,7 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
     r = make_map(c, &c->tm_hk_hi, v.hk_hi, v.hist_cols, v.CAPB, v.H, static_cast<uint64_t>(v.hist_cols) * 2,
                  static_cast<uint64_t>(v.CAPB) * v.hist_cols * 2, 128);
   if (r == FASTAR_OK && v.search_bits == 8)
-    r = make_map_codes(c, &c->tm_pool_k8, v.pool_k8, PT, static_cast<uint64_t>(v.H) * v.CAPB, PT * 128, v.PT);
+    r = make_map_codes(c, &c->tm_pool_k8, v.pool_k8, PT, static_cast<uint64_t>(v.pool_pages), PT * 128, v.PT);
   if (r == FASTAR_OK &&
       (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
        cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
@@ -332,6 +338,32 @@ int fastar_cache_destroy(fastar_cache_t* c) {
   return FASTAR_OK;
 }
 
+// Shared page pool: the live pages of every head, gathered into the [H][CAP][row_bytes] host layout (rows past a
+// head's pages are zero).  Runs of consecutive pages go in one copy.  Synchronises the stream.
+static bool export_paged(const CacheView& v, const void* pool, size_t row_bytes, void* host, cudaStream_t st) {
+  std::vector<int32_t> pt(static_cast<size_t>(v.H) * v.CAPB), len(v.H);
+  if (cudaMemcpyAsync(pt.data(), v.page_table, pt.size() * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return false;
+  if (cudaMemcpyAsync(len.data(), v.len, len.size() * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return false;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return false;
+  std::memset(host, 0, static_cast<size_t>(v.H) * v.CAP * row_bytes);
+  const size_t page_bytes = static_cast<size_t>(v.PT) * row_bytes;
+  for (int h = 0; h < v.H; ++h) {
+    const int held = (len[h] + v.PT - 1) / v.PT;
+    const int32_t* pth = pt.data() + static_cast<size_t>(h) * v.CAPB;
+    for (int p = 0; p < held;) {
+      int run = 1;
+      while (p + run < held && pth[p + run] == pth[p] + run) ++run;
+      if (pth[p] < 0 || pth[p] + run > v.pool_pages) return false;
+      if (cudaMemcpyAsync(static_cast<uint8_t*>(host) + (static_cast<size_t>(h) * v.CAP + static_cast<size_t>(p) * v.PT) * row_bytes,
+                          static_cast<const uint8_t*>(pool) + static_cast<size_t>(pth[p]) * page_bytes, run * page_bytes,
+                          cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return false;
+      p += run;
+    }
+  }
+  return cudaStreamSynchronize(st) == cudaSuccess;
+}
+
 int fastar_cache_export(fastar_cache_t* c, uint16_t* host_k, uint16_t* host_v, int32_t* count, int32_t* stamp, uint32_t* code,
                         int32_t* len, int32_t* now, void* stream) {
   if (!c) return FASTAR_ERR_INVALID_ARG;
@@ -340,8 +372,13 @@ int fastar_cache_export(fastar_cache_t* c, uint16_t* host_k, uint16_t* host_v, i
   const CacheView& v = c->v;
   const size_t pool = static_cast<size_t>(v.H) * v.CAP * v.D * 2, meta = static_cast<size_t>(v.H) * v.CAP * 4;
   bool ok = true;
-  if (host_k) ok &= cudaMemcpyAsync(host_k, v.pool_k, pool, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (host_v) ok &= cudaMemcpyAsync(host_v, v.pool_v, pool, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (v.pool_shared) {
+    if (host_k) ok &= export_paged(v, v.pool_k, static_cast<size_t>(v.D) * 2, host_k, st);
+    if (host_v) ok &= export_paged(v, v.pool_v, static_cast<size_t>(v.D) * 2, host_v, st);
+  } else {
+    if (host_k) ok &= cudaMemcpyAsync(host_k, v.pool_k, pool, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (host_v) ok &= cudaMemcpyAsync(host_v, v.pool_v, pool, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  }
   if (count) ok &= cudaMemcpyAsync(count, v.count, meta, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (stamp) ok &= cudaMemcpyAsync(stamp, v.stamp, meta, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (code) ok &= cudaMemcpyAsync(code, v.kcode, meta, cudaMemcpyDeviceToHost, st) == cudaSuccess;
@@ -367,7 +404,9 @@ int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_code
   DeviceGuard guard(c->desc.device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool ok = true;
-  if (host_cache_codes)
+  if (host_cache_codes && v.pool_shared)
+    ok &= export_paged(v, v.pool_k8, 128, host_cache_codes, st);
+  else if (host_cache_codes)
     ok &= cudaMemcpyAsync(host_cache_codes, v.pool_k8, static_cast<size_t>(v.H) * v.CAP * 128, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (host_new_codes)
     ok &= cudaMemcpy2DAsync(host_new_codes, static_cast<size_t>(n) * 128, v.k8_new, static_cast<size_t>(v.max_tokens) * 128,
@@ -411,6 +450,7 @@ int fastar_cache_export_annca_codes(fastar_cache_t* c, uint8_t* host_q_codes, ui
 int fastar_cache_import(fastar_cache_t* c, const uint16_t* host_k, const uint16_t* host_v, const int32_t* count,
                         const int32_t* stamp, const int32_t* len, int32_t now, void* stream) {
   if (!c || !host_k || !host_v || !len || now < 0) return FASTAR_ERR_INVALID_ARG;
+  if (c->v.pool_shared) return FASTAR_ERR_UNSUPPORTED_SHAPE;      // a shared pool is filled by updates only
   for (int h = 0; h < c->v.H; ++h)
     if (len[h] < 0 || len[h] > c->v.CAP) return FASTAR_ERR_INVALID_ARG;
   DeviceGuard guard(c->desc.device);

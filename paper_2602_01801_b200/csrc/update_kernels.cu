@@ -239,6 +239,7 @@ int launch_prep_codes_strided(const CacheView& c, const __nv_bfloat16* x, int n,
 __global__ void __launch_bounds__(256) match_count_kernel(const CacheView c, int n, float tau) {
   const int h = blockIdx.y;
   const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
+  int mine = 0;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
     const unsigned long long b = c.best[tb + i];
     int j = -1;
@@ -251,6 +252,12 @@ __global__ void __launch_bounds__(256) match_count_kernel(const CacheView c, int
     c.match[tb + i] = matched ? j : -1;
     c.sim[tb + i] = s;
     if (matched) atomicAdd(c.cnt + static_cast<int64_t>(h) * c.CAP + j, 1);
+    mine += matched ? 1 : 0;
+  }
+  if (c.pool_shared) {                       // the planner of every head needs every head's number of unmatched tokens
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+    if ((threadIdx.x & 31) == 0 && mine > 0) atomicAdd(c.n_match + h, mine);
   }
 }
 
@@ -321,7 +328,33 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
     u_run += tot;
   }
   const int U = u_run;
-  const int A = min(U, c.CAP - L);
+  // Slot limit of this head.  Shared page pool: the free pages go to the heads in head order, each asking for what its
+  // unmatched tokens need up to the capacity.  Every head's planner repeats the same short scan over the heads before
+  // it (lengths, matched counts and the pool's fill are only written by the kernels that follow), so the CTAs need no
+  // exchange.  A head's pages are never returned, so a head holds ceil(length / page) of them.
+  __shared__ int s_limit, s_grant, s_base;
+  if (tid == 0) {
+    int limit = c.CAP, grant = 0, base = 0;
+    if (c.pool_shared) {
+      int next = *c.next_free;
+      for (int g = 0; g <= h; ++g) {
+        const int Lg = c.len[g], Ug = n - c.n_match[g];
+        const int held = (Lg + c.PT - 1) / c.PT;
+        const int asked = (min(c.CAP, Lg + Ug) + c.PT - 1) / c.PT - held;
+        const int got = min(asked, c.pool_pages - next);
+        if (g == h) { grant = got; base = next; limit = min(c.CAP, (held + got) * c.PT); }
+        next += got;
+      }
+    }
+    s_limit = limit; s_grant = grant; s_base = base;
+  }
+  __syncthreads();
+  const int limit = s_limit, grant = s_grant;
+  if (grant > 0) {
+    const int held = (L + c.PT - 1) / c.PT;
+    for (int p = tid; p < grant; p += blockDim.x) c.page_table[static_cast<int64_t>(h) * c.CAPB + held + p] = s_base + p;
+  }
+  const int A = min(U, limit - L);
   const int E = U - A;
   int ok = 1;
   // Eviction.  evictable = live, past the sink prefix, stamp < now, not touched by this update (cnt == 0); its key
@@ -448,7 +481,8 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
     pr.len_old = L;
     pr.len_new = ok ? L + A : L;
     pr.evicted_tokens = evicted_tokens;
-    pr.pad[0] = pr.pad[1] = pr.pad[2] = 0;
+    pr.pages_granted = grant;
+    pr.pad[0] = pr.pad[1] = 0;
     c.plan[h] = pr;
   }
 }
@@ -563,6 +597,7 @@ __global__ void __launch_bounds__(256) key_hist_kernel(const CacheView c, int us
   if (b == 0 && threadIdx.x == 0 && use_plan) {
     const PlanRec pr = c.plan[h];
     c.len[h] = pr.len_new;
+    if (c.pool_shared && pr.pages_granted > 0) atomicAdd(c.next_free, pr.pages_granted);
     if (stats_out) {
       fastar_update_stats s;
       s.matched = pr.n_matched;
@@ -734,17 +769,19 @@ __global__ void reset_meta_kernel(const CacheView c) {
     c.log2m[q] = -INFINITY;
     c.rnorm[q] = 0.f;
     c.kcode[q] = 0;
-    if (q < static_cast<int64_t>(c.H) * c.CAPB) c.page_table[q] = static_cast<int32_t>(q);
+    // one full set of pages per head: the identity; a shared pool: no page handed out yet (entries of pages a head
+    // does not hold stay at page 0, a valid address that only masked-out slots ever read)
+    if (q < static_cast<int64_t>(c.H) * c.CAPB) c.page_table[q] = c.pool_shared ? 0 : static_cast<int32_t>(q);
     if (q < c.H) c.len[q] = 0;
-    if (q == 0) { *c.now = 0; *c.status = 0; }
+    if (q == 0) { *c.now = 0; *c.status = 0; *c.next_free = 0; }
   }
 }
 int launch_reset(const CacheView& c, cudaStream_t st) {
-  const size_t pool = static_cast<size_t>(c.H) * c.CAP * c.D * sizeof(__nv_bfloat16);
+  const size_t pool = static_cast<size_t>(c.pool_pages) * c.PT * c.D * sizeof(__nv_bfloat16);
   if (cudaMemsetAsync(c.pool_k, 0, pool, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   if (cudaMemsetAsync(c.pool_v, 0, pool, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   if (cudaMemsetAsync(c.hk, 0, static_cast<size_t>(c.H) * c.CAPB * c.hist_cols * 2, st) != cudaSuccess) return FASTAR_ERR_CUDA;
-  if (c.pool_k8 && cudaMemsetAsync(c.pool_k8, 0, static_cast<size_t>(c.H) * c.CAP * 128, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (c.pool_k8 && cudaMemsetAsync(c.pool_k8, 0, static_cast<size_t>(c.pool_pages) * c.PT * 128, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   reset_meta_kernel<<<296, 256, 0, st>>>(c);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }

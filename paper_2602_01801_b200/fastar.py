@@ -26,7 +26,7 @@ class FastarError(RuntimeError):
 class CacheDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("num_heads", "head_dim", "capacity", "page_tokens", "n_sink", "lsh_tables",
                                          "lsh_bits", "max_tokens", "max_prompt_tokens", "max_frames", "dtype", "device",
-                                         "search_bits", "representative", "weighted_histograms")]
+                                         "search_bits", "representative", "weighted_histograms", "pool_pages")]
 
 
 class UpdateStats(C.Structure):
@@ -109,7 +109,7 @@ class Cache:
     def __init__(self, num_heads: int, head_dim: int, capacity: int, page_tokens: int, lsh_proj: np.ndarray,
                  lsh_tables: int = 4, lsh_bits: int = 8, max_tokens: int = 4096, max_prompt_tokens: int = 512,
                  max_frames: int = 8, n_sink: int = 0, fp32: bool = False, device: int = 0, search_bits: int = 16,
-                 representative: str = "last", weighted_histograms: bool = False):
+                 representative: str = "last", weighted_histograms: bool = False, pool_pages: int = 0):
         import torch
         self.lib = load_library()
         self.torch = torch
@@ -119,7 +119,8 @@ class Cache:
         self.dtype = torch.float32 if fp32 else torch.bfloat16
         self.desc = CacheDesc(num_heads, head_dim, capacity, page_tokens, n_sink, lsh_tables, lsh_bits, max_tokens,
                               max_prompt_tokens, max_frames, FP32 if fp32 else BF16, device, search_bits,
-                              {"last": 0, "mean": 1}[representative], 1 if weighted_histograms else 0)
+                              {"last": 0, "mean": 1}[representative], 1 if weighted_histograms else 0, pool_pages)
+        self.pool_pages = pool_pages             # 0 = one full set of pages per head; else a pool shared by the heads
         self.weighted_histograms = weighted_histograms
         self.search_bits = search_bits           # 16 = bf16 keys, 8 = fp8 direction codes, 1 = LSH sign bits (Hamming)
         self.representative = representative

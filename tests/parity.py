@@ -47,7 +47,7 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
                  sim: np.ndarray, dest: np.ndarray, stats: np.ndarray, post: Dict[str, np.ndarray], h: int,
                  rows: Optional[np.ndarray] = None, codes: Optional[Tuple[np.ndarray, np.ndarray]] = None,
                  probe: Optional[np.ndarray] = None, representative: str = "last",
-                 probe_codes: Optional[np.ndarray] = None, hamming=None) -> O.HeadCache:
+                 probe_codes: Optional[np.ndarray] = None, hamming=None, slot_limit: Optional[int] = None) -> O.HeadCache:
     """Stages T1-T4 for one head.  `pre` is the oracle cache before the call (left untouched), `post` the
     exported state after it.  `rows` restricts the T1 brute force to a sample of tokens (full size cases).
     `codes` = (codes of the new keys [n][128], codes of the pre-call cache [>= L][128]) as the GPU computed them
@@ -123,7 +123,7 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
     # T3/T4: teacher-forced merge
     ref = pre.copy()
     res = O.tempcache_update(ref, K64, V64, frame_len, tau, forced=(np.where(matched, match, 0), sim.astype(np.float64), matched),
-                             representative=representative)
+                             representative=representative, slot_limit=slot_limit)
     st = res["stats"]
     assert np.array_equal(dest, res["dest"]), "T3/T4: destination slots"
     assert int(post["len"][h]) == ref.L == st["length"], "T4: length"

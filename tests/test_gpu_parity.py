@@ -17,12 +17,12 @@ def _gpu():
 
 
 def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16, representative="last",
-               weighted_histograms=False):
+               weighted_histograms=False, pool_pages=0):
     torch, fastar = _gpu()
     return fastar.Cache(cfg.num_heads, cfg.head_dim, capacity or cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables,
                         cfg.lsh_bits, max_tokens=max_tokens or cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64),
                         max_frames=max(cfg.frames_per_chunk, 4), n_sink=n_sink, fp32=fp32, search_bits=search_bits,
-                        representative=representative, weighted_histograms=weighted_histograms)
+                        representative=representative, weighted_histograms=weighted_histograms, pool_pages=pool_pages)
 
 
 def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=None, lsh=None):
@@ -41,6 +41,14 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
     synced = P.oracle_heads_from_export(post, heads[0].n_sink)
     post_codes = cache.export_search_codes(K.shape[1]) if (q8 or sign) else None
     probe_codes = cache.export_probe_codes(K.shape[1]) if (q8 and probe is not None) else None
+    limits = [None] * K.shape[0]
+    if cache.pool_pages:
+        # shared page pool: the oracle hands out the free pages from the lengths it holds and the numbers of unmatched
+        # tokens (the match decisions are the GPU's, checked below; the grant rule is the oracle's)
+        used = getattr(cache, "pages_used", 0)
+        grants, limits = O.page_grants([hc.L for hc in heads], [(match[h] < 0).sum() for h in range(K.shape[0])],
+                                       cache.pool_pages - used, cache.PT, cache.CAP)
+        cache.pages_used = used + sum(grants)
     for h in range(K.shape[0]):
         codes = None
         hamming = None
@@ -65,7 +73,8 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
             codes = (post_codes["new"][h], pre_codes[h])
         ref = P.check_update(heads[h], K[h], V[h], frame_len, tau, match[h], sim[h], dest[h], stats[h], post, h, codes=codes,
                              probe=None if probe is None else probe[h], representative=cache.representative,
-                             probe_codes=probe_codes[h] if (q8 and probe is not None) else None, hamming=hamming)
+                             probe_codes=probe_codes[h] if (q8 and probe is not None) else None, hamming=hamming,
+                             slot_limit=limits[h])
         # teacher forcing across steps: the next step starts from the state the GPU holds (its merged values
         # may sit one bf16 ulp away from the oracle's), the oracle's counters are carried over
         synced[h].evicted_tokens, synced[h].inserted_tokens = ref.evicted_tokens, ref.inserted_tokens
@@ -339,6 +348,54 @@ def test_eviction_and_sink_and_capacity_error():
     assert int(res["stats"][0, 6]) == 0
     for key in ("k", "v", "count", "stamp", "len"):
         assert np.array_equal(before[key], after[key]), key
+
+
+@pytest.mark.parametrize("d,page,search_bits", [(128, 128, 16), (64, 64, 16), (128, 128, 8)])
+def test_shared_page_pool_across_ragged_heads(d, page, search_bits):
+    # (Numbers for 64-slot pages; with 128-slot pages every token count doubles.)
+    # Four heads, 16 pages of 64 slots each would be a full set (64 pages); the pool has 30.  Update 1 appends 300
+    # tokens per head (5 pages each, 20 used).  Update 2: head 0 merges everything, head 1 is all new (asks 5, gets 5),
+    # head 2 half new (asks 3, gets 3), head 3 all new (asks 5, gets the last 2: appends up to 448 slots and replaces
+    # its own oldest slots beyond).  Update 3 finds the pool empty: head 0, all new now, fills its fifth page and evicts.
+    # Every update is checked stage by stage against the oracle under the oracle's own page grants; AnnSA then reads
+    # the pools through a page table that is no longer the identity.
+    torch, fastar = _gpu()
+    H, s = 4, page // 64
+    n = 300 * s
+    cfg = synth.small_config(num_heads=H, head_dim=d, block=page, capacity=16 * page, keep_blocks=4, prior_chunks=0)
+    w = synth.Workload(cfg)
+    cache = make_cache(cfg, w, max_tokens=n, search_bits=search_bits, pool_pages=30)
+    heads = [O.HeadCache(cfg.capacity, d) for _ in range(H)]
+    rng = np.random.default_rng(77)
+    fresh = lambda: synth.round_bf16(rng.standard_normal((n, d)).astype(np.float32))
+    K1 = np.stack([fresh() for _ in range(H)])
+    V = lambda: np.stack([fresh() for _ in range(H)])
+    again = lambda Kh, cnt: synth.round_bf16(1.25 * Kh[rng.permutation(n)[:cnt]])      # same directions: these merge
+    post = gpu_update_checked(cache, heads, K1, V(), n // 2, 2.0)
+    assert [hc.L for hc in heads] == [300 * s] * 4 and cache.pages_used == 20
+    K2 = np.stack([again(K1[0], n), fresh(), np.concatenate([again(K1[2], n // 2), fresh()[: n - n // 2]]), fresh()])
+    post = gpu_update_checked(cache, heads, K2, V(), n // 2, 0.9)
+    assert [hc.L for hc in heads] == [300 * s, 600 * s, 450 * s, 448 * s] and cache.pages_used == 30
+    assert heads[3].evicted_tokens == 152 * s and heads[1].evicted_tokens == 0
+    K3 = np.stack([fresh(), again(K2[1], n), again(K1[2], n), again(K2[3], n)])
+    post = gpu_update_checked(cache, heads, K3, V(), n // 2, 0.9)
+    assert [hc.L for hc in heads] == [320 * s, 600 * s, 450 * s, 448 * s] and cache.pages_used == 30
+    assert heads[0].evicted_tokens == 560 * s              # 280 slots, each holding two merged tokens since update 2
+    Q = np.stack([fresh() for _ in range(H)])
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.capacity // page)                     # dense over the paged pools
+    # a full-size pool is the cache without the option
+    with pytest.raises(fastar.FastarError):
+        make_cache(cfg, w, max_tokens=n, pool_pages=65)
+    # import needs one full set of pages per head
+    st = cache.export_state()
+    with pytest.raises(fastar.FastarError):
+        cache.import_state(st["k"], st["v"], st["len"], st["count"], st["stamp"], int(st["now"][0]))
+    # a head that gets no page and has no slot to replace: its update is rejected, the others go through
+    cache2 = make_cache(cfg, w, max_tokens=n, pool_pages=12)
+    res = cache2.update(fastar.to_device(K1), fastar.to_device(V()), n // 2, 2.0)
+    assert cache2.status() == fastar.ERR_CAPACITY
+    assert res["stats"][:, 6].tolist() == [1, 1, 0, 0] and cache2.export_state(kv=False)["len"].tolist() == [n, n, 0, 0]
 
 
 def test_empty_cache_and_selector_bypass():
