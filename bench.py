@@ -212,7 +212,7 @@ def run_ours(args, cfg):
     cache = fastar.Cache(H, D, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
                          max_prompt_tokens=cfg.prompt_tokens, max_frames=max(cfg.frames_per_chunk, 1), device=local,
                          search_bits=args.search_bits, representative=args.representative,
-                         weighted_histograms=args.weighted_histograms)
+                         weighted_histograms=args.weighted_histograms, pool_pages=args.pool_pages)
     for ci in range(cfg.prior_chunks):
         _, K, V = w.chunk(ci)
         cache.update(fastar.to_device(K, device=local), fastar.to_device(V, device=local), cfg.frame_len, 2.0, outputs=False)
@@ -405,7 +405,7 @@ def run_ours(args, cfg):
             "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": {16: "bf16", 8: "bf16 (correspondence search on fp8 e4m3 codes)",
                       1: "bf16 (correspondence search on LSH sign bits as fp8 +-1)"}[args.search_bits], "data": "synthetic",
-            "config": {"workload": describe(cfg) + ({16: "", 8: " search=8bit", 1: " search=hamming"}[args.search_bits]) + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else "") + (" weighted-histograms" if args.weighted_histograms else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
+            "config": {"workload": describe(cfg) + ({16: "", 8: " search=8bit", 1: " search=hamming"}[args.search_bits]) + (" correspondence=query-probe" if args.probe else "") + (" representative=mean-key" if args.representative == "mean" else "") + (" weighted-histograms" if args.weighted_histograms else "") + (f" pool-pages={args.pool_pages}" if args.pool_pages else ""), "l2": "flushed between timed steps by restoring the cache snapshot "
                        f"({cache.workspace_bytes >> 20} MiB copy, untimed)", "parallelism": (f"heads sharded over {world} ranks (rank 0: heads {head_lo}..{head_hi - 1})" if sharded
                                        else "replicas" if world > 1 else "1 GPU"),
                        "cuda_graph": graph is not None},
@@ -449,6 +449,8 @@ def main():
                     help="also time AnnSA with the chunk's own un-cached K/V segment and the query-probe update, each alone")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
                     help="N > 1: independent replicas of the workload (default, weak scaling) or its heads split over the ranks")
+    ap.add_argument("--pool-pages", type=int, default=0,
+                    help="pages in the K/V pools shared by all heads (0 = one full set per head)")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a captured CUDA graph")
     ap.add_argument("--mode", default="step", choices=["step", "rollout", "sweep"],
                     help="step = the one-line contract; rollout = c2 long rollout + dense baseline; sweep = c4 roofline sweep")
