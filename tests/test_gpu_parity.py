@@ -670,6 +670,9 @@ def _random_case(seed):
     opts = dict(fp32=bool(rng.random() < 0.3), search_bits=int(rng.choice([16, 8, 1])), probe=bool(rng.random() < 0.4),
                 representative=str(rng.choice(["last", "mean"])), block_q=int(rng.choice([64, 128])),
                 n_sink=int(rng.integers(0, 3)) * 16, weighted=bool(rng.random() < 0.3))
+    # sometimes a page pool shared by the heads, 70 % or 85 % of a full set: the last heads run out of pages first
+    pool = float(rng.choice([0.0, 0.0, 0.7, 0.85]))
+    opts["pool_pages"] = max(cfg.num_heads, int(pool * cfg.num_heads * (cap // pt))) if pool else 0
     return cfg, opts
 
 
@@ -684,7 +687,7 @@ def test_random_shapes_and_options(seed):
     w = synth.Workload(cfg)
     lsh = (w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits)
     cache = make_cache(cfg, w, o["fp32"], o["n_sink"], search_bits=o["search_bits"], representative=o["representative"],
-                       weighted_histograms=o["weighted"])
+                       weighted_histograms=o["weighted"], pool_pages=o["pool_pages"])
     heads = [O.HeadCache(cfg.capacity, cfg.head_dim, o["n_sink"]) for _ in range(cfg.num_heads)]
     for ci in range(cfg.prior_chunks):
         _, K, V = w.chunk(ci)
