@@ -44,7 +44,8 @@ def run_rollout(args):
     H, D, n = cfg.num_heads, cfg.head_dim, cfg.chunk_tokens
     R = w.lsh_projection()
     cache = fastar.Cache(H, D, cfg.capacity, cfg.block, R, cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
-                         max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk)
+                         max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk,
+                         pool_pages=getattr(args, "pool_pages", 0))
     dense_cap = -(-chunks * n // 128) * 128
     dense = None
     if not args.no_dense:
