@@ -417,7 +417,9 @@ def run_ours(args, cfg):
         line["variants"] = variants
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            heads = 2 if cfg.num_heads >= 2 else 1
+            # about 10-15 s of oracle time: its cost per head is close to 1.2e-8 s x new tokens x cached keys
+            per_head = 1.2e-8 * n * max(cfg.prior_chunks * n, 1)
+            heads = int(max(1, min(cfg.num_heads, round(12.0 / per_head))))
             times, cores = oracle_step_sample(cfg, heads, 1)
             per_full = float(np.mean(times)) * cfg.num_heads / heads
             line["cpu_baseline"] = {"value": n / per_full, "unit": "tok/s", "cores": cores, "kind": "oracle",
