@@ -117,7 +117,7 @@ typedef struct {
   int32_t evicted_tokens;    /* sum of the victims' multiplicities */
   int32_t length;            /* live slots after the update */
   int32_t ok;                /* 1 = applied, 0 = rejected (FASTAR_ERR_CAPACITY), cache unchanged */
-  int32_t reserved;
+  int32_t pages_granted;     /* shared page pool: pages this head took from the pool in this update (else 0) */
 } fastar_update_stats;
 
 /* Bytes of device workspace a cache with this description needs (0 on an invalid description).
@@ -141,7 +141,9 @@ int fastar_cache_destroy(fastar_cache_t* cache);
 
 /* Copy the cache state to host buffers (any pointer may be NULL to skip it) and synchronise
  * the stream.  host_k/host_v: bf16 bit patterns [H][CAP][d]; count (multiplicity m), stamp,
- * code (LSH code, 8 bits per table, table t in byte t): [H][CAP]; len: [H]; now: [1]. */
+ * code (LSH code, 8 bits per table, table t in byte t): [H][CAP]; len: [H]; now: [1].
+ * The layout is logical (slot s of head h at [h][s]) whatever the page table: with a shared page pool
+ * (pool_pages) the live pages of every head are gathered and the rows past them are zero. */
 int fastar_cache_export(fastar_cache_t* cache, uint16_t* host_k, uint16_t* host_v, int32_t* count,
                         int32_t* stamp, uint32_t* code, int32_t* len, int32_t* now, void* stream);
 

@@ -607,7 +607,7 @@ __global__ void __launch_bounds__(256) key_hist_kernel(const CacheView c, int us
       s.evicted_tokens = pr.evicted_tokens;
       s.length = pr.len_new;
       s.ok = pr.ok;
-      s.reserved = 0;
+      s.pages_granted = pr.pages_granted;
       stats_out[h] = s;
     }
     if (h == 0 && advance_clock) *c.now = *c.now + 1;

@@ -31,7 +31,7 @@ class CacheDesc(C.Structure):
 
 class UpdateStats(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("matched", "touched", "appended", "evicted_slots", "evicted_tokens", "length",
-                                         "ok", "reserved")]
+                                         "ok", "pages_granted")]
 
 
 # name -> (restype, argtypes); mirrors include/fastar.h one to one

@@ -49,6 +49,9 @@ def gpu_update_checked(cache, heads, K, V, frame_len, tau, fp32=False, probe=Non
         grants, limits = O.page_grants([hc.L for hc in heads], [(match[h] < 0).sum() for h in range(K.shape[0])],
                                        cache.pool_pages - used, cache.PT, cache.CAP)
         cache.pages_used = used + sum(grants)
+        assert stats[:, 7].tolist() == grants, "pages granted per head"
+    else:
+        assert not stats[:, 7].any()
     for h in range(K.shape[0]):
         codes = None
         hamming = None
@@ -395,6 +398,7 @@ def test_shared_page_pool_across_ragged_heads(d, page, search_bits):
     cache2 = make_cache(cfg, w, max_tokens=n, pool_pages=12)
     res = cache2.update(fastar.to_device(K1), fastar.to_device(V()), n // 2, 2.0)
     assert cache2.status() == fastar.ERR_CAPACITY
+    assert res["stats"][:, 7].tolist() == [5, 5, 2, 0]          # a rejected head keeps the pages it was granted
     assert res["stats"][:, 6].tolist() == [1, 1, 0, 0] and cache2.export_state(kv=False)["len"].tolist() == [n, n, 0, 0]
 
 
