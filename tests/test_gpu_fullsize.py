@@ -22,7 +22,8 @@ def _oracle_blocks(Q, hc, sel, blocks, bq, bk):
     return out
 
 
-def test_c1_full_size_step_sampled():
+@pytest.mark.parametrize("pool_pages", [0, 2700])      # 2700 of 3072 pages shared by the heads: a non-identity page table
+def test_c1_full_size_step_sampled(pool_pages):
     import torch
     from paper_2602_01801_b200 import fastar
 
@@ -30,7 +31,8 @@ def test_c1_full_size_step_sampled():
     w = synth.Workload(cfg)
     H, n = cfg.num_heads, cfg.chunk_tokens
     cache = fastar.Cache(H, cfg.head_dim, cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables, cfg.lsh_bits,
-                         max_tokens=n, max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk)
+                         max_tokens=n, max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk,
+                         pool_pages=pool_pages)
     for ci in range(cfg.prior_chunks):
         _, K, V = w.chunk(ci)
         cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, 2.0, outputs=False)
