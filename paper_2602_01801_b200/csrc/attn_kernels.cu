@@ -537,18 +537,14 @@ static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
                        const CUtensorMap& tsv, const CacheView& c, const AttnArgs& a, dim3 grid, cudaStream_t st) {
   using SM = AttnSmem<D, BKT>;
   auto kern = attn_kernel<D, BKT, GATHER, SEG>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
-      return FASTAR_ERR_CUDA;
-    configured = true;
-  }
+  const int cfg = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), SM::total);
+  if (cfg != FASTAR_OK) return cfg;
   kern<<<grid, kAttnThreads, SM::total, st>>>(tq, tk, tv, tsk, tsv, c, a);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
 // tm_seg_k / tm_seg_v: maps of the un-cached segment (box {64, page_tokens, 1}); nullptr when a.seg_tiles == 0.
-int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
+int launch_attention_paged_v1(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
                            const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
                            const AttnArgs& a, cudaStream_t st) {
   if (a.seg_tiles > 0 && (!tm_seg_k || !tm_seg_v || !a.seg_bias)) return FASTAR_ERR_INVALID_ARG;

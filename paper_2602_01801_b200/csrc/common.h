@@ -105,6 +105,10 @@ inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int
   return (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D;
 }
 
+// Raises a kernel's dynamic shared-memory limit once per (kernel, device); safe from several host threads.
+// The attribute is per device, so a process that drives several GPUs sets it on each (fastar_api.cu).
+int ensure_dynamic_smem(const void* kernel, int bytes);
+
 // ---- launchers implemented in the .cu files (all asynchronous on `st`) -----------------------
 // Each returns the number of kernels it launched (for the launch counter) or a negative status.
 
@@ -156,6 +160,9 @@ struct AttnArgs {
 int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
                            const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
                            const AttnArgs& a, cudaStream_t st);
+int launch_attention_paged_v1(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
+                           const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
+                           const AttnArgs& a, cudaStream_t st);   // TEMP
 int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st);
 
 // update_kernels.cu

@@ -3,8 +3,12 @@
 #include <cudaTypedefs.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "common.h"
@@ -39,6 +43,21 @@ struct fastar_cache {
     if (copy) cudaStreamDestroy(copy);
   }
 };
+
+namespace fastar {
+int ensure_dynamic_smem(const void* kernel, int bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, int> done;      // (kernel, device ordinal) -> bytes already granted
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FASTAR_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  int& have = done[std::make_pair(kernel, dev)];
+  if (have >= bytes) return FASTAR_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return FASTAR_ERR_CUDA;
+  have = bytes;
+  return FASTAR_OK;
+}
+}  // namespace fastar
 
 namespace {
 
@@ -644,6 +663,10 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
     c->launches += 1;
   }
+  if (std::getenv("FASTAR_S5_V1"))   // TEMP
+    ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged_v1(v, tm_q, c->tm_pool_k, c->tm_pool_v, k_seg ? &tm_sk : nullptr,
+                                                     k_seg ? &tm_sv : nullptr, a, st));
+  else
   ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, k_seg ? &tm_sk : nullptr,
                                                      k_seg ? &tm_sv : nullptr, a, st));
   return FASTAR_OK;

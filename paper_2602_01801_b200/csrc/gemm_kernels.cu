@@ -339,12 +339,8 @@ static int launch_gemm(const CUtensorMap& tm_a, const CUtensorMap& tm_b, const C
                        cudaStream_t st) {
   using SM = GemmSmem<EPI, A_RES, NST>;
   auto kern = gemm_kernel<EPI, A_RES, NST, A_TMEM, RAW>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::total) != cudaSuccess)
-      return FASTAR_ERR_CUDA;
-    configured = true;
-  }
+  const int cfg = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), SM::total);
+  if (cfg != FASTAR_OK) return cfg;
   kern<<<grid, kGemmThreads, SM::total, st>>>(tm_a, tm_b, c, g);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
@@ -580,12 +576,8 @@ template <bool RAW>
 static int launch_t1_pair(const CUtensorMap& tm_a, const CUtensorMap& tm_b_half, const CacheView& c, const GemmArgs& g,
                           dim3 grid, cudaStream_t st) {
   auto kern = t1_pair_kernel<RAW>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::total) != cudaSuccess)
-      return FASTAR_ERR_CUDA;
-    configured = true;
-  }
+  const int cfg = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), PairSmem::total);
+  if (cfg != FASTAR_OK) return cfg;
   kern<<<grid, kGemmThreads, PairSmem::total, st>>>(tm_a, tm_b_half, c, g);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }

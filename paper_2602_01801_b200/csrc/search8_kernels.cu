@@ -469,15 +469,10 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 }
 
 static int configure_search8() {
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(search8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess ||
-        cudaFuncSetAttribute(search8_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess ||
-        cudaFuncSetAttribute(search8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total) != cudaSuccess)
-      return FASTAR_ERR_CUDA;
-    configured = true;
-  }
-  return FASTAR_OK;
+  int r = ensure_dynamic_smem(reinterpret_cast<const void*>(search8_kernel<false>), Smem::total);
+  if (r == FASTAR_OK) r = ensure_dynamic_smem(reinterpret_cast<const void*>(search8_kernel<false, true>), Smem::total);
+  if (r == FASTAR_OK) r = ensure_dynamic_smem(reinterpret_cast<const void*>(search8_kernel<true>), Smem::total);
+  return r;
 }
 
 // Splits of the B range that fill whole waves of 2 CTAs per SM.

@@ -551,12 +551,8 @@ int launch_probe_cosine(const CacheView& c, const __nv_bfloat16* k_new, int n, i
 
 int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_t st) {
   (void)frame_len;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 8) != cudaSuccess)
-      return FASTAR_ERR_CUDA;
-    configured = true;
-  }
+  const int cfg = ensure_dynamic_smem(reinterpret_cast<const void*>(plan_kernel), 16384 * 8);
+  if (cfg != FASTAR_OK) return cfg;
   const dim3 grid((n + 255) / 256, c.H);
   match_count_kernel<<<grid, 256, 0, st>>>(c, n, tau);
   plan_kernel<<<c.H, 1024, 16384 * 8, st>>>(c, n);
