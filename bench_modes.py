@@ -9,6 +9,7 @@ from __future__ import annotations
 import dataclasses
 import json
 import os
+import sys
 import time
 
 import numpy as np
@@ -144,6 +145,7 @@ def run_sweep(args):
             cache.annsa(dq, base.block, max(1, nkb // 4))              # warm-up (module load, attributes)
             for den in (4, 8, 16, 32):
                 keep = max(1, nkb // den)
+                sys.stderr.write(f"sweep: d={d} L={L} keep={keep}\n")
                 cache.profile(True)
                 reps = 5
                 for _ in range(reps):

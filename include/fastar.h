@@ -233,6 +233,17 @@ int fastar_annsa_attention(fastar_cache_t* cache, const void* q, void* out, int3
  * frames are what streaming caches usually pin. */
 int fastar_cache_set_forced_blocks(fastar_cache_t* cache, int32_t sink_blocks, int32_t recent_blocks);
 
+/* Which kernel runs the bf16 correspondence search of fastar_tempcache_update (Section 5.2, finding the top-1
+ * cached key; host-side setting, takes effect from the next update; default FASTAR_T1_AUTO).  All three compute the
+ * same arg-max; AUTO picks single CTAs or CTA pairs from how well their grids fill the GPU.  The other values exist
+ * so that every variant can be run and checked on any shape: SINGLE = one CTA per 128 new keys, PAIR = two CTAs
+ * sharing every key tile (tcgen05 cta_group::2), TS = SINGLE with the new keys held in tensor memory. */
+#define FASTAR_T1_AUTO   0
+#define FASTAR_T1_SINGLE 1
+#define FASTAR_T1_PAIR   2
+#define FASTAR_T1_TS     3
+int fastar_cache_set_similarity_kernel(fastar_cache_t* cache, int32_t kind);
+
 /* AnnSA over the cache and an un-cached segment (Eq. 1, Section 3: the attended set is the keys and
  * values of the frames being generated concatenated with those of the earlier frames; the former
  * enter the cache only when fastar_tempcache_update is called, so attention can run on every
@@ -320,12 +331,22 @@ int64_t fastar_launch_count(const fastar_cache_t* cache);
  * The first call on each device looks up the array's device address and clears its header with a
  * synchronous copy; make that first call before any stream capture starts.  All calls share the one
  * array, which keeps the previous call's contents: each call clears the part it uses on `stream`, and
- * calls that overlap on the GPU (other streams or threads) race -- serialise them. */
+ * calls that overlap on the GPU (other streams or threads) race -- serialise them.
+ * Errors only the device can see (a bounded wait of the relevance kernel that ran out) go to a status
+ * word in the array's header: the selection kernel then writes -1 into every entry of sel_out instead of
+ * ranking unfinished accumulators, and fastar_noalloc_last_status reports the code; the word stays set, and
+ * later calls keep writing -1, until that function has read and cleared it.  Exactly keep_tokens
+ * entries are written per (head, frame) for any input bit patterns, non-finite keys included. */
 #define FASTAR_NOALLOC_MAX_WORDS (512 * 1024)
 int fastar_annca_select_noalloc(const void* q, const void* k_prompt, int32_t num_heads, int32_t head_dim, int32_t nq,
                                 int32_t frame_len, int32_t np, int32_t keep_tokens, int64_t head_stride,
                                 int64_t token_stride, int64_t prompt_head_stride, int64_t prompt_token_stride,
                                 int32_t* sel_out, void* stream);
+
+/* Device status of the allocation-free call above (the paper has no counterpart): synchronises `stream`,
+ * returns FASTAR_OK or the first error a kernel of fastar_annca_select_noalloc recorded on the current
+ * device since the last read, and clears it.  Allocates nothing; not for use during stream capture. */
+int fastar_noalloc_last_status(void* stream);
 
 /* Measurement aid (no counterpart in the paper).  While enabled, every hot kernel launch is bracketed
  * by a pair of CUDA events recorded on the launching stream.  fastar_profile_read synchronises the

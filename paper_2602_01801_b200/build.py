@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libfastar.so")
-SOURCES = ["gemm_kernels.cu", "attn_kernels.cu", "attn_paged_kernel.cu", "update_kernels.cu", "commit_kernel.cu", "search8_kernels.cu", "fastar_api.cu", "noalloc_select.cu"]
+SOURCES = ["gemm_kernels.cu", "attn_kernels.cu", "update_kernels.cu", "commit_kernel.cu", "search8_kernels.cu", "fastar_api.cu", "noalloc_select.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 

@@ -205,9 +205,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       auto load_tile = [&](bool is_k, int j, int blk, int page) {
         if (lane != 0) return;
         const int s = (is_k ? 0 : 2) + (j & 1);
-#ifdef FASTAR_PHASE_TIMING
-        reinterpret_cast<volatile long long*>(sgen + SM::bar_off + kBarBytes + 8)[s] = clock64();
-#endif
         const bool seg = SEG && page < 0;   // rows past the segment's end arrive as zeros and carry a -inf bias
         const CUtensorMap* tm = seg ? (is_k ? &tm_sk : &tm_sv) : (is_k ? &tm_k : &tm_v);
         mbar_arrive_expect_tx(bar_r_full + 8 * s, SM::kv_bytes);
@@ -315,20 +312,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, BKT, 0);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
       bool ok = mbar_wait(bar_q_full, 0, abort_flag, c.status);
-      PT_DECL
       auto issue_s = [&](int j) -> bool {
         const int s = j & 1, g = j & 1, i = j >> 1;      // key stage, softmax group, tile index inside the group
         if (!mbar_wait(bar_r_full + 8 * s, i & 1, abort_flag, c.status)) return false;
-#ifdef FASTAR_PHASE_TIMING
-        if (clock64() - pt_t > 100) {     // the tile was late: time since its load was issued
-          pt_acc[6] += clock64() - reinterpret_cast<volatile long long*>(sgen + SM::bar_off + kBarBytes + 8)[s];
-          pt_acc[7] += 1000;          // printed value / 1000 = late tiles per iteration
-        }
-#endif
-        PT_MARK(0)
         // S[g] is free once group g holds the logits of its previous tile (j - 2) in registers
         if (i > 0 && !mbar_wait(bar_s_empty + 8 * g, (i - 1) & 1, abort_flag, c.status)) return false;
-        PT_MARK(1)
         tc_fence_after();
         const uint32_t kt = ring_s + s * SM::kv_bytes;
 #pragma unroll
@@ -339,7 +327,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         umma_commit(bar_r_empty + 8 * s);
         umma_commit(bar_s_full + 8 * g);
-        PT_MARK(2)
         return true;
       };
       if (ok) ok = issue_s(0);
@@ -349,10 +336,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const int s = 2 + (j & 1), g = j & 1, i = j >> 1;   // value stage, softmax group, tile index inside the group
         ok = mbar_wait(bar_p_full + 8 * g, i & 1, abort_flag, c.status);
         if (!ok) break;
-        PT_MARK(3)
         ok = mbar_wait(bar_r_full + 8 * s, i & 1, abort_flag, c.status);
         if (!ok) break;
-        PT_MARK(4)
         tc_fence_after();
         const uint32_t vt = ring_s + s * SM::kv_bytes;
         const uint32_t pt = p_s + g * SM::p_bytes;
@@ -364,9 +349,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         umma_commit(bar_r_empty + 8 * s);
         umma_commit(bar_pv_done + 8 * g);
-        PT_MARK(5)
       }
-      PT_FLUSH("attn mma (wait K, wait S buffer, issue QK, wait P, wait V, issue PV)", nt)
     }
   } else {
     // ================================================================== softmax groups + epilogue (256 threads)
@@ -381,14 +364,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
     bool ok = true;
     const int n_mine = (nt - g + 1) >> 1;               // tiles of this group
-    PT_DECL
     for (int i = 0; i < n_mine && ok; ++i) {
       const int j = 2 * i + g, b4 = j % NB;
       ok = mbar_wait(bar_b_full + 8 * b4, (j / NB) & 1, abort_flag, c.status) &&
            mbar_wait(bar_s_full + 8 * g, i & 1, abort_flag, c.status);
       ok = __all_sync(0xffffffffu, ok);          // TMEM loads below are warp-collective
       if (!ok) break;
-      PT_MARK(0)
       tc_fence_after();
       // the whole logits row of this tile, kept in registers
       float x[BKT];
@@ -410,7 +391,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       tc_fence_before();
       mbar_arrive_warp(bar_s_empty + 8 * g);           // S[g] and the bias are consumed
-      PT_MARK(1)
       // row maximum: independent chains of 3-input maxima
       float mx0 = x[0], mx1 = x[1], mx2 = x[2], mx3 = x[3];
 #pragma unroll
@@ -431,7 +411,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         resc = i > 0;
       }
       const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
-      PT_MARK(2)
       // P[g] and O_g are free once the group's previous P.V (tile j - 2) has completed
       if (i > 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + 8 * g, (i - 1) & 1, abort_flag, c.status));
@@ -450,7 +429,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           tmem_wait_st();
         }
       }
-      PT_MARK(3)
       // exponentials -> bf16 P (K-major, 128-byte swizzle); 4 independent row-sum chains
 #pragma unroll
       for (int q = 0; q < BKT / 8; ++q) {
@@ -466,13 +444,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                      "r"(pack_bf16x2(p[2], p[3])), "r"(pack_bf16x2(p[4], p[5])), "r"(pack_bf16x2(p[6], p[7]))
                      : "memory");
       }
-      PT_MARK(4)
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive_warp(bar_p_full + 8 * g);
-      PT_MARK(5)
     }
-    if (threadIdx.x == 0) { PT_FLUSH("attn softmax group 0 (wait S, load, max, wait PV, exp, arrive)", n_mine) }
     // ---- the two groups meet: (m, l) of every row through shared memory, then O = combination of O_0, O_1 ----
     if (ok && n_mine > 0) ok = mbar_wait(bar_pv_done + 8 * g, (n_mine - 1) & 1, abort_flag, c.status);
     ok = __all_sync(0xffffffffu, ok);
@@ -544,7 +519,7 @@ static int launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
 }
 
 // tm_seg_k / tm_seg_v: maps of the un-cached segment (box {64, page_tokens, 1}); nullptr when a.seg_tiles == 0.
-int launch_attention_paged_v1(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
+int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
                            const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
                            const AttnArgs& a, cudaStream_t st) {
   if (a.seg_tiles > 0 && (!tm_seg_k || !tm_seg_v || !a.seg_bias)) return FASTAR_ERR_INVALID_ARG;

@@ -115,7 +115,7 @@ int ensure_dynamic_smem(const void* kernel, int bytes);
 // gemm_kernels.cu
 // tm_pool_k: one page per box; tm_pool_k_half: 64 key rows per box (what one CTA of a pair fetches)
 int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k,
-                         const CUtensorMap& tm_pool_k_half, int n, cudaStream_t st);
+                         const CUtensorMap& tm_pool_k_half, int n, int force, cudaStream_t st);
 int launch_c1_relevance(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_kp, int nq, int np, int frame_len,
                         int n_frames, cudaStream_t st);
 int launch_s3_scores(const CacheView& c, const CUtensorMap& tm_hq, const CUtensorMap& tm_hk, int nqb, cudaStream_t st);
@@ -160,9 +160,6 @@ struct AttnArgs {
 int launch_attention_paged(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
                            const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
                            const AttnArgs& a, cudaStream_t st);
-int launch_attention_paged_v1(const CacheView& c, const CUtensorMap& tm_q, const CUtensorMap& tm_pool_k,
-                           const CUtensorMap& tm_pool_v, const CUtensorMap* tm_seg_k, const CUtensorMap* tm_seg_v,
-                           const AttnArgs& a, cudaStream_t st);   // TEMP
 int launch_attention_gather(const CacheView& c, const CUtensorMap& tm_q, const AttnArgs& a, cudaStream_t st);
 
 // update_kernels.cu

@@ -3,7 +3,6 @@
 #include <cudaTypedefs.h>
 
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -31,6 +30,7 @@ struct fastar_cache {
   size_t bytes;
   // second stream of the host-tensor step (uploads of q and the prompt, AnnCA, its download) and its fork/join events
   int force_sink_blocks = 0, force_recent_blocks = 0;    // AnnSA selector option (fastar_cache_set_forced_blocks)
+  int t1_kernel = FASTAR_T1_AUTO;                        // fastar_cache_set_similarity_kernel
   cudaStream_t side = nullptr, copy = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_q = nullptr, ev_join = nullptr, ev_p = nullptr, ev_v = nullptr;
   ~fastar_cache() {
@@ -414,6 +414,12 @@ int fastar_cache_set_forced_blocks(fastar_cache_t* c, int32_t sink_blocks, int32
   return FASTAR_OK;
 }
 
+int fastar_cache_set_similarity_kernel(fastar_cache_t* c, int32_t kind) {
+  if (!c || kind < FASTAR_T1_AUTO || kind > FASTAR_T1_TS) return FASTAR_ERR_INVALID_ARG;
+  c->t1_kernel = kind;
+  return FASTAR_OK;
+}
+
 int fastar_cache_export_search_codes(fastar_cache_t* c, uint8_t* host_cache_codes, uint8_t* host_new_codes, int32_t n,
                                      void* stream) {
   if (!c) return FASTAR_ERR_INVALID_ARG;
@@ -544,10 +550,10 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
   } else if (q_probe) {
     CacheView vr = v;
     vr.raw_dot = 1;
-    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(vr, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(vr, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, c->t1_kernel, st));
     ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
   } else {
-    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, st));
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, c->t1_kernel, st));
   }
   ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
   if (v_ready && !v_converted && cudaStreamWaitEvent(st, v_ready, 0) != cudaSuccess) return FASTAR_ERR_CUDA;
@@ -663,10 +669,6 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     if (cudaGetLastError() != cudaSuccess) return FASTAR_ERR_CUDA;
     c->launches += 1;
   }
-  if (std::getenv("FASTAR_S5_V1"))   // TEMP
-    ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged_v1(v, tm_q, c->tm_pool_k, c->tm_pool_v, k_seg ? &tm_sk : nullptr,
-                                                     k_seg ? &tm_sv : nullptr, a, st));
-  else
   ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, k_seg ? &tm_sk : nullptr,
                                                      k_seg ? &tm_sv : nullptr, a, st));
   return FASTAR_OK;

@@ -11,8 +11,6 @@
 #include "common.h"
 #include "ptx.cuh"
 
-#include <cstdlib>
-#include <cstring>
 
 namespace fastar {
 
@@ -174,19 +172,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         if (A_RES) ok = mbar_wait(bar_afull, 0, abort_flag, c.status);
         if (A_TMEM && ok) ok = mbar_wait(bar_atm, 0, abort_flag, c.status);
         int it = 0;
-        PT_DECL
         for (int tl = 0; tl < ntl && ok; ++tl) {
           const int buf = A_TMEM ? 0 : (tl & 1), bph = A_TMEM ? (tl & 1) : ((tl >> 1) & 1);
           ok = mbar_wait(bar_tempty + 8 * buf, bph ^ 1, abort_flag, c.status);
           if (!ok) break;
-          PT_MARK(0)
           tc_fence_after();
           const uint32_t d_t = tmem + buf * 128;
           for (int kc = 0; kc < nkc; ++kc, ++it) {
             const int s = it % NST;
             ok = mbar_wait(bar_full + 8 * s, (it / NST) & 1, abort_flag, c.status);
             if (!ok) break;
-            PT_MARK(1)
             tc_fence_after();
             const uint32_t st_s = ring_s + s * SM::stage_bytes;
             const uint32_t a_c = A_RES ? a_s + kc * kChunkBytes : st_s;
@@ -199,11 +194,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
               else umma_ss(d_t, ad, bd, idesc, (kc | k4) != 0);
             }
             umma_commit(bar_empty + 8 * s);
-            PT_MARK(2)
           }
           if (ok) umma_commit(bar_tfull + 8 * buf);
         }
-        PT_FLUSH("gemm mma (wait tmem, wait smem, issue)", ntl)
       }
     } else {
       // ------------------------------------------------------------------ epilogue (256 threads)
@@ -238,7 +231,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           mbar_arrive_warp(bar_atm);
         }
       }
-      PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
         const int buf = A_TMEM ? 0 : (tl & 1), bph = A_TMEM ? (tl & 1) : ((tl >> 1) & 1), rbuf = tl & 1;
@@ -257,7 +249,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         }
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bph, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
-        PT_MARK(0)
         tc_fence_after();
         uint32_t vv[2][32];
         tmem_ld32(tmem + lane_addr + buf * 128 + wg * 64, vv[0]);
@@ -265,7 +256,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive_warp(bar_tempty + 8 * buf);      // the scores are in registers: release the accumulator
-        PT_MARK(1)
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
@@ -314,9 +304,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             }
           }
         }
-        PT_MARK(2)
       }
-      if (threadIdx.x == 0) { PT_FLUSH("gemm epilogue (wait acc, tmem loads, compute, arrive)", ntl) }
       if (EPI == EPI_ARGMAX && ok && row < g.rows_a && best_j >= 0) {
         const float sim = RAW ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
@@ -470,19 +458,16 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         constexpr uint32_t idesc = make_idesc_bf16(256, 128, 0);
         bool ok = mbar_wait(bar_afull, 0, abort_flag, c.status);
         int it = 0;
-        PT_DECL
         for (int tl = 0; tl < ntl && ok; ++tl) {
           const int buf = tl & 1;
           ok = mbar_wait(bar_tempty + 8 * buf, ((tl >> 1) & 1) ^ 1, abort_flag, c.status);
           if (!ok) break;
-          PT_MARK(0)
           tc_fence_after();
           const uint32_t d_t = tmem + buf * 128;
           for (int kc = 0; kc < nkc; ++kc, ++it) {
             const int s = it % NST;
             ok = mbar_wait(bar_full + 8 * s, (it / NST) & 1, abort_flag, c.status);
             if (!ok) break;
-            PT_MARK(1)
             tc_fence_after();
             const uint32_t a_c = a_s + kc * kChunkBytes;
             const uint32_t b_c = ring_s + s * SM::stage_bytes;
@@ -493,11 +478,9 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
               umma_ss_pair(d_t, ad, bd, idesc, (kc | k4) != 0);
             }
             umma_commit_pair(bar_empty + 8 * s);
-            PT_MARK(2)
           }
           if (ok) umma_commit_pair(bar_tfull + 8 * buf);
         }
-        PT_FLUSH("t1 pair mma (wait tmem, wait smem, issue)", ntl)
       }
     } else {
       // ------------------------------------------------------------------ epilogue (256 threads, both CTAs)
@@ -512,7 +495,6 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       // latency is not paid between two tiles
       const float* rn_h = c.rnorm + static_cast<int64_t>(h) * c.CAP;
       float rn_next = (wg == 0 && !RAW && t0 * 128 + r < L) ? rn_h[t0 * 128 + r] : 0.f;
-      PT_DECL
       for (int tl = 0; tl < ntl && ok; ++tl) {
         const int t = t0 + tl;
         const int buf = tl & 1;
@@ -527,7 +509,6 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int valid_cols = min(128, L - t * 128);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (tl >> 1) & 1, abort_flag, c.status));
         if (!ok) break;                              // warp-uniform: TMEM loads are warp-collective
-        PT_MARK(0)
         tc_fence_after();
         uint32_t vv[2][32];
         const uint32_t acc = tmem + lane_addr + buf * 128 + wg * 64;
@@ -540,7 +521,6 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           if (rank == 0) mbar_arrive(bar_tempty + 8 * buf);
           else mbar_arrive_cluster(lead_tempty + 8 * buf);
         }
-        PT_MARK(1)
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
@@ -548,9 +528,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           else chunk_argmax(vv[c2], reinterpret_cast<const float4*>(rn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
                             t * 128 + cc * 32, best, best_j);
         }
-        PT_MARK(2)
       }
-      if (threadIdx.x == 0 && rank == 0) { PT_FLUSH("t1 pair epilogue (wait acc, tmem loads, compute)", ntl) }
       if (ok && row < g.rows_a && best_j >= 0) {
         const float sim = RAW ? best : best * c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
         const unsigned long long key = (static_cast<unsigned long long>(float_to_ordered(sim)) << 32) |
@@ -600,9 +578,9 @@ static int pick_splits(int ctas_per_split, int slots, int max_splits, double* ef
 // T1.  Two kernels: single CTAs of 128 rows, and CTA pairs (256 rows, half the operand traffic per SM).  The pair
 // kernel is the faster one when both fill their waves equally well (about 10 % at 16k new keys against a 130k-key
 // cache); with few row tiles the padding to an even tile count and the coarser grid can cost more than it gains, so
-// the launcher compares the wave efficiencies.  FASTAR_T1_KERNEL=single|pair|ts in the environment forces one (tests).
+// the launcher compares the wave efficiencies.  `force` (fastar_cache_set_similarity_kernel) picks one regardless.
 int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUtensorMap& tm_pool_k,
-                         const CUtensorMap& tm_pool_k_half, int n, cudaStream_t st) {
+                         const CUtensorMap& tm_pool_k_half, int n, int force, cudaStream_t st) {
   GemmArgs g{};
   g.rows_a = n;
   g.nkc = c.D / 64;
@@ -622,11 +600,9 @@ int launch_t1_similarity(const CacheView& c, const CUtensorMap& tm_a, const CUte
   eff_pair *= static_cast<double>(tiles_single) / tiles_pair;
   // ts = the single-CTA kernel with the new keys held in tensor memory (A operand from TMEM)
   enum { SINGLE, PAIR, TS } kind = eff_pair >= 0.96 * eff_single ? PAIR : SINGLE;
-  if (const char* force = std::getenv("FASTAR_T1_KERNEL")) {
-    if (std::strcmp(force, "pair") == 0) kind = PAIR;
-    else if (std::strcmp(force, "single") == 0) kind = SINGLE;
-    else if (std::strcmp(force, "ts") == 0) kind = TS;
-  }
+  if (force == FASTAR_T1_PAIR) kind = PAIR;
+  else if (force == FASTAR_T1_SINGLE) kind = SINGLE;
+  else if (force == FASTAR_T1_TS) kind = TS;
   if (kind == TS)
     return c.raw_dot ? launch_gemm<EPI_ARGMAX, true, 4, true, true>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st)
                      : launch_gemm<EPI_ARGMAX, true, 4, true, false>(tm_a, tm_pool_k, c, g, dim3(tiles_single, c.H, splits_single), st);

@@ -27,27 +27,35 @@ constexpr int kNoAllocMaxHeads = 128;
 static __device__ __align__(256) uint32_t g_noalloc_scratch[kNoAllocHeaderWords + kNoAllocMaxWords];
 
 // Per row (head, frame): keep the k largest accumulators (ties -> lower index), ascending.  Reads the
-// file-scope array directly; `rel_words_off` is the offset of the accumulators inside it.
+// file-scope array directly; `rel_words_off` is the offset of the accumulators inside it.  The accumulators
+// are ranked as the raw order-preserving words, exactly as the regular entry point's top-k does: unsigned
+// integers are totally ordered, so exactly min(keep, np) entries are taken whatever the bit patterns (NaN or
+// infinite relevances included).  A word that no atomicMax reached stays 0 and ranks below every real value.
+// If the relevance kernel recorded an error in the header's status word, the row is filled with -1 instead.
 __global__ void __launch_bounds__(256) noalloc_topk_kernel(int rel_words_off, int n_frames, int np, int keep,
                                                            int32_t* __restrict__ sel_out) {
-  extern __shared__ float vals[];
+  extern __shared__ uint32_t vals[];
   __shared__ int red[8];
   __shared__ int run_s;
   const int f = blockIdx.x, h = blockIdx.y;
+  int32_t* orow = sel_out + (static_cast<int64_t>(h) * n_frames + f) * keep;
+  if (g_noalloc_scratch[0] != 0u) {                   // uniform for the CTA: the status word is not written by this kernel
+    for (int i = threadIdx.x; i < keep; i += blockDim.x) orow[i] = -1;
+    return;
+  }
   const uint32_t* src = g_noalloc_scratch + rel_words_off + (static_cast<int64_t>(h) * n_frames + f) * np;
-  for (int i = threadIdx.x; i < np; i += blockDim.x) vals[i] = ordered_to_float(src[i]);
+  for (int i = threadIdx.x; i < np; i += blockDim.x) vals[i] = src[i];
   if (threadIdx.x == 0) run_s = 0;
   __syncthreads();
-  int32_t* orow = sel_out + (static_cast<int64_t>(h) * n_frames + f) * keep;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int i0 = 0; i0 < np; i0 += blockDim.x) {
     const int i = i0 + threadIdx.x;
     int take = 0;
     if (i < np) {
-      const float v = vals[i];
+      const uint32_t v = vals[i];
       int rank = 0;
       for (int j = 0; j < np; ++j) {
-        const float u = vals[j];
+        const uint32_t u = vals[j];
         rank += (u > v || (u == v && j < i)) ? 1 : 0;
       }
       take = rank < keep ? 1 : 0;
@@ -63,7 +71,8 @@ __global__ void __launch_bounds__(256) noalloc_topk_kernel(int rel_words_off, in
     __syncthreads();
     int base = run_s;
     for (int w = 0; w < warp; ++w) base += red[w];
-    if (take) orow[base + inc - 1] = i;
+    const int pos = base + inc - 1;
+    if (take && pos < keep) orow[pos] = i;
     __syncthreads();
     if (threadIdx.x == 0) {
       int tot = 0;
@@ -158,11 +167,25 @@ extern "C" int fastar_annca_select_noalloc(const void* q, const void* k_prompt, 
     r = encode_map(&tm_kp, k_prompt, head_dim, np, num_heads, static_cast<uint64_t>(prompt_token_stride) * 2,
                    static_cast<uint64_t>(prompt_head_stride) * 2);
   if (r != FASTAR_OK) return r;
-  // the accumulators are maxima: the part this call uses must start at zero
+  // the accumulators are maxima: the part this call uses must start at zero (0 is below the word of every float)
   if (cudaMemsetAsync(v.rel, 0, static_cast<size_t>(num_heads) * F * np * 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
   r = launch_c1_relevance(v, tm_q, tm_kp, nq, np, frame_len, static_cast<int>(F), st);
   if (r < 0) return r;
   noalloc_topk_kernel<<<dim3(static_cast<unsigned>(F), num_heads), 256, np * 4, st>>>(kNoAllocHeaderWords, static_cast<int>(F), np,
                                                                                     keep_tokens, sel_out);
   return cudaGetLastError() == cudaSuccess ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
+extern "C" int fastar_noalloc_last_status(void* stream) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FASTAR_ERR_CUDA;
+  uint32_t* base = nullptr;
+  const int r = setup_device(dev, &base);
+  if (r != FASTAR_OK) return r;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int status = 0;
+  if (cudaMemcpyAsync(&status, base, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaMemsetAsync(base, 0, 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  return status;
 }

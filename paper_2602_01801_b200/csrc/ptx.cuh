@@ -7,7 +7,6 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdio.h>
 
 namespace fastar {
 
@@ -288,41 +287,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
-
-// 32 lanes x 16 consecutive 32-bit columns
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-
-// ---------------------------------------------------------------------------------------------
-// Optional per-phase cycle counters (compiled in only with -DFASTAR_PHASE_TIMING): CTA (0,0,0) prints the
-// cycles each role spent between marks, per loop iteration.  For finding where a tile's time goes.
-// ---------------------------------------------------------------------------------------------
-#ifdef FASTAR_PHASE_TIMING
-__device__ __forceinline__ unsigned long long pt_globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-#define PT_DECL long long pt_t = clock64(); const long long pt_c0 = pt_t; const unsigned long long pt_g0 = pt_globaltimer(); \
-  long long pt_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#define PT_MARK(i) { const long long n__ = clock64(); pt_acc[i] += n__ - pt_t; pt_t = n__; }
-#define PT_FLUSH(name, iters)                                                                                        \
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iters) > 0)                                          \
-    printf("%s: per-iteration cycles %lld %lld %lld %lld %lld %lld %lld %lld (iterations %d) total %lld cycles %llu ns\n", name, \
-           pt_acc[0] / (iters), pt_acc[1] / (iters), pt_acc[2] / (iters), pt_acc[3] / (iters), pt_acc[4] / (iters),  \
-           pt_acc[5] / (iters), pt_acc[6] / (iters), pt_acc[7] / (iters), static_cast<int>(iters),                   \
-           static_cast<long long>(clock64() - pt_c0), pt_globaltimer() - pt_g0);
-#else
-#define PT_DECL
-#define PT_MARK(i)
-#define PT_FLUSH(name, iters)
-#endif
 
 // ---------------------------------------------------------------------------------------------
 // small numeric helpers

@@ -43,6 +43,7 @@ SIGNATURES = {
     "fastar_cache_destroy": (C.c_int, [_vp]),
     "fastar_cache_export": (C.c_int, [_vp] * 9),
     "fastar_cache_set_forced_blocks": (C.c_int, [_vp, _i32, _i32]),
+    "fastar_cache_set_similarity_kernel": (C.c_int, [_vp, _i32]),
     "fastar_cache_export_search_codes": (C.c_int, [_vp, _vp, _vp, _i32, _vp]),
     "fastar_cache_export_probe_codes": (C.c_int, [_vp, _vp, _i32, _vp]),
     "fastar_cache_export_annca_codes": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _vp]),
@@ -60,6 +61,7 @@ SIGNATURES = {
     "fastar_last_device_status": (C.c_int, [_vp, _vp]),
     "fastar_launch_count": (C.c_int64, [_vp]),
     "fastar_annca_select_noalloc": (C.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp]),
+    "fastar_noalloc_last_status": (C.c_int, [_vp]),
     "fastar_profile_enable": (C.c_int, [_vp, _i32]),
     "fastar_profile_read": (C.c_int, [_vp, _vp, _vp, _vp]),
     "fastar_status_string": (C.c_char_p, [C.c_int]),
@@ -182,6 +184,11 @@ class Cache:
     def set_forced_blocks(self, sink_blocks: int = 0, recent_blocks: int = 0) -> None:
         """AnnSA selector option: always keep the first / the last live key blocks of every head (within the budget)."""
         _check(self.lib.fastar_cache_set_forced_blocks(self.handle, sink_blocks, recent_blocks), "fastar_cache_set_forced_blocks")
+
+    def set_similarity_kernel(self, kind: str = "auto") -> None:
+        """Which kernel runs the bf16 correspondence search: "auto" (default), "single", "pair" or "ts"."""
+        _check(self.lib.fastar_cache_set_similarity_kernel(self.handle, {"auto": 0, "single": 1, "pair": 2, "ts": 3}[kind]),
+               "fastar_cache_set_similarity_kernel")
 
     def export_search_codes(self, n_new: int = 0) -> Dict[str, np.ndarray]:
         """8-bit search only: the code rows of every slot [H][CAP][128] and of the last update's n_new keys."""
@@ -369,6 +376,11 @@ def annca_select_noalloc(q, k_prompt, frame_len: int, keep_tokens: int, sel_out=
                                                q.stride(0), q.stride(1), k_prompt.stride(0), k_prompt.stride(1),
                                                sel_out.data_ptr(), _stream()), "fastar_annca_select_noalloc")
     return sel_out
+
+
+def noalloc_last_status() -> int:
+    """Device status of the allocation-free selection on the current device (0 = ok); synchronises and clears it."""
+    return load_library().fastar_noalloc_last_status(_stream())
 
 
 # ---- helpers for moving synthetic numpy data (bf16-exact float32) onto the device ---------------

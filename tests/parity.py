@@ -214,14 +214,36 @@ def check_selection(qcodes: np.ndarray, kcodes: np.ndarray, nq: int, L: int, blo
     return want
 
 
+_SCALED_ABS_BOUND = False
+
+
+class scaled_abs_bound:
+    """Within this context check_attention lets the absolute bound grow with the size of the outputs (see there).
+    Only the seeded random-shape cases use it; the workload configurations are held to the fixed 2e-2."""
+
+    def __enter__(self):
+        global _SCALED_ABS_BOUND
+        self.prev, _SCALED_ABS_BOUND = _SCALED_ABS_BOUND, True
+
+    def __exit__(self, *exc):
+        global _SCALED_ABS_BOUND
+        _SCALED_ABS_BOUND = self.prev
+
+
 def check_attention(got: np.ndarray, want: np.ndarray, what: str) -> None:
     """max-abs 2e-2 and relative L2 1e-2 (the stated bar for bf16 inputs with fp32 accumulation).  The absolute bound
-    is meant for outputs of the workloads' size (|o| below 4 with N(0, 1) values); bf16 numbers in [4, 8) are
-    2^-5 = 0.031 apart, so for larger outputs, which only the random-shape cases produce, it scales with max|o| / 4."""
+    assumes outputs of the workloads' size (|o| below 4 with N(0, 1) values): bf16 numbers in [4, 8) are 2^-5 = 0.031
+    apart, so a bf16 result cannot meet 2e-2 there.  Inside `scaled_abs_bound()` (random-shape cases with very few
+    clusters produce such outputs) the bound scales with max|o| / 4, and an error above 2e-2 that it lets through
+    is printed."""
     got = got.astype(np.float64)
     err = np.max(np.abs(got - want))
     rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
-    abs_tol = ATT_MAX_ABS * max(1.0, float(np.max(np.abs(want))) / 4.0)
+    abs_tol = ATT_MAX_ABS
+    if _SCALED_ABS_BOUND:
+        abs_tol = ATT_MAX_ABS * max(1.0, float(np.max(np.abs(want))) / 4.0)
+        if ATT_MAX_ABS < err <= abs_tol:
+            print(f"{what}: max-abs {err:.3e} above {ATT_MAX_ABS} accepted under the scaled bound {abs_tol:.3e} (max|o| = {np.max(np.abs(want)):.2f})")
     assert err <= abs_tol and rel <= ATT_REL_L2, f"{what}: max-abs {err:.3e} (<= {abs_tol:.3e}), rel-L2 {rel:.3e} (<= {ATT_REL_L2})"
 
 

@@ -17,7 +17,14 @@ def _gpu():
 
 
 def make_cache(cfg, w, fp32=False, n_sink=0, capacity=None, max_tokens=None, search_bits=16, representative="last",
-               weighted_histograms=False, pool_pages=0):
+               weighted_histograms=False, pool_pages=0, t1_kernel="auto"):
+    torch, fastar = _gpu()
+    cache = _make_cache(cfg, w, fp32, n_sink, capacity, max_tokens, search_bits, representative, weighted_histograms, pool_pages)
+    cache.set_similarity_kernel(t1_kernel)
+    return cache
+
+
+def _make_cache(cfg, w, fp32, n_sink, capacity, max_tokens, search_bits, representative, weighted_histograms, pool_pages):
     torch, fastar = _gpu()
     return fastar.Cache(cfg.num_heads, cfg.head_dim, capacity or cfg.capacity, cfg.block, w.lsh_projection(), cfg.lsh_tables,
                         cfg.lsh_bits, max_tokens=max_tokens or cfg.chunk_tokens, max_prompt_tokens=max(cfg.prompt_tokens, 64),
@@ -129,9 +136,9 @@ def gpu_annca_checked(cache, cfg, Q, Kp, Vp, keep, fp32=False):
     return res
 
 
-def full_step(cfg, fp32=False, tau=None, n_sink=0, search_bits=16):
+def full_step(cfg, fp32=False, tau=None, n_sink=0, search_bits=16, t1_kernel="auto"):
     w = synth.Workload(cfg)
-    cache = make_cache(cfg, w, fp32, n_sink, search_bits=search_bits)
+    cache = make_cache(cfg, w, fp32, n_sink, search_bits=search_bits, t1_kernel=t1_kernel)
     heads = [O.HeadCache(cfg.capacity, cfg.head_dim, n_sink) for _ in range(cfg.num_heads)]
     for ci in range(cfg.prior_chunks):                 # prior chunks enter un-merged (tau > 1): plain append
         _, K, V = w.chunk(ci)
@@ -171,13 +178,12 @@ def test_other_tile_shapes(d, pt):
 
 @pytest.mark.parametrize("kernel", ["single", "pair", "ts"])
 @pytest.mark.parametrize("d,pt", [(128, 128), (64, 64)])
-def test_both_similarity_kernels(kernel, d, pt, monkeypatch):
+def test_both_similarity_kernels(kernel, d, pt):
     # The launcher picks the single-CTA or the CTA-pair similarity kernel from the grid's wave efficiency; force each
     # one in turn so that both are checked against the oracle (ragged row tiles, ragged cache lengths, two updates).
     # "ts" is the single-CTA kernel with the new keys held in tensor memory (A operand from TMEM), an option.
-    monkeypatch.setenv("FASTAR_T1_KERNEL", kernel)
     cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
-    cache, w, heads, post, _, _ = full_step(cfg)
+    cache, w, heads, post, _, _ = full_step(cfg, t1_kernel=kernel)
     Q, K, V = w.chunk(cfg.prior_chunks + 1)
     post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)
     assert post["count"].max() > 1
@@ -185,14 +191,13 @@ def test_both_similarity_kernels(kernel, d, pt, monkeypatch):
 
 @pytest.mark.parametrize("d,pt,fp32,kernel", [(128, 128, False, "single"), (64, 64, True, "single"), (128, 128, False, "pair"),
                                                (64, 64, False, "pair")])
-def test_query_probe_correspondence(d, pt, fp32, kernel, monkeypatch):
-    monkeypatch.setenv("FASTAR_T1_KERNEL", kernel)
+def test_query_probe_correspondence(d, pt, fp32, kernel):
     # The slot is chosen by the token's QUERY (highest attention score over the cache), the merge decision by the key
     # cosine of that slot.  Prior chunks enter un-merged; then two merging chunks, each probed with its own queries;
     # AnnSA runs on the result.  An empty cache and the 8-bit refusal are covered too.
     cfg = synth.small_config(head_dim=d, block=pt, capacity=2048, keep_blocks=5, num_heads=3)
     w = synth.Workload(cfg)
-    cache = make_cache(cfg, w, fp32)
+    cache = make_cache(cfg, w, fp32, t1_kernel=kernel)
     heads = [O.HeadCache(cfg.capacity, cfg.head_dim) for _ in range(cfg.num_heads)]
     Q, K, V = w.chunk(0)
     post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, fp32, probe=Q)      # empty cache: all appended
@@ -685,6 +690,11 @@ def test_random_shapes_and_options(seed):
     # Seeded random cases over head dim, page size, frame shape (row counts that are no multiple of anything), cache
     # capacity (some evict), LSH shape, budgets, threshold, input dtype, search width, correspondence rule and
     # representative: a whole step plus two more updates, every stage checked against the oracle.
+    with P.scaled_abs_bound():                   # very few clusters can give |o| > 4, where bf16 is coarser than 2e-2
+        _run_random_case(seed)
+
+
+def _run_random_case(seed):
     cfg, o = _random_case(1000 + seed)
     if o["search_bits"] == 1:
         o["probe"] = False                       # the Hamming search compares keys with keys

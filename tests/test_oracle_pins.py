@@ -363,6 +363,34 @@ def test_density_and_recall_definitions():
     assert 0 < O.attention_recall(Q, c, sel, 8, 16) < 1
 
 
+def test_attention_recall_against_python_loop_brute_force():
+    # Section 4.2 measures how much of the dense attention mass the kept keys hold.  Pinned by brute force over
+    # (query, slot) pairs in Python loops on a cache with multiplicities above 1 and a ragged last key block: the
+    # weight of slot j for query i is m_j exp(q_i.k_j / sqrt d) / sum over all live slots, summed over the slots of
+    # the query block's selected blocks.  A missing log m term or a wrong block slice changes the value.
+    import math
+    d, L, bq, bk = 4, 27, 5, 8                                     # 4 key blocks, the last one holds 3 slots
+    c = O.HeadCache(32, d)
+    m = np.array([1 + (7 * j) % 5 for j in range(L)], np.int64)    # multiplicities 1..5
+    c.load(_rng(30).standard_normal((L, d)), _rng(31).standard_normal((L, d)), m=m)
+    Q = _rng(32).standard_normal((12, d))                          # 3 query blocks, the last one holds 2 rows
+    sel = np.array([[0, 3], [1, 3], [2, 3]])
+    tot = 0.0
+    for i in range(Q.shape[0]):
+        w = [float(m[j]) * math.exp(sum(Q[i, t] * c.K[j, t] for t in range(d)) / math.sqrt(d)) for j in range(L)]
+        kept = 0.0
+        for b in sel[i // bq]:
+            for j in range(b * bk, min((b + 1) * bk, L)):
+                kept += w[j]
+        tot += kept / sum(w)
+    want = tot / Q.shape[0]
+    assert O.attention_recall(Q, c, sel, bq, bk) == pytest.approx(want, rel=1e-12)
+    # the bias matters on this cache: the same quantity without multiplicities is a different number
+    c1 = O.HeadCache(32, d)
+    c1.load(c.K[:L].copy(), c.V[:L].copy())
+    assert abs(O.attention_recall(Q, c1, sel, bq, bk) - want) > 1e-3
+
+
 def test_c0_workload_behaves_as_designed():
     cfg = synth.CONFIGS["c0"]
     w = synth.Workload(cfg)
