@@ -234,11 +234,16 @@ def run_ours(args, cfg):
     def step():
         # AnnCA reads no cache state and has its own scratch, so it runs on a second stream beside the update
         # (its small kernels fill the SMs the update's planning kernels leave idle); joined before the step ends.
+        # So does the query side of AnnSA's selector (codes and block histograms of the queries).
         main = torch.cuda.current_stream()
         ca_stream.wait_stream(main)
         with torch.cuda.stream(ca_stream):
+            cache.annsa_prepare(dq, cfg.block)
+            prepared = torch.cuda.Event()
+            prepared.record()
             cache.annca(dq, dkp, dvp, cfg.frame_len, cfg.keep_prompt, out=out_ca)
         cache.update(dk, dv, cfg.frame_len, cfg.tau, outputs=False, probe=dq if args.probe else None)
+        main.wait_event(prepared)
         cache.annsa(dq, cfg.block, cfg.keep_blocks, out=out_sa)
         main.wait_stream(ca_stream)
 

@@ -21,7 +21,7 @@
  *     void* (0 = the legacy default stream).  All work is enqueued on that stream and the
  *     call returns without synchronising unless stated otherwise.
  *   - Ownership: the caller owns every tensor and the workspace buffer; the library owns only
- *     the small host object behind fastar_cache_t (with two CUDA streams and five events created and
+ *     the small host object behind fastar_cache_t (with two CUDA streams and six events created and
  *     destroyed with it).  Nothing here allocates device memory.
  *   - Tensors are [head][token][channel] with element strides `head_stride`, `token_stride`
  *     (channel stride 1).  Strides in bytes must be multiples of 16 and base pointers 16-byte
@@ -224,6 +224,16 @@ int fastar_annsa_attention(fastar_cache_t* cache, const void* q, void* out, int3
                            int64_t head_stride, int64_t token_stride, int32_t block_q, int32_t keep_blocks,
                            int32_t* sel_out, int32_t* nsel_out, uint32_t* qcode_out, float* scores_out,
                            const int32_t* sel_in, const int32_t* nsel_in, void* stream);
+
+/* The query side of AnnSA's selector ahead of time (Section 5.1: the bucket ids of the queries; Section 5.4: their
+ * per-block counts): codes of the nq queries and the bucket histogram of every query block, written to the cache's
+ * scratch.  It reads no cache state, so it may be issued on another stream while fastar_tempcache_update runs; the
+ * next fastar_annsa_attention call with the same q, nq, strides and block_q (and a selecting keep_blocks) then
+ * starts at the block scores.  The caller orders the two calls (same stream, or an event between the streams) and
+ * issues nothing else that hashes queries for AnnSA on this cache in between; any other AnnSA call discards the
+ * prepared state.  Results are identical with or without this call. */
+int fastar_annsa_prepare(fastar_cache_t* cache, const void* q, int32_t nq, int64_t head_stride, int64_t token_stride,
+                         int32_t block_q, void* stream);
 
 /* AnnSA selector option (host-side setting, takes effect from the next AnnSA call; default 0, 0 = the
  * plain rule): the first `sink_blocks` and the last `recent_blocks` live key blocks of every head are

@@ -98,6 +98,9 @@ struct CacheView {
   uint32_t* code_q_ca;             // [H][max_tokens]
   uint32_t* code_p_ca;             // [H][max_prompt]
   int32_t* nselp;                  // [H][max_frames]
+  // AnnSA's query codes (their own array: fastar_annsa_prepare may run beside an update, which hashes its keys into code_new)
+  uint32_t* code_q_sa;             // [H][max_tokens]
+  __nv_bfloat16* stage_prep;       // fp32 caches: bf16 copy of the queries hashed by fastar_annsa_prepare (null for bf16)
 };
 
 inline __host__ __device__ int64_t slot_row_offset(const CacheView& c, const int32_t* page_table_h, int slot) {
@@ -174,7 +177,7 @@ int launch_plan(const CacheView& c, int n, int frame_len, float tau, cudaStream_
 int launch_commit(const CacheView& c, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new, int n, int frame_len,
                   int64_t hs, int64_t ts, cudaStream_t st);
 int launch_finalize_hist(const CacheView& c, fastar_update_stats* stats_out, int advance_clock, cudaStream_t st);
-int launch_query_hist(const CacheView& c, int nq, int block_q, cudaStream_t st);
+int launch_query_hist(const CacheView& c, const uint32_t* codes, int nq, int block_q, cudaStream_t st);
 int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, int force_recent, cudaStream_t st);
 int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st);
 int launch_reset(const CacheView& c, cudaStream_t st);

@@ -31,6 +31,9 @@ struct fastar_cache {
   // second stream of the host-tensor step (uploads of q and the prompt, AnnCA, its download) and its fork/join events
   int force_sink_blocks = 0, force_recent_blocks = 0;    // AnnSA selector option (fastar_cache_set_forced_blocks)
   int t1_kernel = FASTAR_T1_AUTO;                        // fastar_cache_set_similarity_kernel
+  // queries whose codes and block histograms fastar_annsa_prepare has already produced (consumed by the next matching AnnSA call)
+  struct { const void* q = nullptr; int32_t nq = 0, block_q = 0; int64_t hs = 0, ts = 0; bool valid = false; } prep;
+  cudaEvent_t ev_prep = nullptr;
   cudaStream_t side = nullptr, copy = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_q = nullptr, ev_join = nullptr, ev_p = nullptr, ev_v = nullptr;
   ~fastar_cache() {
@@ -39,6 +42,7 @@ struct fastar_cache {
     if (ev_join) cudaEventDestroy(ev_join);
     if (ev_p) cudaEventDestroy(ev_p);
     if (ev_v) cudaEventDestroy(ev_v);
+    if (ev_prep) cudaEventDestroy(ev_prep);
     if (side) cudaStreamDestroy(side);
     if (copy) cudaStreamDestroy(copy);
   }
@@ -165,6 +169,8 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.code_q_ca = reinterpret_cast<uint32_t*>(take(H * MT * 4));
   t.code_p_ca = reinterpret_cast<uint32_t*>(take(H * MP * 4));
   t.nselp = reinterpret_cast<int32_t*>(take(H * t.max_frames * 4));
+  t.code_q_sa = reinterpret_cast<uint32_t*>(take(H * MT * 4));
+  t.stage_prep = d.dtype == FASTAR_FP32 ? reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2)) : nullptr;
   for (int i = 0; i < 2; ++i) t.stage_out[i] = take(H * MT * D * esz);
   for (int i = 0; i < 5; ++i) t.stage_in_raw[i] = d.dtype == FASTAR_FP32 ? take(H * (i < 3 ? MT : MP) * D * 4) : nullptr;
   cur = (cur + 1023) & ~static_cast<size_t>(1023);
@@ -313,6 +319,7 @@ int fastar_cache_create(fastar_cache_t** out, const fastar_cache_desc* desc, con
        cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_p, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_v, cudaEventDisableTiming) != cudaSuccess ||
+       cudaEventCreateWithFlags(&c->ev_prep, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_q, cudaEventDisableTiming) != cudaSuccess ||
        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
@@ -619,8 +626,13 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     a.sel_head_stride = static_cast<int64_t>(nqb) * keep_blocks;
     a.keep = keep_blocks;
   } else if (!dense) {
-    ACCK(FASTAR_K_HASH, launch_prep_codes(v, qb, nq, qhs, qts, v.code_new, nullptr, st));
-    ACCK(FASTAR_K_QUERY_HIST, launch_query_hist(v, nq, block_q, st));
+    const bool prepared = c->prep.valid && c->prep.q == q && c->prep.nq == nq && c->prep.block_q == block_q &&
+                          c->prep.hs == head_stride && c->prep.ts == token_stride;
+    c->prep.valid = false;
+    if (!prepared) {
+      ACCK(FASTAR_K_HASH, launch_prep_codes(v, qb, nq, qhs, qts, v.code_q_sa, nullptr, st));
+      ACCK(FASTAR_K_QUERY_HIST, launch_query_hist(v, v.code_q_sa, nq, block_q, st));
+    }
     ACCK(FASTAR_K_S3_SCORES, launch_s3_scores(v, c->tm_hq, c->tm_hk, nqb, st));
     if (v.hist_weighted) {                   // the high digits of the weighted histograms, into their own score array
       CacheView vh = v;
@@ -640,7 +652,7 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
     }
     if (nsel_out && cudaMemcpyAsync(nsel_out, v.nsel, static_cast<size_t>(v.H) * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return FASTAR_ERR_CUDA;
-    if (qcode_out && cudaMemcpy2DAsync(qcode_out, static_cast<size_t>(nq) * 4, v.code_new, static_cast<size_t>(v.max_tokens) * 4,
+    if (qcode_out && cudaMemcpy2DAsync(qcode_out, static_cast<size_t>(nq) * 4, v.code_q_sa, static_cast<size_t>(v.max_tokens) * 4,
                                        static_cast<size_t>(nq) * 4, v.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return FASTAR_ERR_CUDA;
     if (scores_out && v.hist_weighted) {
@@ -671,6 +683,32 @@ static int annsa_impl(fastar_cache_t* c, const void* q, const void* k_seg, const
   }
   ACCK(FASTAR_K_S5_ATTENTION, launch_attention_paged(v, tm_q, c->tm_pool_k, c->tm_pool_v, k_seg ? &tm_sk : nullptr,
                                                      k_seg ? &tm_sv : nullptr, a, st));
+  return FASTAR_OK;
+}
+
+int fastar_annsa_prepare(fastar_cache_t* c, const void* q, int32_t nq, int64_t head_stride, int64_t token_stride, int32_t block_q,
+                         void* stream) {
+  if (!c || !q || nq < 1) return FASTAR_ERR_INVALID_ARG;
+  if (block_q != 64 && block_q != 128) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (nq > c->v.max_tokens) return FASTAR_ERR_UNSUPPORTED_SHAPE;
+  if (token_stride < c->v.D || head_stride < 0) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const CacheView& v = c->v;
+  c->prep.valid = false;
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  int64_t qhs = head_stride, qts = token_stride;
+  if (c->desc.dtype == FASTAR_FP32) {          // own staging buffer: an update or another attention call may be converting too
+    if ((reinterpret_cast<uintptr_t>(q) & 15) || (qhs & 3) || (qts & 3)) return FASTAR_ERR_INVALID_ARG;
+    ACCK(FASTAR_K_CONVERT, launch_convert_f32_to_bf16(static_cast<const float*>(q), v.stage_prep, v.H, nq, v.D, qhs, qts, st));
+    qb = v.stage_prep;
+    qhs = static_cast<int64_t>(nq) * v.D;
+    qts = v.D;
+  }
+  ACCK(FASTAR_K_HASH, launch_prep_codes(v, qb, nq, qhs, qts, v.code_q_sa, nullptr, st));
+  ACCK(FASTAR_K_QUERY_HIST, launch_query_hist(v, v.code_q_sa, nq, block_q, st));
+  c->prep.q = q; c->prep.nq = nq; c->prep.block_q = block_q; c->prep.hs = head_stride; c->prep.ts = token_stride;
+  c->prep.valid = true;
   return FASTAR_OK;
 }
 
@@ -868,6 +906,11 @@ int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const 
   bool copies_ok = upload(0, st) && upload(2, sd);
   copies_ok = copies_ok && cudaEventRecord(c->ev_q, sd) == cudaSuccess && upload(3, sd) && upload(4, sd) &&
               cudaEventRecord(c->ev_p, sd) == cudaSuccess && cudaStreamWaitEvent(sc, c->ev_p, 0) == cudaSuccess && upload(1, sc);
+  // the query-side selector work (codes, block histograms) needs only q: it runs on the side stream, behind the uploads
+  // (the host link is the bottleneck) and before AnnCA
+  const bool sparse_sa = keep_blocks < v.CAPB;
+  if (copies_ok && sparse_sa && fastar_annsa_prepare(c, dsrc[2], n, static_cast<int64_t>(n) * v.D, v.D, block_q, sd) != FASTAR_OK) copies_ok = false;
+  if (cudaEventRecord(c->ev_prep, sd) != cudaSuccess) copies_ok = false;
   // recorded even after a failed copy: the update below waits on it
   copies_ok = (cudaEventRecord(c->ev_v, sc) == cudaSuccess) && copies_ok;
   if (!copies_ok) r = FASTAR_ERR_CUDA;
@@ -880,7 +923,7 @@ int fastar_attention_step_host(fastar_cache_t* c, const void* k_new_host, const 
     r = fastar_annca_attention(c, dsrc[2], dsrc[3], dsrc[4], v.stage_out[1], n, frame_len, np, keep_tokens, hs, ts, phs, ts, nullptr,
                                nullptr, nullptr, sd);
   if (r == FASTAR_OK && cudaMemcpyAsync(out_ca_host, v.stage_out[1], obytes, cudaMemcpyDeviceToHost, sd) != cudaSuccess) r = FASTAR_ERR_CUDA;
-  if (r == FASTAR_OK && cudaStreamWaitEvent(st, c->ev_q, 0) != cudaSuccess) r = FASTAR_ERR_CUDA;
+  if (r == FASTAR_OK && cudaStreamWaitEvent(st, c->ev_prep, 0) != cudaSuccess) r = FASTAR_ERR_CUDA;
   if (r == FASTAR_OK)
     r = fastar_annsa_attention(c, dsrc[2], v.stage_out[0], n, hs, ts, block_q, keep_blocks, nullptr, nullptr, nullptr, nullptr, nullptr,
                                nullptr, st);

@@ -616,7 +616,7 @@ int launch_finalize_hist(const CacheView& c, fastar_update_stats* stats_out, int
 }
 
 // S2 (query side)
-__global__ void __launch_bounds__(128) query_hist_kernel(const CacheView c, int nq, int block_q) {
+__global__ void __launch_bounds__(128) query_hist_kernel(const CacheView c, const uint32_t* __restrict__ codes, int nq, int block_q) {
   extern __shared__ int hist[];
   const int a = blockIdx.x, h = blockIdx.y;
   for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) hist[q] = 0;
@@ -624,16 +624,16 @@ __global__ void __launch_bounds__(128) query_hist_kernel(const CacheView c, int 
   const int r0 = a * block_q, r1 = min(nq, r0 + block_q);
   const int nb = 1 << c.B;
   for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x) {
-    const uint32_t code = c.code_new[static_cast<int64_t>(h) * c.max_tokens + r];
+    const uint32_t code = codes[static_cast<int64_t>(h) * c.max_tokens + r];
     for (int t = 0; t < c.T; ++t) atomicAdd(&hist[t * nb + ((code >> (8 * t)) & 0xFFu)], 1);
   }
   __syncthreads();
   __nv_bfloat16* dst = c.hq + (static_cast<int64_t>(h) * c.max_qb + a) * c.hist_cols;
   for (int q = threadIdx.x; q < c.hist_cols; q += blockDim.x) dst[q] = __float2bfloat16(static_cast<float>(hist[q]));
 }
-int launch_query_hist(const CacheView& c, int nq, int block_q, cudaStream_t st) {
+int launch_query_hist(const CacheView& c, const uint32_t* codes, int nq, int block_q, cudaStream_t st) {
   const int nqb = (nq + block_q - 1) / block_q;
-  query_hist_kernel<<<dim3(nqb, c.H), 128, c.hist_cols * 4, st>>>(c, nq, block_q);
+  query_hist_kernel<<<dim3(nqb, c.H), 128, c.hist_cols * 4, st>>>(c, codes, nq, block_q);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 

@@ -50,6 +50,7 @@ SIGNATURES = {
     "fastar_cache_import": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp]),
     "fastar_tempcache_update": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
     "fastar_tempcache_update_probe": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp, _vp, _vp, _vp, _vp]),
+    "fastar_annsa_prepare": (C.c_int, [_vp, _vp, _i32, _i64, _i64, _i32, _vp]),
     "fastar_annsa_attention": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "fastar_annsa_attention_segment": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _i64, _i64, _i32, _i32, _vp, _vp,
                                                  _vp]),
@@ -264,6 +265,13 @@ class Cache:
                                                 _ptr(res.get("dest")), _ptr(res.get("stats")), _stream()),
                "fastar_tempcache_update")
         return res
+
+    def annsa_prepare(self, q, block_q: int) -> None:
+        """Hashes the queries and builds their block histograms on the current stream (no cache state is read): the next
+        annsa() call on the same q / block_q skips that work.  Order the two calls with an event if the streams differ."""
+        H, nq, _ = q.shape
+        hs, ts = self._strides(q)
+        _check(self.lib.fastar_annsa_prepare(self.handle, q.data_ptr(), nq, hs, ts, block_q, _stream()), "fastar_annsa_prepare")
 
     def annsa(self, q, block_q: int, keep_blocks: int, sel_in=None, nsel_in=None, debug: bool = False, out=None):
         torch = self.torch

@@ -119,6 +119,70 @@ def test_c2_style_rollout_invariants():
     assert evicted.sum() > 0 and np.all(lens[-1] == cfg.capacity)
 
 
+def test_c2_rollout_at_full_size_against_the_oracle_at_checkpoints():
+    """The long rollout of the benchmark's config 2 at its full size (12 heads, 4680-token chunks, capacity 32768), run
+    past the point where the cache is full: 126 chunks.  Every chunk: the token bookkeeping (sum of multiplicities +
+    evicted = inserted, length bounded).  At the checkpoints -- chunks 0, 1, 2, every tenth, 117-119 and the eviction
+    tail 120-125 -- the state before the chunk is handed to the oracle, which replays the chunk: top-1 and threshold on
+    sampled tokens, the merge / append / eviction bookkeeping in full, codes, block scores and selections in full and
+    the attention on sampled query blocks, for three heads.  Multiplicities reach the hundreds here, which is where the
+    log2 m bias and the bf16 running mean of the values would drift if they were wrong."""
+    import torch
+    from paper_2602_01801_b200 import fastar
+
+    cfg = synth.CONFIGS["c2"]
+    w = synth.Workload(cfg)
+    H, n = cfg.num_heads, cfg.chunk_tokens
+    R = w.lsh_projection()
+    cache = fastar.Cache(H, cfg.head_dim, cfg.capacity, cfg.block, R, cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
+                         max_prompt_tokens=cfg.prompt_tokens, max_frames=cfg.frames_per_chunk)
+    chunks = 126
+    checkpoints = {0, 1, 2, 117, 118, 119} | set(range(9, 120, 10)) | set(range(120, chunks))
+    heads_checked = [0, 6, 11]
+    rng = np.random.default_rng(2)
+    nqb = -(-n // cfg.block)
+    evicted = np.zeros(H, np.int64)
+    m_max, evicting_checkpoints = 0, 0
+    for ci in range(chunks):
+        Q, K, V = w.chunk(ci)
+        check = ci in checkpoints
+        pre = cache.export_state() if check else None
+        res = cache.update(fastar.to_device(K), fastar.to_device(V), cfg.frame_len, cfg.tau)
+        a = cache.annsa(fastar.to_device(Q), cfg.block, cfg.keep_blocks, debug=check)
+        assert cache.status() == 0
+        stats = res["stats"].cpu().numpy()
+        evicted += stats[:, 4]
+        light = cache.export_state(kv=False)
+        for h in range(H):
+            L = int(light["len"][h])
+            assert L <= cfg.capacity and L == int(stats[h, 5]) and int(stats[h, 6]) == 1
+            assert int(light["count"][h, :L].sum()) + int(evicted[h]) == (ci + 1) * n, f"chunk {ci} head {h}: token count"
+            assert int(stats[h, 0]) + int(stats[h, 2]) + int(stats[h, 3]) == n
+        if not check:
+            continue
+        post = cache.export_state()
+        match, sim, dest = (res[k].cpu().numpy() for k in ("match", "sim", "dest"))
+        pre_heads = P.oracle_heads_from_export(pre)
+        post_heads = P.oracle_heads_from_export(post)
+        out = a["out"].float().cpu().numpy()
+        evicting_checkpoints += int(stats[heads_checked, 3].sum() > 0)
+        for h in heads_checked:
+            rows = np.sort(rng.choice(n, 64, replace=False))
+            P.check_update(pre_heads[h], K[h], V[h], cfg.frame_len, cfg.tau, match[h], sim[h], dest[h], stats[h], post, h, rows=rows)
+            hc = post_heads[h]
+            m_max = max(m_max, int(hc.m[: hc.L].max()))
+            qcodes = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, a["qcode"][h].cpu().numpy().view(np.uint32))
+            kcodes = P.check_codes(P.bits_to_f64(post["k"][h, : hc.L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][h, : hc.L])
+            sel = P.check_selection(qcodes, kcodes, n, hc.L, cfg.block, cfg.block, cfg.lsh_bits, cfg.keep_blocks,
+                                    a["scores"][h].cpu().numpy(), a["sel"][h].cpu().numpy(), int(a["nsel"][h]))
+            blocks = [int(rng.integers(0, nqb - 1)), nqb - 1]          # a random block and the ragged last one
+            for blk, want in _oracle_blocks(Q[h], hc, sel, blocks, cfg.block, cfg.block).items():
+                rws = slice(blk * cfg.block, min((blk + 1) * cfg.block, n))
+                P.check_attention(out[h][rws], want, f"c2 chunk {ci} head {h} block {blk}")
+    assert m_max > 50, "the rollout never built large multiplicities"
+    assert evicted.sum() > 0 and evicting_checkpoints >= 3, "the eviction tail was not reached"
+
+
 def test_c1_full_size_update_with_eight_bit_search_sampled():
     """The 8-bit quantised correspondence search at full c1 size: quantiser and top-1 on sampled tokens of three heads
     (the oracle's scores of the GPU's codes), merge bookkeeping in full for those heads, invariants for all heads."""

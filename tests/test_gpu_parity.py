@@ -407,6 +407,36 @@ def test_shared_page_pool_across_ragged_heads(d, page, search_bits):
     assert res["stats"][:, 6].tolist() == [1, 1, 0, 0] and cache2.export_state(kv=False)["len"].tolist() == [n, n, 0, 0]
 
 
+@pytest.mark.parametrize("fp32", [False, True])
+def test_annsa_prepare_gives_identical_results(fp32):
+    # The query side of the selector computed ahead of time, on another stream beside the update: selection, codes,
+    # scores and outputs must be bit-identical to the plain call, and the oracle comparison holds as for it.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(head_dim=128 if not fp32 else 64, block=128 if not fp32 else 64, capacity=2048, keep_blocks=3, num_heads=3)
+    cache, w, heads, post, _, _ = full_step(cfg, fp32)
+    Q, K, V = w.chunk(cfg.prior_chunks + 1)
+    dq = fastar.to_device(Q, fp32)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        cache.annsa_prepare(dq, cfg.block)
+        done = torch.cuda.Event()
+        done.record()
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau, fp32)       # runs while / after the preparation
+    torch.cuda.current_stream().wait_event(done)
+    a = cache.annsa(dq, cfg.block, cfg.keep_blocks, debug=True)
+    b = cache.annsa(dq, cfg.block, cfg.keep_blocks, debug=True)                        # nothing prepared any more: the plain path
+    assert cache.status() == 0
+    for k in ("out", "sel", "nsel", "qcode", "scores"):
+        assert torch.equal(a[k], b[k]), k
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks, fp32)
+    # a call with other arguments discards the prepared state instead of using it
+    cache.annsa_prepare(dq, cfg.block)
+    c2 = cache.annsa(dq[:, : cfg.frame_len].contiguous(), cfg.block, cfg.keep_blocks, debug=True)
+    d2 = cache.annsa(dq[:, : cfg.frame_len].contiguous(), cfg.block, cfg.keep_blocks, debug=True)
+    assert torch.equal(c2["out"], d2["out"]) and torch.equal(c2["sel"], d2["sel"])
+
+
 def test_empty_cache_and_selector_bypass():
     torch, fastar = _gpu()
     cfg = synth.small_config(prior_chunks=1)
