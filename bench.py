@@ -464,12 +464,13 @@ def main():
     ap.add_argument("--chunks", type=int, default=120)
     ap.add_argument("--denoise-steps", type=int, default=0,
                     help="rollout mode: denoising steps per chunk, each attending to the cache plus the chunk's own un-cached K/V")
+    ap.add_argument("--sweep-point", default=None, help="sweep mode: run the single point 'd,L,den' (e.g. 128,131072,32)")
     ap.add_argument("--out", default=None)
     ap.add_argument("--no-dense", action="store_true")
     args = ap.parse_args()
     if args.mode != "step":
         import bench_modes
-        args.out = args.out or os.path.join(ROOT, "gpurun_out", "c2_rollout.json" if args.mode == "rollout" else "c4_sweep.json")
+        args.out = args.out or ("c2_rollout.json" if args.mode == "rollout" else "c4_sweep.json")
         (bench_modes.run_rollout if args.mode == "rollout" else bench_modes.run_sweep)(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

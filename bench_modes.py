@@ -1,8 +1,8 @@
 """Extra measurement modes of bench.py (not the one-line contract): the c2 long rollout with its dense
 baseline and the c4 roofline sweep.  Each writes a small JSON report and prints a text table.
 
-  python bench.py --mode rollout [--chunks 120] [--out gpurun_out/c2_rollout.json]
-  python bench.py --mode sweep   [--out gpurun_out/c4_sweep.json]
+  python bench.py --mode rollout [--chunks 120] [--out c2_rollout.json]
+  python bench.py --mode sweep   [--out c4_sweep.json] [--sweep-point d,L,den]
 """
 from __future__ import annotations
 
@@ -125,9 +125,35 @@ def run_sweep(args):
     from paper_2602_01801_b200 import fastar
 
     peak_tf, peak_gb, kind = _peaks()
+    nominal_tf, nominal_gb = 2250.0, 8000.0                    # B200 dense bf16 and HBM3e, for context beside the measured peaks
     rows = []
+    points = None
+    if getattr(args, "sweep_point", None):                      # "d,L,den": one point only (what an ncu capture runs)
+        pd, pL, pden = (int(x) for x in args.sweep_point.split(","))
+        points = {(pd, pL): pden}
+    rng = np.random.default_rng(4)
+
+    def time_s5(cache, dq, snap, base, keep, reps=5):
+        cache.profile(True)
+        for _ in range(reps):
+            cache.workspace.copy_(snap)
+            cache.annsa(dq, base.block, keep)
+        prof = cache.profile_read()
+        cache.profile(False)
+        ms = prof["s5_attention"]["ms"] / reps
+        sel_ms = sum(prof[k]["ms"] for k in ("hash", "query_hist", "s3_scores", "topk_blocks")) / reps
+        # compulsory bytes from the selection that ran: Q and O once, K, V and the bias of every key block that at
+        # least one query block of the head selected (each is fetched from HBM once and then found in L2)
+        dbg = cache.annsa(dq, base.block, keep, debug=True)
+        sel, nsel = dbg["sel"].cpu().numpy(), dbg["nsel"].cpu().numpy()
+        uniq = sum(int(np.unique(sel[h][:, : nsel[h]]).size) for h in range(sel.shape[0]))
+        tiles = sum(int(sel[h].shape[0]) * int(nsel[h]) for h in range(sel.shape[0]))
+        return ms, sel_ms, uniq, tiles
+
     for d in (128, 64):
         for L in (4096, 16384, 65536, 131072):
+            if points is not None and (d, L) not in points:
+                continue
             base = synth.sweep_config(L, d, 8)
             w = synth.Workload(base)
             H, n = base.num_heads, base.chunk_tokens
@@ -143,23 +169,40 @@ def run_sweep(args):
             snap = cache.workspace.clone()
             nkb = L // base.block
             cache.annsa(dq, base.block, max(1, nkb // 4))              # warm-up (module load, attributes)
-            for den in (4, 8, 16, 32):
+
+            def s5_row(den, variant=None):
                 keep = max(1, nkb // den)
-                sys.stderr.write(f"sweep: d={d} L={L} keep={keep}\n")
-                cache.profile(True)
-                reps = 5
-                for _ in range(reps):
-                    cache.workspace.copy_(snap)
-                    cache.annsa(dq, base.block, keep)
-                prof = cache.profile_read()
-                cache.profile(False)
-                ms = prof["s5_attention"]["ms"] / reps
-                sel_ms = sum(prof[k]["ms"] for k in ("hash", "query_hist", "s3_scores", "topk_blocks")) / reps
+                ms, sel_ms, uniq, tiles = time_s5(cache, dq, snap, base, keep)
                 flops = 4.0 * n * keep * base.block * d * H
-                unique = 2.0 * n * d * 2 * H + min(2.0 * L * d * 2 * H, 2.0 * (n // base.block) * keep * base.block * d * 2 * H) + 4.0 * L * H
-                rows.append(dict(kernel="s5_attention", L=L, d=d, keep=keep, fraction=f"1/{den}", ms=ms, selector_ms=sel_ms,
-                                 tflops=flops / (ms * 1e-3) / 1e12, frac_tensor=flops / (ms * 1e-3) / 1e12 / peak_tf,
-                                 gbs=unique / (ms * 1e-3) / 1e9, frac_hbm=unique / (ms * 1e-3) / 1e9 / peak_gb))
+                unique = 2.0 * n * d * 2 * H + uniq * base.block * (2.0 * d * 2 + 4.0)
+                row = dict(kernel="s5_attention", L=L, d=d, keep=keep, fraction=f"1/{den}", ms=ms, selector_ms=sel_ms,
+                           tflops=flops / (ms * 1e-3) / 1e12, frac_tensor=flops / (ms * 1e-3) / 1e12 / peak_tf,
+                           frac_tensor_nominal=flops / (ms * 1e-3) / 1e12 / nominal_tf,
+                           unique_blocks=uniq, tile_loads=tiles, unique_bytes=unique,
+                           gbs=unique / (ms * 1e-3) / 1e9, frac_hbm=unique / (ms * 1e-3) / 1e9 / peak_gb,
+                           frac_hbm_nominal=unique / (ms * 1e-3) / 1e9 / nominal_gb)
+                if variant:
+                    row["variant"] = variant
+                rows.append(row)
+
+            for den in ((points[(d, L)],) if points is not None else (4, 8, 16, 32)):
+                sys.stderr.write(f"sweep: d={d} L={L} 1/{den}\n")
+                s5_row(den)
+            if points is not None:
+                del cache, snap
+                torch.cuda.empty_cache()
+                continue
+            # the same cache with multiplicities drawn from 1..8 (an imported, merged state): the bias is live on every tile
+            st = cache.export_state()
+            cnt = rng.integers(1, 9, size=st["count"].shape).astype(np.int32)
+            cache.import_state(st["k"][:, :L], st["v"][:, :L], st["len"], count=cnt[:, :L], now=int(st["now"][0]) + 1)
+            assert cache.status() == 0
+            snap_m = cache.workspace.clone()
+            snap, snap_keep = snap_m, snap
+            s5_row(8, variant="imported multiplicities 1..8")
+            snap = snap_keep
+            cache.workspace.copy_(snap)
+            del st, cnt, snap_m
             cache.profile(True)
             reps = 3
             for _ in range(reps):
@@ -173,7 +216,9 @@ def run_sweep(args):
             rows.append(dict(kernel="t1_similarity", L=L, d=d, keep=None, fraction=None, ms=ms,
                              update_ms=sum(v["ms"] for v in prof.values()) / reps,
                              tflops=flops / (ms * 1e-3) / 1e12, frac_tensor=flops / (ms * 1e-3) / 1e12 / peak_tf,
-                             gbs=byts / (ms * 1e-3) / 1e9, frac_hbm=byts / (ms * 1e-3) / 1e9 / peak_gb))
+                             frac_tensor_nominal=flops / (ms * 1e-3) / 1e12 / nominal_tf,
+                             gbs=byts / (ms * 1e-3) / 1e9, frac_hbm=byts / (ms * 1e-3) / 1e9 / peak_gb,
+                             frac_hbm_nominal=byts / (ms * 1e-3) / 1e9 / nominal_gb))
             assert cache.status() == 0
             del cache, snap
             torch.cuda.empty_cache()
@@ -182,11 +227,12 @@ def run_sweep(args):
     os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
     with open(args.out, "w") as f:
         json.dump(report, f)
-    print(f"{'kernel':<14} {'L':>7} {'d':>4} {'keep':>6} {'ms':>8} {'TFLOP/s':>8} {'of peak':>8} {'GB/s':>8} {'of peak':>8}  bound")
+    print(f"{'kernel':<14} {'L':>7} {'d':>4} {'keep':>9} {'ms':>8} {'TFLOP/s':>8} {'of meas.':>8} {'of nom.':>8} {'GB/s':>8} {'of meas.':>8} {'of nom.':>8}  bound")
     for r in rows:
         bound = "tensor" if r["frac_tensor"] >= r["frac_hbm"] else "hbm"
         if r["ms"] < 0.012:
             bound = "launch latency"
         keep = "-" if r["keep"] is None else f"{r['keep']}({r['fraction']})"
-        print(f"{r['kernel']:<14} {r['L']:>7} {r['d']:>4} {keep:>6} {r['ms']:>8.4f} {r['tflops']:>8.1f} {r['frac_tensor']:>8.3f} "
-              f"{r['gbs']:>8.0f} {r['frac_hbm']:>8.3f}  {bound}")
+        print(f"{r['kernel']:<14} {r['L']:>7} {r['d']:>4} {keep:>9} {r['ms']:>8.4f} {r['tflops']:>8.1f} {r['frac_tensor']:>8.3f} "
+              f"{r['frac_tensor_nominal']:>8.3f} {r['gbs']:>8.0f} {r['frac_hbm']:>8.3f} {r['frac_hbm_nominal']:>8.3f}  {bound}"
+              + (f"  [{r['variant']}]" if r.get("variant") else ""))

@@ -50,6 +50,7 @@ extern "C" {
 #define FASTAR_ERR_TIMEOUT            -5   /* a bounded device-side wait gave up */
 #define FASTAR_ERR_NOT_SM100          -6
 #define FASTAR_ERR_WORKSPACE          -7   /* workspace buffer too small or misaligned */
+#define FASTAR_ERR_BOUNDS             -8   /* range-checking build only: a computed index left its array (access redirected) */
 
 typedef struct fastar_cache fastar_cache_t;          /* opaque host object */
 
@@ -381,6 +382,13 @@ enum {
 };
 int fastar_profile_enable(fastar_cache_t* cache, int32_t on);
 int fastar_profile_read(fastar_cache_t* cache, float* ms_by_kind, int32_t* launches_by_kind, void* stream);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper): launches one small CTA that waits, with
+ * a limit of limit_us microseconds, on an mbarrier nobody ever arrives on -- no copy or MMA is in flight -- while a
+ * second warp waits on another one and must be released by the first warp's abort flag.  The kernel returns by itself
+ * and leaves FASTAR_ERR_TIMEOUT in the cache's device status word (read it with fastar_last_device_status); this is
+ * the path every kernel of the library takes if one of its waits ever ran out.  1 <= limit_us <= 1000000. */
+int fastar_selftest_bounded_wait(fastar_cache_t* cache, int32_t limit_us, void* stream);
 
 const char* fastar_status_string(int status);
 

@@ -158,7 +158,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int i = qq / CPR, ch = qq % CPR;
       uint4 val = make_uint4(0, 0, 0, 0);
       if (i < keep_n) {
-        const int idx = list[i];
+        const int idx = FASTAR_IDX(list[i], a.np, c.status);
         val = *reinterpret_cast<const uint4*>((which ? vp_h : kp_h) + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
       }
       const uint32_t off = which * 2 * SM::kv_bytes + (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);
@@ -194,8 +194,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       auto fetch = [&](int j0, int& blk, int& page) {
         const int jj = j0 + lane;
         if (jj < ntc) {
-          blk = list ? list[jj] : jj;
-          page = pt_h[blk];
+          blk = FASTAR_IDX(list ? list[jj] : jj, c.CAPB, c.status);
+          page = FASTAR_IDX(pt_h[blk], c.pool_pages, c.status);
         } else if (SEG && jj < nt) {        // tile of the un-cached segment: its index, no page
           blk = jj - ntc;
           page = -1;
@@ -279,7 +279,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const int tok = j * BKT + i;
           uint4 val = make_uint4(0, 0, 0, 0);
           if (tok < keep_n) {
-            const int idx = list[tok];
+            const int idx = FASTAR_IDX(list[tok], a.np, c.status);
             val = *reinterpret_cast<const uint4*>(src_h + static_cast<int64_t>(idx) * a.p_token_stride + ch * 8);
           }
           const uint32_t off = (ch >> 3) * (BKT * 128) + i * 128 + (((ch & 7) ^ (i & 7)) << 4);

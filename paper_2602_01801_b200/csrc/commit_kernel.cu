@@ -79,8 +79,8 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
 
   if (w < pr.n_seg) {
     const int g = p1 - p0;
-    const int slot = slot_g;
-    const int page = pt_h[slot / c.PT];
+    const int slot = FASTAR_IDX(slot_g, c.CAP, c.status);
+    const int page = FASTAR_IDX(pt_h[slot / c.PT], c.pool_pages, c.status);
     const int m_old = c.count[sb + slot];
     const int mine = (p0 + sl < p1) ? c.order[tb + p0 + sl] : 0x7fffffff;
     const int64_t ro = (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D + sl * 8;
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
     }
     int best_i;
     if (g == 1) {
-      best_i = __shfl_sync(mask, mine, sub * LPR);
+      best_i = FASTAR_IDX(__shfl_sync(mask, mine, sub * LPR), n, c.status);
       float f[8];
       unpack8(*reinterpret_cast<const uint4*>(vh + best_i * ts + sl * 8), f);
 #pragma unroll
@@ -245,8 +245,8 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
       c.kcode[sb + slot] = code;
     }
   } else if (w - pr.n_seg < pr.n_unmatched) {
-    const int i = c.ulist[tb + (w - pr.n_seg)];
-    const int slot = c.dest[tb + i];
+    const int i = FASTAR_IDX(c.ulist[tb + (w - pr.n_seg)], n, c.status);
+    const int slot = FASTAR_IDX(c.dest[tb + i], c.CAP, c.status);
     const uint4 krow = *reinterpret_cast<const uint4*>(kh + i * ts + sl * 8);
     const uint4 vrow = *reinterpret_cast<const uint4*>(vh + i * ts + sl * 8);
     uint4 code8 = make_uint4(0u, 0u, 0u, 0u);
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(256) commit_kernel(const CacheView c, const __
       rn = c.rnorm_new[tb + i];
       code = c.code_new[tb + i];
     }
-    const int page = pt_h[slot / c.PT];
+    const int page = FASTAR_IDX(pt_h[slot / c.PT], c.pool_pages, c.status);
     const int64_t ro = (static_cast<int64_t>(page) * c.PT + (slot % c.PT)) * c.D + sl * 8;
     *reinterpret_cast<uint4*>(c.pool_k + ro) = krow;
     *reinterpret_cast<uint4*>(c.pool_v + ro) = vrow;

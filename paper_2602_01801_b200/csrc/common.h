@@ -156,6 +156,7 @@ struct AttnArgs {
   // rows (0 for a token, -inf past its end), seg_tiles * page_tokens floats
   int seg_tiles;
   const float* seg_bias;
+  int np;                  // gather mode: prompt tokens (range of the kept indices)
   // gather mode: kept tokens of every frame, [H][keep_frames_stride] (nullptr: `keep` for all frames)
   const int32_t* keep_frames;
   int keep_frames_stride;
@@ -182,6 +183,7 @@ int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, in
 int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st);
 int launch_reset(const CacheView& c, cudaStream_t st);
 int launch_import_derive(const CacheView& c, cudaStream_t st);
+int launch_bounded_wait_selftest(const CacheView& c, int limit_us, int* released, cudaStream_t st);
 int launch_copy_outputs(const CacheView& c, int n, int32_t* match_out, float* sim_out, int32_t* dest_out, cudaStream_t st);
 int launch_decode_rel(const CacheView& c, int n_frames, int np, float scale, float* rel_out, cudaStream_t st);
 

@@ -759,6 +759,7 @@ int fastar_annca_attention(fastar_cache_t* c, const void* q, const void* k_promp
   a.block_q = 128;
   a.rows_per_frame = frame_len;
   a.keep = keep;
+  a.np = np;
   a.n_frames = F;
   a.kp = kpb;
   a.vp = vpb;
@@ -839,6 +840,7 @@ int fastar_annca_attention_lsh(fastar_cache_t* c, const void* q, const void* k_p
   a.block_q = 128;
   a.rows_per_frame = frame_len;
   a.keep = np;                      // upper bound; the kept count of every frame comes from keep_frames
+  a.np = np;
   a.keep_frames = v.nselp;
   a.keep_frames_stride = v.max_frames;
   a.n_frames = F;
@@ -950,6 +952,19 @@ int fastar_last_device_status(fastar_cache_t* c, void* stream) {
   return status;
 }
 
+int fastar_selftest_bounded_wait(fastar_cache_t* c, int32_t limit_us, void* stream) {
+  if (!c || limit_us < 1 || limit_us > 1000000) return FASTAR_ERR_INVALID_ARG;
+  DeviceGuard guard(c->desc.device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* released = c->v.nsel;                 // a scratch word: 1 = the second warp left through the abort flag
+  if (cudaMemsetAsync(released, 0, 4, st) != cudaSuccess) return FASTAR_ERR_CUDA;
+  ACC(launch_bounded_wait_selftest(c->v, limit_us, released, st));
+  int rel = 0;
+  if (cudaMemcpyAsync(&rel, released, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return FASTAR_ERR_CUDA;
+  return rel == 1 ? FASTAR_OK : FASTAR_ERR_CUDA;
+}
+
 int64_t fastar_launch_count(const fastar_cache_t* c) { return c ? c->launches : 0; }
 
 int fastar_profile_enable(fastar_cache_t* c, int32_t on) {
@@ -985,6 +1000,7 @@ const char* fastar_status_string(int status) {
     case FASTAR_ERR_TIMEOUT: return "a bounded device-side wait gave up";
     case FASTAR_ERR_NOT_SM100: return "device is not compute capability 10.x";
     case FASTAR_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case FASTAR_ERR_BOUNDS: return "range-checking build: a computed index left its array";
     default: return "unknown status";
   }
 }

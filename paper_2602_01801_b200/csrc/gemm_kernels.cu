@@ -133,8 +133,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       for (int tl = 0; tl < ntl; ++tl) {
         const int t = t0 + tl;
         if (EPI == EPI_ARGMAX && (tl & 31) == 0 && tl + lane < ntl) {
-          pg0 = pt_h[(t + lane) * pages_per_tile];
-          pg1 = pages_per_tile == 2 ? pt_h[(t + lane) * pages_per_tile + 1] : 0;
+          pg0 = FASTAR_IDX(pt_h[(t + lane) * pages_per_tile], c.pool_pages, c.status);
+          pg1 = pages_per_tile == 2 ? FASTAR_IDX(pt_h[(t + lane) * pages_per_tile + 1], c.pool_pages, c.status) : 0;
         }
         const int page0 = __shfl_sync(0xffffffffu, pg0, tl & 31);
         const int page1 = __shfl_sync(0xffffffffu, pg1, tl & 31);
@@ -440,7 +440,7 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int pg = 0;
       for (int tl = 0; tl < ntl; ++tl) {
         const int t = t0 + tl;
-        if ((tl & 31) == 0 && tl + lane < ntl) pg = pt_h[(t + lane) * pages_per_tile + page_sel];
+        if ((tl & 31) == 0 && tl + lane < ntl) pg = FASTAR_IDX(pt_h[(t + lane) * pages_per_tile + page_sel], c.pool_pages, c.status);
         const int page = __shfl_sync(0xffffffffu, pg, tl & 31);
         if (lane == 0 && ok) {
           for (int kc = 0; kc < nkc; ++kc, ++it) {

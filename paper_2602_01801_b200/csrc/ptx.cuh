@@ -15,10 +15,27 @@ namespace fastar {
 // ---------------------------------------------------------------------------------------------
 constexpr int kErrCapacity = -3;
 constexpr int kErrTimeout = -5;
+constexpr int kErrBounds = -8;
 
 __device__ __forceinline__ void record_status(int* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
+
+// Range checks of computed indices (slot, block, page, token, output position), compiled in with -DFASTAR_DEBUG_BOUNDS:
+// a violation is recorded in the status word and the index is replaced by 0, so the access that follows stays inside
+// the array and the kernel runs to its end.  The regular build passes the index through.
+#ifdef FASTAR_DEBUG_BOUNDS
+__device__ __forceinline__ int checked_index(int idx, int n, int* status) {
+  if (idx < 0 || idx >= n) {
+    record_status(status, kErrBounds);
+    return 0;
+  }
+  return idx;
+}
+#define FASTAR_IDX(idx, n, status) ::fastar::checked_index((idx), (n), (status))
+#else
+#define FASTAR_IDX(idx, n, status) (idx)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -82,7 +99,8 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 // Bounded wait.  `abort_flag` is a shared-memory word every role of the CTA polls, so that one
 // role giving up releases the others quickly.  Returns false when the wait was abandoned.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -91,7 +109,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       uint64_t t = global_timer_ns();
       if (t0 == 0) t0 = t;
-      else if (t - t0 > kWaitLimitNs) {
+      else if (t - t0 > limit_ns) {
         *abort_flag = 1;
         record_status(status, kErrTimeout);
         return false;

@@ -320,8 +320,8 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       for (int tl = 0; tl < ntl; ++tl) {
         const int t = t0 + tl;
         if (!COLMAX && (tl & 31) == 0 && tl + lane < ntl) {      // page ids of 32 tiles with one coalesced load
-          pg0 = pt_h[(t + lane) * pages_per_tile];
-          pg1 = pages_per_tile == 2 ? pt_h[(t + lane) * pages_per_tile + 1] : 0;
+          pg0 = FASTAR_IDX(pt_h[(t + lane) * pages_per_tile], c.pool_pages, c.status);
+          pg1 = pages_per_tile == 2 ? FASTAR_IDX(pt_h[(t + lane) * pages_per_tile + 1], c.pool_pages, c.status) : 0;
         }
         const int page0 = __shfl_sync(0xffffffffu, pg0, tl & 31);
         const int page1 = __shfl_sync(0xffffffffu, pg1, tl & 31);

@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(256) match_count_kernel(const CacheView c, int
     int j = -1;
     float s = 0.f;
     if (b != 0ull) {
-      j = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull));
+      j = FASTAR_IDX(static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull)), c.CAP, c.status);
       s = ordered_to_float(static_cast<uint32_t>(b >> 32));
     }
     const bool matched = j >= 0 && s >= tau;
@@ -465,7 +465,8 @@ __global__ void __launch_bounds__(1024) plan_kernel(const CacheView c, int n) {
   __syncthreads();
   // destinations (matched tokens get theirs in the scatter kernel)
   if (ok) {
-    for (int k = tid; k < U; k += blockDim.x) c.dest[tb + c.ulist[tb + k]] = k < A ? L + k : c.victims[tb + k - A];
+    for (int k = tid; k < U; k += blockDim.x)
+      c.dest[tb + FASTAR_IDX(c.ulist[tb + k], n, c.status)] = FASTAR_IDX(k < A ? L + k : c.victims[tb + k - A], c.CAP, c.status);
   } else {
     for (int i = tid; i < n; i += blockDim.x) c.dest[tb + i] = -1;
     if (tid == 0) record_status(c.status, kErrCapacity);
@@ -494,7 +495,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(const CacheView c, int n) 
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
     const int j = c.match[tb + i];
     if (j >= 0) {
-      const int pos = atomicAdd(c.cur + static_cast<int64_t>(h) * c.CAP + j, 1);
+      const int pos = FASTAR_IDX(atomicAdd(c.cur + static_cast<int64_t>(h) * c.CAP + FASTAR_IDX(j, c.CAP, c.status), 1), n, c.status);
       c.order[tb + pos] = i;
       c.dest[tb + i] = j;
     }
@@ -519,7 +520,7 @@ __global__ void __launch_bounds__(256) probe_cosine_kernel(const CacheView c, co
     const int64_t tb = static_cast<int64_t>(h) * c.max_tokens;
     const unsigned long long b = c.best[tb + i];
     if (b == 0ull) continue;                         // empty cache: nothing was ranked (same for all 16 lanes)
-    const int j = static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull));
+    const int j = FASTAR_IDX(static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(b & 0xFFFFFFFFull)), c.CAP, c.status);
     float dot = 0.f;
     if (e8 * 8 < c.D) {
       const uint4 a = *reinterpret_cast<const uint4*>(k_new + h * hs + i * ts + e8 * 8);
@@ -645,7 +646,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
                                                    const int32_t* __restrict__ len, int len_div, int n_fixed, int keep,
                                                    int32_t* __restrict__ out, int64_t out_head_stride, int out_row_stride,
                                                    int out_fill, int32_t* __restrict__ nsel, int force_first, int force_last,
-                                                   const float* __restrict__ src_hi) {
+                                                   const float* __restrict__ src_hi, int* status) {
   extern __shared__ uint32_t vals[];     // ranking keys: larger key = better entry
   __shared__ int red[32];
   const int row = blockIdx.x, h = blockIdx.y;
@@ -684,7 +685,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
     }
     int tot;
     const int pos = run + block_exscan(take, red, &tot);
-    if (take) orow[pos] = i;
+    if (take) orow[FASTAR_IDX(pos, k, status)] = i;
     run += tot;
   }
   for (int i = k + threadIdx.x; i < out_fill; i += blockDim.x) orow[i] = -1;
@@ -694,7 +695,7 @@ int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, in
   topk_kernel<false><<<dim3(nqb, c.H), 256, c.CAPB * 4, st>>>(c.scores, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB, c.len,
                                                             c.PT, 0, keep, c.sel, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB,
                                                             min(keep, c.CAPB), c.nsel, force_sink, force_recent,
-                                                            c.hist_weighted ? c.scores_hi : nullptr);
+                                                            c.hist_weighted ? c.scores_hi : nullptr, c.status);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 // ---------------------------------------------------------------------------------------------
@@ -749,7 +750,7 @@ int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaS
   topk_kernel<true><<<dim3(n_frames, c.H), 256, np * 4, st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
                                                              c.max_prompt, nullptr, 1, np, keep, c.selp,
                                                              static_cast<int64_t>(c.max_frames) * c.max_prompt, c.max_prompt,
-                                                             min(keep, np), nullptr, 0, 0, nullptr);
+                                                             min(keep, np), nullptr, 0, 0, nullptr, c.status);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
@@ -821,6 +822,36 @@ int launch_import_derive(const CacheView& c, cudaStream_t st) {
   int r2 = launch_finalize_hist(c, nullptr, -1, st);
   if (r2 < 0) return r2;
   return r + 1 + r2 + r3;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded waits: warp 0 waits on a barrier that never completes and gives up after `limit_ns`
+// (status word <- time-out, abort flag set); warp 1 waits on a second dead barrier with the full limit and must be
+// released by the abort flag.  `released` receives 1 when it was.  Nothing is in flight, so the CTA simply returns.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns, int* released) {
+  __shared__ __align__(8) unsigned long long bars[2];
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars[0]), 1);
+    mbar_init(smem_u32(&bars[1]), 1);
+    abort_word = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5;
+  if (warp == 0) {
+    const bool ok = mbar_wait(smem_u32(&bars[0]), 0, abort_flag, status, limit_ns);
+    if (ok && threadIdx.x == 0) record_status(status, FASTAR_ERR_CUDA);      // cannot happen: nobody arrives
+  } else {
+    const bool ok = mbar_wait(smem_u32(&bars[1]), 0, abort_flag, nullptr);
+    if (threadIdx.x == 32) *released = ok ? 0 : 1;
+  }
+}
+int launch_bounded_wait_selftest(const CacheView& c, int limit_us, int* released, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(c.status, static_cast<unsigned long long>(limit_us) * 1000ull, released);
+  return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
 int launch_copy_outputs(const CacheView& c, int n, int32_t* match_out, float* sim_out, int32_t* dest_out, cudaStream_t st) {

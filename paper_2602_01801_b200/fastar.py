@@ -13,7 +13,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "lib
 _lib = None
 
 OK = 0
-ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_SM100, ERR_WORKSPACE = range(-1, -8, -1)
+ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_SM100, ERR_WORKSPACE, ERR_BOUNDS = range(-1, -9, -1)
 BF16, FP32 = 0, 1
 
 
@@ -60,6 +60,7 @@ SIGNATURES = {
                                              _vp]),
     "fastar_attention_step_host": (C.c_int, [_vp] * 8 + [_i32, _i32, _i32, _f32, _i32, _i32, _i32, _i32, _vp]),
     "fastar_last_device_status": (C.c_int, [_vp, _vp]),
+    "fastar_selftest_bounded_wait": (C.c_int, [_vp, _i32, _vp]),
     "fastar_launch_count": (C.c_int64, [_vp]),
     "fastar_annca_select_noalloc": (C.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _vp, _vp]),
     "fastar_noalloc_last_status": (C.c_int, [_vp]),
@@ -153,6 +154,11 @@ class Cache:
 
     def status(self) -> int:
         return self.lib.fastar_last_device_status(self.handle, _stream())
+
+    def selftest_bounded_wait(self, limit_us: int = 1000) -> None:
+        """Lets a device-side wait run out on purpose (a barrier nobody signals, nothing in flight); afterwards
+        status() returns ERR_TIMEOUT once."""
+        _check(self.lib.fastar_selftest_bounded_wait(self.handle, int(limit_us), _stream()), "fastar_selftest_bounded_wait")
 
     def launch_count(self) -> int:
         return self.lib.fastar_launch_count(self.handle)

@@ -183,6 +183,54 @@ def test_c2_rollout_at_full_size_against_the_oracle_at_checkpoints():
     assert evicted.sum() > 0 and evicting_checkpoints >= 3, "the eviction tail was not reached"
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_c4_sweep_shapes_long_lists_and_imported_multiplicities(d):
+    """The shapes of the roofline sweep (benchmark config 4) that nothing else reaches: 131072 cached keys in 1024
+    key blocks, 8 heads, 4096 queries, kept fractions 1/4 (lists of 256 tiles) and 1/32, head dim 64 and 128.  The
+    cache is imported with multiplicities drawn from 1..8, so the log m bias is live on every tile.  Codes, block
+    scores and selections are checked in full for two heads, the attention on sampled query blocks."""
+    import torch
+    from paper_2602_01801_b200 import fastar
+
+    L = 131072
+    cfg = synth.sweep_config(L, d, 4)
+    w = synth.Workload(cfg)
+    H, n = cfg.num_heads, cfg.chunk_tokens
+    R = w.lsh_projection()
+    cache = fastar.Cache(H, d, cfg.capacity, cfg.block, R, cfg.lsh_tables, cfg.lsh_bits, max_tokens=n,
+                         max_prompt_tokens=cfg.prompt_tokens, max_frames=1)
+    ks, vs = [], []
+    for ci in range(cfg.prior_chunks):
+        _, K, V = w.chunk(ci)
+        ks.append(fastar.bf16_bits(K))
+        vs.append(fastar.bf16_bits(V))
+    kb, vb = np.concatenate(ks, axis=1), np.concatenate(vs, axis=1)
+    rng = np.random.default_rng(4)
+    count = rng.integers(1, 9, size=(H, L)).astype(np.int32)
+    cache.import_state(kb, vb, np.full(H, L, np.int32), count=count, now=1)
+    assert cache.status() == 0
+    post = cache.export_state()
+    assert np.array_equal(post["count"][:, :L], count) and np.all(post["len"] == L)
+    Q, _, _ = w.chunk(cfg.prior_chunks)
+    dq = fastar.to_device(Q)
+    heads = P.oracle_heads_from_export(post)
+    nqb = n // cfg.block
+    for keep in (L // cfg.block // 4, L // cfg.block // 32):
+        a = cache.annsa(dq, cfg.block, keep, debug=True)
+        assert cache.status() == 0
+        out = a["out"].float().cpu().numpy()
+        for h in (0, H - 1):
+            hc = heads[h]
+            qcodes = P.check_codes(Q[h], R, cfg.lsh_tables, cfg.lsh_bits, a["qcode"][h].cpu().numpy().view(np.uint32))
+            kcodes = P.check_codes(P.bits_to_f64(post["k"][h, :L]), R, cfg.lsh_tables, cfg.lsh_bits, post["code"][h, :L])
+            sel = P.check_selection(qcodes, kcodes, n, L, cfg.block, cfg.block, cfg.lsh_bits, keep, a["scores"][h].cpu().numpy(),
+                                    a["sel"][h].cpu().numpy(), int(a["nsel"][h]))
+            blocks = [0, int(rng.integers(1, nqb - 1)), nqb - 1]
+            for blk, want in _oracle_blocks(Q[h], hc, sel, blocks, cfg.block, cfg.block).items():
+                rows = slice(blk * cfg.block, (blk + 1) * cfg.block)
+                P.check_attention(out[h][rows], want, f"c4 d={d} keep={keep} head {h} block {blk}")
+
+
 def test_c1_full_size_update_with_eight_bit_search_sampled():
     """The 8-bit quantised correspondence search at full c1 size: quantiser and top-1 on sampled tokens of three heads
     (the oracle's scores of the GPU's codes), merge bookkeeping in full for those heads, invariants for all heads."""

@@ -437,6 +437,23 @@ def test_annsa_prepare_gives_identical_results(fp32):
     assert torch.equal(c2["out"], d2["out"]) and torch.equal(c2["sel"], d2["sel"])
 
 
+def test_a_bounded_wait_that_runs_out_reports_a_timeout_and_leaves_the_context_usable():
+    # Every device-side wait of the library gives up after a time limit, sets the CTA's abort flag (which releases the
+    # other roles) and records FASTAR_ERR_TIMEOUT.  The self-test kernel makes that happen on purpose, harmlessly: a
+    # barrier nobody signals, a 1 ms limit, nothing in flight.  The status is reported once and work goes on.
+    torch, fastar = _gpu()
+    cfg = synth.small_config(num_heads=2, capacity=1024)
+    cache, w, heads, post, _, _ = full_step(cfg)
+    cache.selftest_bounded_wait(1000)
+    assert cache.status() == fastar.ERR_TIMEOUT
+    assert cache.status() == 0
+    Q, K, V = w.chunk(cfg.prior_chunks + 1)
+    post = gpu_update_checked(cache, heads, K, V, cfg.frame_len, cfg.tau)       # the cache still works and still matches
+    gpu_annsa_checked(cache, cfg, w, Q, post, cfg.keep_blocks)
+    with pytest.raises(fastar.FastarError):
+        cache.selftest_bounded_wait(0)
+
+
 def test_empty_cache_and_selector_bypass():
     torch, fastar = _gpu()
     cfg = synth.small_config(prior_chunks=1)
