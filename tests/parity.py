@@ -3,7 +3,7 @@ oracle.  This module imports only the oracle and numpy; it never touches the CUD
 two implementations stay independent.  Near-ties have several correct answers, hence the stages:
 
   T1  accept j iff cos_oracle(i, j) >= best_i - 1e-4                  (bit-equal wherever the margin is larger)
-      (8-bit search: the quantiser is checked byte by byte, then the scores of the codes produced, margin 5e-4)
+      (8-bit search: the quantiser is checked byte by byte, then the scores of the codes produced, same margin)
   T2  matched flags agree wherever |best_i - tau| > 1e-4
   T3/T4  the decisions taken are fed to the oracle's merge -> dest, len, count, stamp, K rows bit-exact,
          V rows within one bf16 ulp
@@ -21,7 +21,11 @@ import numpy as np
 from oracle import fastar_oracle as O
 
 MARGIN = 1e-4
-MARGIN_Q8 = 5e-4      # 8-bit search: the fp8 tensor-core accumulation is not bit-exact fp32
+# 8-bit search: the scores the GPU forms from its codes (tcgen05 kind::f8f6f4, fp32 accumulation) differ from the oracle's
+# fp64 scores of the same codes by at most 1.4e-7 (measured over the small cases and the full c1 size; Q8_OBSERVED
+# below keeps the running maximum), so the 8-bit search is held to the same tie window as the bf16 search.
+MARGIN_Q8 = 1e-4
+Q8_OBSERVED = {"max_abs_diff": 0.0}   # largest |GPU score - oracle score of the same codes| seen by check_update (8-bit search)
 ATT_MAX_ABS = 2e-2
 ATT_REL_L2 = 1e-2
 
@@ -59,7 +63,7 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
     matched = match >= 0
     idx = np.arange(n) if rows is None else rows
     margin = MARGIN if codes is None else MARGIN_Q8
-    sim_tol = 2e-5 if codes is None else MARGIN_Q8
+    sim_tol = 2e-5
     if pre.L > 0 and hamming is not None:
         # integer ranking: the slot is the arg-min of the Hamming distance of the GPU's own sign bits, exactly
         codes_new, codes_cache, bits = hamming
@@ -114,6 +118,8 @@ def check_update(pre: O.HeadCache, K_new: np.ndarray, V_new: np.ndarray, frame_l
         ui = mi[uniq[mi]]
         assert np.array_equal(match[idx][ui], np.argmax(cosm[ui], axis=1)), "T1: index differs outside the tie window"
         # the similarity reported is the cosine of the best slot
+        if codes is not None:
+            Q8_OBSERVED["max_abs_diff"] = max(Q8_OBSERVED["max_abs_diff"], float(np.max(np.abs(sim[idx] - cbest))))
         assert np.max(np.abs(sim[idx] - cbest)) <= sim_tol, "T1: similarity value"
         # T2
         far = np.abs(cbest - tau) > margin
