@@ -79,12 +79,12 @@ typedef struct {
                               * then ranks prompt tokens by max_i code(q_i).code(k_p) |q_i| |k_p| / (256 sqrt d)
                               * (codes of its queries and prompt keys are made per call); the attention over
                               * the kept tokens uses the bf16 tensors.
-                              * 1 = the LSH flavour (Section 5.1, "LSH"): the code row of a key holds the T*b sign
+                              * 1 = the LSH flavour (Section 5.1, LSH): the code row of a key holds the T*b sign
                               * bits of the shared projection as +1 / -1; TempCache's correspondence is the live
                               * slot at the smallest Hamming distance (ties: lowest slot) and the threshold is
                               * applied to the exact cosine of that slot.  AnnCA is not affected (use
                               * fastar_annca_attention_lsh for its LSH flavour); the probe update is refused. */
-  int32_t representative;    /* key a merged slot keeps (Appendix C, "Representative selection"):
+  int32_t representative;    /* key a merged slot keeps (Appendix C, on the choice of the representative):
                               * FASTAR_REP_LAST_KEY (0, the paper's choice) = the key of its newest matching
                               * token; FASTAR_REP_MEAN_KEY (1, the ablation's alternative) = the count-weighted
                               * mean (m_j K_j + sum k_i)/(m_j + g), summed in fp32 in ascending token order and
@@ -194,7 +194,7 @@ int fastar_tempcache_update(fastar_cache_t* cache, const void* k_new, const void
                             int32_t* match_out, float* sim_out, int32_t* dest_out,
                             fastar_update_stats* stats_out, void* stream);
 
-/* TempCache update with query-probe correspondence (Section 5.2, "Finding temporal correspondences":
+/* TempCache update with query-probe correspondence (Section 5.2, the paragraph on how correspondences are found:
  * the corresponding token of a current-frame query is the cached key with the highest attention
  * score).  As fastar_tempcache_update, except that the slot is chosen by the probe rows,
  *   j*_i = argmax_j <q_i, K_j> over live slots (ties: lowest slot),

@@ -13,15 +13,15 @@ steps; there is no blocking, fusion or reordering beyond the stated algorithm.
 Paper passages followed
   * Eq. 1 (Section 3)            dense cached attention            -> dense_attention
   * Section 5.1                  attention over a candidate set    -> sparse_attention
-  * Section 5.2 "Finding temporal correspondences"  top-1 key      -> top1_cosine
+  * Section 5.2 (how correspondences are found)  top-1 key      -> top1_cosine
   * Section 5.2 (same paragraph) query-probe form: highest attention
                                  score of the token's query             -> top1_query_probe
-  * Section 5.1 "quantised similarity search"  8-bit codes         -> key_codes_e4m3, top1_quantized,
+  * Section 5.1 (quantised search)  8-bit codes         -> key_codes_e4m3, top1_quantized,
                                                                       prompt_relevance_quantized
   * Section 5.2 / Appendix C     threshold merge, last-key representative,
                                  mean value, multiplicity m        -> tempcache_update
   * Lemma 1 (Section 5.2, Appendix A)  + log m bias                -> sparse_attention
-  * Section 5.1 "LSH"            shared random projection, buckets -> lsh_codes
+  * Section 5.1 (LSH)            shared random projection, buckets -> lsh_codes
   * Section 5.4 (AnnSA)          same-bucket rule, block-sparse    -> block_histograms,
                                                                       block_scores, topk_lowest_index
   * Section 5.3 (AnnCA)          prompt token kept iff a current-frame query
@@ -30,9 +30,9 @@ Paper passages followed
                                  of the frame                      -> prompt_bucket_selection, annca_lsh
   * Eq. 1 (Section 3)            attended set = current frames' K/V joined
                                  with the cache                    -> sparse_attention_with_segment
-  * Appendix C "Representative selection"  mean key (ablation)     -> tempcache_update(representative="mean")
+  * Appendix C (choice of the representative)  mean key (ablation)     -> tempcache_update(representative="mean")
   * selector option (no passage) forced sink / recent blocks       -> select_blocks
-  * Section 4 / Section 6 "Metrics"  recall, density              -> attention_recall, density
+  * Section 4 / Section 6 (metrics)  recall, density              -> attention_recall, density
 
 Pinned by tests/test_oracle_pins.py: Lemma exactness, brute-force nearest
 neighbour, cache invariants, reduction to dense attention (checked against
@@ -145,7 +145,7 @@ def top1_cosine(K_new: np.ndarray, cache: HeadCache) -> Tuple[np.ndarray, np.nda
 
 
 # ---------------------------------------------------------------------------------------------------
-# 8-bit quantised similarity search (Section 5.1 "quantised similarity search", 8 bits being the
+# 8-bit quantised similarity search (Section 5.1 (quantised search), 8 bits being the
 # paper's default, Section 6 / Appendix C bit-width ablation).  Reading taken here: a key is scaled
 # to unit length, multiplied by E4M3_SCALE and every component is rounded to an 8-bit float
 # (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448;
@@ -216,11 +216,11 @@ def probe_scores_quantized(codes_q: np.ndarray, codes_k: np.ndarray, K_cache: np
 
 
 def top1_query_probe(Q_new: np.ndarray, K_new: np.ndarray, cache: HeadCache, search_bits: int = 16) -> Tuple[np.ndarray, np.ndarray]:
-    """Correspondence read off the attention scores (Section 5.2, "Finding temporal correspondences"):
+    """Correspondence read off the attention scores (Section 5.2, where correspondences are found):
     the token corresponding to query q_i is the live cached key with the highest score <q_i, k_j>
     (softmax and the 1/sqrt(d) scale are monotone, so this is the highest attention weight; ties ->
     smallest slot).  Returns (j*, cos(k_i, k_j*)): the similarity the merge threshold is applied to is
-    that of the keys (Appendix C, "key-similarity threshold").  j* = -1, c* = 0 on an empty cache.
+    that of the keys (Appendix C, on the similarity threshold).  j* = -1, c* = 0 on an empty cache.
     search_bits = 8 ranks with probe_scores_quantized instead of the exact dot products; the cosine of the
     winner is always exact."""
     Q_new = np.asarray(Q_new, np.float64)
@@ -249,7 +249,7 @@ def hamming_distances(codes_a: np.ndarray, codes_b: np.ndarray, bits: int) -> np
 
 def top1_hamming(K_new: np.ndarray, cache: HeadCache, R: np.ndarray, tables: int, bits: int,
                  codes_new: Optional[np.ndarray] = None, codes_cache: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
-    """The LSH flavour of the correspondence search (Section 5.1 "LSH", Section 5.2): keys are compared through the
+    """The LSH flavour of the correspondence search (Section 5.1 (LSH), Section 5.2): keys are compared through the
     T*b sign bits of the shared random projection; the corresponding token of a new key is the live cached key at
     the smallest Hamming distance (ties -> smallest slot).  Returns (j*, cos(k_i, k_j*)): the merge threshold is
     applied to the exact cosine of that key.  codes_*: bucket ids computed elsewhere (staged parity)."""

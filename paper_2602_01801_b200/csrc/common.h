@@ -85,7 +85,7 @@ struct CacheView {
   float* kpn_ca;                   // [H][max_prompt]  |k_p|
   uint8_t* q8_probe;               // [H][max_tokens][128]  codes of the probe rows of a query-probe update
   float* qn_probe;                 // [H][max_tokens]  their norms (written by the quantiser, not used)
-  // Query-probe correspondence (Section 5.2, "the key with the highest attention score"): the similarity kernels
+  // Query-probe correspondence (Section 5.2: a query corresponds to the cached key it attends to most): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
   int hist_weighted;               // key histograms count a slot m times (selector option); high digits in hk_hi / scores_hi

@@ -1,4 +1,4 @@
-// 8-bit quantised correspondence search for TempCache (paper Section 5.1, "quantised similarity search": 8 bits is
+// 8-bit quantised correspondence search for TempCache (paper Section 5.1 on the quantised search: 8 bits is
 // the paper's default; Section 5.2 uses it for the top-1 lookup).
 //
 // A key's search code is its direction in fp8 e4m3: x / |x| * 16, every component rounded to nearest even,
