@@ -44,6 +44,8 @@ def load_peaks():
 def workload_config(name: str) -> synth.WorkloadConfig:
     if name == "small":
         return synth.small_config()
+    if name == "c4":               # one point of the roofline sweep: 8 heads, d = 128, 65 536 cached keys, keep 1/8
+        return synth.sweep_config(65536, 128, 8)
     return synth.CONFIGS[name]
 
 
@@ -447,7 +449,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c1", choices=["c1", "c3", "c0", "small"])
+    ap.add_argument("--workload", default="c1", choices=["c1", "c3", "c4", "c0", "small"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--search-bits", type=int, default=16, choices=[16, 8, 1],
                     help="TempCache correspondence search on the bf16 keys (16, default) or on their 8-bit codes (8)")
