@@ -116,18 +116,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
   if (valid_rows <= 0) return;          // uniform for the CTA; nothing allocated yet
 
-  if (threadIdx.x == 0) {
-    mbar_init(bar_q_full, 1);
-    for (int s = 0; s < RS; ++s) { mbar_init(bar_r_full + 8 * s, 1); mbar_init(bar_r_empty + 8 * s, 1); }
-    for (int s = 0; s < NB; ++s) mbar_init(bar_b_full + 8 * s, 1);
-    for (int g = 0; g < 2; ++g) {
-      mbar_init(bar_s_full + 8 * g, 1);
-      mbar_init(bar_s_empty + 8 * g, 4);       // one arrival per warp of the group
-      mbar_init(bar_p_full + 8 * g, 4);
-      mbar_init(bar_pv_done + 8 * g, 1);
+  // one thread per barrier: q_full, r_full[RS], r_empty[RS], b_full[NB], s_full[2], s_empty[2], p_full[2], pv_done[2], xchg
+  {
+    constexpr int kNumBars = 1 + 2 * RS + NB + 8 + 1;
+    static_assert(kNumBars * 8 == kBarBytes, "barrier table");
+    const int b = threadIdx.x;
+    if (b < kNumBars) {
+      const int grp = b - (1 + 2 * RS + NB);          // index inside the last nine
+      mbar_init(bar + 8 * b, grp < 0 ? 1u : (grp == 8 ? 8u : ((grp >= 2 && grp < 6) ? 4u : 1u)));
     }
-    mbar_init(bar_xchg, 8);
-    *abort_flag = 0;
+    if (threadIdx.x == 0) *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == kProducerWarp && lane == 0) {
