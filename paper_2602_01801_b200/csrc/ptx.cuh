@@ -69,15 +69,28 @@ __device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// HINT_NS > 0: the suspend-time hint of try_wait, in nanoseconds (how long the hardware may park the thread before
+// it answers "not yet"; the thread still wakes as soon as the phase completes).  0: the default limit.
+template <uint32_t HINT_NS = 0>
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
+  if constexpr (HINT_NS > 0) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(HINT_NS)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+  }
   return ok;
 }
 // Non-blocking test (try_wait may suspend the thread for a while before it answers; a loop that watches two
@@ -99,12 +112,13 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 // Bounded wait.  `abort_flag` is a shared-memory word every role of the CTA polls, so that one
 // role giving up releases the others quickly.  Returns false when the wait was abandoned.
+template <uint32_t HINT_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           uint64_t limit_ns = kWaitLimitNs) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait<HINT_NS>(bar, parity)) return true;
   uint64_t t0 = 0;
   for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait<HINT_NS>(bar, parity)) return true;
     if ((it & 255u) == 0) {
       if (*abort_flag) return false;
       uint64_t t = global_timer_ns();
@@ -338,16 +352,25 @@ __device__ __forceinline__ void fmul2(float& x0, float& x1, float a0, float a1, 
 }
 // Maximum of 32 scores x[j] = acc[j] * rn[j] and, only when it beats `best`, its first column.
 // acc: raw accumulator bits; rn: 32 floats (16-byte aligned, shared or registers via pointer).
-__device__ __forceinline__ void chunk_argmax(const uint32_t (&acc)[32], const float4* rn4, int valid, int jbase, float& best,
-                                             int& best_j) {
+// MASK: columns >= valid do not count (only the last tile of a cache has any; the caller peels that tile off so that
+// the common path carries no masking code).  SCALE = false ranks the scores as they are (rn4 unused).
+template <bool MASK, bool SCALE>
+__device__ __forceinline__ void chunk_argmax_t(const uint32_t (&acc)[32], const float4* rn4, int valid, int jbase, float& best,
+                                               int& best_j) {
   float x[32];
+  if (SCALE) {
 #pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    const float4 r = rn4[u];
-    fmul2(x[4 * u], x[4 * u + 1], __uint_as_float(acc[4 * u]), __uint_as_float(acc[4 * u + 1]), r.x, r.y);
-    fmul2(x[4 * u + 2], x[4 * u + 3], __uint_as_float(acc[4 * u + 2]), __uint_as_float(acc[4 * u + 3]), r.z, r.w);
+    for (int u = 0; u < 8; ++u) {
+      const float4 r = rn4[u];
+      fmul2(x[4 * u], x[4 * u + 1], __uint_as_float(acc[4 * u]), __uint_as_float(acc[4 * u + 1]), r.x, r.y);
+      fmul2(x[4 * u + 2], x[4 * u + 3], __uint_as_float(acc[4 * u + 2]), __uint_as_float(acc[4 * u + 3]), r.z, r.w);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(acc[j]);
   }
-  if (valid < 32) {
+  if (MASK) {
+    if (valid <= 0) return;
 #pragma unroll
     for (int j = 0; j < 32; ++j)
       if (j >= valid) x[j] = -INFINITY;
@@ -366,32 +389,6 @@ __device__ __forceinline__ void chunk_argmax(const uint32_t (&acc)[32], const fl
     best_j = jbase + idx;
   }
 }
-
-// The same without the per-column factor (scores ranked as they are).
-__device__ __forceinline__ void chunk_argmax_plain(const uint32_t (&acc)[32], int valid, int jbase, float& best, int& best_j) {
-  float x[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(acc[j]);
-  if (valid < 32) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (j >= valid) x[j] = -INFINITY;
-  }
-  float m[11];
-#pragma unroll
-  for (int j = 0; j < 10; ++j) m[j] = fmax3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
-  m[10] = fmaxf(x[30], x[31]);
-  const float a0 = fmax3(m[0], m[1], m[2]), a1 = fmax3(m[3], m[4], m[5]), a2 = fmax3(m[6], m[7], m[8]);
-  const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
-  if (cm > best) {
-    best = cm;
-    int idx = 31;
-#pragma unroll
-    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;
-    best_j = jbase + idx;
-  }
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);

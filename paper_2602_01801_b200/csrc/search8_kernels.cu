@@ -51,64 +51,6 @@ __device__ __forceinline__ void umma_ss_f8(uint32_t d_tmem, uint64_t adesc, uint
       : "memory");
 }
 
-// Maximum of 32 raw scores and, only when it beats `best`, its first column.
-__device__ __forceinline__ void chunk_argmax_raw(const uint32_t (&acc)[32], int valid, int jbase, float& best, int& best_j) {
-  float x[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(acc[j]);
-  if (valid < 32) {                                  // only the last tile of a cache has columns to mask
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (j >= valid) x[j] = -INFINITY;
-  }
-  float m[11];
-#pragma unroll
-  for (int j = 0; j < 10; ++j) m[j] = fmax3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
-  m[10] = fmaxf(x[30], x[31]);
-  const float a0 = fmax3(m[0], m[1], m[2]), a1 = fmax3(m[3], m[4], m[5]), a2 = fmax3(m[6], m[7], m[8]);
-  const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
-  if (cm > best) {
-    best = cm;
-    int idx = 31;
-#pragma unroll
-    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;   // first (lowest) column of the maximum
-    best_j = jbase + idx;
-  }
-}
-
-// The same on scores scaled by the norm of their column's key (query-probe ranking: the codes carry directions, the
-// attention score also depends on |k_j|).  kn = |k_j| of the 32 columns (shared memory, the same for every lane).
-__device__ __forceinline__ void chunk_argmax_scaled(const uint32_t (&acc)[32], const float4* __restrict__ kn, int valid, int jbase,
-                                                    float& best, int& best_j) {
-  float x[32];
-#pragma unroll
-  for (int q = 0; q < 8; ++q) {
-    const float4 k4 = kn[q];
-    x[4 * q] = __uint_as_float(acc[4 * q]) * k4.x;
-    x[4 * q + 1] = __uint_as_float(acc[4 * q + 1]) * k4.y;
-    x[4 * q + 2] = __uint_as_float(acc[4 * q + 2]) * k4.z;
-    x[4 * q + 3] = __uint_as_float(acc[4 * q + 3]) * k4.w;
-  }
-  if (valid < 32) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (j >= valid) x[j] = -INFINITY;
-  }
-  float m[11];
-#pragma unroll
-  for (int j = 0; j < 10; ++j) m[j] = fmax3(x[3 * j], x[3 * j + 1], x[3 * j + 2]);
-  m[10] = fmaxf(x[30], x[31]);
-  const float a0 = fmax3(m[0], m[1], m[2]), a1 = fmax3(m[3], m[4], m[5]), a2 = fmax3(m[6], m[7], m[8]);
-  const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
-  if (cm > best) {
-    best = cm;
-    int idx = 31;
-#pragma unroll
-    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;
-    best_j = jbase + idx;
-  }
-}
-
 }  // namespace
 
 // Half a warp per row: |x|, then the code of x / |x| * 16 (an all-zero row gets an all-zero code and norm 0).
@@ -418,36 +360,42 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive_warp(bar_tempty + 8 * buf);      // the scores are in registers: release the accumulator
+        if (!COLMAX) {
+          // COLNORM: scores scaled by |k_j| of their column's key (the codes carry directions, the attention score
+          // also depends on the norm).  Only the last tile of a cache has columns to mask.
+          const float4* kn4 = reinterpret_cast<const float4*>(kn_s + buf * 128 + wg * 64);
+          const int jb = t * 128 + wg * 64;
+          if (valid_cols >= 128) {
+            chunk_argmax_t<false, COLNORM>(vv[0], kn4, 32, jb, best, best_j);
+            chunk_argmax_t<false, COLNORM>(vv[1], kn4 + 8, 32, jb + 32, best, best_j);
+          } else {
+            chunk_argmax_t<true, COLNORM>(vv[0], kn4, valid_cols - wg * 64, jb, best, best_j);
+            chunk_argmax_t<true, COLNORM>(vv[1], kn4 + 8, valid_cols - wg * 64 - 32, jb + 32, best, best_j);
+          }
+          continue;
+        }
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
           const int cc = wg * 2 + c2;
-          if (!COLMAX) {
-            if (COLNORM)
-              chunk_argmax_scaled(vv[c2], reinterpret_cast<const float4*>(kn_s + buf * 128 + cc * 32), valid_cols - cc * 32,
-                                  t * 128 + cc * 32, best, best_j);
-            else
-              chunk_argmax_raw(vv[c2], valid_cols - cc * 32, t * 128 + cc * 32, best, best_j);
-          } else {
-            for (int f = f_lo; f <= f_hi; ++f) {       // empty when the warp has no valid row
-              float x[32];
+          for (int f = f_lo; f <= f_hi; ++f) {         // empty when the warp has no valid row
+            float x[32];
 #pragma unroll
-              for (int j = 0; j < 32; ++j) x[j] = (f_r == f) ? __uint_as_float(vv[c2][j]) * qn : -INFINITY;
-              // butterfly: after it, lane l holds the maximum of column l over the 32 rows
+            for (int j = 0; j < 32; ++j) x[j] = (f_r == f) ? __uint_as_float(vv[c2][j]) * qn : -INFINITY;
+            // butterfly: after it, lane l holds the maximum of column l over the 32 rows
 #pragma unroll
-              for (int o = 16, w = 32; o >= 1; o >>= 1, w >>= 1) {
-                const bool up = (lane & o) != 0;
+            for (int o = 16, w = 32; o >= 1; o >>= 1, w >>= 1) {
+              const bool up = (lane & o) != 0;
 #pragma unroll
-                for (int j = 0; j < w / 2; ++j) {
-                  const float send = up ? x[j] : x[j + w / 2];
-                  const float keep = up ? x[j + w / 2] : x[j];
-                  x[j] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, o));
-                }
+              for (int j = 0; j < w / 2; ++j) {
+                const float send = up ? x[j] : x[j + w / 2];
+                const float keep = up ? x[j + w / 2] : x[j];
+                x[j] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, o));
               }
-              const int col = t * 128 + cc * 32 + lane;
-              if (col < g.cols_b)
-                atomicMax(c.rel + (static_cast<int64_t>(h) * c.max_frames + f) * c.max_prompt + col,
-                          float_to_ordered(x[0] * kn[c2]));
             }
+            const int col = t * 128 + cc * 32 + lane;
+            if (col < g.cols_b)
+              atomicMax(c.rel + (static_cast<int64_t>(h) * c.max_frames + f) * c.max_prompt + col,
+                        float_to_ordered(x[0] * kn[c2]));
           }
         }
       }
