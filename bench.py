@@ -272,7 +272,9 @@ def run_ours(args, cfg):
                 step()
             torch.cuda.current_stream().wait_stream(side)
             graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
+            # captured on the step's own high-priority stream: the kernel nodes keep the priorities of the streams
+            # they were captured on, so AnnCA's nodes stay below the update's inside the graph as well
+            with torch.cuda.graph(graph, stream=torch.cuda.current_stream()):
                 step()
             cache.workspace.copy_(snap)
             graph.replay()
