@@ -9,9 +9,9 @@ import sys
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 SCRIPT = r"""
-import ctypes, itertools
-from paper_2602_01801_b200 import build, fastar
-fastar._LIB_PATH = build.build_library(host_sanitizers=True)
+import ctypes, itertools, sys
+from paper_2602_01801_b200 import fastar
+fastar._LIB_PATH = sys.argv[1]
 lib = fastar.load_library()
 for code in range(-12, 3):
     assert isinstance(lib.fastar_status_string(code), bytes)
@@ -56,9 +56,13 @@ print("HOST-SANITIZERS-OK")
 
 
 def test_host_side_is_clean_under_asan_and_ubsan():
+    # the instrumented library is built here, without the preload: the compiler's own processes must not inherit it
+    sys.path.insert(0, ROOT)
+    from paper_2602_01801_b200 import build
+    lib_path = build.build_library(host_sanitizers=True)
     runtime = subprocess.run(["gcc", "-print-file-name=libasan.so"], capture_output=True, text=True).stdout.strip()
     assert os.path.isabs(runtime) and os.path.exists(runtime), "no AddressSanitizer runtime beside gcc"
     env = dict(os.environ, LD_PRELOAD=runtime, ASAN_OPTIONS="detect_leaks=0:protect_shadow_gap=0:abort_on_error=1",
                UBSAN_OPTIONS="halt_on_error=1:print_stacktrace=1")
-    r = subprocess.run([sys.executable, "-c", SCRIPT], cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
+    r = subprocess.run([sys.executable, "-c", SCRIPT, lib_path], cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0 and "HOST-SANITIZERS-OK" in r.stdout, r.stdout[-1500:] + r.stderr[-4000:]
