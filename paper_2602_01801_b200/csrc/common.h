@@ -88,6 +88,10 @@ struct CacheView {
   // Query-probe correspondence (Section 5.2: a query corresponds to the cached key it attends to most): the similarity kernels
   // rank cached keys by the plain dot product with the probe rows instead of the cosine.
   int raw_dot;
+  // Similarity below which the update does not need the slot of the arg-max (its threshold minus a margin): a row
+  // whose running maximum is still below it is appended whatever its best slot is, so the search kernels skip the
+  // column search for it.  -inf: the slot is always needed (query-probe and Hamming rankings, which a cosine pass follows).
+  float search_floor;
   int hist_weighted;               // key histograms count a slot m times (selector option); high digits in hk_hi / scores_hi
   __nv_bfloat16* hk_hi;            // [H][CAPB][hist_cols]  entry >> 8 (entry & 255 is in hk)
   float* scores_hi;                // [H][max_qb][CAPB]  HQ . HK_hi^T

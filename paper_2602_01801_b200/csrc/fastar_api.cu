@@ -153,6 +153,7 @@ size_t carve(const fastar_cache_desc& d, uint8_t* base, CacheView* v) {
   t.stage[5] = reinterpret_cast<__nv_bfloat16*>(take(H * MT * D * 2));
   t.search_bits = (d.search_bits == 8 || d.search_bits == 1) ? 8 : 16;     // both keep a pool of 128-byte code rows
   t.sign_codes = d.search_bits == 1 ? 1 : 0;
+  t.search_floor = -INFINITY;                // set per update (fastar_tempcache_update knows the threshold)
   t.rep_mean = d.representative == FASTAR_REP_MEAN_KEY ? 1 : 0;
   t.hist_weighted = d.weighted_histograms ? 1 : 0;
   t.hk_hi = t.hist_weighted ? reinterpret_cast<__nv_bfloat16*>(take(H * t.CAPB * t.hist_cols * 2)) : nullptr;
@@ -541,6 +542,11 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
   // packed arg-max words and per-slot match counts start at zero (adjacent in the workspace: one memset)
   if (cudaMemsetAsync(v.best, 0, reinterpret_cast<uint8_t*>(v.cnt) - reinterpret_cast<uint8_t*>(v.best) + static_cast<size_t>(v.H) * v.CAP * 4, st) != cudaSuccess)
     return FASTAR_ERR_CUDA;
+  // A row whose best similarity stays below the threshold is appended whatever its best slot is: the search kernels
+  // skip the column search for running maxima below tau minus a margin that covers their rounding (the similarity
+  // itself is always exact).  Rankings that a cosine pass follows need the slot in every case.
+  CacheView vs = v;
+  vs.search_floor = (q_probe || v.sign_codes) ? -INFINITY : tau - 1e-3f;
   if (v.search_bits == 8) {
     // correspondence search on the 8-bit codes: quantise the new keys, then the fp8 contraction with the arg-max fused
     CUtensorMap tm_a8;
@@ -551,16 +557,16 @@ static int update_impl(fastar_cache_t* c, const void* q_probe, const void* k_new
     if (v.sign_codes) ACCK(FASTAR_K_HASH, launch_sign_rows(v, v.code_new, n, v.max_tokens, v.k8_new, v.max_tokens, st));
     else ACCK(FASTAR_K_HASH, launch_quantize_keys(v, kb, n, khs, kts, v.rnorm_new, v.max_tokens, v.k8_new, v.max_tokens, st));
     if (q_probe) ACCK(FASTAR_K_HASH, launch_quantize_rows(v, pb, n, phs, pts, v.q8_probe, v.max_tokens, v.qn_probe, v.max_tokens, st));
-    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(v, tm_a8, c->tm_pool_k8, n, q_probe != nullptr, st));
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity_fp8(vs, tm_a8, c->tm_pool_k8, n, q_probe != nullptr, st));
     // query-probe and Hamming rankings are not similarities: the threshold is applied to the exact key cosine of the winner
     if (q_probe || v.sign_codes) ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
   } else if (q_probe) {
-    CacheView vr = v;
+    CacheView vr = vs;
     vr.raw_dot = 1;
     ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(vr, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, c->t1_kernel, st));
     ACCK(FASTAR_K_PLAN, launch_probe_cosine(v, kb, n, khs, kts, st));
   } else {
-    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(v, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, c->t1_kernel, st));
+    ACCK(FASTAR_K_T1_SIMILARITY, launch_t1_similarity(vs, tm_a, c->tm_pool_k, c->tm_pool_k_half, n, c->t1_kernel, st));
   }
   ACCK(FASTAR_K_PLAN, launch_plan(v, n, frame_len, tau, st));
   if (v_ready && !v_converted && cudaStreamWaitEvent(st, v_ready, 0) != cudaSuccess) return FASTAR_ERR_CUDA;

@@ -214,6 +214,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
       float best = -INFINITY;
       int best_j = -1;
+      // the cosine of this row's key reaches the update's search floor when |k_i| cos does floor * |k_i|
+      float need_from = -INFINITY;
+      if (EPI == EPI_ARGMAX && !RAW && row < g.rows_a && c.search_floor > -INFINITY) {
+        const float rn_i = c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        if (rn_i > 0.f) need_from = c.search_floor / rn_i;
+      }
       float rn_next = 0.f;                           // 1/|k| of the next tile's keys, loaded one tile ahead
       bool ok = true;
       if (A_TMEM && wg == 0) {
@@ -269,11 +275,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           const float4* rn4 = reinterpret_cast<const float4*>(rn_s + rbuf * 128 + wg * 64);
           const int jb = t * 128 + wg * 64;
           if (valid_cols >= 128) {
-            chunk_argmax_t<false, !RAW>(vv[0], rn4, 32, jb, best, best_j);
-            chunk_argmax_t<false, !RAW>(vv[1], rn4 + 8, 32, jb + 32, best, best_j);
+            chunk_argmax_t<false, !RAW>(vv[0], rn4, 32, jb, need_from, best, best_j);
+            chunk_argmax_t<false, !RAW>(vv[1], rn4 + 8, 32, jb + 32, need_from, best, best_j);
           } else {
-            chunk_argmax_t<true, !RAW>(vv[0], rn4, valid_cols - wg * 64, jb, best, best_j);
-            chunk_argmax_t<true, !RAW>(vv[1], rn4 + 8, valid_cols - wg * 64 - 32, jb + 32, best, best_j);
+            chunk_argmax_t<true, !RAW>(vv[0], rn4, valid_cols - wg * 64, jb, need_from, best, best_j);
+            chunk_argmax_t<true, !RAW>(vv[1], rn4 + 8, valid_cols - wg * 64 - 32, jb + 32, need_from, best, best_j);
           }
           continue;
         }
@@ -505,6 +511,11 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
       float best = -INFINITY;
       int best_j = -1;
+      float need_from = -INFINITY;                   // as in the single-CTA kernel
+      if (!RAW && row < g.rows_a && c.search_floor > -INFINITY) {
+        const float rn_i = c.rnorm_new[static_cast<int64_t>(h) * c.max_tokens + row];
+        if (rn_i > 0.f) need_from = c.search_floor / rn_i;
+      }
       bool ok = true;
       // 1/|k| of the tile's cache keys goes through shared memory; the global load runs one tile ahead so that its
       // latency is not paid between two tiles
@@ -540,11 +551,11 @@ t1_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const float4* rn4 = reinterpret_cast<const float4*>(rn_s + buf * 128 + wg * 64);
         const int jb = t * 128 + wg * 64;
         if (valid_cols >= 128) {
-          chunk_argmax_t<false, !RAW>(vv[0], rn4, 32, jb, best, best_j);
-          chunk_argmax_t<false, !RAW>(vv[1], rn4 + 8, 32, jb + 32, best, best_j);
+          chunk_argmax_t<false, !RAW>(vv[0], rn4, 32, jb, need_from, best, best_j);
+          chunk_argmax_t<false, !RAW>(vv[1], rn4 + 8, 32, jb + 32, need_from, best, best_j);
         } else {
-          chunk_argmax_t<true, !RAW>(vv[0], rn4, valid_cols - wg * 64, jb, best, best_j);
-          chunk_argmax_t<true, !RAW>(vv[1], rn4 + 8, valid_cols - wg * 64 - 32, jb + 32, best, best_j);
+          chunk_argmax_t<true, !RAW>(vv[0], rn4, valid_cols - wg * 64, jb, need_from, best, best_j);
+          chunk_argmax_t<true, !RAW>(vv[1], rn4 + 8, valid_cols - wg * 64 - 32, jb + 32, need_from, best, best_j);
         }
       }
       if (ok && row < g.rows_a && best_j >= 0) {

@@ -354,9 +354,11 @@ __device__ __forceinline__ void fmul2(float& x0, float& x1, float a0, float a1, 
 // acc: raw accumulator bits; rn: 32 floats (16-byte aligned, shared or registers via pointer).
 // MASK: columns >= valid do not count (only the last tile of a cache has any; the caller peels that tile off so that
 // the common path carries no masking code).  SCALE = false ranks the scores as they are (rn4 unused).
+// need_from: running maxima below it need no column (the caller's row is not a match candidate yet): the chunk's first
+// slot stands in, which keeps best_j a live slot.
 template <bool MASK, bool SCALE>
-__device__ __forceinline__ void chunk_argmax_t(const uint32_t (&acc)[32], const float4* rn4, int valid, int jbase, float& best,
-                                               int& best_j) {
+__device__ __forceinline__ void chunk_argmax_t(const uint32_t (&acc)[32], const float4* rn4, int valid, int jbase, float need_from,
+                                               float& best, int& best_j) {
   float x[32];
   if (SCALE) {
 #pragma unroll
@@ -383,10 +385,13 @@ __device__ __forceinline__ void chunk_argmax_t(const uint32_t (&acc)[32], const 
   const float cm = fmax3(fmax3(a0, a1, a2), m[9], m[10]);
   if (cm > best) {
     best = cm;
-    int idx = 31;
+    best_j = jbase;
+    if (cm >= need_from) {
+      int idx = 31;
 #pragma unroll
-    for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;   // first (lowest) column of the maximum
-    best_j = jbase + idx;
+      for (int j = 30; j >= 0; --j) idx = (x[j] == cm) ? j : idx;   // first (lowest) column of the maximum
+      best_j = jbase + idx;
+    }
   }
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {

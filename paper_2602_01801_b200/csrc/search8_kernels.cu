@@ -315,6 +315,8 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
       float best = -INFINITY;
       int best_j = -1;
+      // the scores are 256 x the quantised similarity (both code rows carry the factor 16)
+      const float need_from = (!COLMAX && !COLNORM && c.search_floor > -INFINITY) ? c.search_floor * (kCodeScale * kCodeScale) : -INFINITY;
       float rn_next = 0.f;
       bool ok = true;
       // COLMAX: |q| of this thread's row and the range of frames the warp's 32 rows fall in
@@ -366,11 +368,11 @@ search8_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const float4* kn4 = reinterpret_cast<const float4*>(kn_s + buf * 128 + wg * 64);
           const int jb = t * 128 + wg * 64;
           if (valid_cols >= 128) {
-            chunk_argmax_t<false, COLNORM>(vv[0], kn4, 32, jb, best, best_j);
-            chunk_argmax_t<false, COLNORM>(vv[1], kn4 + 8, 32, jb + 32, best, best_j);
+            chunk_argmax_t<false, COLNORM>(vv[0], kn4, 32, jb, need_from, best, best_j);
+            chunk_argmax_t<false, COLNORM>(vv[1], kn4 + 8, 32, jb + 32, need_from, best, best_j);
           } else {
-            chunk_argmax_t<true, COLNORM>(vv[0], kn4, valid_cols - wg * 64, jb, best, best_j);
-            chunk_argmax_t<true, COLNORM>(vv[1], kn4 + 8, valid_cols - wg * 64 - 32, jb + 32, best, best_j);
+            chunk_argmax_t<true, COLNORM>(vv[0], kn4, valid_cols - wg * 64, jb, need_from, best, best_j);
+            chunk_argmax_t<true, COLNORM>(vv[1], kn4 + 8, valid_cols - wg * 64 - 32, jb + 32, need_from, best, best_j);
           }
           continue;
         }
