@@ -646,8 +646,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
                                                    const int32_t* __restrict__ len, int len_div, int n_fixed, int keep,
                                                    int32_t* __restrict__ out, int64_t out_head_stride, int out_row_stride,
                                                    int out_fill, int32_t* __restrict__ nsel, int force_first, int force_last,
-                                                   const float* __restrict__ src_hi, int* status) {
-  extern __shared__ uint32_t vals[];     // ranking keys: larger key = better entry
+                                                   const float* __restrict__ src_hi, int* status, int sort_np2) {
+  extern __shared__ __align__(16) uint32_t vals[];     // ranking keys: larger key = better entry
   __shared__ int red[32];
   const int row = blockIdx.x, h = blockIdx.y;
   const int n = len ? (len[h] + len_div - 1) / len_div : n_fixed;
@@ -670,11 +670,28 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
   }
   __syncthreads();
   int32_t* orow = out + static_cast<int64_t>(h) * out_head_stride + static_cast<int64_t>(row) * out_row_stride;
+  // Rows that fit: sort (key, -index) in shared memory, flag the k largest, then list the flagged entries in index
+  // order.  Ranking every entry against every other one, the general path below, costs n^2 / 256 steps per thread,
+  // which at 512 key blocks was 0.2 ms of a 8 ms step.
+  if (sort_np2 > 0) {
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(vals + ((n + 3) & ~3));   // 16-byte aligned, behind vals
+    for (int i = threadIdx.x; i < sort_np2; i += blockDim.x)
+      keys[i] = i < n ? (static_cast<unsigned long long>(vals[i]) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(i)) : 0ull;
+    __syncthreads();
+    bitonic_sort_smem(keys, sort_np2);             // ascending: the k best entries are the last k
+    for (int i = threadIdx.x; i < n; i += blockDim.x) vals[i] = 0u;
+    __syncthreads();
+    for (int p = threadIdx.x; p < k; p += blockDim.x)
+      vals[FASTAR_IDX(static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(keys[sort_np2 - 1 - p] & 0xFFFFFFFFull)), n, status)] = 1u;
+    __syncthreads();
+  }
   int run = 0;
   for (int i0 = 0; i0 < n; i0 += blockDim.x) {
     const int i = i0 + threadIdx.x;
     int take = 0;
-    if (i < n) {
+    if (i < n && sort_np2 > 0) {
+      take = static_cast<int>(vals[i]);
+    } else if (i < n) {
       const uint32_t v = vals[i];
       int rank = 0;
       for (int j = 0; j < n; ++j) {
@@ -691,11 +708,21 @@ __global__ void __launch_bounds__(256) topk_kernel(const void* __restrict__ src,
   for (int i = k + threadIdx.x; i < out_fill; i += blockDim.x) orow[i] = -1;
   if (nsel && row == 0 && threadIdx.x == 0) nsel[h] = k;
 }
+// Shared memory of the sorting path for rows of up to n entries (0: rows too long, rank by counting): the keys behind
+// the 32-bit values.
+static int topk_sort_np2(int n) {
+  int np2 = 1;
+  while (np2 < n) np2 <<= 1;
+  return np2 <= 2048 ? np2 : 0;                    // 16 KB of keys at most
+}
+static size_t topk_smem(int n, int np2) { return static_cast<size_t>((n + 3) & ~3) * 4 + static_cast<size_t>(np2) * 8; }
+
 int launch_topk_blocks(const CacheView& c, int nqb, int keep, int force_sink, int force_recent, cudaStream_t st) {
-  topk_kernel<false><<<dim3(nqb, c.H), 256, c.CAPB * 4, st>>>(c.scores, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB, c.len,
+  const int np2 = topk_sort_np2(c.CAPB);
+  topk_kernel<false><<<dim3(nqb, c.H), 256, topk_smem(c.CAPB, np2), st>>>(c.scores, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB, c.len,
                                                             c.PT, 0, keep, c.sel, static_cast<int64_t>(c.max_qb) * c.CAPB, c.CAPB,
                                                             min(keep, c.CAPB), c.nsel, force_sink, force_recent,
-                                                            c.hist_weighted ? c.scores_hi : nullptr, c.status);
+                                                            c.hist_weighted ? c.scores_hi : nullptr, c.status, np2);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 // ---------------------------------------------------------------------------------------------
@@ -747,10 +774,11 @@ int launch_bucket_select(const CacheView& c, int nq, int frame_len, int n_frames
 }
 
 int launch_topk_prompt(const CacheView& c, int n_frames, int np, int keep, cudaStream_t st) {
-  topk_kernel<true><<<dim3(n_frames, c.H), 256, np * 4, st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
-                                                             c.max_prompt, nullptr, 1, np, keep, c.selp,
-                                                             static_cast<int64_t>(c.max_frames) * c.max_prompt, c.max_prompt,
-                                                             min(keep, np), nullptr, 0, 0, nullptr, c.status);
+  const int np2 = topk_sort_np2(np);
+  topk_kernel<true><<<dim3(n_frames, c.H), 256, topk_smem(np, np2), st>>>(c.rel, static_cast<int64_t>(c.max_frames) * c.max_prompt,
+                                                                         c.max_prompt, nullptr, 1, np, keep, c.selp,
+                                                                         static_cast<int64_t>(c.max_frames) * c.max_prompt, c.max_prompt,
+                                                                         min(keep, np), nullptr, 0, 0, nullptr, c.status, np2);
   return cudaGetLastError() == cudaSuccess ? 1 : FASTAR_ERR_CUDA;
 }
 
