@@ -732,7 +732,7 @@ def _random_case(seed):
     return cfg, opts
 
 
-@pytest.mark.parametrize("seed", list(range(12)))
+@pytest.mark.parametrize("seed", list(range(32)))
 def test_random_shapes_and_options(seed):
     # Seeded random cases over head dim, page size, frame shape (row counts that are no multiple of anything), cache
     # capacity (some evict), LSH shape, budgets, threshold, input dtype, search width, correspondence rule and
